@@ -1,0 +1,214 @@
+/*
+ * CPU oracle for the in-context video KV-cache retrieval hot path.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, double-precision
+ * statement of what the five steps compute; the CUDA library never includes,
+ * links or calls it, and it shares no code with the CUDA path.  Only the test
+ * suite, the smoke check and the benchmark's CPU-baseline leg may load it.
+ *
+ * Steps, in the paper's order (Section "ReKV", internal retrieval):
+ *   1. frame representative  = mean of the frame's N_f key vectors, heads
+ *      concatenated                     (internal-retrieval paragraph)
+ *   2. question vector       = mean of the question's N_q query vectors;
+ *      score = cosine similarity, tau=1 (Eq. 2 with tau = 1)
+ *   3. keep the r most similar frames   (Eq. 2 paragraph, "r most relevant")
+ *   4. the retrieved K/V, R, are brought together as the context
+ *   5. O = Attn(Q, R_k, R_v)            (Eq. 3)
+ *
+ * Readings where the paper is silent (each also listed in the design notes):
+ *   - GQA: the G query heads of one KV group are averaged so that question
+ *     and frame vectors share D' = H_kv * D.
+ *   - norms are clamped at 1e-8; NaN scores rank below every number.
+ *   - the last W visible frames (the recent window) are always in the
+ *     context and are not candidates for retrieval.
+ *   - ties go to the lower frame index; selected frames are emitted in
+ *     ascending frame order (temporal order).
+ *   - Attn = softmax(Q K^T / sqrt(D)) V, no mask (all context precedes the
+ *     question), query head h reads KV head floor(h / G).
+ *
+ * Arithmetic: bf16 inputs are widened exactly; every sum is a double; each
+ * stored result is rounded once (to float, and for attention also to bf16).
+ *
+ * Parity pins: every function below is pinned by tests/test_oracle_pins.py
+ * (closed forms, brute force, library routines, invariants).  The paper's
+ * accuracy / recall / latency tables need its datasets and weights and stay
+ * "parity unpinned".
+ */
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <vector>
+
+namespace {
+
+inline double bf16_to_double(uint16_t b) {
+  uint32_t u = (uint32_t)b << 16;
+  float f;
+  std::memcpy(&f, &u, 4);
+  return (double)f;
+}
+
+inline uint16_t float_to_bf16_rne(float x) {
+  uint32_t u;
+  std::memcpy(&u, &x, 4);
+  if ((u & 0x7F800000u) == 0x7F800000u && (u & 0x007FFFFFu)) return (uint16_t)((u >> 16) | 0x40);  // NaN
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return (uint16_t)(u >> 16);
+}
+
+}  // namespace
+
+extern "C" {
+
+/* Step 1.  k: one layer of one frame, token-major [n_tokens][n_kv_heads][head_dim] bf16.
+ * rep[h*head_dim + d] = (1/N_f) * sum_t k[t][h][d], rounded once to float. */
+void oracle_pool_frame(const uint16_t* k, int n_tokens, int n_kv_heads, int head_dim, float* rep) {
+  const int dp = n_kv_heads * head_dim;
+  for (int c = 0; c < dp; ++c) {
+    double s = 0.0;
+    for (int t = 0; t < n_tokens; ++t) s += bf16_to_double(k[(long)t * dp + c]);
+    rep[c] = (float)(s / (double)n_tokens);
+  }
+}
+
+/* Step 2a.  q: one layer of one question, [n_q][n_q_heads][head_dim] bf16.
+ * qa[g*head_dim + d] = mean over the question's tokens and over the G query heads of KV group g. */
+void oracle_question_vector(const uint16_t* q, int n_q, int n_q_heads, int n_kv_heads, int head_dim, double* qa) {
+  const int G = n_q_heads / n_kv_heads;
+  std::vector<double> qbar((size_t)n_q_heads * head_dim, 0.0);
+  for (int h = 0; h < n_q_heads; ++h)
+    for (int d = 0; d < head_dim; ++d) {
+      double s = 0.0;
+      for (int n = 0; n < n_q; ++n) s += bf16_to_double(q[((long)n * n_q_heads + h) * head_dim + d]);
+      qbar[(size_t)h * head_dim + d] = s / (double)n_q;
+    }
+  for (int g = 0; g < n_kv_heads; ++g)
+    for (int d = 0; d < head_dim; ++d) {
+      double s = 0.0;
+      for (int j = 0; j < G; ++j) s += qbar[(size_t)(g * G + j) * head_dim + d];
+      qa[g * head_dim + d] = s / (double)G;
+    }
+}
+
+/* Step 2b.  scores[f] = <qa, rep_f> / (max(|qa|,eps) * max(|rep_f|,eps)), tau = 1.
+ * reps: [n_frames][n_kv_heads*head_dim] float (as stored by step 1). */
+void oracle_score(const uint16_t* q, int n_q, int n_q_heads, int n_kv_heads, int head_dim, const float* reps,
+                  int n_frames, float* scores) {
+  const int dp = n_kv_heads * head_dim;
+  const double eps = 1e-8;
+  std::vector<double> qa(dp);
+  oracle_question_vector(q, n_q, n_q_heads, n_kv_heads, head_dim, qa.data());
+  double qn = 0.0;
+  for (int c = 0; c < dp; ++c) qn += qa[c] * qa[c];
+  qn = std::max(std::sqrt(qn), eps);
+  for (int f = 0; f < n_frames; ++f) {
+    const float* r = reps + (long)f * dp;
+    double dot = 0.0, rn = 0.0;
+    for (int c = 0; c < dp; ++c) {
+      dot += qa[c] * (double)r[c];
+      rn += (double)r[c] * (double)r[c];
+    }
+    rn = std::max(std::sqrt(rn), eps);
+    scores[f] = (float)(dot / (qn * rn));
+  }
+}
+
+/* Step 3.  Candidates are frames [0, n_visible - window).  Order by (score descending, index
+ * ascending), keep k_eff = min(k, #candidates), write them in ascending index order, pad idx_out
+ * (length k) with -1.  *gap_out = score of the last kept minus score of the best rejected
+ * (+inf if nothing is rejected or nothing kept).  Returns k_eff. */
+int oracle_select(const float* scores, int n_visible, int window, int k, int32_t* idx_out, double* gap_out) {
+  int n_cand = std::max(n_visible - window, 0);
+  int k_eff = std::max(std::min(k, n_cand), 0);
+  std::vector<int32_t> order(n_cand);
+  for (int i = 0; i < n_cand; ++i) order[i] = i;
+  auto key = [&](int i) {
+    float s = scores[i];
+    return std::isnan(s) ? -std::numeric_limits<double>::infinity() : (double)s;
+  };
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+    double sa = key(a), sb = key(b);
+    if (sa != sb) return sa > sb;
+    return a < b;
+  });
+  double gap = std::numeric_limits<double>::infinity();
+  if (k_eff > 0 && k_eff < n_cand) gap = key(order[k_eff - 1]) - key(order[k_eff]);
+  if (gap_out) *gap_out = gap;
+  std::vector<int32_t> sel(order.begin(), order.begin() + k_eff);
+  std::sort(sel.begin(), sel.end());
+  for (int i = 0; i < k; ++i) idx_out[i] = i < k_eff ? sel[i] : -1;
+  return k_eff;
+}
+
+/* Step 4.  cache: one layer's K (or V), token-major frames [n_frames][n_tokens][n_kv_heads][head_dim].
+ * Context frame list = idx[0..k_eff) (ascending) followed by frames max(n_visible-window,0) .. n_visible-1.
+ * ctx: [n_kv_heads][n_ctx_frames*n_tokens][head_dim].  Returns the number of context frames. */
+int oracle_gather(const uint16_t* cache, int n_tokens, int n_kv_heads, int head_dim, const int32_t* idx, int k_eff,
+                  int n_visible, int window, uint16_t* ctx) {
+  std::vector<int> frames;
+  for (int i = 0; i < k_eff; ++i) frames.push_back(idx[i]);
+  for (int f = std::max(n_visible - window, 0); f < n_visible; ++f) frames.push_back(f);
+  const int nf = (int)frames.size();
+  const long n_ctx = (long)nf * n_tokens;
+  for (int h = 0; h < n_kv_heads; ++h)
+    for (int j = 0; j < nf; ++j)
+      for (int t = 0; t < n_tokens; ++t)
+        for (int d = 0; d < head_dim; ++d)
+          ctx[((long)h * n_ctx + (long)j * n_tokens + t) * head_dim + d] =
+              cache[(((long)frames[j] * n_tokens + t) * n_kv_heads + h) * head_dim + d];
+  return nf;
+}
+
+/* Step 5.  q: [n_q][n_q_heads][head_dim]; k_ctx, v_ctx: [n_kv_heads][n_ctx][head_dim]; all bf16.
+ * out_f32 (and out_bf16, nullable): [n_q][n_q_heads][head_dim].
+ * probs (nullable): [n_q][n_q_heads][n_ctx] doubles, the softmax rows, for the row-sum pin. */
+void oracle_attend(const uint16_t* q, int n_q, int n_q_heads, int n_kv_heads, int head_dim, const uint16_t* k_ctx,
+                   const uint16_t* v_ctx, long n_ctx, float* out_f32, uint16_t* out_bf16, double* probs) {
+  const int G = n_q_heads / n_kv_heads;
+  const double scale = 1.0 / std::sqrt((double)head_dim);
+  const long rows = (long)n_q * n_q_heads;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long row = 0; row < rows; ++row) {
+    const int h = (int)(row % n_q_heads);
+    const int g = h / G;
+    const uint16_t* qv = q + row * head_dim;
+    const uint16_t* kh = k_ctx + (long)g * n_ctx * head_dim;
+    const uint16_t* vh = v_ctx + (long)g * n_ctx * head_dim;
+    std::vector<double> qd(head_dim), logit((size_t)n_ctx), acc(head_dim, 0.0);
+    for (int d = 0; d < head_dim; ++d) qd[d] = bf16_to_double(qv[d]);
+    double m = -std::numeric_limits<double>::infinity();
+    for (long j = 0; j < n_ctx; ++j) {
+      double s = 0.0;
+      for (int d = 0; d < head_dim; ++d) s += qd[d] * bf16_to_double(kh[j * head_dim + d]);
+      logit[j] = s * scale;
+      m = std::max(m, logit[j]);
+    }
+    double z = 0.0;
+    for (long j = 0; j < n_ctx; ++j) {
+      logit[j] = std::exp(logit[j] - m);
+      z += logit[j];
+    }
+    for (long j = 0; j < n_ctx; ++j) {
+      const double p = logit[j] / z;
+      if (probs) probs[row * n_ctx + j] = p;
+      for (int d = 0; d < head_dim; ++d) acc[d] += p * bf16_to_double(vh[j * head_dim + d]);
+    }
+    for (int d = 0; d < head_dim; ++d) {
+      const float o = (float)acc[d];
+      out_f32[row * head_dim + d] = o;
+      if (out_bf16) out_bf16[row * head_dim + d] = float_to_bf16_rne(o);
+    }
+  }
+}
+
+/* Bytes of K/V cache for a stream: 2 (K and V) * L * T * M * H * D * bytes_per_element
+ * (the appendix's cache-size expression; fp16/bf16 -> 2 bytes). */
+double oracle_kv_cache_bytes(int n_layers, long n_frames, int tokens_per_frame, int n_kv_heads, int head_dim,
+                             int bytes_per_element) {
+  return 2.0 * (double)n_layers * (double)n_frames * (double)tokens_per_frame * (double)n_kv_heads *
+         (double)head_dim * (double)bytes_per_element;
+}
+
+}  // extern "C"

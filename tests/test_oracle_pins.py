@@ -1,0 +1,306 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, independent of the oracle's own code.
+
+Each oracle function is checked against closed forms, brute force, invariants or a library
+routine, chosen so that a dropped term, a wrong sign/index or a transposed operand fails.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import rekv_oracle as orc
+from paper_2503_00540_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf16(x):
+    return torch.as_tensor(x, dtype=torch.float32).to(torch.bfloat16).contiguous()
+
+
+# ----------------------------------------------------------------------------- cache size (appendix formula)
+def test_kv_cache_size_matches_printed_values():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "kv_cache_size.txt")) if l.strip() and not l.startswith("#")]
+    assert len(rows) == 2
+    for name, L, T, M, H, D, b, printed in rows:
+        got = orc.kv_cache_bytes(int(L), int(T), int(M), int(H), int(D), int(b))
+        assert round(got / 2**30, 1) == float(printed), (name, got / 2**30)
+    # term-by-term: doubling any factor doubles the size
+    base = orc.kv_cache_bytes(28, 1800, 196, 4, 128, 2)
+    assert base == 2 * 28 * 1800 * 196 * 4 * 128 * 2
+    assert orc.kv_cache_bytes(56, 1800, 196, 4, 128, 2) == 2 * base
+
+
+# ----------------------------------------------------------------------------- step 1: frame representative
+def test_pool_constant_frame_is_that_constant():
+    k = bf16(torch.full((16, 2, 128), 0.375))
+    assert torch.equal(orc.pool_frame(k), torch.full((256,), 0.375))
+
+
+def test_pool_ramp_is_midpoint_and_heads_concatenate_in_order():
+    n_tok, H, D = 9, 2, 4
+    k = torch.zeros(n_tok, H, D)
+    for t in range(n_tok):
+        for h in range(H):
+            for d in range(D):
+                k[t, h, d] = t * (h + 1) + d  # exact in bf16 (small integers)
+    rep = orc.pool_frame(bf16(k))
+    want = torch.tensor([[4.0 * (h + 1) + d for d in range(D)] for h in range(H)]).reshape(-1)
+    assert torch.equal(rep, want)
+
+
+def test_pool_brute_force_double_loop():
+    k = synth.frame(2503, synth.K, 5, 1, 16, 2, 128)[0]
+    rep = orc.pool_frame(k)
+    kd = k.double().numpy()
+    want = np.zeros(256)
+    for h in range(2):
+        for d in range(128):
+            acc = 0.0
+            for t in range(16):
+                acc += kd[t, h, d]
+            want[h * 128 + d] = acc / 16
+    np.testing.assert_allclose(rep.numpy(), want.astype(np.float32), rtol=0, atol=0)
+
+
+# ----------------------------------------------------------------------------- step 2: question vector + cosine
+def test_question_vector_brute_force_gqa_grouping():
+    q = synth.question(7, 0, 1, 5, 8, 128)[0]  # [5][8][128], G = 4 with 2 kv heads
+    qa = orc.question_vector(q, 2).numpy()
+    qd = q.double().numpy()
+    for g in range(2):
+        for d in (0, 17, 127):
+            want = np.mean([qd[n, h, d] for n in range(5) for h in range(4 * g, 4 * g + 4)])
+            assert abs(qa[g * 128 + d] - want) < 1e-15
+
+
+def _q_from_vector(vec, n_q, Hq, Hkv, D):
+    """A question whose every token/head in group g equals vec[g] (so its question vector is vec)."""
+    G = Hq // Hkv
+    q = torch.zeros(n_q, Hq, D)
+    for h in range(Hq):
+        q[:, h, :] = vec[h // G]
+    return bf16(q)
+
+
+def test_score_closed_forms_parallel_antiparallel_orthogonal():
+    Hq, Hkv, D = 8, 2, 128
+    torch.manual_seed(0)
+    r = bf16(torch.randn(Hkv, D)).float()
+    reps = torch.stack([r.reshape(-1), -r.reshape(-1), torch.zeros(Hkv * D), 3.0 * r.reshape(-1)]).contiguous()
+    # an orthogonal vector: swap pairs with a sign flip
+    orth = r.reshape(-1).clone().reshape(-1, 2).flip(1)
+    orth[:, 0] = -orth[:, 0]
+    reps[2] = orth.reshape(-1)
+    q = _q_from_vector(r, 3, Hq, Hkv, D)
+    s = orc.score(q, reps, Hkv)
+    assert abs(s[0].item() - 1.0) < 1e-6
+    assert abs(s[1].item() + 1.0) < 1e-6
+    assert abs(s[2].item()) < 1e-6
+    assert abs(s[3].item() - 1.0) < 1e-6  # scale invariance in the frame vector
+
+
+def test_score_scale_invariance_in_question_and_zero_norm_clamp():
+    Hq, Hkv, D = 8, 2, 128
+    q = synth.question(3, 1, 1, 6, Hq, D)[0]
+    reps = torch.randn(10, Hkv * D, generator=torch.Generator().manual_seed(1))
+    reps[4] = 0.0
+    s1 = orc.score(q, reps, Hkv)
+    s2 = orc.score(bf16(q.float() * 4.0), reps, Hkv)  # *4 is exact in bf16
+    assert torch.equal(s1, s2)
+    assert s1[4].item() == 0.0 and torch.isfinite(s1).all()
+
+
+def test_score_matches_library_cosine_and_repeat_k_reading_ranks_equal():
+    Hq, Hkv, D, T = 8, 2, 128, 40
+    G = Hq // Hkv
+    q = synth.question(11, 2, 1, 7, Hq, D)[0]
+    reps = torch.stack([orc.pool_frame(synth.frame(11, synth.K, f, 1, 16, Hkv, D)[0]) for f in range(T)])
+    s = orc.score(q, reps, Hkv)
+    # library routine on independently pooled vectors
+    qbar = q.double().mean(0)  # [Hq][D]
+    qa = qbar.reshape(Hkv, G, D).mean(1).reshape(-1)
+    lib = torch.nn.functional.cosine_similarity(qa[None, :], reps.double(), dim=1)
+    assert torch.allclose(s.double(), lib, atol=1e-7, rtol=0)
+    # the other natural GQA reading: concatenate all H_q query heads, repeat each key head G times
+    q_cat = qbar.reshape(-1)
+    reps_rep = reps.double().reshape(T, Hkv, 1, D).expand(T, Hkv, G, D).reshape(T, -1)
+    alt = torch.nn.functional.cosine_similarity(q_cat[None, :], reps_rep, dim=1)
+    assert torch.equal(torch.argsort(alt, descending=True, stable=True), torch.argsort(lib, descending=True, stable=True))
+
+
+# ----------------------------------------------------------------------------- step 3: selection
+def _brute_select(scores, n_vis, W, k):
+    cand = list(range(max(n_vis - W, 0)))
+    key = lambda f: (-(scores[f] if not math.isnan(scores[f]) else -math.inf), f)
+    order = sorted(cand, key=key)
+    return sorted(order[:min(k, len(cand))])
+
+
+def test_select_brute_force_and_nestedness():
+    g = torch.Generator().manual_seed(5)
+    for trial in range(20):
+        T = int(torch.randint(1, 64, (1,), generator=g))
+        W = int(torch.randint(0, 6, (1,), generator=g))
+        s = torch.randn(T, generator=g)
+        prev = set()
+        for k in range(0, T + 2):
+            idx, k_eff, gap = orc.select(s, T, W, k)
+            want = _brute_select(s.tolist(), T, W, k)
+            assert k_eff == len(want)
+            assert idx[:k_eff].tolist() == want
+            assert (idx[k_eff:] == -1).all()
+            assert prev <= set(want)
+            prev = set(want)
+            assert gap >= 0
+
+
+def test_select_ties_go_to_lowest_index_and_nan_ranks_last():
+    s = torch.tensor([0.5, 0.7, 0.5, 0.7, 0.5, float("nan"), 0.1])
+    idx, k_eff, gap = orc.select(s, 7, 0, 3)
+    assert idx.tolist() == [0, 1, 3] and k_eff == 3 and gap == 0.0
+    idx, k_eff, _ = orc.select(s, 7, 0, 6)
+    assert idx.tolist() == [0, 1, 2, 3, 4, 6]
+    idx, k_eff, _ = orc.select(s, 7, 0, 7)
+    assert idx.tolist() == [0, 1, 2, 3, 4, 5, 6]
+
+
+def test_select_window_excluded_and_degenerate_counts():
+    s = torch.tensor([0.1, 0.9, 0.2, 0.95, 0.99])
+    idx, k_eff, _ = orc.select(s, 5, 2, 2)  # frames 3, 4 are the window
+    assert idx.tolist() == [1, 2] and k_eff == 2
+    idx, k_eff, gap = orc.select(s, 5, 2, 8)
+    assert idx.tolist() == [0, 1, 2, -1, -1, -1, -1, -1] and k_eff == 3 and gap == math.inf
+    idx, k_eff, _ = orc.select(s, 2, 4, 3)  # fewer visible frames than the window
+    assert k_eff == 0 and idx.tolist() == [-1, -1, -1]
+    idx, k_eff, _ = orc.select(s, 4, 2, 2)  # n_visible cuts the stream
+    assert idx.tolist() == [0, 1]
+
+
+def test_select_permutation_invariance():
+    g = torch.Generator().manual_seed(9)
+    s = torch.randn(50, generator=g)
+    perm = torch.randperm(50, generator=g)
+    idx, k_eff, _ = orc.select(s, 50, 0, 12)
+    idx_p, k_eff_p, _ = orc.select(s[perm].contiguous(), 50, 0, 12)
+    # position j of the permuted array holds original frame perm[j]
+    assert sorted(perm[idx_p[:k_eff_p].long()].tolist()) == idx[:k_eff].tolist()
+
+
+def test_planted_needle_frame_is_retrieved():
+    """Adding a multiple of one frame's representative to every question token makes that frame win."""
+    L, Hq, Hkv, D, Nf, T = 1, 8, 2, 128, 16, 64
+    G = Hq // Hkv
+    cache = orc.OracleCache(L, Hq, Hkv, D, Nf, window=4)
+    for f in range(T):
+        cache.append(synth.frame(2503, synth.K, f, L, Nf, Hkv, D), synth.frame(2503, synth.V, f, L, Nf, Hkv, D))
+    target = 23
+    q = synth.question(2503, 0, L, 16, Hq, D).float()
+    rep = cache.reps[target][0].reshape(Hkv, D)
+    for h in range(Hq):
+        q[0, :, h, :] += 8.0 * rep[h // G]
+    scores, idx, k_eff, _ = cache.retrieve(bf16(q), 1, T)
+    assert k_eff == 1 and idx[0, 0].item() == target
+
+
+# ----------------------------------------------------------------------------- step 4: gather
+def test_gather_is_a_pure_copy_in_temporal_order():
+    L, Hkv, D, Nf, T, W = 1, 2, 128, 16, 20, 3
+    cacheK = torch.stack([synth.frame(1, synth.K, f, L, Nf, Hkv, D)[0] for f in range(T)]).contiguous()
+    idx = torch.tensor([2, 7, 11, -1], dtype=torch.int32)
+    ctx = orc.gather(cacheK, idx, 3, 18, W)  # n_visible = 18 -> window frames 15, 16, 17
+    frames = [2, 7, 11, 15, 16, 17]
+    assert ctx.shape == (Hkv, len(frames) * Nf, D)
+    for h in range(Hkv):
+        for j, f in enumerate(frames):
+            assert torch.equal(ctx[h, j * Nf:(j + 1) * Nf], cacheK[f, :, h, :])
+
+
+# ----------------------------------------------------------------------------- step 5: attention (Eq. 3)
+def _rand_ctx(seed, Hkv, n_ctx, D):
+    g = torch.Generator().manual_seed(seed)
+    return bf16(torch.randn(Hkv, n_ctx, D, generator=g)), bf16(torch.randn(Hkv, n_ctx, D, generator=g))
+
+
+def test_attend_softmax_rows_sum_to_one_and_ones_value_gives_ones():
+    q = synth.question(1, 0, 1, 4, 8, 128)[0]
+    k, _ = _rand_ctx(0, 2, 37, 128)
+    v = bf16(torch.ones(2, 37, 128))
+    out, out_b, probs = orc.attend(q, k, v, want_probs=True)
+    assert torch.allclose(probs.sum(-1), torch.ones(4, 8, dtype=torch.float64), atol=1e-14)
+    assert (probs >= 0).all()
+    assert torch.allclose(out, torch.ones_like(out), atol=1e-6)
+
+
+def test_attend_single_token_returns_its_value_and_equal_keys_give_mean_value():
+    q = synth.question(1, 1, 1, 3, 8, 128)[0]
+    k, v = _rand_ctx(1, 2, 1, 128)
+    out, _, _ = orc.attend(q, k, v)
+    for h in range(8):
+        assert torch.equal(out[:, h, :], v[h // 4, 0].float().expand(3, 128))
+    k2 = bf16(torch.randn(2, 1, 128, generator=torch.Generator().manual_seed(3))).expand(2, 9, 128).contiguous()
+    _, v2 = _rand_ctx(2, 2, 9, 128)
+    out2, _, _ = orc.attend(q, k2, v2)
+    for h in range(8):
+        want = v2[h // 4].double().mean(0).float()
+        assert torch.allclose(out2[0, h], want, atol=1e-6)
+
+
+def test_attend_matches_library_sdpa_with_gqa_head_repeat():
+    Hq, Hkv, D, n_ctx, n_q = 8, 2, 128, 83, 5
+    q = synth.question(4, 2, 1, n_q, Hq, D)[0]
+    k, v = _rand_ctx(4, Hkv, n_ctx, D)
+    out, out_b, _ = orc.attend(q, k, v)
+    qd = q.double().permute(1, 0, 2)[None]  # [1][Hq][n_q][D]
+    kd = k.double().repeat_interleave(Hq // Hkv, dim=0)[None]
+    vd = v.double().repeat_interleave(Hq // Hkv, dim=0)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(qd, kd, vd)[0].permute(1, 0, 2)
+    assert torch.allclose(out.double(), ref, atol=2e-7, rtol=0)
+    assert torch.equal(out_b, out.to(torch.bfloat16))
+
+
+def test_full_retrieval_equals_full_attention_over_all_visible_frames():
+    """k >= number of candidates: the retrieved context is every visible frame, so the whole
+    five-step path must equal plain attention over the visible stream."""
+    L, Hq, Hkv, D, Nf, T, W = 1, 8, 2, 128, 16, 24, 4
+    cache = orc.OracleCache(L, Hq, Hkv, D, Nf, window=W)
+    for f in range(T):
+        cache.append(synth.frame(540, synth.K, f, L, Nf, Hkv, D), synth.frame(540, synth.V, f, L, Nf, Hkv, D))
+    q = synth.question(540, 0, L, 6, Hq, D)
+    n_vis = 21
+    res = cache.question(q, top_k=64, n_visible=n_vis)
+    assert res["k_eff"] == n_vis - W
+    assert res["idx"][0, :n_vis - W].tolist() == list(range(n_vis - W))
+    k_all = cache.layer_cache(0, "k")[:n_vis].permute(2, 0, 1, 3).reshape(Hkv, n_vis * Nf, D)
+    v_all = cache.layer_cache(0, "v")[:n_vis].permute(2, 0, 1, 3).reshape(Hkv, n_vis * Nf, D)
+    assert torch.equal(res["k_ctx"][0], k_all) and torch.equal(res["v_ctx"][0], v_all)
+    qd = q[0].double().permute(1, 0, 2)[None]
+    kd = k_all.double().repeat_interleave(Hq // Hkv, dim=0)[None]
+    vd = v_all.double().repeat_interleave(Hq // Hkv, dim=0)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(qd, kd, vd)[0].permute(1, 0, 2)
+    assert torch.allclose(res["out"][0].double(), ref, atol=2e-7, rtol=0)
+
+
+def test_attention_is_invariant_to_context_order():
+    q = synth.question(8, 0, 1, 2, 8, 128)[0]
+    k, v = _rand_ctx(8, 2, 40, 128)
+    perm = torch.randperm(40, generator=torch.Generator().manual_seed(0))
+    a, _, _ = orc.attend(q, k, v)
+    b, _, _ = orc.attend(q, k[:, perm].contiguous(), v[:, perm].contiguous())
+    assert torch.allclose(a, b, atol=1e-6)
+
+
+# ----------------------------------------------------------------------------- input generator
+def test_synthetic_inputs_have_the_stated_distribution():
+    k = synth.frame(2503, synth.K, 0, 2, 196, 4, 128, off_scale=0.0).float()
+    assert abs(k.mean().item()) < 0.01 and abs(k.std().item() - 1.0) < 0.01
+    ko = synth.frame(2503, synth.K, 0, 2, 196, 4, 128, off_scale=0.5).float()
+    off = ko.mean(1)  # per (layer, head, dim) frame mean ~ N(0, 0.5^2 + 1/196)
+    assert abs(off.std().item() - math.sqrt(0.25 + 1 / 196)) < 0.03
+    # stateless: a layer slice equals the same layer generated alone
+    k1 = synth.frame(2503, synth.K, 0, 1, 196, 4, 128, off_scale=0.5, layer0=1)
+    assert torch.equal(k1[0], synth.frame(2503, synth.K, 0, 2, 196, 4, 128, off_scale=0.5)[1])
+    lens = synth.question_lengths(7, 64, 24, 64)
+    assert min(lens) >= 24 and max(lens) <= 64 and len(set(lens)) > 10
