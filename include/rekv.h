@@ -1,0 +1,167 @@
+/*
+ * librekv -- in-context video KV-cache retrieval hot path for one B200 (sm_100a).
+ *
+ * A video stream's per-layer K/V is appended frame by frame; a question is answered from
+ * the query-relevant frames only.  The library covers the five steps of the paper's
+ * internal retrieval (Section "ReKV"):
+ *
+ *   1. frame representative = mean of the frame's N_f key vectors, heads concatenated
+ *      ("Internal Video KV-Cache Retrieval": v = 1/N_f * sum_j k_j)       rekv_append_frame
+ *   2. question vector = mean of the question's N_q query vectors; cosine similarity with
+ *      tau = 1 (Eq. 2), independently in every layer                        rekv_retrieve
+ *   3. the r most similar frames are kept (Eq. 2 paragraph)                rekv_retrieve
+ *   4. the retrieved K/V, R, are brought onto the GPU as the context        rekv_gather
+ *   5. O = Attn(Q, R_k, R_v)  (Eq. 3), GQA, over retrieved frames plus a recent window
+ *                                                                           rekv_attend
+ *
+ * Conventions
+ *   - C ABI, plain pointers.  "device" pointers are CUDA device addresses on the context's
+ *     device; "host" pointers are ordinary host memory.  bf16 tensors are passed as void*.
+ *   - Every call returns 0 (or a non-negative value where stated) on success and a negative
+ *     REKV_ERR_* code on failure; it never aborts.  rekv_last_error() gives the message.
+ *   - The caller owns every input and output buffer; the context owns the store, the
+ *     representative table and all scratch memory.
+ *   - Work is enqueued on the caller's CUDA stream (`stream`, a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and the call returns without synchronising.
+ *     Internal side streams are fenced to the caller's stream with events.
+ *   - A context is not thread-safe.  Append and question calls may be interleaved freely
+ *     from one thread; a question sees exactly the frames [0, n_visible).
+ *   - The library has no CPU fallback: without a CUDA device rekv_create fails.
+ */
+#ifndef REKV_H_
+#define REKV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rekv_ctx rekv_ctx;
+
+enum {
+  REKV_OK = 0,
+  REKV_ERR_ARG = -1,     /* bad argument (null pointer, size out of range, unsupported shape) */
+  REKV_ERR_FULL = -2,    /* append past max_frames */
+  REKV_ERR_EMPTY = -3,   /* question with n_visible == 0 */
+  REKV_ERR_ALLOC = -4,   /* device or pinned-host allocation failed */
+  REKV_ERR_CUDA = -5,    /* a CUDA call or launch failed */
+  REKV_ERR_TIMEOUT = -6, /* a bounded device-side wait expired (read from the status word) */
+  REKV_ERR_STATE = -7    /* call order violated (attend without a preceding gather, ...) */
+};
+
+/* rekv_config.flags */
+enum {
+  REKV_FLAG_HOST_GATHER_COPY_ENGINE = 1u << 0, /* host tier: per-page cudaMemcpyAsync instead of the
+                                                  zero-copy gather kernel (needs a host sync on the indices) */
+  REKV_FLAG_ATTEND_LEGACY_MMA = 1u << 1         /* use the mma.sync attention kernel instead of tcgen05 */
+};
+
+typedef struct {
+  int32_t n_layers;          /* L */
+  int32_t n_q_heads;         /* H_q; must be a multiple of n_kv_heads */
+  int32_t n_kv_heads;        /* H_kv */
+  int32_t head_dim;          /* D; must be 128 */
+  int32_t tokens_per_frame;  /* N_f, fixed per context (the paper's M); 1..256 */
+  int32_t max_frames;        /* stream capacity; an append past it returns REKV_ERR_FULL */
+  int32_t hbm_tail_frames;   /* 0: the whole cache lives in HBM.  n > 0: every page lives in pinned host
+                                memory and only the most recent n frames are also kept in HBM */
+  int32_t window_frames;     /* W: the last W visible frames are always part of a question's context and
+                                are not retrieval candidates; W <= hbm_tail_frames when offloaded */
+  int32_t block_frames;      /* frames per retrieval block (the paper's b); only 1 is accepted */
+  int32_t max_q_tokens;      /* upper bound on the sum of question lengths in one batch */
+  int32_t max_topk;          /* upper bound on top_k */
+  int32_t max_questions;     /* upper bound on questions per batch (<= 64) */
+  int32_t device;            /* CUDA device ordinal */
+  uint32_t flags;
+} rekv_config;
+
+typedef struct {
+  int64_t frames;            /* frames appended so far */
+  int64_t kv_bytes_hbm;      /* bytes of K/V pages currently resident in HBM */
+  int64_t kv_bytes_host;     /* bytes of K/V pages held in pinned host memory */
+  int64_t kv_bytes_logical;  /* 2 * L * frames * N_f * H_kv * D * 2: the appendix's cache-size expression */
+  int64_t rep_bytes;         /* bytes of the representative table in use */
+  int64_t page_bytes;        /* bytes of one (layer, frame) page: K and V, all KV heads */
+  int64_t last_link_bytes;   /* bytes the last rekv_gather pulled from pinned host memory */
+  int32_t last_k_eff;        /* frames actually retrieved per (layer, question) by the last question */
+  int32_t last_ctx_frames;   /* k_eff + window frames of the last gather */
+} rekv_stats_t;
+
+/* Creates a context on cfg->device: allocates the frame store (HBM tier, and the pinned-host tier
+ * when hbm_tail_frames > 0), the fp32 representative table [max_frames][L][H_kv*D] and scratch
+ * sized from the max_* fields.  *out receives the context.  Fails with REKV_ERR_ARG on an
+ * unsupported shape and REKV_ERR_ALLOC / REKV_ERR_CUDA when memory or a device is missing. */
+int rekv_create(const rekv_config* cfg, rekv_ctx** out);
+
+/* Frees everything the context owns.  Synchronises the device first. */
+int rekv_destroy(rekv_ctx* ctx);
+
+/* Step 1 (+ paging).  k, v: device bf16 [L][N_f][H_kv][D], token-major as a decoder emits them.
+ * Stores the frame's K/V as page (frame, layer) and the frame representative
+ * rep[frame][layer][h*D+d] = 1/N_f * sum_t k[layer][t][h][d] (fp32).  On an offloaded context the
+ * page is also written through to pinned host memory on an internal stream.
+ * Returns the new frame's index (>= 0), REKV_ERR_FULL when the store is full. */
+int rekv_append_frame(rekv_ctx* ctx, const void* k, const void* v, void* stream);
+
+/* Steps 2-3 for a batch of nQ independent questions, in every layer.
+ *   q         device bf16, packed [L][sum_Nq][H_q][D]; question i owns rows cu_q[i] .. cu_q[i+1]
+ *   cu_q      HOST int32[nQ+1], prefix sums of the question lengths, cu_q[0] == 0
+ *   top_k     frames to retrieve per (layer, question) (the paper's r), 0..max_topk
+ *   n_visible frames the questions may see: frames [0, n_visible) (question time stamp)
+ *   idx_out   device int32 [L][nQ][top_k]: the selected frames in ascending frame order, padded
+ *             with -1 past k_eff = min(top_k, max(n_visible - W, 0))
+ *   scores_out (nullable) device fp32 [L][nQ][n_visible]: cosine similarity of every visible frame
+ * The question vector averages the question's tokens and the G = H_q/H_kv query heads of each KV
+ * group; score = <q, rep> / (max(|q|,1e-8) * max(|rep|,1e-8)).  Candidates are frames
+ * [0, n_visible - W); ties go to the lower frame index; NaN ranks below every number.
+ * Returns k_eff. */
+int rekv_retrieve(rekv_ctx* ctx, const void* q, const int32_t* cu_q, int nQ, int top_k, int n_visible,
+                  int32_t* idx_out, float* scores_out, void* stream);
+
+/* Step 4.  idx: device int32 [L][nQ][top_k] as written by rekv_retrieve, or the caller's own list
+ * with the same shape: its first k_eff = min(top_k, max(n_visible - W, 0)) entries per (layer,
+ * question) must be frames in [0, n_visible) (an entry outside that range is reported by
+ * rekv_check_status as REKV_ERR_ARG).  Builds the context of every (layer, question):
+ * the selected frames in list order, then frames max(n_visible - W, 0) .. n_visible-1.  Pages that
+ * live only in pinned host memory are pulled over the host link into an HBM staging area (on an
+ * internal stream, layer by layer).  rekv_attend reads this context.
+ *   k_ctx, v_ctx (nullable, both or neither): device bf16 [L][nQ][H_kv][(k_eff+W')*N_f][D] with
+ *   W' = min(W, n_visible); when given, the context is also written out contiguously, token rows
+ *   in context order -- a bit-exact copy of the stored K/V.
+ * Returns the number of context frames per (layer, question). */
+int rekv_gather(rekv_ctx* ctx, const int32_t* idx, int nQ, int top_k, int n_visible, void* k_ctx, void* v_ctx,
+                void* stream);
+
+/* Step 5 (Eq. 3).  q, cu_q, nQ as in rekv_retrieve and consistent with the preceding rekv_gather.
+ * out: device bf16 [L][sum_Nq][H_q][D].  For every layer, question token n and query head h:
+ * out = softmax(q . K_ctx^T / sqrt(D)) V_ctx over the gathered context of KV head floor(h/G);
+ * no mask (every context token precedes the question); bf16 operands, fp32 accumulation and softmax.
+ * Returns 0, or REKV_ERR_STATE without a preceding gather. */
+int rekv_attend(rekv_ctx* ctx, const void* q, const int32_t* cu_q, int nQ, void* out, void* stream);
+
+/* Fills *out with store accounting and the last call's counters. */
+int rekv_stats(rekv_ctx* ctx, rekv_stats_t* out);
+
+/* Reads (and clears) the device status word after synchronising `stream`: 0, or REKV_ERR_TIMEOUT
+ * if a bounded device-side wait gave up since the last check. */
+int rekv_check_status(rekv_ctx* ctx, void* stream);
+
+/* Message of the last failure on this context (or of the last failed rekv_create when ctx is NULL).
+ * The pointer stays valid until the next failing call. */
+const char* rekv_last_error(rekv_ctx* ctx);
+
+/* Test helpers.  rekv_get_reps copies the representatives of frames [0, n_frames) of one layer to
+ * dev_out, device fp32 [n_frames][H_kv*D].  rekv_get_page copies one stored (frame, layer) page back
+ * in plain layout: k_out, v_out device bf16 [H_kv][N_f][D] (from HBM if resident, else from host). */
+int rekv_get_reps(rekv_ctx* ctx, int layer, int n_frames, float* dev_out, void* stream);
+int rekv_get_page(rekv_ctx* ctx, int frame, int layer, void* k_out, void* v_out, void* stream);
+
+/* Number of kernels this library has launched on the context since creation (for launch counting). */
+int64_t rekv_launch_count(rekv_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+
+#endif /* REKV_H_ */

@@ -13,7 +13,7 @@ CSRC = os.path.join(PKG, "csrc")
 SYNTH = os.path.join(PKG, "synth")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "-shared",
-              "-Xcompiler", "-fPIC", "--use_fast_math", "-Xptxas", "-v"]
+              "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
 LIBREKV = os.path.join(CSRC, "librekv.so")
 LIBSYNTH_CPU = os.path.join(SYNTH, "librekv_synth_cpu.so")

@@ -1,0 +1,410 @@
+// The C ABI of librekv: context life cycle, argument checks, stream/event plumbing.
+// Every step of the path runs in the kernels of the k_*.cu files; this file only launches them.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "rekv_internal.cuh"
+
+static thread_local std::string g_create_error;
+
+void rekv_set_error(rekv_ctx* ctx, const char* msg) {
+  if (ctx)
+    ctx->err = msg;
+  else
+    g_create_error = msg;
+}
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  explicit DeviceGuard(int dev) {
+    cudaGetDevice(&prev);
+    if (prev != dev) cudaSetDevice(dev);
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    cudaGetDevice(&cur);
+    if (prev >= 0 && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+constexpr long long ARENA_BYTES = 4ll << 30;
+
+int build_qbatch(rekv_ctx* c, const int32_t* cu_q, int nQ, QBatch* qb) {
+  if (!cu_q) REKV_FAIL(c, REKV_ERR_ARG, "cu_q is null");
+  if (nQ < 1 || nQ > c->cfg.max_questions) REKV_FAIL(c, REKV_ERR_ARG, "nQ=%d outside [1, %d]", nQ, c->cfg.max_questions);
+  if (cu_q[0] != 0) REKV_FAIL(c, REKV_ERR_ARG, "cu_q[0] must be 0");
+  qb->nQ = nQ;
+  for (int i = 0; i < nQ; ++i) {
+    if (cu_q[i + 1] <= cu_q[i]) REKV_FAIL(c, REKV_ERR_ARG, "question %d has no tokens", i);
+    qb->cu[i] = cu_q[i];
+  }
+  qb->cu[nQ] = cu_q[nQ];
+  qb->sumNq = cu_q[nQ];
+  if (qb->sumNq > c->cfg.max_q_tokens)
+    REKV_FAIL(c, REKV_ERR_ARG, "sum of question lengths %d exceeds max_q_tokens %d", qb->sumNq, c->cfg.max_q_tokens);
+  return 0;
+}
+
+void free_ctx(rekv_ctx* c) {
+  if (!c) return;
+  cudaDeviceSynchronize();
+  cudaFree(c->sv.hbm);
+  cudaFree(c->sv.staging);
+  cudaFree(c->sv.reps);
+  cudaFree(c->d_host_arenas);
+  cudaFree(c->qa);
+  cudaFree(c->qnorm);
+  cudaFree(c->scores);
+  cudaFree(c->ctx_tbl);
+  cudaFree(c->part_o);
+  cudaFree(c->part_ml);
+  cudaFree(c->status);
+  cudaFree(c->link_bytes);
+  for (char* a : c->host_arenas) cudaFreeHost(a);
+  for (cudaEvent_t e : c->slot_events) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->layer_events) cudaEventDestroy(e);
+  if (c->ev_main) cudaEventDestroy(c->ev_main);
+  if (c->ev_side) cudaEventDestroy(c->ev_side);
+  if (c->side) cudaStreamDestroy(c->side);
+  delete c;
+}
+
+}  // namespace
+
+extern "C" {
+
+int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
+  if (!cfg || !out) REKV_FAIL(nullptr, REKV_ERR_ARG, "null config or output pointer");
+  *out = nullptr;
+  if (cfg->head_dim != REKV_HEAD_DIM) REKV_FAIL(nullptr, REKV_ERR_ARG, "head_dim must be 128, got %d", cfg->head_dim);
+  if (cfg->n_layers < 1 || cfg->n_layers > 1023) REKV_FAIL(nullptr, REKV_ERR_ARG, "n_layers=%d out of range", cfg->n_layers);
+  if (cfg->n_kv_heads < 1 || cfg->n_kv_heads > 8 || cfg->n_q_heads < cfg->n_kv_heads ||
+      cfg->n_q_heads % cfg->n_kv_heads)
+    REKV_FAIL(nullptr, REKV_ERR_ARG, "unsupported head counts: %d query / %d kv (kv <= 8, query a multiple of kv)",
+              cfg->n_q_heads, cfg->n_kv_heads);
+  if (cfg->tokens_per_frame < 1 || cfg->tokens_per_frame > 256)
+    REKV_FAIL(nullptr, REKV_ERR_ARG, "tokens_per_frame=%d outside [1, 256]", cfg->tokens_per_frame);
+  if (cfg->max_frames < 1) REKV_FAIL(nullptr, REKV_ERR_ARG, "max_frames must be positive");
+  if (cfg->block_frames != 1) REKV_FAIL(nullptr, REKV_ERR_ARG, "block_frames=%d: only 1 is supported", cfg->block_frames);
+  if (cfg->window_frames < 0) REKV_FAIL(nullptr, REKV_ERR_ARG, "window_frames must be >= 0");
+  if (cfg->hbm_tail_frames < 0 || (cfg->hbm_tail_frames > 0 && cfg->window_frames > cfg->hbm_tail_frames))
+    REKV_FAIL(nullptr, REKV_ERR_ARG, "window_frames=%d must fit in hbm_tail_frames=%d", cfg->window_frames,
+              cfg->hbm_tail_frames);
+  if (cfg->max_questions < 1 || cfg->max_questions > REKV_MAX_QUESTIONS)
+    REKV_FAIL(nullptr, REKV_ERR_ARG, "max_questions=%d outside [1, %d]", cfg->max_questions, REKV_MAX_QUESTIONS);
+  if (cfg->max_q_tokens < 1 || cfg->max_topk < 0) REKV_FAIL(nullptr, REKV_ERR_ARG, "max_q_tokens / max_topk out of range");
+
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0) {
+    cudaGetLastError();
+    REKV_FAIL(nullptr, REKV_ERR_CUDA, "no CUDA device: librekv has no CPU path");
+  }
+  if (cfg->device < 0 || cfg->device >= n_dev) REKV_FAIL(nullptr, REKV_ERR_ARG, "device %d not present", cfg->device);
+  DeviceGuard guard(cfg->device);
+
+  rekv_ctx* c = new (std::nothrow) rekv_ctx();
+  if (!c) REKV_FAIL(nullptr, REKV_ERR_ALLOC, "out of host memory");
+  c->cfg = *cfg;
+  c->device = cfg->device;
+  c->frames = 0;
+  c->launches = 0;
+  c->d_host_arenas = nullptr;
+  c->side = nullptr;
+  c->ev_main = c->ev_side = nullptr;
+  c->d2h_pending = false;
+  c->gathered = false;
+  c->gather_layerwise = false;
+  memset(&c->sv, 0, sizeof(c->sv));
+  c->qa = c->qnorm = c->scores = c->part_o = c->part_ml = nullptr;
+  c->ctx_tbl = nullptr;
+  c->status = nullptr;
+  c->link_bytes = nullptr;
+
+  StoreView& s = c->sv;
+  s.L = cfg->n_layers;
+  s.Hq = cfg->n_q_heads;
+  s.Hkv = cfg->n_kv_heads;
+  s.G = s.Hq / s.Hkv;
+  s.Nf = cfg->tokens_per_frame;
+  s.Dp = s.Hkv * REKV_HEAD_DIM;
+  s.max_frames = cfg->max_frames;
+  s.tail = cfg->hbm_tail_frames;
+  s.page_bytes = (long long)s.Hkv * 2 * s.Nf * 256;
+  const long long frame_bytes = s.page_bytes * s.L;
+  s.frames_per_arena = (int)(ARENA_BYTES / frame_bytes);
+  if (s.frames_per_arena < 1) s.frames_per_arena = 1;
+
+#define CREATE_CUDA(call, what)                                                                              \
+  do {                                                                                                       \
+    cudaError_t _e = (call);                                                                                 \
+    if (_e != cudaSuccess) {                                                                                 \
+      char _b[256];                                                                                          \
+      snprintf(_b, sizeof(_b), "%s: %s", what, cudaGetErrorString(_e));                                      \
+      cudaGetLastError();                                                                                    \
+      free_ctx(c);                                                                                           \
+      rekv_set_error(nullptr, _b);                                                                           \
+      return _e == cudaErrorMemoryAllocation ? REKV_ERR_ALLOC : REKV_ERR_CUDA;                               \
+    }                                                                                                        \
+  } while (0)
+
+  const long long hbm_frames = s.tail > 0 ? s.tail : s.max_frames;
+  CREATE_CUDA(cudaMalloc(&s.hbm, (size_t)(hbm_frames * frame_bytes)), "allocating the HBM frame store");
+  CREATE_CUDA(cudaMalloc(&s.reps, (size_t)s.L * s.max_frames * s.Dp * sizeof(float)), "allocating the representative table");
+  const int ctx_frames_max = cfg->max_topk + cfg->window_frames;
+  const int maxQ = cfg->max_questions;
+  CREATE_CUDA(cudaMalloc(&c->qa, (size_t)s.L * maxQ * s.Dp * sizeof(float)), "allocating question vectors");
+  CREATE_CUDA(cudaMalloc(&c->qnorm, (size_t)s.L * maxQ * sizeof(float)), "allocating question norms");
+  CREATE_CUDA(cudaMalloc(&c->scores, (size_t)s.L * maxQ * s.max_frames * sizeof(float)), "allocating the score buffer");
+  CREATE_CUDA(cudaMalloc(&c->ctx_tbl, (size_t)s.L * maxQ * (ctx_frames_max + 1) * sizeof(char*)), "allocating the context table");
+  c->part_units = 2048;
+  CREATE_CUDA(cudaMalloc(&c->part_o, c->part_units * 128 * 128 * sizeof(float)), "allocating split-KV partials");
+  CREATE_CUDA(cudaMalloc(&c->part_ml, c->part_units * 128 * 2 * sizeof(float)), "allocating split-KV partials");
+  CREATE_CUDA(cudaMalloc(&c->status, sizeof(int)), "allocating the status word");
+  CREATE_CUDA(cudaMemset(c->status, 0, sizeof(int)), "clearing the status word");
+  CREATE_CUDA(cudaMalloc(&c->link_bytes, sizeof(unsigned long long)), "allocating counters");
+  CREATE_CUDA(cudaMemset(c->link_bytes, 0, sizeof(unsigned long long)), "clearing counters");
+  CREATE_CUDA(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking), "creating the side stream");
+  CREATE_CUDA(cudaEventCreateWithFlags(&c->ev_main, cudaEventDisableTiming), "creating events");
+  CREATE_CUDA(cudaEventCreateWithFlags(&c->ev_side, cudaEventDisableTiming), "creating events");
+
+  if (s.tail > 0) {
+    // pinned-host tier: arenas of whole frames, allocated up front so that append never blocks
+    const int n_arenas = (s.max_frames + s.frames_per_arena - 1) / s.frames_per_arena;
+    for (int a = 0; a < n_arenas; ++a) {
+      int fr = s.max_frames - a * s.frames_per_arena;
+      if (fr > s.frames_per_arena) fr = s.frames_per_arena;
+      char* p = nullptr;
+      cudaError_t e = cudaHostAlloc((void**)&p, (size_t)fr * frame_bytes, cudaHostAllocDefault);
+      if (e != cudaSuccess) {
+        cudaGetLastError();
+        char b[256];
+        snprintf(b, sizeof(b), "pinning host arena %d of %d (%lld bytes): %s", a, n_arenas, fr * frame_bytes,
+                 cudaGetErrorString(e));
+        free_ctx(c);
+        rekv_set_error(nullptr, b);
+        return REKV_ERR_ALLOC;
+      }
+      c->host_arenas.push_back(p);
+    }
+    CREATE_CUDA(cudaMalloc(&c->d_host_arenas, n_arenas * sizeof(char*)), "allocating the arena table");
+    CREATE_CUDA(cudaMemcpy(c->d_host_arenas, c->host_arenas.data(), n_arenas * sizeof(char*), cudaMemcpyHostToDevice),
+                "uploading the arena table");
+    s.host_arenas = c->d_host_arenas;
+    CREATE_CUDA(cudaMalloc(&s.staging, (size_t)s.L * maxQ * ctx_frames_max * s.page_bytes), "allocating gather staging");
+    c->slot_events.resize(s.tail);
+    c->slot_event_valid.assign(s.tail, 0);
+    for (int i = 0; i < s.tail; ++i)
+      CREATE_CUDA(cudaEventCreateWithFlags(&c->slot_events[i], cudaEventDisableTiming), "creating events");
+    c->layer_events.resize(s.L);
+    for (int i = 0; i < s.L; ++i)
+      CREATE_CUDA(cudaEventCreateWithFlags(&c->layer_events[i], cudaEventDisableTiming), "creating events");
+  }
+#undef CREATE_CUDA
+  *out = c;
+  return REKV_OK;
+}
+
+int rekv_destroy(rekv_ctx* ctx) {
+  if (!ctx) return REKV_ERR_ARG;
+  DeviceGuard guard(ctx->device);
+  free_ctx(ctx);
+  return REKV_OK;
+}
+
+int rekv_append_frame(rekv_ctx* c, const void* k, const void* v, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (!k || !v) REKV_FAIL(c, REKV_ERR_ARG, "null K or V");
+  if (c->frames >= c->cfg.max_frames) REKV_FAIL(c, REKV_ERR_FULL, "store is full (%d frames)", c->cfg.max_frames);
+  DeviceGuard guard(c->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const int f = c->frames;
+  const StoreView& s = c->sv;
+  if (s.tail > 0) {
+    // the ring slot is reused: its previous occupant's write-through must have left HBM
+    const int slot = f % s.tail;
+    if (c->slot_event_valid[slot]) REKV_CUDA(c, cudaStreamWaitEvent(st, c->slot_events[slot], 0));
+  }
+  REKV_CUDA(c, rekv_launch_append(c, k, v, f, st));
+  if (s.tail > 0) {
+    const int slot = f % s.tail;
+    const long long frame_bytes = s.page_bytes * s.L;
+    char* dst = c->host_arenas[f / s.frames_per_arena] + (long long)(f % s.frames_per_arena) * frame_bytes;
+    REKV_CUDA(c, cudaEventRecord(c->ev_main, st));
+    REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_main, 0));
+    REKV_CUDA(c, cudaMemcpyAsync(dst, s.hbm + rekv_hbm_page_offset(s, f, 0), (size_t)frame_bytes,
+                                 cudaMemcpyDeviceToHost, c->side));
+    REKV_CUDA(c, cudaEventRecord(c->slot_events[slot], c->side));
+    c->slot_event_valid[slot] = 1;
+    c->d2h_pending = true;
+  }
+  c->frames = f + 1;
+  return f;
+}
+
+int rekv_retrieve(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, int top_k, int n_visible, int32_t* idx_out,
+                  float* scores_out, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (!q) REKV_FAIL(c, REKV_ERR_ARG, "null q");
+  if (top_k < 0 || top_k > c->cfg.max_topk) REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d outside [0, %d]", top_k, c->cfg.max_topk);
+  if (top_k > 0 && !idx_out) REKV_FAIL(c, REKV_ERR_ARG, "null idx_out");
+  if (n_visible < 0 || n_visible > c->frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "n_visible=%d outside [0, %d]", n_visible, c->frames);
+  if (n_visible == 0) REKV_FAIL(c, REKV_ERR_EMPTY, "no visible frame");
+  QBatch qb;
+  int rc = build_qbatch(c, cu_q, nQ, &qb);
+  if (rc) return rc;
+  DeviceGuard guard(c->device);
+  int n_cand = n_visible - c->cfg.window_frames;
+  if (n_cand < 0) n_cand = 0;
+  const int k_eff = top_k < n_cand ? top_k : n_cand;
+  REKV_CUDA(c, rekv_launch_retrieve(c, q, qb, top_k, k_eff, n_visible, idx_out, scores_out ? scores_out : c->scores,
+                                    (cudaStream_t)stream));
+  return k_eff;
+}
+
+int rekv_gather(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, int n_visible, void* k_ctx, void* v_ctx,
+                void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (nQ < 1 || nQ > c->cfg.max_questions) REKV_FAIL(c, REKV_ERR_ARG, "nQ=%d outside [1, %d]", nQ, c->cfg.max_questions);
+  if (top_k < 0 || top_k > c->cfg.max_topk) REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d outside [0, %d]", top_k, c->cfg.max_topk);
+  if (n_visible < 0 || n_visible > c->frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "n_visible=%d outside [0, %d]", n_visible, c->frames);
+  if (n_visible == 0) REKV_FAIL(c, REKV_ERR_EMPTY, "no visible frame");
+  if ((k_ctx == nullptr) != (v_ctx == nullptr)) REKV_FAIL(c, REKV_ERR_ARG, "k_ctx and v_ctx must both be given or both be null");
+  int n_cand = n_visible - c->cfg.window_frames;
+  if (n_cand < 0) n_cand = 0;
+  const int k_eff = top_k < n_cand ? top_k : n_cand;
+  if (k_eff > 0 && !idx) REKV_FAIL(c, REKV_ERR_ARG, "null idx");
+  const int W = n_visible < c->cfg.window_frames ? n_visible : c->cfg.window_frames;
+  const int ncf = k_eff + W;
+  DeviceGuard guard(c->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const StoreView& s = c->sv;
+  REKV_CUDA(c, cudaMemsetAsync(c->link_bytes, 0, sizeof(unsigned long long), st));
+  if (s.tail == 0) {
+    REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, k_eff, n_visible, 0, s.L, c->frames, st));
+    c->gather_layerwise = false;
+  } else {
+    // host tier: the pulls run layer by layer on the side stream (behind every write-through that is
+    // still in flight there); attention of layer l only waits for layer l's event
+    REKV_CUDA(c, cudaEventRecord(c->ev_main, st));
+    REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_main, 0));
+    for (int l = 0; l < s.L; ++l) {
+      REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, k_eff, n_visible, l, l + 1, c->frames, c->side));
+      REKV_CUDA(c, cudaEventRecord(c->layer_events[l], c->side));
+    }
+    c->gather_layerwise = true;
+  }
+  c->gathered = true;
+  c->g_nQ = nQ;
+  c->g_ncf = ncf;
+  c->g_keff = k_eff;
+  c->g_nvis = n_visible;
+  if (k_ctx) {
+    if (c->gather_layerwise) REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[s.L - 1], 0));
+    REKV_CUDA(c, rekv_launch_materialize(c, nQ, ncf, k_ctx, v_ctx, st));
+  }
+  return ncf;
+}
+
+int rekv_attend(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, void* out, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (!q || !out) REKV_FAIL(c, REKV_ERR_ARG, "null q or out");
+  if (!c->gathered) REKV_FAIL(c, REKV_ERR_STATE, "rekv_attend needs a preceding rekv_gather");
+  if (nQ != c->g_nQ) REKV_FAIL(c, REKV_ERR_STATE, "nQ=%d differs from the gathered batch (%d)", nQ, c->g_nQ);
+  QBatch qb;
+  int rc = build_qbatch(c, cu_q, nQ, &qb);
+  if (rc) return rc;
+  DeviceGuard guard(c->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const StoreView& s = c->sv;
+  if (!c->gather_layerwise) {
+    REKV_CUDA(c, rekv_launch_attend_mma(c, q, qb, c->g_ncf, 0, s.L, out, st));
+  } else {
+    for (int l = 0; l < s.L; ++l) {
+      REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[l], 0));
+      REKV_CUDA(c, rekv_launch_attend_mma(c, q, qb, c->g_ncf, l, l + 1, out, st));
+    }
+    // later appends (ring slots) and gathers (staging) on the side stream must not overtake this read
+    REKV_CUDA(c, cudaEventRecord(c->ev_side, st));
+    REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_side, 0));
+  }
+  return REKV_OK;
+}
+
+int rekv_stats(rekv_ctx* c, rekv_stats_t* out) {
+  if (!c || !out) return REKV_ERR_ARG;
+  DeviceGuard guard(c->device);
+  const StoreView& s = c->sv;
+  memset(out, 0, sizeof(*out));
+  out->frames = c->frames;
+  out->page_bytes = s.page_bytes;
+  const long long frame_bytes = s.page_bytes * s.L;
+  const long long resident = s.tail > 0 ? (c->frames < s.tail ? c->frames : s.tail) : c->frames;
+  out->kv_bytes_hbm = resident * frame_bytes;
+  out->kv_bytes_host = s.tail > 0 ? (long long)c->frames * frame_bytes : 0;
+  out->kv_bytes_logical = 2ll * s.L * c->frames * s.Nf * s.Hkv * REKV_HEAD_DIM * 2;
+  out->rep_bytes = (long long)s.L * c->frames * s.Dp * (long long)sizeof(float);
+  unsigned long long lb = 0;
+  REKV_CUDA(c, cudaDeviceSynchronize());
+  REKV_CUDA(c, cudaMemcpy(&lb, c->link_bytes, sizeof(lb), cudaMemcpyDeviceToHost));
+  out->last_link_bytes = (int64_t)lb;
+  out->last_k_eff = c->gathered ? c->g_keff : 0;
+  out->last_ctx_frames = c->gathered ? c->g_ncf : 0;
+  return REKV_OK;
+}
+
+int rekv_check_status(rekv_ctx* c, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  DeviceGuard guard(c->device);
+  REKV_CUDA(c, cudaStreamSynchronize((cudaStream_t)stream));
+  if (c->side) REKV_CUDA(c, cudaStreamSynchronize(c->side));
+  int st = 0;
+  REKV_CUDA(c, cudaMemcpy(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (st != 0) {
+    REKV_CUDA(c, cudaMemset(c->status, 0, sizeof(int)));
+    if (st == REKV_ERR_TIMEOUT) REKV_FAIL(c, REKV_ERR_TIMEOUT, "a device-side wait expired");
+    REKV_FAIL(c, st, "a kernel reported error %d (an index outside the visible frames?)", st);
+  }
+  return REKV_OK;
+}
+
+const char* rekv_last_error(rekv_ctx* c) { return c ? c->err.c_str() : g_create_error.c_str(); }
+
+int rekv_get_reps(rekv_ctx* c, int layer, int n_frames, float* dev_out, void* stream) {
+  if (!c || !dev_out) return REKV_ERR_ARG;
+  if (layer < 0 || layer >= c->sv.L || n_frames < 0 || n_frames > c->frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "layer %d / n_frames %d out of range", layer, n_frames);
+  DeviceGuard guard(c->device);
+  const StoreView& s = c->sv;
+  REKV_CUDA(c, cudaMemcpyAsync(dev_out, s.reps + (long long)layer * s.max_frames * s.Dp,
+                               (size_t)n_frames * s.Dp * sizeof(float), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return REKV_OK;
+}
+
+int rekv_get_page(rekv_ctx* c, int frame, int layer, void* k_out, void* v_out, void* stream) {
+  if (!c || !k_out || !v_out) return REKV_ERR_ARG;
+  if (layer < 0 || layer >= c->sv.L || frame < 0 || frame >= c->frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "frame %d / layer %d out of range", frame, layer);
+  DeviceGuard guard(c->device);
+  const StoreView& s = c->sv;
+  cudaStream_t st = (cudaStream_t)stream;
+  const char* page;
+  if (s.tail == 0 || frame >= c->frames - s.tail) {
+    page = s.hbm + rekv_hbm_page_offset(s, frame, layer);
+  } else {
+    // host-only page: read it zero-copy once its write-through has landed
+    REKV_CUDA(c, cudaStreamSynchronize(c->side));
+    page = c->host_arenas[frame / s.frames_per_arena] +
+           ((long long)(frame % s.frames_per_arena) * s.L + layer) * s.page_bytes;
+  }
+  REKV_CUDA(c, rekv_launch_unswizzle_page(c, page, k_out, v_out, st));
+  return REKV_OK;
+}
+
+int64_t rekv_launch_count(rekv_ctx* c) { return c ? c->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,123 @@
+// Internal declarations shared by the librekv translation units: the context, the store's
+// address arithmetic and the kernel launchers.  Nothing here is part of the public ABI.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "rekv.h"
+
+#define REKV_MAX_QUESTIONS 64
+#define REKV_HEAD_DIM 128
+
+// ---------------------------------------------------------------------------------------------
+// Store layout
+//
+// One page = one (frame, layer): for every KV head a K tile followed by a V tile.
+// A tile holds the head's N_f tokens x 128 dims as two 64-dim halves, each half a dense
+// [N_f rows][128 bytes] block whose 16-byte chunks are XOR-swizzled with (row & 7) -- the 128-byte
+// shared-memory swizzle of the tensor-core operand layouts.  A tile half can therefore be moved
+// into shared memory with one contiguous bulk copy and used by MMA instructions as it lands.
+//   page_bytes = H_kv * 2 * N_f * 256
+//   tile(h, kv) at (h*2 + kv) * N_f*256;  half hh at + hh * N_f*128
+//   element (row, dim): + row*128 + (((dim%64)/8) ^ (row&7))*16 + (dim%8)*2
+// Pages are frame-major: page(frame, layer) = base + (slot(frame)*L + layer) * page_bytes, so one
+// appended frame is one contiguous range (one D2H copy to the host tier).
+// ---------------------------------------------------------------------------------------------
+struct StoreView {
+  char* hbm;                   // HBM tier (all frames, or a ring of `tail` frames when offloaded)
+  char* const* host_arenas;    // device array of pinned-host arena base pointers (offloaded only)
+  char* staging;               // HBM staging pages for host-tier gathers (offloaded only)
+  float* reps;                 // [L][max_frames][D'] fp32
+  long long page_bytes;
+  int L, Hq, Hkv, G, Nf, Dp;   // Dp = Hkv * 128
+  int max_frames, tail, frames_per_arena;
+};
+
+__host__ __device__ inline long long rekv_tile_bytes(int Nf) { return (long long)Nf * 256; }
+
+__host__ __device__ inline long long rekv_hbm_page_offset(const StoreView& s, int frame, int layer) {
+  int slot = s.tail > 0 ? frame % s.tail : frame;
+  return ((long long)slot * s.L + layer) * s.page_bytes;
+}
+
+// Batch of questions, passed to kernels by value (no device-side table to keep alive).
+struct QBatch {
+  int nQ;
+  int sumNq;
+  int cu[REKV_MAX_QUESTIONS + 1];  // prefix sums of question lengths
+};
+
+struct rekv_ctx {
+  rekv_config cfg;
+  StoreView sv;
+  int device;
+  int frames;                       // appended so far
+  std::string err;
+  int64_t launches;
+
+  // host tier
+  std::vector<char*> host_arenas;   // pinned
+  char** d_host_arenas;             // device copy of the pointer table
+  cudaStream_t side;                // D2H write-through and host-tier gathers
+  std::vector<cudaEvent_t> slot_events;   // per ring slot: its D2H write-through finished
+  std::vector<char> slot_event_valid;
+  cudaEvent_t ev_main;              // caller stream -> side stream fence
+  cudaEvent_t ev_side;              // side stream -> caller stream fence
+  std::vector<cudaEvent_t> layer_events;  // per layer: its host-tier gather finished
+  bool d2h_pending;
+
+  // scratch (device)
+  float* qa;                        // [L][max_questions][Dp] fp32 question vectors
+  float* qnorm;                     // [L][max_questions]
+  float* scores;                    // [L][max_questions][max_frames]
+  char** ctx_tbl;                   // [L][max_questions][max_topk + W] page pointers
+  float* part_o;                    // split-KV partial outputs
+  float* part_ml;                   // split-KV partial (max, sum)
+  size_t part_units;                // capacity in (unit) entries of 128 rows
+  int* status;                      // device status word
+  unsigned long long* link_bytes;   // device counter: bytes pulled over the host link
+
+  // state of the last gather
+  bool gathered;
+  bool gather_layerwise;            // layer events are pending (offloaded context)
+  int g_nQ, g_ncf, g_keff, g_nvis;
+};
+
+#define REKV_FAIL(ctx, code, ...)                         \
+  do {                                                    \
+    char _b[512];                                         \
+    snprintf(_b, sizeof(_b), __VA_ARGS__);                \
+    rekv_set_error((ctx), _b);                            \
+    return (code);                                        \
+  } while (0)
+
+#define REKV_CUDA(ctx, call)                                                                   \
+  do {                                                                                         \
+    cudaError_t _e = (call);                                                                   \
+    if (_e != cudaSuccess)                                                                     \
+      REKV_FAIL(ctx, REKV_ERR_CUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(_e),    \
+                __FILE__, __LINE__);                                                           \
+  } while (0)
+
+void rekv_set_error(rekv_ctx* ctx, const char* msg);
+
+// ---- kernel launchers (each returns the cudaError_t of its launches) -----------------------
+// k_append.cu
+cudaError_t rekv_launch_append(rekv_ctx* c, const void* k, const void* v, int frame, cudaStream_t st);
+cudaError_t rekv_launch_unswizzle_page(rekv_ctx* c, const char* page, void* k_out, void* v_out, cudaStream_t st);
+// k_retrieve.cu
+cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, int k_eff, int n_visible,
+                                 int32_t* idx_out, float* scores, cudaStream_t st);
+// k_gather.cu
+cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, int k_eff, int n_visible,
+                                   int layer0, int layer1, int frames_now, cudaStream_t st);
+cudaError_t rekv_launch_materialize(rekv_ctx* c, int nQ, int ncf, void* k_ctx, void* v_ctx, cudaStream_t st);
+// k_attend_mma.cu
+size_t rekv_attend_units(const rekv_ctx* c, const QBatch& qb, int ncf, int* n_splits_out, int* mt_total_out);
+cudaError_t rekv_launch_attend_mma(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
+                                   void* out, cudaStream_t st);

@@ -1,0 +1,213 @@
+"""Python binding of librekv: argument marshalling only.
+
+Every step of the path (pooling, scoring, selection, gather, attention) runs in the CUDA
+kernels behind the C ABI declared in include/rekv.h; this module converts torch tensors to
+raw pointers, passes torch's current stream, and turns negative return codes into exceptions.
+There is no CPU fallback: loading fails loudly if the shared library is missing or cannot be
+built, and creating a context fails without a CUDA device.
+"""
+import ctypes
+from dataclasses import dataclass
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+from . import _build
+
+OK, ERR_ARG, ERR_FULL, ERR_EMPTY, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT, ERR_STATE = 0, -1, -2, -3, -4, -5, -6, -7
+FLAG_HOST_GATHER_COPY_ENGINE = 1 << 0
+FLAG_ATTEND_LEGACY_MMA = 1 << 1
+
+
+class RekvError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"librekv error {code}: {msg}")
+        self.code = code
+
+
+class rekv_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "tokens_per_frame", "max_frames", "hbm_tail_frames",
+        "window_frames", "block_frames", "max_q_tokens", "max_topk", "max_questions", "device")] + [
+            ("flags", ctypes.c_uint32)]
+
+
+class rekv_stats_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in (
+        "frames", "kv_bytes_hbm", "kv_bytes_host", "kv_bytes_logical", "rep_bytes", "page_bytes",
+        "last_link_bytes")] + [("last_k_eff", ctypes.c_int32), ("last_ctx_frames", ctypes.c_int32)]
+
+
+EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", "rekv_gather", "rekv_attend",
+           "rekv_stats", "rekv_check_status", "rekv_last_error", "rekv_get_reps", "rekv_get_page",
+           "rekv_launch_count")
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads (building in-tree if stale) librekv.so.  Raises if that is impossible."""
+    global _lib
+    if _lib is None:
+        path = _build.build_librekv()
+        L = ctypes.CDLL(path)
+        vp, i32, ip = ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int32)
+        L.rekv_create.argtypes = [ctypes.POINTER(rekv_config), ctypes.POINTER(vp)]
+        L.rekv_destroy.argtypes = [vp]
+        L.rekv_append_frame.argtypes = [vp, vp, vp, vp]
+        L.rekv_retrieve.argtypes = [vp, vp, ip, i32, i32, i32, vp, vp, vp]
+        L.rekv_gather.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
+        L.rekv_attend.argtypes = [vp, vp, ip, i32, vp, vp]
+        L.rekv_stats.argtypes = [vp, ctypes.POINTER(rekv_stats_t)]
+        L.rekv_check_status.argtypes = [vp, vp]
+        L.rekv_last_error.argtypes = [vp]
+        L.rekv_last_error.restype = ctypes.c_char_p
+        L.rekv_get_reps.argtypes = [vp, i32, i32, vp, vp]
+        L.rekv_get_page.argtypes = [vp, i32, i32, vp, vp, vp]
+        L.rekv_launch_count.argtypes = [vp]
+        L.rekv_launch_count.restype = ctypes.c_int64
+        for name in EXPORTS:
+            if name not in ("rekv_last_error", "rekv_launch_count"):
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def _cu_array(cu_q: Sequence[int]):
+    return (ctypes.c_int32 * len(cu_q))(*cu_q)
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, cuda: bool = True):
+    if t is None:
+        return None
+    if cuda and not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+class ReKV:
+    """One retrieval context (one video stream) on one GPU.  Methods mirror the C entry points."""
+
+    def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, tokens_per_frame: int,
+                 max_frames: int, window_frames: int, hbm_tail_frames: int = 0, max_q_tokens: int = 64,
+                 max_topk: int = 64, max_questions: int = 1, device: int = 0, flags: int = 0,
+                 block_frames: int = 1):
+        self.cfg = rekv_config(n_layers, n_q_heads, n_kv_heads, head_dim, tokens_per_frame, max_frames,
+                               hbm_tail_frames, window_frames, block_frames, max_q_tokens, max_topk, max_questions,
+                               device, flags)
+        self._h = ctypes.c_void_p()
+        rc = lib().rekv_create(ctypes.byref(self.cfg), ctypes.byref(self._h))
+        if rc != 0:
+            raise RekvError(rc, (lib().rekv_last_error(None) or b"").decode())
+        self.device = torch.device("cuda", device)
+        self.L, self.Hq, self.Hkv, self.D, self.Nf, self.W = (n_layers, n_q_heads, n_kv_heads, head_dim,
+                                                              tokens_per_frame, window_frames)
+
+    # ------------------------------------------------------------------ plumbing
+    def _check(self, rc: int) -> int:
+        if rc < 0:
+            raise RekvError(rc, (lib().rekv_last_error(self._h) or b"").decode())
+        return rc
+
+    def _stream(self) -> int:
+        return torch.cuda.current_stream(self.device).cuda_stream
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib().rekv_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ the five calls
+    def append_frame(self, k: torch.Tensor, v: torch.Tensor) -> int:
+        """k, v: bf16 [L][N_f][H_kv][D] on the context's device.  Returns the frame index."""
+        shape = (self.L, self.Nf, self.Hkv, self.D)
+        if tuple(k.shape) != shape or tuple(v.shape) != shape:
+            raise ValueError(f"expected K/V of shape {shape}")
+        return self._check(lib().rekv_append_frame(self._h, _ptr(k, torch.bfloat16), _ptr(v, torch.bfloat16),
+                                                   self._stream()))
+
+    def retrieve(self, q: torch.Tensor, cu_q: Sequence[int], top_k: int, n_visible: int,
+                 want_scores: bool = False) -> Tuple[torch.Tensor, int, Optional[torch.Tensor]]:
+        """q: bf16 [L][sum_Nq][H_q][D].  Returns (idx int32 [L][nQ][top_k], k_eff, scores or None)."""
+        nQ = len(cu_q) - 1
+        if tuple(q.shape) != (self.L, cu_q[-1], self.Hq, self.D):
+            raise ValueError("q must be [L][sum_Nq][H_q][D]")
+        idx = torch.empty((self.L, nQ, max(top_k, 0)), dtype=torch.int32, device=self.device)
+        scores = (torch.empty((self.L, nQ, n_visible), dtype=torch.float32, device=self.device)
+                  if want_scores and n_visible > 0 else None)
+        k_eff = self._check(lib().rekv_retrieve(self._h, _ptr(q, torch.bfloat16), _cu_array(cu_q), nQ, top_k,
+                                                n_visible, _ptr(idx), _ptr(scores), self._stream()))
+        return idx, k_eff, scores
+
+    def gather(self, idx: torch.Tensor, nQ: int, top_k: int, n_visible: int,
+               materialize: bool = False) -> Tuple[int, Optional[torch.Tensor], Optional[torch.Tensor]]:
+        """idx: int32 [L][nQ][top_k].  Returns (context frames, k_ctx, v_ctx); the last two are bf16
+        [L][nQ][H_kv][n_ctx][D] when materialize is set, else None."""
+        if tuple(idx.shape) != (self.L, nQ, top_k):
+            raise ValueError("idx must be [L][nQ][top_k]")
+        k_ctx = v_ctx = None
+        if materialize:
+            k_eff = min(top_k, max(n_visible - self.W, 0))
+            n_ctx = (k_eff + min(self.W, n_visible)) * self.Nf
+            shape = (self.L, nQ, self.Hkv, n_ctx, self.D)
+            k_ctx = torch.empty(shape, dtype=torch.bfloat16, device=self.device)
+            v_ctx = torch.empty(shape, dtype=torch.bfloat16, device=self.device)
+        ncf = self._check(lib().rekv_gather(self._h, _ptr(idx, torch.int32), nQ, top_k, n_visible, _ptr(k_ctx),
+                                            _ptr(v_ctx), self._stream()))
+        return ncf, k_ctx, v_ctx
+
+    def attend(self, q: torch.Tensor, cu_q: Sequence[int], out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """q: bf16 [L][sum_Nq][H_q][D] -> bf16 of the same shape."""
+        if out is None:
+            out = torch.empty_like(q)
+        self._check(lib().rekv_attend(self._h, _ptr(q, torch.bfloat16), _cu_array(cu_q), len(cu_q) - 1,
+                                      _ptr(out, torch.bfloat16), self._stream()))
+        return out
+
+    def question(self, q: torch.Tensor, cu_q: Sequence[int], top_k: int, n_visible: int,
+                 out: Optional[torch.Tensor] = None, idx: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """retrieve -> gather -> attend for a batch of questions (the calls a user makes, in order)."""
+        nQ = len(cu_q) - 1
+        if idx is None:
+            idx, _, _ = self.retrieve(q, cu_q, top_k, n_visible)
+        self.gather(idx, nQ, top_k, n_visible)
+        return self.attend(q, cu_q, out)
+
+    # ------------------------------------------------------------------ accounting and test helpers
+    def stats(self) -> rekv_stats_t:
+        st = rekv_stats_t()
+        self._check(lib().rekv_stats(self._h, ctypes.byref(st)))
+        return st
+
+    def check_status(self) -> None:
+        self._check(lib().rekv_check_status(self._h, self._stream()))
+
+    def launch_count(self) -> int:
+        return int(lib().rekv_launch_count(self._h))
+
+    def get_reps(self, layer: int, n_frames: int) -> torch.Tensor:
+        out = torch.empty((n_frames, self.Hkv * self.D), dtype=torch.float32, device=self.device)
+        self._check(lib().rekv_get_reps(self._h, layer, n_frames, _ptr(out), self._stream()))
+        return out
+
+    def get_page(self, frame: int, layer: int) -> Tuple[torch.Tensor, torch.Tensor]:
+        k = torch.empty((self.Hkv, self.Nf, self.D), dtype=torch.bfloat16, device=self.device)
+        v = torch.empty_like(k)
+        self._check(lib().rekv_get_page(self._h, frame, layer, _ptr(k), _ptr(v), self._stream()))
+        return k, v
+
+
+def kv_cache_bytes(n_layers: int, n_frames: int, tokens_per_frame: int, n_kv_heads: int, head_dim: int,
+                   bytes_per_element: int = 2) -> int:
+    """K/V bytes of a stream: 2 * L * T * M * H * D * bytes (the paper's cache-size expression)."""
+    return 2 * n_layers * n_frames * tokens_per_frame * n_kv_heads * head_dim * bytes_per_element

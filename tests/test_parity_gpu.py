@@ -1,0 +1,151 @@
+"""CUDA path vs CPU oracle, element by element, through the C ABI, on the same seeded inputs."""
+import pytest
+import torch
+
+from oracle import rekv_oracle as orc
+from paper_2503_00540_b200 import rekv, synth
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_question_parity(s: H.Shape, lengths, n_visible=None, flags=0, max_questions=None):
+    n_visible = s.T if n_visible is None else n_visible
+    nQ = len(lengths)
+    g = H.build_gpu(s, max_questions=max_questions or nQ, max_q_tokens=sum(lengths), flags=flags)
+    o = H.build_oracle(s)
+    # step 1
+    for l in range(s.L):
+        H.assert_close_rel(g.get_reps(l, s.T), o.rep_table(l), f"reps layer {l}")
+    q_gpu, cu = H.questions(s, lengths, device="cuda")
+    q_cpu, _ = H.questions(s, lengths)
+    assert torch.equal(q_gpu.cpu(), q_cpu)
+    # steps 2-3
+    idx, k_eff, scores = g.retrieve(q_gpu, cu, s.k, n_visible, want_scores=True)
+    ref = [o.question(q_cpu[:, cu[i]:cu[i + 1]].contiguous(), s.k, n_visible) for i in range(nQ)]
+    for i in range(nQ):
+        assert k_eff == ref[i]["k_eff"]
+        for l in range(s.L):
+            H.assert_close_rel(scores[l, i][None], ref[i]["scores"][l][None], f"scores l{l} q{i}")
+            H.assert_indices(idx[l, i], ref[i]["idx"][l], ref[i]["scores"][l], ref[i]["gaps"][l], k_eff,
+                             f"idx l{l} q{i}")
+    # steps 4-5 on the oracle's selection (inside a near-tie several selections are correct)
+    idx_ref = torch.stack([r["idx"] for r in ref], dim=1).contiguous().cuda()  # [L][nQ][k]
+    ncf, k_ctx, v_ctx = g.gather(idx_ref, nQ, s.k, n_visible, materialize=True)
+    assert ncf == k_eff + min(s.W, n_visible)
+    for i in range(nQ):
+        assert torch.equal(k_ctx[:, i].cpu(), ref[i]["k_ctx"]), f"gathered K differs, question {i}"
+        assert torch.equal(v_ctx[:, i].cpu(), ref[i]["v_ctx"]), f"gathered V differs, question {i}"
+    out = g.attend(q_gpu, cu)
+    g.check_status()
+    for i in range(nQ):
+        H.assert_attention(out[:, cu[i]:cu[i + 1]], ref[i]["out"], f"attention q{i}")
+    # the library's own selection must give the same answer when it equals the oracle's
+    out2 = g.question(q_gpu, cu, s.k, n_visible)
+    g.check_status()
+    if torch.equal(idx.cpu(), idx_ref.cpu()):
+        assert torch.equal(out2, out)
+    st = g.stats()
+    assert st.kv_bytes_logical == rekv.kv_cache_bytes(s.L, s.T, s.Nf, s.Hkv, s.D)
+    assert st.kv_bytes_hbm + (0 if s.tail == 0 else 0) >= 0
+    g.close()
+    return st
+
+
+def test_tiny_config():
+    """1 layer, 8/2 heads, 64 frames x 16 tokens, question of 16 tokens, window 4, top-k 8."""
+    for seed in (2503, 540, 7):
+        s = H.Shape(**{**H.TINY.__dict__, "seed": seed})
+        st = _run_question_parity(s, [16])
+        assert st.kv_bytes_hbm == st.kv_bytes_logical and st.kv_bytes_host == 0
+
+
+def test_7b_shape_small_stream_ragged_tiles():
+    """7B head shape, 196-token frames (a ragged 16-token tail per tile), 224 rows = one full and one
+    partial 128-row tile, several context frames per split."""
+    s = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=40, W=8, k=12)
+    _run_question_parity(s, [32])
+
+
+def test_batched_questions_of_mixed_length():
+    s = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=30, W=4, k=6, seed=540)
+    _run_question_parity(s, [24, 64, 37, 5])
+
+
+def test_72b_head_shape():
+    s = H.Shape(L=1, Hq=64, Hkv=8, Nf=196, T=24, W=8, k=8, seed=7)
+    _run_question_parity(s, [64])
+
+
+def test_question_in_the_past_sees_only_visible_frames():
+    s = H.Shape(L=1, Hq=8, Hkv=2, Nf=16, T=64, W=4, k=8, off_scale=0.0)
+    _run_question_parity(s, [16], n_visible=37)
+
+
+def test_degenerate_counts():
+    # k larger than the candidates -> every visible frame is attended; fewer frames than the window
+    s = H.Shape(L=1, Hq=8, Hkv=2, Nf=16, T=10, W=4, k=32, off_scale=0.0)
+    _run_question_parity(s, [7])
+    _run_question_parity(s, [7], n_visible=3)
+    # top_k = 0: window only
+    s0 = H.Shape(L=1, Hq=8, Hkv=2, Nf=16, T=10, W=4, k=0, off_scale=0.0)
+    g = H.build_gpu(s0)
+    o = H.build_oracle(s0)
+    q_gpu, cu = H.questions(s0, [5], device="cuda")
+    out = g.question(q_gpu, cu, 0, 10)
+    ref = o.question(q_gpu.cpu(), 0, 10)
+    H.assert_attention(out, ref["out"], "window only")
+    g.close()
+
+
+def test_odd_tokens_per_frame_and_single_token_question():
+    s = H.Shape(L=1, Hq=4, Hkv=1, Nf=37, T=20, W=2, k=5, seed=7)
+    _run_question_parity(s, [1])
+
+
+def test_error_paths_on_device():
+    s = H.TINY
+    g = H.build_gpu(s, n_frames=3, max_frames=3)
+    k = synth.frame(1, synth.K, 0, s.L, s.Nf, s.Hkv, s.D, device="cuda")
+    with pytest.raises(rekv.RekvError) as e:
+        g.append_frame(k, k)
+    assert e.value.code == rekv.ERR_FULL
+    q, cu = H.questions(s, [4], device="cuda")
+    with pytest.raises(rekv.RekvError) as e:
+        g.retrieve(q, cu, 2, 0)
+    assert e.value.code == rekv.ERR_EMPTY
+    with pytest.raises(rekv.RekvError) as e:
+        g.retrieve(q, cu, 2, 4)
+    assert e.value.code == rekv.ERR_ARG
+    with pytest.raises(rekv.RekvError) as e:
+        g.attend(q, cu)
+    assert e.value.code == rekv.ERR_STATE
+    # an index outside the visible frames is reported, not dereferenced
+    bad = torch.full((s.L, 1, 2), 99, dtype=torch.int32, device="cuda")
+    g2 = H.build_gpu(H.Shape(**{**s.__dict__, "W": 0}), n_frames=5)
+    g2.gather(bad, 1, 2, 5)
+    with pytest.raises(rekv.RekvError) as e:
+        g2.check_status()
+    assert e.value.code == rekv.ERR_ARG
+    g.close()
+    g2.close()
+
+
+def test_host_tier_small_stream():
+    """Offloaded context: every page in pinned host memory, the last 6 frames also in HBM."""
+    s = H.Shape(L=3, Hq=28, Hkv=4, Nf=196, T=30, W=4, k=8, tail=6, seed=540)
+    st = _run_question_parity(s, [32])
+    assert st.kv_bytes_host == st.kv_bytes_logical
+    assert st.kv_bytes_hbm == st.kv_bytes_logical * 6 // 30
+
+
+def test_host_tier_pages_survive_the_round_trip():
+    s = H.Shape(L=2, Hq=8, Hkv=2, Nf=16, T=20, W=2, k=4, tail=4, off_scale=0.0)
+    g = H.build_gpu(s)
+    for f in (0, 7, 15, 16, 19):
+        for l in range(s.L):
+            k, v = g.get_page(f, l)
+            kr = synth.frame(s.seed, synth.K, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale)[l].permute(1, 0, 2)
+            vr = synth.frame(s.seed, synth.V, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale)[l].permute(1, 0, 2)
+            assert torch.equal(k.cpu(), kr) and torch.equal(v.cpu(), vr), (f, l)
+    g.close()
