@@ -1,0 +1,358 @@
+#!/usr/bin/env python
+"""Benchmark of the retrieval hot path on one B200 (replicas only at N > 1: the path does not shard).
+
+A step = append one frame (step 1: page + pool) and answer one question (steps 2-5: retrieve, gather,
+attend over all layers) on the 7B-shape, HBM-resident, 1800-frame synthetic stream.  The headline
+value is the per-question retrieve+gather+attend latency; the append time is reported beside it.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle, as it stands, on the host
+cores on a bounded sample of the same workload.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+# BASELINE configs[1]: Qwen2-7B-like decoder, 1-hour stream at 0.5 fps
+WORKLOAD = dict(name="7b_hbm_1800f", L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503,
+                off_scale=0.5)
+N_ROTATE = 8  # distinct questions rotated through the timed steps
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.split(",") for r in open(self.f.name).read().strip().splitlines() if r.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[1]))
+                mx.append(float(r[2]))
+                for n, v in zip(names, r[5:9]):
+                    if v.strip().lower() == "active":
+                        reasons.add(n)
+            except Exception:
+                continue
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def algorithmic_bytes(w):
+    """Bytes the method must move per question (all layers): representatives once, Q in / O out, the
+    (k + W) context frames' K and V once."""
+    page = w["Hkv"] * 2 * w["Nf"] * w["D"] * 2
+    reps = w["L"] * w["T"] * w["Hkv"] * w["D"] * 4
+    qo = 2 * w["L"] * w["Nq"] * w["Hq"] * w["D"] * 2
+    kv = w["L"] * (w["k"] + w["W"]) * page
+    return dict(reps=reps, q_out=qo, kv=kv, total=reps + qo + kv, attend_kernel=kv + qo)
+
+
+def attention_flops(w):
+    return 4.0 * w["L"] * w["Nq"] * w["Hq"] * (w["k"] + w["W"]) * w["Nf"] * w["D"]
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle arm
+class OracleArm:
+    """The CPU oracle, as it stands, on the first `n_layers` layers of the workload.
+
+    Set-up (untimed) computes those layers' representatives (step 1) for the whole stream.  run() times
+    steps 2-5 of one question; the frames it selects are regenerated from the seeded generator instead
+    of holding the 20 GB cache (input generation, excluded from the timing)."""
+
+    def __init__(self, w, n_layers):
+        from oracle import rekv_oracle as orc
+        from paper_2503_00540_b200 import synth
+        self.w, self.Ls, self.orc, self.synth = w, n_layers, orc, synth
+        self.cores = len(os.sched_getaffinity(0))
+        self.reps = torch.empty(n_layers, w["T"], w["Hkv"] * w["D"], dtype=torch.float32)
+        for f in range(w["T"]):
+            kf = synth.frame(w["seed"], synth.K, f, n_layers, w["Nf"], w["Hkv"], w["D"], w["off_scale"])
+            for l in range(n_layers):
+                self.reps[l, f] = orc.pool_frame(kf[l])
+
+    def run(self, question_id=0):
+        w, orc, synth = self.w, self.orc, self.synth
+        q = synth.question(w["seed"], question_id, self.Ls, w["Nq"], w["Hq"], w["D"])
+        t0 = time.perf_counter()
+        t_gen = 0.0
+        for l in range(self.Ls):
+            s = orc.score(q[l].contiguous(), self.reps[l].contiguous(), w["Hkv"])
+            idx, k_eff, _ = orc.select(s, w["T"], w["W"], w["k"])
+            t1 = time.perf_counter()
+            frames = idx[:k_eff].tolist() + list(range(w["T"] - w["W"], w["T"]))
+            ck = torch.stack([synth.frame(w["seed"], synth.K, f, 1, w["Nf"], w["Hkv"], w["D"], w["off_scale"],
+                                          layer0=l)[0] for f in frames]).contiguous()
+            cv = torch.stack([synth.frame(w["seed"], synth.V, f, 1, w["Nf"], w["Hkv"], w["D"], w["off_scale"],
+                                          layer0=l)[0] for f in frames]).contiguous()
+            t_gen += time.perf_counter() - t1
+            sub_idx = torch.arange(k_eff, dtype=torch.int32)
+            kc = orc.gather(ck, sub_idx, k_eff, len(frames), w["W"])
+            vc = orc.gather(cv, sub_idx, k_eff, len(frames), w["W"])
+            orc.attend(q[l].contiguous(), kc, vc)
+        dt = time.perf_counter() - t0 - t_gen
+        return dt, dt * w["L"] / self.Ls
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    Ls = 2
+    arm = OracleArm(w, Ls)
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt, scaled = arm.run(i % N_ROTATE)
+        if i >= args.warmup:
+            times.append(scaled)
+    cores = arm.cores
+    val = sum(times) / len(times) * 1e6
+    line = {
+        "impl": "reference", "metric": "question_latency_us", "value": val, "unit": "us", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": val / 1e3, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w["name"], "layers": w["L"], "frames": w["T"], "tokens_per_frame": w["Nf"],
+                   "q_tokens": w["Nq"], "top_k": w["k"], "window": w["W"]},
+        "cpu_baseline": {"value": val, "unit": "us", "cores": cores, "kind": "oracle",
+                         "sample": f"steps 2-5 of one question on {Ls} of {w['L']} layers per step, "
+                                   f"scaled x{w['L'] // Ls}"},
+        "e2e": {"value": val, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------ CUDA arm
+def run_cuda(args, w):
+    import torch.distributed as dist
+    from paper_2503_00540_b200 import rekv, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    K, Wu = args.steps, args.warmup
+    n_total_steps = 2 * (K + Wu) + 4
+    T0 = w["T"] - n_total_steps  # the stream ends at ~T frames after all appends
+
+    g = rekv.ReKV(w["L"], w["Hq"], w["Hkv"], w["D"], w["Nf"], w["T"] + 8, w["W"], max_q_tokens=w["Nq"],
+                  max_topk=w["k"], max_questions=1, device=local, flags=rekv.FLAG_TIMING)
+    kf = torch.empty((w["L"], w["Nf"], w["Hkv"], w["D"]), dtype=torch.bfloat16, device=dev)
+    vf = torch.empty_like(kf)
+    for f in range(T0):
+        synth.frame(w["seed"], synth.K, f, w["L"], w["Nf"], w["Hkv"], w["D"], w["off_scale"], device=dev, out=kf)
+        synth.frame(w["seed"], synth.V, f, w["L"], w["Nf"], w["Hkv"], w["D"], w["off_scale"], device=dev, out=vf)
+        g.append_frame(kf, vf)
+    # the frames appended inside the timed steps, and the rotating questions, resident in HBM
+    n_new = n_total_steps
+    new_k = [synth.frame(w["seed"], synth.K, T0 + i, w["L"], w["Nf"], w["Hkv"], w["D"], w["off_scale"], device=dev)
+             for i in range(n_new)]
+    new_v = [synth.frame(w["seed"], synth.V, T0 + i, w["L"], w["Nf"], w["Hkv"], w["D"], w["off_scale"], device=dev)
+             for i in range(n_new)]
+    qs = [synth.question(w["seed"], i, w["L"], w["Nq"], w["Hq"], w["D"], device=dev) for i in range(N_ROTATE)]
+    cu = [0, w["Nq"]]
+    out = torch.empty_like(qs[0])
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream(dev)
+    state = {"next": 0}
+
+    def step_device(i, ev=None):
+        j = state["next"]
+        state["next"] += 1
+        if ev:
+            ev[0].record(stream)
+        nf = g.append_frame(new_k[j], new_v[j])
+        if ev:
+            ev[1].record(stream)
+        g.question(qs[i % N_ROTATE], cu, w["k"], nf + 1, out=out)
+        if ev:
+            ev[2].record(stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ----
+    for i in range(Wu):
+        step_device(i)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    att_us = []
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    l0 = g.launch_count()
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record(stream)
+    for i in range(K):
+        step_device(i, evs[i])
+    t_end.record(stream)
+    barrier()
+    launches = g.launch_count() - l0
+    clocks = sampler.stop()
+    total_ms = t_begin.elapsed_time(t_end)
+    q_us = [e[1].elapsed_time(e[2]) * 1e3 for e in evs]
+    a_us = [e[0].elapsed_time(e[1]) * 1e3 for e in evs]
+    g.check_status()
+
+    # attention-kernel duration (library-internal events), sampled over a few more questions
+    for i in range(min(K, 8)):
+        g.question(qs[i % N_ROTATE], cu, w["k"], g.stats().frames, out=out)
+        torch.cuda.synchronize()
+        att_us.append(g.stats().last_attend_kernel_us)
+
+    # ---- end to end: inputs in pinned host memory, result read back, every step ----
+    hk = [t.cpu().pin_memory() for t in new_k[:2]]
+    hv = [t.cpu().pin_memory() for t in new_v[:2]]
+    hq = [t.cpu().pin_memory() for t in qs]
+    hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    dq = torch.empty_like(qs[0])
+
+    def step_e2e(i, ev=None):
+        j = state["next"]
+        state["next"] += 1
+        kf.copy_(hk[i % 2], non_blocking=True)
+        vf.copy_(hv[i % 2], non_blocking=True)
+        nf = g.append_frame(kf, vf)
+        if ev:
+            ev[0].record(stream)
+        dq.copy_(hq[i % N_ROTATE], non_blocking=True)
+        g.question(dq, cu, w["k"], nf + 1, out=out)
+        hout.copy_(out, non_blocking=True)
+        if ev:
+            ev[1].record(stream)
+
+    for i in range(Wu):
+        step_e2e(i)
+    evs2 = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K)]
+    barrier()
+    for i in range(K):
+        step_e2e(i, evs2[i])
+    barrier()
+    e2e_us = [e[0].elapsed_time(e[1]) * 1e3 for e in evs2]
+    g.check_status()
+
+    def mean(x):
+        return sum(x) / len(x)
+
+    vals = torch.tensor([mean(q_us), total_ms / K, mean(e2e_us), mean(a_us), mean(att_us)], dtype=torch.float64,
+                        device=dev)
+    if world > 1:
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+    q_lat, ms_step, e2e_lat, app_us, att_kernel_us = vals.tolist()
+
+    if rank == 0:
+        peaks = measured_peaks()
+        ab = algorithmic_bytes(w)
+        fl = attention_flops(w)
+        achieved = ab["attend_kernel"] / (att_kernel_us * 1e-6) / 1e9
+        line = {
+            "metric": "question_latency_us", "value": q_lat, "unit": "us", "n_gpus": world, "steps": K, "warmup": Wu,
+            "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w["name"], "layers": w["L"], "q_heads": w["Hq"], "kv_heads": w["Hkv"],
+                       "frames": w["T"], "tokens_per_frame": w["Nf"], "q_tokens": w["Nq"], "top_k": w["k"],
+                       "window": w["W"], "cache_gb": 2 * w["L"] * w["T"] * w["Nf"] * w["Hkv"] * w["D"] * 2 / 1e9,
+                       "l2": "inputs larger than L2: each question streams 0.93 GB, 8 questions rotate",
+                       "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "step": "append 1 frame + 1 question (retrieve, gather, attend; all layers)"},
+            "question": {"bytes": ab["total"], "gbs": ab["total"] / (q_lat * 1e-6) / 1e9,
+                         "hbm_frac": ab["total"] / (q_lat * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                         "frames_scored_per_s": None, "questions_per_s_all_gpus": world * 1e6 / q_lat},
+            "append_us": app_us,
+            "roofline": {"kernel": "attention (step 5)", "bound": "hbm", "achieved": achieved,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                         "traffic": None, "peak_source": peaks["source"], "kernel_us": att_kernel_us,
+                         "tensor_tflops": fl / (att_kernel_us * 1e-6) / 1e12,
+                         "tensor_frac": fl / (att_kernel_us * 1e-6) / 1e12 / peaks["bf16_tflops"]},
+            "e2e": {"value": e2e_lat, "unit": "us",
+                    "h2d_bytes_per_step": 2 * kf.numel() * 2 + dq.numel() * 2, "d2h_bytes_per_step": out.numel() * 2},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            arm = OracleArm(w, w["L"])
+            dt, scaled = arm.run(0)
+            line["cpu_baseline"] = {"value": scaled * 1e6, "unit": "us", "cores": arm.cores, "kind": "oracle",
+                                    "sample": f"steps 2-5 of one whole question, all {w['L']} layers "
+                                              f"({dt:.1f} s of CPU work; pooling and input generation untimed)"}
+        print(json.dumps(line))
+    g.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=None, help="profiling only: fewer layers than the workload")
+    ap.add_argument("--frames", type=int, default=None, help="profiling only: a shorter stream")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    w = dict(WORKLOAD)
+    if args.layers or args.frames:
+        w["L"] = args.layers or w["L"]
+        w["T"] = args.frames or w["T"]
+        w["name"] = f"{w['name']}_reduced_L{w['L']}_T{w['T']}_for_profiling"
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_cuda(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -54,7 +54,9 @@ enum {
 enum {
   REKV_FLAG_HOST_GATHER_COPY_ENGINE = 1u << 0, /* host tier: per-page cudaMemcpyAsync instead of the
                                                   zero-copy gather kernel (needs a host sync on the indices) */
-  REKV_FLAG_ATTEND_LEGACY_MMA = 1u << 1         /* use the mma.sync attention kernel instead of tcgen05 */
+  REKV_FLAG_ATTEND_LEGACY_MMA = 1u << 1,        /* use the mma.sync attention kernel instead of tcgen05 */
+  REKV_FLAG_TIMING = 1u << 2                    /* bracket the attention kernel with CUDA events on the caller's
+                                                  stream; rekv_stats then reports its duration */
 };
 
 typedef struct {
@@ -86,10 +88,12 @@ typedef struct {
   int64_t last_link_bytes;   /* bytes the last rekv_gather pulled from pinned host memory */
   int32_t last_k_eff;        /* frames actually retrieved per (layer, question) by the last question */
   int32_t last_ctx_frames;   /* k_eff + window frames of the last gather */
+  double last_attend_kernel_us; /* device time of the last attention kernel launch (REKV_FLAG_TIMING, HBM
+                                   tier), without the split-KV merge; 0 when not measured */
 } rekv_stats_t;
 
 /* Creates a context on cfg->device: allocates the frame store (HBM tier, and the pinned-host tier
- * when hbm_tail_frames > 0), the fp32 representative table [max_frames][L][H_kv*D] and scratch
+ * when hbm_tail_frames > 0), the fp32 representative table [L][max_frames][H_kv*D] and scratch
  * sized from the max_* fields.  *out receives the context.  Fails with REKV_ERR_ARG on an
  * unsupported shape and REKV_ERR_ALLOC / REKV_ERR_CUDA when memory or a device is missing. */
 int rekv_create(const rekv_config* cfg, rekv_ctx** out);
@@ -99,7 +103,7 @@ int rekv_destroy(rekv_ctx* ctx);
 
 /* Step 1 (+ paging).  k, v: device bf16 [L][N_f][H_kv][D], token-major as a decoder emits them.
  * Stores the frame's K/V as page (frame, layer) and the frame representative
- * rep[frame][layer][h*D+d] = 1/N_f * sum_t k[layer][t][h][d] (fp32).  On an offloaded context the
+ * rep[layer][frame][h*D+d] = 1/N_f * sum_t k[layer][t][h][d] (fp32).  On an offloaded context the
  * page is also written through to pinned host memory on an internal stream.
  * Returns the new frame's index (>= 0), REKV_ERR_FULL when the store is full. */
 int rekv_append_frame(rekv_ctx* ctx, const void* k, const void* v, void* stream);

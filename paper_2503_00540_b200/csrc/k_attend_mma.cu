@@ -339,16 +339,8 @@ int choose_splits(long long base, int ncf, size_t cap_units) {
 
 }  // namespace
 
-size_t rekv_attend_units(const rekv_ctx* c, const QBatch& qb, int ncf, int* n_splits_out, int* mt_total_out) {
-  const int MT = total_mtiles(qb, c->sv.G);
-  (void)ncf;
-  if (mt_total_out) *mt_total_out = MT;
-  if (n_splits_out) *n_splits_out = 1;
-  return (size_t)MT;
-}
-
 cudaError_t rekv_launch_attend_mma(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
-                                   void* out, cudaStream_t st) {
+                                   void* out, cudaStream_t st, bool timed) {
   const StoreView& s = c->sv;
   AttParams p;
   p.q = (const __nv_bfloat16*)q;
@@ -377,7 +369,12 @@ cudaError_t rekv_launch_attend_mma(rekv_ctx* c, const void* q, const QBatch& qb,
     attr_set = true;
   }
   if (smem > 227 * 1024) return cudaErrorInvalidValue;
+  if (timed) cudaEventRecord(c->ev_t0, st);
   attend_mma_kernel<<<(unsigned)(base * p.n_splits), ATT_THREADS, smem, st>>>(p);
+  if (timed) {
+    cudaEventRecord(c->ev_t1, st);
+    c->timing_valid = true;
+  }
   c->launches += 1;
   if (p.n_splits > 1) {
     combine_kernel<<<dim3(p.MT, s.Hkv, layer1 - layer0), 128, 0, st>>>(p);

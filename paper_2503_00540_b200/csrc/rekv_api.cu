@@ -68,6 +68,8 @@ void free_ctx(rekv_ctx* c) {
   for (cudaEvent_t e : c->layer_events) cudaEventDestroy(e);
   if (c->ev_main) cudaEventDestroy(c->ev_main);
   if (c->ev_side) cudaEventDestroy(c->ev_side);
+  if (c->ev_t0) cudaEventDestroy(c->ev_t0);
+  if (c->ev_t1) cudaEventDestroy(c->ev_t1);
   if (c->side) cudaStreamDestroy(c->side);
   delete c;
 }
@@ -114,6 +116,8 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   c->d_host_arenas = nullptr;
   c->side = nullptr;
   c->ev_main = c->ev_side = nullptr;
+  c->ev_t0 = c->ev_t1 = nullptr;
+  c->timing_valid = false;
   c->d2h_pending = false;
   c->gathered = false;
   c->gather_layerwise = false;
@@ -169,6 +173,8 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   CREATE_CUDA(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking), "creating the side stream");
   CREATE_CUDA(cudaEventCreateWithFlags(&c->ev_main, cudaEventDisableTiming), "creating events");
   CREATE_CUDA(cudaEventCreateWithFlags(&c->ev_side, cudaEventDisableTiming), "creating events");
+  CREATE_CUDA(cudaEventCreate(&c->ev_t0), "creating events");
+  CREATE_CUDA(cudaEventCreate(&c->ev_t1), "creating events");
 
   if (s.tail > 0) {
     // pinned-host tier: arenas of whole frames, allocated up front so that append never blocks
@@ -322,11 +328,11 @@ int rekv_attend(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, void* o
   cudaStream_t st = (cudaStream_t)stream;
   const StoreView& s = c->sv;
   if (!c->gather_layerwise) {
-    REKV_CUDA(c, rekv_launch_attend_mma(c, q, qb, c->g_ncf, 0, s.L, out, st));
+    REKV_CUDA(c, rekv_launch_attend_mma(c, q, qb, c->g_ncf, 0, s.L, out, st, (c->cfg.flags & REKV_FLAG_TIMING) != 0));
   } else {
     for (int l = 0; l < s.L; ++l) {
       REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[l], 0));
-      REKV_CUDA(c, rekv_launch_attend_mma(c, q, qb, c->g_ncf, l, l + 1, out, st));
+      REKV_CUDA(c, rekv_launch_attend_mma(c, q, qb, c->g_ncf, l, l + 1, out, st, false));
     }
     // later appends (ring slots) and gathers (staging) on the side stream must not overtake this read
     REKV_CUDA(c, cudaEventRecord(c->ev_side, st));
@@ -352,6 +358,11 @@ int rekv_stats(rekv_ctx* c, rekv_stats_t* out) {
   REKV_CUDA(c, cudaDeviceSynchronize());
   REKV_CUDA(c, cudaMemcpy(&lb, c->link_bytes, sizeof(lb), cudaMemcpyDeviceToHost));
   out->last_link_bytes = (int64_t)lb;
+  if (c->timing_valid) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->ev_t0, c->ev_t1) == cudaSuccess) out->last_attend_kernel_us = 1e3 * ms;
+    cudaGetLastError();
+  }
   out->last_k_eff = c->gathered ? c->g_keff : 0;
   out->last_ctx_frames = c->gathered ? c->g_ncf : 0;
   return REKV_OK;

@@ -70,6 +70,8 @@ struct rekv_ctx {
   cudaEvent_t ev_side;              // side stream -> caller stream fence
   std::vector<cudaEvent_t> layer_events;  // per layer: its host-tier gather finished
   bool d2h_pending;
+  cudaEvent_t ev_t0, ev_t1;         // REKV_FLAG_TIMING: around the attention kernel
+  bool timing_valid;
 
   // scratch (device)
   float* qa;                        // [L][max_questions][Dp] fp32 question vectors
@@ -118,6 +120,5 @@ cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int 
                                    int layer0, int layer1, int frames_now, cudaStream_t st);
 cudaError_t rekv_launch_materialize(rekv_ctx* c, int nQ, int ncf, void* k_ctx, void* v_ctx, cudaStream_t st);
 // k_attend_mma.cu
-size_t rekv_attend_units(const rekv_ctx* c, const QBatch& qb, int ncf, int* n_splits_out, int* mt_total_out);
 cudaError_t rekv_launch_attend_mma(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
-                                   void* out, cudaStream_t st);
+                                   void* out, cudaStream_t st, bool timed);

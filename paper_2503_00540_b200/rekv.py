@@ -17,6 +17,7 @@ from . import _build
 OK, ERR_ARG, ERR_FULL, ERR_EMPTY, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT, ERR_STATE = 0, -1, -2, -3, -4, -5, -6, -7
 FLAG_HOST_GATHER_COPY_ENGINE = 1 << 0
 FLAG_ATTEND_LEGACY_MMA = 1 << 1
+FLAG_TIMING = 1 << 2
 
 
 class RekvError(RuntimeError):
@@ -35,7 +36,8 @@ class rekv_config(ctypes.Structure):
 class rekv_stats_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in (
         "frames", "kv_bytes_hbm", "kv_bytes_host", "kv_bytes_logical", "rep_bytes", "page_bytes",
-        "last_link_bytes")] + [("last_k_eff", ctypes.c_int32), ("last_ctx_frames", ctypes.c_int32)]
+        "last_link_bytes")] + [("last_k_eff", ctypes.c_int32), ("last_ctx_frames", ctypes.c_int32),
+                                       ("last_attend_kernel_us", ctypes.c_double)]
 
 
 EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", "rekv_gather", "rekv_attend",
