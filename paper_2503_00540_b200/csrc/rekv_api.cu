@@ -327,12 +327,18 @@ int rekv_attend(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, void* o
   DeviceGuard guard(c->device);
   cudaStream_t st = (cudaStream_t)stream;
   const StoreView& s = c->sv;
+  if (c->g_ncf == 0) {  // no context at all (W == 0 and nothing retrieved): the output is defined as zero
+    REKV_CUDA(c, cudaMemsetAsync(out, 0, (size_t)s.L * qb.sumNq * s.Hq * REKV_HEAD_DIM * 2, st));
+    return REKV_OK;
+  }
+  const bool legacy = (c->cfg.flags & REKV_FLAG_ATTEND_LEGACY_MMA) != 0;
+  auto launch = legacy ? rekv_launch_attend_mma : rekv_launch_attend_tc5;
   if (!c->gather_layerwise) {
-    REKV_CUDA(c, rekv_launch_attend_mma(c, q, qb, c->g_ncf, 0, s.L, out, st, (c->cfg.flags & REKV_FLAG_TIMING) != 0));
+    REKV_CUDA(c, launch(c, q, qb, c->g_ncf, 0, s.L, out, st, (c->cfg.flags & REKV_FLAG_TIMING) != 0));
   } else {
     for (int l = 0; l < s.L; ++l) {
       REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[l], 0));
-      REKV_CUDA(c, rekv_launch_attend_mma(c, q, qb, c->g_ncf, l, l + 1, out, st, false));
+      REKV_CUDA(c, launch(c, q, qb, c->g_ncf, l, l + 1, out, st, false));
     }
     // later appends (ring slots) and gathers (staging) on the side stream must not overtake this read
     REKV_CUDA(c, cudaEventRecord(c->ev_side, st));

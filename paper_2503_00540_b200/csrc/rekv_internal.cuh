@@ -122,3 +122,6 @@ cudaError_t rekv_launch_materialize(rekv_ctx* c, int nQ, int ncf, void* k_ctx, v
 // k_attend_mma.cu
 cudaError_t rekv_launch_attend_mma(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
                                    void* out, cudaStream_t st, bool timed);
+// k_attend_tc5.cu
+cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
+                                   void* out, cudaStream_t st, bool timed);

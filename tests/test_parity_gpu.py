@@ -8,6 +8,9 @@ from tests import harness as H
 
 pytestmark = pytest.mark.gpu
 
+# both attention kernels are checked: the tcgen05 one (default) and the mma.sync one
+ATT = [pytest.param(0, id="tcgen05"), pytest.param(rekv.FLAG_ATTEND_LEGACY_MMA, id="mma_sync")]
+
 
 def _run_question_parity(s: H.Shape, lengths, n_visible=None, flags=0, max_questions=None):
     n_visible = s.T if n_visible is None else n_visible
@@ -52,29 +55,33 @@ def _run_question_parity(s: H.Shape, lengths, n_visible=None, flags=0, max_quest
     return st
 
 
-def test_tiny_config():
+@pytest.mark.parametrize("flags", ATT)
+def test_tiny_config(flags):
     """1 layer, 8/2 heads, 64 frames x 16 tokens, question of 16 tokens, window 4, top-k 8."""
     for seed in (2503, 540, 7):
         s = H.Shape(**{**H.TINY.__dict__, "seed": seed})
-        st = _run_question_parity(s, [16])
+        st = _run_question_parity(s, [16], flags=flags)
         assert st.kv_bytes_hbm == st.kv_bytes_logical and st.kv_bytes_host == 0
 
 
-def test_7b_shape_small_stream_ragged_tiles():
+@pytest.mark.parametrize("flags", ATT)
+def test_7b_shape_small_stream_ragged_tiles(flags):
     """7B head shape, 196-token frames (a ragged 16-token tail per tile), 224 rows = one full and one
     partial 128-row tile, several context frames per split."""
     s = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=40, W=8, k=12)
-    _run_question_parity(s, [32])
+    _run_question_parity(s, [32], flags=flags)
 
 
-def test_batched_questions_of_mixed_length():
+@pytest.mark.parametrize("flags", ATT)
+def test_batched_questions_of_mixed_length(flags):
     s = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=30, W=4, k=6, seed=540)
-    _run_question_parity(s, [24, 64, 37, 5])
+    _run_question_parity(s, [24, 64, 37, 5], flags=flags)
 
 
-def test_72b_head_shape():
+@pytest.mark.parametrize("flags", ATT)
+def test_72b_head_shape(flags):
     s = H.Shape(L=1, Hq=64, Hkv=8, Nf=196, T=24, W=8, k=8, seed=7)
-    _run_question_parity(s, [64])
+    _run_question_parity(s, [64], flags=flags)
 
 
 def test_question_in_the_past_sees_only_visible_frames():
