@@ -183,6 +183,8 @@ def run_cuda(args, w):
     n_total_steps = 2 * (K + Wu) + 4
     T0 = w["T"] - n_total_steps  # the stream ends at ~T frames after all appends
 
+    if args.debug:
+        rekv.lib().rekv_debug_set(args.debug)
     g = rekv.ReKV(w["L"], w["Hq"], w["Hkv"], w["D"], w["Nf"], w["T"] + 8, w["W"], max_q_tokens=w["Nq"],
                   max_topk=w["k"], max_questions=1, device=local, flags=rekv.FLAG_TIMING)
     kf = torch.empty((w["L"], w["Nf"], w["Hkv"], w["D"]), dtype=torch.bfloat16, device=dev)
@@ -339,6 +341,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--debug", type=int, default=0)
     ap.add_argument("--layers", type=int, default=None, help="profiling only: fewer layers than the workload")
     ap.add_argument("--frames", type=int, default=None, help="profiling only: a shorter stream")
     args = ap.parse_args()

@@ -40,6 +40,8 @@ struct TcParams {
   int per;          // (unit, frame) steps per CTA
   long long total;  // units * ncf
   float scale_log2;
+  int debug;
+  long long* trace;
 };
 
 struct UnitInfo {
@@ -67,9 +69,21 @@ __device__ __forceinline__ UnitInfo decode_unit(const TcParams& p, long long u) 
   return ui;
 }
 
+// barrier slots after the K/V ring: full[b], empty[b], s_full[t], p_ready[t], pv_done[t]
 struct Bars {
-  uint32_t full[KV_BUFS], empty[KV_BUFS], s_full[2], p_ready[2], pv_done[2];
+  uint32_t base;
+  __device__ __forceinline__ uint32_t full(uint32_t b) const { return base + 8 * b; }
+  __device__ __forceinline__ uint32_t empty(uint32_t b) const { return base + 8 * (KV_BUFS + b); }
+  __device__ __forceinline__ uint32_t s_full(uint32_t t) const { return base + 8 * (2 * KV_BUFS + t); }
+  __device__ __forceinline__ uint32_t p_ready(uint32_t t) const { return base + 8 * (2 * KV_BUFS + 2 + t); }
+  __device__ __forceinline__ uint32_t pv_done(uint32_t t) const { return base + 8 * (2 * KV_BUFS + 4 + t); }
 };
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 
 __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParams p) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -81,17 +95,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   const uint32_t s_kv = s_base + 2 * Q_TILE_BYTES;   // ring of KV_BUFS tiles
   const uint32_t s_bar = s_kv + KV_BUFS * tile_bytes;
   Bars bars;
-#pragma unroll
-  for (int i = 0; i < KV_BUFS; ++i) {
-    bars.full[i] = s_bar + 8 * i;
-    bars.empty[i] = s_bar + 8 * (KV_BUFS + i);
-  }
-#pragma unroll
-  for (int t = 0; t < 2; ++t) {
-    bars.s_full[t] = s_bar + 8 * (2 * KV_BUFS + t);
-    bars.p_ready[t] = s_bar + 8 * (2 * KV_BUFS + 2 + t);
-    bars.pv_done[t] = s_bar + 8 * (2 * KV_BUFS + 4 + t);
-  }
+  bars.base = s_bar;
   volatile uint32_t* s_tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + (s_bar - s_base) + 8 * (2 * KV_BUFS + 6));
   volatile uint32_t* s_abort = s_tmem_slot + 1;
 
@@ -111,13 +115,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   }
   if (tid == 0) {
     for (int i = 0; i < KV_BUFS; ++i) {
-      mbar_init(bars.full[i], 1);
-      mbar_init(bars.empty[i], 1);
+      mbar_init(bars.full(i), 1);
+      mbar_init(bars.empty(i), 1);
     }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(bars.s_full[t], 1);
-      mbar_init(bars.p_ready[t], 128);
-      mbar_init(bars.pv_done[t], 1);
+      mbar_init(bars.s_full(t), 1);
+      mbar_init(bars.p_ready(t), 4);  // one arrival per softmax warp
+      mbar_init(bars.pv_done(t), 1);
     }
     *s_abort = 0;
     fence_barrier_init();
@@ -131,7 +135,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem_slot;
-  const uint32_t col_o[2] = {0u, 128u}, col_s[2] = {256u, 384u};
+  auto col_o = [](int t) { return (uint32_t)t * 128u; };
+  auto col_s = [](int t) { return 256u + (uint32_t)t * 128u; };
 
   auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
     for (uint32_t it = 0; it < (1u << 22); ++it) {
@@ -153,6 +158,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   uint32_t ring = 0;    // K/V tiles moved so far (K and V of a frame are consecutive ring entries)
   uint32_t chunk_cnt[2] = {0u, 0u};  // token chunks processed so far, per row tile (barrier phases)
 
+  if (p.debug & 64) pos = end;
   while (pos < end) {
     const long long u = pos / p.ncf;
     const int f0 = (int)(pos - u * p.ncf);
@@ -185,68 +191,110 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
 
     if (warp == 0) {
       // ================= copy producer =================
-      if (lane == 0) {
-        for (int fi = 0; fi < nfr; ++fi) {
-          const char* kt = pages[fi] + (long long)(ui.g * 2) * p.Nf * 256;
+      // the whole warp walks the ring (uniform control flow); one elected lane issues the copies
+      for (int fi = 0; fi < nfr; ++fi) {
+        const char* kt = pages[fi] + (long long)(ui.g * 2) * p.Nf * 256;
+        bool stop = false;
 #pragma unroll
-          for (int kv = 0; kv < 2; ++kv) {
-            const uint32_t r = ring + 2 * fi + kv;
-            const uint32_t b = r % KV_BUFS, use = r / KV_BUFS;
-            if (use > 0 && !wait(bars.empty[b], (use - 1) & 1)) break;
-            const uint32_t dst = s_kv + b * tile_bytes;
-            mbar_expect_tx(bars.full[b], 2u * half_bytes);
-            bulk_g2s(dst, kt + (long long)kv * 2 * half_bytes, half_bytes, bars.full[b]);
-            bulk_g2s(dst + half_stride, kt + (long long)kv * 2 * half_bytes + half_bytes, half_bytes, bars.full[b]);
+        for (int kv = 0; kv < 2; ++kv) {
+          const uint32_t r = ring + 2 * fi + kv;
+          const uint32_t b = r % KV_BUFS, use = r / KV_BUFS;
+          if (use > 0 && !wait(bars.empty(b), (use - 1) & 1)) {
+            stop = true;
+            break;
           }
-          if (*s_abort) break;
+          const uint32_t dst = s_kv + b * tile_bytes;
+          const char* src = kt + (long long)kv * 2 * half_bytes;
+          if (elect_one()) {
+            if (p.debug & 2) {
+              mbar_arrive(bars.full(b));
+            } else {
+              mbar_expect_tx(bars.full(b), 2u * half_bytes);
+              bulk_g2s(dst, src, half_bytes, bars.full(b));
+              bulk_g2s(dst + half_stride, src + half_bytes, half_bytes, bars.full(b));
+            }
+          }
+          __syncwarp();
         }
+        if (stop || *s_abort) break;
       }
-      __syncwarp();
     } else if (warp == 1) {
       // ================= MMA issuer =================
-      if (lane == 0) {
+      // Descriptors are built once; per instruction only the 14-bit start-address field advances.
+      {
+        const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);  // SBO = 1024 B, version, SWIZZLE_128B
+        const uint32_t lbo_v = ((half_stride >> 4) & 0x3FFFu) << 16;      // pitch of V's two 64-dim blocks
+        const uint32_t lbo_k = 1u << 16;                                  // unused for K-major operands
+        const uint32_t half16 = half_stride >> 4;
+        const int tiles = ui.tiles;
         bool ok = true;
-        auto issue_s = [&](int t, int i) {
-          const int fi = i / cpf, part = i - fi * cpf;
-          const uint32_t r = ring + 2 * fi, b = r % KV_BUFS;
-          const int tok0 = part ? p.NA : 0, N = part ? p.NB : p.NA;
-          if (part == 0 && t == 0) ok = ok && wait(bars.full[b], (r / KV_BUFS) & 1);
-          if (!ok) return;
-          tc_fence_after();
-          const uint32_t kb = s_kv + b * tile_bytes + tok0 * 128;
-          const uint32_t qb = s_q + t * Q_TILE_BYTES;
-          const uint32_t idesc = idesc_bf16(128, N, 0);
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint64_t ad = smem_desc_sw128(qb + (kk >> 2) * (Q_TILE_BYTES / 2) + (kk & 3) * 32, 16, 1024);
-            const uint64_t bd = smem_desc_sw128(kb + (kk >> 2) * half_stride + (kk & 3) * 32, 16, 1024);
-            mma_ss(tmem + col_s[t], ad, bd, idesc, kk > 0);
+        const bool trm = (p.debug & 256) && blockIdx.x == 0 && lane == 0;
+#define REKV_DESC(lo) (((uint64_t)desc_hi << 32) | (uint64_t)(lo))
+#define REKV_ISSUE_S(T, I)                                                                                    \
+  do {                                                                                                        \
+    const int fi_ = (I) / cpf, part_ = (I) - fi_ * cpf;                                                       \
+    const uint32_t r_ = ring + 2 * fi_, b_ = r_ % KV_BUFS;                                                    \
+    const uint32_t tok0_ = part_ ? p.NA : 0, N_ = part_ ? p.NB : p.NA;                                        \
+    if (part_ == 0 && (T) == 0) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                                 \
+    if (ok) {                                                                                                 \
+      tc_fence_after();                                                                                       \
+      const uint32_t k_lo = ((s_kv + b_ * tile_bytes + tok0_ * 128u) >> 4) | lbo_k;                           \
+      const uint32_t q_lo = ((s_q + (T) * Q_TILE_BYTES) >> 4) | lbo_k;                                        \
+      const uint32_t idesc_ = idesc_bf16(128, N_, 0);                                                         \
+      const uint32_t d_ = tmem + col_s(T);                                                                    \
+      if (elect_one()) {                                                                                      \
+      if (!(p.debug & 16)) {                                                                                  \
+      _Pragma("unroll") for (int kk = 0; kk < 4; ++kk)                                                        \
+          mma_ss(d_, REKV_DESC(q_lo + 2 * kk), REKV_DESC(k_lo + 2 * kk), idesc_, kk > 0);                     \
+      _Pragma("unroll") for (int kk = 0; kk < 4; ++kk)                                                        \
+          mma_ss(d_, REKV_DESC(q_lo + (Q_TILE_BYTES / 32) + 2 * kk), REKV_DESC(k_lo + half16 + 2 * kk), idesc_, 1); \
+      }                                                                                                       \
+      tc_commit(bars.s_full(T));                                                                              \
+      if (part_ == cpf - 1 && (T) == tiles - 1) tc_commit(bars.empty(b_)); /* K tile no longer needed */      \
+      }                                                                                                       \
+      __syncwarp();                                                                                           \
+    }                                                                                                         \
+  } while (0)
+#define REKV_ISSUE_PV(T, I)                                                                                   \
+  do {                                                                                                        \
+    const int fi_ = (I) / cpf, part_ = (I) - fi_ * cpf;                                                       \
+    const uint32_t r_ = ring + 2 * fi_ + 1, b_ = r_ % KV_BUFS;                                                \
+    const uint32_t tok0_ = part_ ? p.NA : 0, nk_ = (part_ ? p.NB : p.NA) >> 4;                                \
+    if (part_ == 0 && (T) == 0) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                                 \
+    if (trm && (I) < 20) p.trace[((I) * 2 + (T)) * 4 + 0] = clock64();                                        \
+    if (ok && !(p.debug & 8)) ok = wait(bars.p_ready(T), (chunk_cnt[T] + (I)) & 1);                           \
+    if (trm && (I) < 20) p.trace[((I) * 2 + (T)) * 4 + 1] = clock64();                                        \
+    if (ok) {                                                                                                 \
+      tc_fence_after();                                                                                       \
+      const uint32_t v_lo = ((s_kv + b_ * tile_bytes + tok0_ * 128u) >> 4) | lbo_v;                           \
+      const uint32_t d_ = tmem + col_o(T), a_ = tmem + col_s(T);                                              \
+      if (elect_one()) {                                                                                      \
+      if (!(p.debug & 32))                                                                                    \
+      _Pragma("unroll") for (int kk = 0; kk < 8; ++kk)                                                        \
+          if (kk < (int)nk_) mma_ts(d_, a_ + 8 * kk, REKV_DESC(v_lo + 128 * kk), idesc_pv, ((I) > 0) | (kk > 0)); \
+      tc_commit(bars.pv_done(T));                                                                             \
+      if (part_ == cpf - 1 && (T) == tiles - 1) tc_commit(bars.empty(b_)); /* V tile no longer needed */      \
+      }                                                                                                       \
+      __syncwarp();                                                                                           \
+    }                                                                                                         \
+  } while (0)
+        REKV_ISSUE_S(0, 0);
+        if (tiles == 2 && ok) REKV_ISSUE_S(1, 0);
+        for (int i = 0; i < nchunks && ok; ++i) {
+          REKV_ISSUE_PV(0, i);
+          if (trm && i < 20) p.trace[(i * 2 + 0) * 4 + 2] = clock64();
+          if (i + 1 < nchunks && ok) REKV_ISSUE_S(0, i + 1);
+          if (trm && i < 20) p.trace[(i * 2 + 0) * 4 + 3] = clock64();
+          if (tiles == 2 && ok) {
+            REKV_ISSUE_PV(1, i);
+            if (trm && i < 20) p.trace[(i * 2 + 1) * 4 + 2] = clock64();
+            if (i + 1 < nchunks && ok) REKV_ISSUE_S(1, i + 1);
+            if (trm && i < 20) p.trace[(i * 2 + 1) * 4 + 3] = clock64();
           }
-          tc_commit(bars.s_full[t]);
-          if (part == cpf - 1 && t == ui.tiles - 1) tc_commit(bars.empty[b]);  // K tile no longer needed
-        };
-        auto issue_pv = [&](int t, int i) {
-          const int fi = i / cpf, part = i - fi * cpf;
-          const uint32_t r = ring + 2 * fi + 1, b = r % KV_BUFS;
-          const int tok0 = part ? p.NA : 0, N = part ? p.NB : p.NA;
-          if (part == 0 && t == 0) ok = ok && wait(bars.full[b], (r / KV_BUFS) & 1);
-          ok = ok && wait(bars.p_ready[t], (chunk_cnt[t] + i) & 1);
-          if (!ok) return;
-          tc_fence_after();
-          const uint32_t vb = s_kv + b * tile_bytes + tok0 * 128;
-          for (int kk = 0; kk < N / 16; ++kk) {
-            const uint64_t bd = smem_desc_sw128(vb + kk * 2048, half_stride, 1024);
-            mma_ts(tmem + col_o[t], tmem + col_s[t] + kk * 8, bd, idesc_pv, (i > 0 || kk > 0));
-          }
-          tc_commit(bars.pv_done[t]);
-          if (part == cpf - 1 && t == ui.tiles - 1) tc_commit(bars.empty[b]);  // V tile no longer needed
-        };
-        for (int t = 0; t < ui.tiles && ok; ++t) issue_s(t, 0);
-        for (int i = 0; i < nchunks && ok; ++i)
-          for (int t = 0; t < ui.tiles && ok; ++t) {
-            issue_pv(t, i);
-            if (i + 1 < nchunks && ok) issue_s(t, i + 1);
-          }
+        }
+#undef REKV_ISSUE_S
+#undef REKV_ISSUE_PV
+#undef REKV_DESC
       }
       __syncwarp();
     } else {
@@ -255,8 +303,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
       if (t < ui.tiles) {
         const uint32_t lane_base = (uint32_t)((warp & 3) << 5) << 16;
         const int row = ((warp & 3) << 5) | lane;
-        const uint32_t t_s = tmem + lane_base + col_s[t];
-        const uint32_t t_o = tmem + lane_base + col_o[t];
+        const uint32_t t_s = tmem + lane_base + col_s(t);
+        const uint32_t t_o = tmem + lane_base + col_o(t);
         float m_used = -INFINITY, l_sum = 0.f;
         bool ok = true;
         for (int i = 0; i < nchunks && ok; ++i) {
@@ -264,76 +312,163 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
           const int tok0 = part ? p.NA : 0, N = part ? p.NB : p.NA;
           const int nv = min(N, p.Nf - tok0);  // valid tokens of this chunk
           const int npc = N >> 4;
-          if (!wait(bars.s_full[t], (chunk_cnt[t] + i) & 1)) {
+          const bool tr = (p.debug & 256) && blockIdx.x == 0 && (warp == 2 || warp == 6) && lane == 0 && i < 40;
+          if (tr) p.trace[(1 + t) * 256 + i * 4 + 0] = clock64();
+          if (!wait(bars.s_full(t), (chunk_cnt[t] + i) & 1)) {
             ok = false;
             break;
           }
           tc_fence_after();
-          uint32_t sv[8][16];
-#pragma unroll
-          for (int pc = 0; pc < 8; ++pc)
-            if (pc < npc) tmem_ld16(t_s + pc * 16, sv[pc]);
-#pragma unroll
-          for (int pc = 0; pc < 8; ++pc)
-            if (pc < npc) tmem_wait_ld16(sv[pc]);
-          float mx = -INFINITY;
-#pragma unroll
-          for (int pc = 0; pc < 8; ++pc)
-            if (pc < npc) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (pc * 16 + j < nv) mx = fmaxf(mx, __uint_as_float(sv[pc][j]));
-            }
-          mx *= p.scale_log2;
-          float alpha = 1.f;
-          bool need = false;
-          if (i == 0) {
-            m_used = mx;
-          } else if (mx > m_used + RESCALE_THRESHOLD) {
-            need = true;
-            alpha = ex2(m_used - mx);
-            m_used = mx;
+          if (tr) p.trace[(1 + t) * 256 + i * 4 + 1] = clock64();
+          if (p.debug & 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars.p_ready(t));
+            continue;
           }
-          const bool any_need = __any_sync(0xffffffffu, need);
-          float psum = 0.f;
+          // Online softmax, one pass over S.  S is read from TMEM in groups of two 16-column pieces,
+          // the next group's load in flight while the current one is processed.  A group whose
+          // scaled maximum exceeds the maximum in use by more than the threshold (always the very
+          // first group) raises it: P pieces already written for this chunk, this chunk's partial
+          // sums, the running sum and O are rescaled by 2^(m_old - m_new).  This is rare after the
+          // first chunk, so the common path has no second read of S and no rescaling.
+          const float NEG_INF = -INFINITY;
+          float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
+          auto do_group = [&](uint32_t (&a)[16], uint32_t (&b)[16], const int pc0) {
+            const bool has_b = pc0 + 1 < npc;
+            if (pc0 * 16 + 32 > nv) {  // the group that holds the frame's ragged end: mask the pad tokens
 #pragma unroll
-          for (int pc = 0; pc < 8; ++pc)
-            if (pc < npc) {
-              uint32_t pk[8];
-#pragma unroll
-              for (int jj = 0; jj < 8; ++jj) {
-                const int c0 = pc * 16 + 2 * jj;
-                float p0 = c0 < nv ? ex2(fmaf(__uint_as_float(sv[pc][2 * jj]), p.scale_log2, -m_used)) : 0.f;
-                float p1 = c0 + 1 < nv ? ex2(fmaf(__uint_as_float(sv[pc][2 * jj + 1]), p.scale_log2, -m_used)) : 0.f;
-                psum += p0 + p1;
-                pk[jj] = pack_bf16(p0, p1);
+              for (int j = 0; j < 16; ++j) {
+                if (pc0 * 16 + j >= nv) a[j] = __float_as_uint(NEG_INF);
+                if (pc0 * 16 + 16 + j >= nv) b[j] = __float_as_uint(NEG_INF);
               }
-              tmem_st8(t_s + pc * 8, pk);
             }
-          l_sum = l_sum * alpha + psum;
-          if (any_need) {
-            // O of this tile must be at rest: the previous chunk's P V has to be complete
-            if (!wait(bars.pv_done[t], (chunk_cnt[t] + i - 1) & 1)) {
-              ok = false;
-              break;
+            float g0 = max3(__uint_as_float(a[0]), __uint_as_float(a[1]), __uint_as_float(a[2]));
+            float g1 = max3(__uint_as_float(a[3]), __uint_as_float(a[4]), __uint_as_float(a[5]));
+            float g2 = max3(__uint_as_float(a[6]), __uint_as_float(a[7]), __uint_as_float(a[8]));
+            float g3 = max3(__uint_as_float(a[9]), __uint_as_float(a[10]), __uint_as_float(a[11]));
+            g0 = max3(g0, __uint_as_float(a[12]), __uint_as_float(a[13]));
+            g1 = max3(g1, __uint_as_float(a[14]), __uint_as_float(a[15]));
+            if (has_b) {
+              g2 = max3(g2, __uint_as_float(b[0]), __uint_as_float(b[1]));
+              g3 = max3(g3, __uint_as_float(b[2]), __uint_as_float(b[3]));
+              g0 = max3(g0, __uint_as_float(b[4]), __uint_as_float(b[5]));
+              g1 = max3(g1, __uint_as_float(b[6]), __uint_as_float(b[7]));
+              g2 = max3(g2, __uint_as_float(b[8]), __uint_as_float(b[9]));
+              g3 = max3(g3, __uint_as_float(b[10]), __uint_as_float(b[11]));
+              g0 = max3(g0, __uint_as_float(b[12]), __uint_as_float(b[13]));
+              g1 = max3(g1, __uint_as_float(b[14]), __uint_as_float(b[15]));
             }
-            tc_fence_after();
+            const float gm = fmaxf(fmaxf(g0, g1), fmaxf(g2, g3)) * p.scale_log2;
+            const bool need = gm > m_used + RESCALE_THRESHOLD;
+            if (__any_sync(0xffffffffu, need)) {
+              const float alpha = need ? ex2(m_used - gm) : 1.f;  // 0 when nothing has been seen yet
+              if (need) m_used = gm;
+#pragma unroll 1
+              for (int q = 0; q < pc0; ++q) {  // P pieces of this chunk written under the old maximum
+                uint32_t w[8];
+                tmem_ld8(t_s + q * 8, w);
+                tmem_wait_ld8(w);
 #pragma unroll
-            for (int pc = 0; pc < 8; ++pc) {
-              uint32_t o[16];
-              tmem_ld16(t_o + pc * 16, o);
-              tmem_wait_ld16(o);
+                for (int e = 0; e < 8; ++e) {
+                  const float lo = __uint_as_float(w[e] << 16) * alpha, hi = __uint_as_float(w[e] & 0xFFFF0000u) * alpha;
+                  w[e] = pack_bf16(lo, hi);
+                }
+                tmem_st8(t_s + q * 8, w);
+              }
+              l_sum *= alpha;
+              ps0 *= alpha;
+              ps1 *= alpha;
+              ps2 *= alpha;
+              ps3 *= alpha;
+              if (i > 0) {  // O holds earlier chunks; their P V is complete (this chunk's S came after it)
+#pragma unroll 1
+                for (int pc = 0; pc < 8; ++pc) {
+                  uint32_t o[16];
+                  tmem_ld16(t_o + pc * 16, o);
+                  tmem_wait_ld16(o);
 #pragma unroll
-              for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-              tmem_st16(t_o + pc * 16, o);
+                  for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+                  tmem_st16(t_o + pc * 16, o);
+                }
+              }
+            }
+            const float neg_m = -m_used;
+            uint32_t pk[8];
+#pragma unroll
+            for (int jj = 0; jj < 8; jj += 2) {
+              const float p0 = ex2(fmaf(__uint_as_float(a[2 * jj]), p.scale_log2, neg_m));
+              const float p1 = ex2(fmaf(__uint_as_float(a[2 * jj + 1]), p.scale_log2, neg_m));
+              const float p2 = ex2(fmaf(__uint_as_float(a[2 * jj + 2]), p.scale_log2, neg_m));
+              const float p3 = ex2(fmaf(__uint_as_float(a[2 * jj + 3]), p.scale_log2, neg_m));
+              ps0 += p0;
+              ps1 += p1;
+              ps2 += p2;
+              ps3 += p3;
+              pk[jj] = pack_bf16(p0, p1);
+              pk[jj + 1] = pack_bf16(p2, p3);
+            }
+            tmem_st8(t_s + pc0 * 8, pk);
+            if (has_b) {
+#pragma unroll
+              for (int jj = 0; jj < 8; jj += 2) {
+                const float p0 = ex2(fmaf(__uint_as_float(b[2 * jj]), p.scale_log2, neg_m));
+                const float p1 = ex2(fmaf(__uint_as_float(b[2 * jj + 1]), p.scale_log2, neg_m));
+                const float p2 = ex2(fmaf(__uint_as_float(b[2 * jj + 2]), p.scale_log2, neg_m));
+                const float p3 = ex2(fmaf(__uint_as_float(b[2 * jj + 3]), p.scale_log2, neg_m));
+                ps0 += p0;
+                ps1 += p1;
+                ps2 += p2;
+                ps3 += p3;
+                pk[jj] = pack_bf16(p0, p1);
+                pk[jj + 1] = pack_bf16(p2, p3);
+              }
+              tmem_st8(t_s + (pc0 + 1) * 8, pk);
+            }
+          };
+          {
+            uint32_t a0[16], a1[16], b0[16], b1[16];
+            tmem_ld16(t_s, a0);
+            if (npc > 1) {
+              tmem_ld16(t_s + 16, a1);
+              tmem_wait_ld16(a1);
+            }
+            tmem_wait_ld16(a0);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int pa = 4 * h, pb = 4 * h + 2;
+              if (pa < npc) {
+                if (pb < npc) {  // next group in flight while this one is processed
+                  tmem_ld16(t_s + pb * 16, b0);
+                  if (pb + 1 < npc) tmem_ld16(t_s + (pb + 1) * 16, b1);
+                }
+                do_group(a0, a1, pa);
+                if (pb < npc) {
+                  if (pb + 1 < npc) tmem_wait_ld16(b1);
+                  tmem_wait_ld16(b0);
+                  if (pa + 4 < npc) {
+                    tmem_ld16(t_s + (pa + 4) * 16, a0);
+                    if (pa + 5 < npc) tmem_ld16(t_s + (pa + 5) * 16, a1);
+                  }
+                  do_group(b0, b1, pb);
+                  if (pa + 4 < npc) {
+                    if (pa + 5 < npc) tmem_wait_ld16(a1);
+                    tmem_wait_ld16(a0);
+                  }
+                }
+              }
             }
           }
+          l_sum += (ps0 + ps1) + (ps2 + ps3);
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(bars.p_ready[t]);
+          if (tr) p.trace[(1 + t) * 256 + i * 4 + 2] = clock64();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bars.p_ready(t));
+          if (tr) p.trace[(1 + t) * 256 + i * 4 + 3] = clock64();
         }
         // ---- output of this range: final rows, or a partial for the combine kernel ----
-        if (ok && wait(bars.pv_done[t], (chunk_cnt[t] + nchunks - 1) & 1)) {
+        if (ok && wait(bars.pv_done(t), (chunk_cnt[t] + nchunks - 1) & 1) && !(p.debug & 128)) {
           tc_fence_after();
           const int rr = ui.m0 + t * 128 + row;
           const bool valid = rr < ui.rows_q;
@@ -436,6 +571,15 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
 
 }  // namespace
 
+static int g_debug = 0;
+static long long* g_trace = nullptr;
+extern "C" void rekv_debug_set(int v) { g_debug = v; }
+extern "C" int rekv_debug_trace(long long* host, int n) {
+  if (!g_trace) return -1;
+  cudaDeviceSynchronize();
+  return (int)cudaMemcpy(host, g_trace, n * sizeof(long long), cudaMemcpyDeviceToHost);
+}
+
 cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
                                    void* out, cudaStream_t st, bool timed) {
   const StoreView& s = c->sv;
@@ -462,6 +606,12 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   p.ncf = ncf;
   p.layer0 = layer0;
   p.scale_log2 = 1.4426950408889634f / sqrtf(128.f);
+  p.debug = g_debug;
+  if (g_debug & 256) {
+    if (!g_trace) { cudaMalloc(&g_trace, 1024 * sizeof(long long)); }
+    cudaMemsetAsync(g_trace, 0, 1024 * sizeof(long long), st);
+  }
+  p.trace = g_trace;
   int MP = 0;
   for (int i = 0; i < qb.nQ; ++i) MP += ((qb.cu[i + 1] - qb.cu[i]) * s.G + 255) / 256;
   p.MP = MP;
