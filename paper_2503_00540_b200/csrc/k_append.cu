@@ -24,16 +24,28 @@ __global__ void __launch_bounds__(256) append_pool_kernel(const uint4* __restric
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.f;
 
-  for (int t = rg; t < Nf; t += 16) {
-    uint4 x = __ldg(src + (long long)t * Hkv * 16);
-    *reinterpret_cast<uint4*>(tile + t * 128 + ((cc ^ (t & 7)) << 4)) = x;
-    if (kv == 0) {
-      const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&x);
+  // four rows per thread in flight
+  for (int t0 = rg; t0 < Nf; t0 += 64) {
+    uint4 x[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float2 f = __bfloat1622float2(p[i]);
-        acc[2 * i] += f.x;
-        acc[2 * i + 1] += f.y;
+    for (int u = 0; u < 4; ++u) {
+      const int t = t0 + 16 * u;
+      if (t < Nf) x[u] = __ldg(src + (long long)t * Hkv * 16);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int t = t0 + 16 * u;
+      if (t < Nf) {
+        *reinterpret_cast<uint4*>(tile + t * 128 + ((cc ^ (t & 7)) << 4)) = x[u];
+        if (kv == 0) {
+          const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&x[u]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            float2 f = __bfloat1622float2(p[i]);
+            acc[2 * i] += f.x;
+            acc[2 * i + 1] += f.y;
+          }
+        }
       }
     }
   }

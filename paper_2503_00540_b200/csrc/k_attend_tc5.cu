@@ -533,7 +533,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
 }
 
 // Merge the partials of the units that were cut by a CTA boundary.
-// grid = (units, 2 row tiles); 4 warps, a warp per row, float4 per lane.
+// grid = (units, 2 row tiles, 4 row quarters); 4 warps x 8 rows, a warp per row, float4 per lane.
 __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
   const long long u = blockIdx.x;
   const int t = blockIdx.y;
@@ -542,7 +542,8 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
   const UnitInfo ui = decode_unit(p, u);
   if (t >= ui.tiles) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int r = warp; r < 128; r += 4) {
+  for (int k8 = 0; k8 < 8; ++k8) {
+    const int r = blockIdx.z * 32 + warp * 8 + k8;
     const int rr = ui.m0 + t * 128 + r;
     if (rr >= ui.rows_q) break;
     float M = -INFINITY;
@@ -643,7 +644,7 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   }
   c->launches += 1;
   if (p.per != ncf) {
-    combine_tc5_kernel<<<dim3((unsigned)units, 2), 128, 0, st>>>(p);
+    combine_tc5_kernel<<<dim3((unsigned)units, 2, 4), 128, 0, st>>>(p);
     c->launches += 1;
   }
   return cudaGetLastError();

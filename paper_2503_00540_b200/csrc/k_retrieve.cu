@@ -5,42 +5,44 @@
 namespace {
 
 // ---- question vector: mean over the question's tokens and over the G query heads of each KV group
-// grid = (nQ, L); each thread owns dim pairs.  Also writes |q|.
+// grid = (nQ, L, H_kv); 256 threads = 4 token slices x 64 dim pairs: every load instruction of a warp
+// covers 128 contiguous bytes of one (token, head) row.  Writes the group's 128 dims of the question
+// vector and its partial sum of squares (the score kernel adds the H_kv partials).
 __global__ void __launch_bounds__(256) qmean_kernel(const __nv_bfloat162* __restrict__ q, QBatch qb, int Hq, int Hkv,
-                                                    int G, float* __restrict__ qa, float* __restrict__ qnorm,
+                                                    int G, float* __restrict__ qa, float* __restrict__ qsq,
                                                     int maxQ) {
-  const int qi = blockIdx.x, l = blockIdx.y;
+  const int qi = blockIdx.x, l = blockIdx.y, g = blockIdx.z;
   const int Dp = Hkv * 128;
   const int n0 = qb.cu[qi], n1 = qb.cu[qi + 1];
-  float* dst = qa + ((long long)l * maxQ + qi) * Dp;
-  float sq = 0.f;
-  for (int p = threadIdx.x; p < Dp / 2; p += blockDim.x) {
-    const int g = p >> 6, d2 = p & 63;
-    float sx = 0.f, sy = 0.f;
-    for (int n = n0; n < n1; ++n) {
-      const __nv_bfloat162* row = q + (((long long)l * qb.sumNq + n) * Hq + g * G) * 64 + d2;
-      for (int j = 0; j < G; ++j) {
-        float2 f = __bfloat1622float2(row[j * 64]);
-        sx += f.x;
-        sy += f.y;
-      }
+  const int d2 = threadIdx.x & 63, slice = threadIdx.x >> 6;
+  float sx = 0.f, sy = 0.f;
+  for (int n = n0 + slice; n < n1; n += 4) {
+    const __nv_bfloat162* row = q + (((long long)l * qb.sumNq + n) * Hq + g * G) * 64 + d2;
+    for (int j = 0; j < G; ++j) {
+      float2 f = __bfloat1622float2(row[j * 64]);
+      sx += f.x;
+      sy += f.y;
     }
-    const float inv = (float)((n1 - n0) * G);
-    sx = __fdiv_rn(sx, inv);
-    sy = __fdiv_rn(sy, inv);
-    dst[2 * p] = sx;
-    dst[2 * p + 1] = sy;
-    sq += sx * sx + sy * sy;
   }
-  __shared__ float red[8];
-  for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
+  __shared__ float2 part[4][64];
+  __shared__ float red[2];
+  part[slice][d2] = make_float2(sx, sy);
   __syncthreads();
-  if (threadIdx.x == 0) {
-    float s = 0.f;
-    for (int w = 0; w < (blockDim.x >> 5); ++w) s += red[w];
-    qnorm[l * maxQ + qi] = __fsqrt_rn(s);
+  if (threadIdx.x < 64) {
+    const float inv = (float)((n1 - n0) * G);
+    float ax = (part[0][d2].x + part[1][d2].x) + (part[2][d2].x + part[3][d2].x);
+    float ay = (part[0][d2].y + part[1][d2].y) + (part[2][d2].y + part[3][d2].y);
+    ax = __fdiv_rn(ax, inv);
+    ay = __fdiv_rn(ay, inv);
+    float* dst = qa + ((long long)l * maxQ + qi) * Dp + g * 128;
+    dst[2 * d2] = ax;
+    dst[2 * d2 + 1] = ay;
+    float sq = ax * ax + ay * ay;
+    for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
   }
+  __syncthreads();
+  if (threadIdx.x == 0) qsq[((long long)l * maxQ + qi) * Hkv + g] = red[0] + red[1];
 }
 
 // ---- cosine scores.  grid = (frame chunks, L); one warp per frame: the representative row is read
@@ -50,16 +52,22 @@ constexpr int SCORE_FRAMES_PER_CTA = 64;
 constexpr int SCORE_MAX_V4 = 8;  // float4 per lane: D' <= 1024
 
 __global__ void __launch_bounds__(256) score_kernel(const float* __restrict__ reps, const float* __restrict__ qa,
-                                                    const float* __restrict__ qnorm, int nQ, int maxQ, int Dp,
+                                                    const float* __restrict__ qsq, int nQ, int maxQ, int Dp, int Hkv,
                                                     int max_frames, int n_visible, int q_group,
                                                     float* __restrict__ scores) {
   extern __shared__ float4 s_q[];  // [q_group][Dp/4]
+  __shared__ float s_qn[REKV_MAX_QUESTIONS];
   const int l = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int f0 = blockIdx.x * SCORE_FRAMES_PER_CTA;
   const int f1 = min(f0 + SCORE_FRAMES_PER_CTA, n_visible);
   const int nv4 = Dp / 128;  // float4 per lane
   const float eps = 1e-8f;
+  if (threadIdx.x < nQ) {
+    float sq = 0.f;
+    for (int g = 0; g < Hkv; ++g) sq += qsq[((long long)l * maxQ + threadIdx.x) * Hkv + g];
+    s_qn[threadIdx.x] = fmaxf(__fsqrt_rn(sq), eps);
+  }
 
   for (int qg0 = 0; qg0 < nQ; qg0 += q_group) {
     const int qn = min(q_group, nQ - qg0);
@@ -67,113 +75,164 @@ __global__ void __launch_bounds__(256) score_kernel(const float* __restrict__ re
     const float4* src = reinterpret_cast<const float4*>(qa + ((long long)l * maxQ + qg0) * Dp);
     for (int i = threadIdx.x; i < qn * (Dp / 4); i += blockDim.x) s_q[i] = src[i];
     __syncthreads();
-    for (int f = f0 + warp; f < f1; f += 8) {
-      const float4* row = reinterpret_cast<const float4*>(reps + ((long long)l * max_frames + f) * Dp);
-      float4 r[SCORE_MAX_V4];
-      float rn = 0.f;
+    // two frames per iteration: twice the loads in flight per warp
+    for (int f = f0 + warp * 2; f < f1; f += 16) {
+      const bool two = f + 1 < f1;
+      const float4* row0 = reinterpret_cast<const float4*>(reps + ((long long)l * max_frames + f) * Dp);
+      const float4* row1 = row0 + (two ? Dp / 4 : 0);
+      float4 r0[SCORE_MAX_V4], r1[SCORE_MAX_V4];
 #pragma unroll
       for (int i = 0; i < SCORE_MAX_V4; ++i)
         if (i < nv4) {
-          r[i] = __ldg(row + i * 32 + lane);
-          rn += r[i].x * r[i].x + r[i].y * r[i].y + r[i].z * r[i].z + r[i].w * r[i].w;
+          r0[i] = __ldg(row0 + i * 32 + lane);
+          r1[i] = __ldg(row1 + i * 32 + lane);
         }
-      for (int o = 16; o; o >>= 1) rn += __shfl_xor_sync(0xffffffffu, rn, o);
-      rn = fmaxf(__fsqrt_rn(rn), eps);
+      float n0 = 0.f, n1 = 0.f;
+#pragma unroll
+      for (int i = 0; i < SCORE_MAX_V4; ++i)
+        if (i < nv4) {
+          n0 += r0[i].x * r0[i].x + r0[i].y * r0[i].y + r0[i].z * r0[i].z + r0[i].w * r0[i].w;
+          n1 += r1[i].x * r1[i].x + r1[i].y * r1[i].y + r1[i].z * r1[i].z + r1[i].w * r1[i].w;
+        }
+      for (int o = 16; o; o >>= 1) {
+        n0 += __shfl_xor_sync(0xffffffffu, n0, o);
+        n1 += __shfl_xor_sync(0xffffffffu, n1, o);
+      }
+      n0 = fmaxf(__fsqrt_rn(n0), eps);
+      n1 = fmaxf(__fsqrt_rn(n1), eps);
       for (int qi = 0; qi < qn; ++qi) {
-        float dot = 0.f;
+        float d0 = 0.f, d1 = 0.f;
 #pragma unroll
         for (int i = 0; i < SCORE_MAX_V4; ++i)
           if (i < nv4) {
-            float4 a = s_q[qi * (Dp / 4) + i * 32 + lane];
-            dot += r[i].x * a.x + r[i].y * a.y + r[i].z * a.z + r[i].w * a.w;
+            const float4 a = s_q[qi * (Dp / 4) + i * 32 + lane];
+            d0 += r0[i].x * a.x + r0[i].y * a.y + r0[i].z * a.z + r0[i].w * a.w;
+            d1 += r1[i].x * a.x + r1[i].y * a.y + r1[i].z * a.z + r1[i].w * a.w;
           }
-        for (int o = 16; o; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        for (int o = 16; o; o >>= 1) {
+          d0 += __shfl_xor_sync(0xffffffffu, d0, o);
+          d1 += __shfl_xor_sync(0xffffffffu, d1, o);
+        }
         if (lane == 0) {
-          float qn_ = fmaxf(qnorm[l * maxQ + qg0 + qi], eps);
-          scores[((long long)l * nQ + qg0 + qi) * n_visible + f] = __fdiv_rn(dot, qn_ * rn);
+          const float qn_ = s_qn[qg0 + qi];
+          float* dst = scores + ((long long)l * nQ + qg0 + qi) * n_visible + f;
+          dst[0] = __fdiv_rn(d0, qn_ * n0);
+          if (two) dst[1] = __fdiv_rn(d1, qn_ * n1);
         }
       }
     }
   }
 }
 
-// ---- exact top-k by radix select on 64-bit keys (score order, then lower index first).
-__device__ __forceinline__ unsigned long long topk_key(float s, int idx) {
+// ---- exact top-k by radix select on the score keys (score order, then lower index first).
+// Order-preserving 32-bit image of a score: larger score <=> larger key; NaN ranks as -inf, -0 == +0.
+__device__ __forceinline__ unsigned score_key(float s) {
   unsigned u = __float_as_uint(s);
-  if (s != s) u = 0xFF800000u;       // NaN ranks as -inf
-  if (s == 0.f) u = 0u;              // -0 == +0
-  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-  return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)idx);
+  if (s != s) u = 0xFF800000u;
+  if (s == 0.f) u = 0u;
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// grid = (nQ, L), 512 threads.  Candidates are frames [0, n_cand).  Eight 8-bit passes find the
-// k-th largest key exactly (keys are unique), then an ordered compaction emits the selected frames
-// in ascending frame index.
+// grid = (nQ, L), 512 threads.  Candidates are frames [0, n_cand).  Four 8-bit radix passes over the
+// score keys find the k-th largest key T exactly, with the number of candidates above it; one
+// ordered compaction then emits, in ascending frame index, every frame above T and the lowest-index
+// frames equal to T that are still needed (ties go to the lower index).
 __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ scores, int nQ, int n_visible,
                                                    int n_cand, int top_k, int k_eff, int32_t* __restrict__ idx_out) {
   const int qi = blockIdx.x, l = blockIdx.y;
   const float* s = scores + ((long long)l * nQ + qi) * n_visible;
   int32_t* out = idx_out + ((long long)l * nQ + qi) * top_k;
   __shared__ unsigned hist[256];
-  __shared__ unsigned long long s_prefix;
+  __shared__ unsigned s_prefix;
   __shared__ int s_krem;
-  __shared__ int warp_cnt[16];
-  __shared__ int s_base;
+  __shared__ int warp_gt[16], warp_eq[16];
+  __shared__ int s_base_gt, s_base_eq;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   for (int j = k_eff + threadIdx.x; j < top_k; j += blockDim.x) out[j] = -1;
   if (k_eff <= 0) return;
-
   if (threadIdx.x == 0) {
-    s_prefix = 0ull;
+    s_prefix = 0u;
     s_krem = k_eff;
-    s_base = 0;
+    s_base_gt = 0;
+    s_base_eq = 0;
   }
-  for (int pass = 0; pass < 8; ++pass) {
-    const int shift = 56 - 8 * pass;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
     for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
     __syncthreads();
-    const unsigned long long prefix = s_prefix;
-    const unsigned long long mask = pass == 0 ? 0ull : (~0ull << (shift + 8));
+    const unsigned prefix = s_prefix;
+    const unsigned mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
     for (int i = threadIdx.x; i < n_cand; i += blockDim.x) {
-      unsigned long long key = topk_key(s[i], i);
-      if ((key & mask) == prefix) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
+      const unsigned key = score_key(s[i]);
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-      int krem = s_krem;
-      int d = 255;
-      for (; d > 0; --d) {
-        int c = (int)hist[d];
-        if (c >= krem) break;
-        krem -= c;
+    if (warp == 0) {
+      // lane owns bins [8*lane, 8*lane+8); suffix sums over lanes locate the bin of the k-th largest
+      unsigned b[8], tot = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        b[j] = hist[lane * 8 + j];
+        tot += b[j];
       }
-      s_krem = krem;
-      s_prefix = prefix | ((unsigned long long)d << shift);
+      unsigned suf = tot;  // inclusive suffix sum over lanes >= this one
+      for (int o = 1; o < 32; o <<= 1) {
+        unsigned v = __shfl_down_sync(0xffffffffu, suf, o);
+        if (lane + o < 32) suf += v;
+      }
+      const int krem = s_krem;
+      const unsigned ball = __ballot_sync(0xffffffffu, (int)suf >= krem);
+      const int owner = 31 - __clz(ball);  // highest lane whose suffix still reaches krem
+      if (lane == owner) {
+        int above = (int)(suf - tot);  // candidates in higher lanes' bins
+        int d = 7;
+        for (; d > 0; --d) {
+          if (above + (int)b[d] >= krem) break;
+          above += (int)b[d];
+        }
+        s_krem = krem - above;
+        s_prefix = prefix | ((unsigned)(lane * 8 + d) << shift);
+      }
     }
     __syncthreads();
   }
-  const unsigned long long thr = s_prefix;  // the k_eff-th largest key
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned thr = s_prefix;  // key of the k_eff-th largest score
+  const int need_eq = s_krem;     // how many candidates equal to it are selected (lowest indices first)
+  const int n_gt = k_eff - need_eq;
   for (int i0 = 0; i0 < n_cand; i0 += blockDim.x) {
     const int i = i0 + threadIdx.x;
-    const bool sel = i < n_cand && topk_key(s[i], i) >= thr;
-    const unsigned b = __ballot_sync(0xffffffffu, sel);
-    if (lane == 0) warp_cnt[warp] = __popc(b);
-    __syncthreads();
-    int off = s_base;
-    for (int w = 0; w < warp; ++w) off += warp_cnt[w];
-    if (sel) {
-      int pos = off + __popc(b & ((1u << lane) - 1u));
-      if (pos < k_eff) out[pos] = i;
+    const unsigned key = i < n_cand ? score_key(s[i]) : 0u;
+    const bool gt = i < n_cand && key > thr, eq = i < n_cand && key == thr;
+    const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) {
+      warp_gt[warp] = __popc(bg);
+      warp_eq[warp] = __popc(be);
     }
     __syncthreads();
+    int og = s_base_gt, oe = s_base_eq;
+    for (int w = 0; w < warp; ++w) {
+      og += warp_gt[w];
+      oe += warp_eq[w];
+    }
+    const unsigned lower = (1u << lane) - 1u;
+    const int rank_gt = og + __popc(bg & lower), rank_eq = oe + __popc(be & lower);
+    // output position = selected frames before this one = (greater before) + min(equal before, need_eq)
+    if (gt) out[rank_gt + min(rank_eq, need_eq)] = i;
+    if (eq && rank_eq < need_eq) out[rank_gt + rank_eq] = i;
+    __syncthreads();
     if (threadIdx.x == 0) {
-      int t = 0;
-      for (int w = 0; w < 16; ++w) t += warp_cnt[w];
-      s_base += t;
+      int tg = 0, te = 0;
+      for (int w = 0; w < 16; ++w) {
+        tg += warp_gt[w];
+        te += warp_eq[w];
+      }
+      s_base_gt += tg;
+      s_base_eq += te;
     }
     __syncthreads();
   }
+  (void)n_gt;
 }
 
 }  // namespace
@@ -182,8 +241,8 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
                                  int32_t* idx_out, float* scores, cudaStream_t st) {
   const StoreView& s = c->sv;
   const int maxQ = c->cfg.max_questions;
-  qmean_kernel<<<dim3(qb.nQ, s.L), 256, 0, st>>>((const __nv_bfloat162*)q, qb, s.Hq, s.Hkv, s.G, c->qa, c->qnorm,
-                                                maxQ);
+  qmean_kernel<<<dim3(qb.nQ, s.L, s.Hkv), 256, 0, st>>>((const __nv_bfloat162*)q, qb, s.Hq, s.Hkv, s.G, c->qa,
+                                                       c->qnorm, maxQ);
   int q_group = (int)((96 * 1024) / (s.Dp * sizeof(float)));
   if (q_group > qb.nQ) q_group = qb.nQ;
   size_t smem = (size_t)q_group * s.Dp * sizeof(float);
@@ -193,8 +252,8 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
     attr_set = true;
   }
   dim3 grid((n_visible + SCORE_FRAMES_PER_CTA - 1) / SCORE_FRAMES_PER_CTA, s.L);
-  score_kernel<<<grid, 256, smem, st>>>(s.reps, c->qa, c->qnorm, qb.nQ, maxQ, s.Dp, s.max_frames, n_visible, q_group,
-                                        scores);
+  score_kernel<<<grid, 256, smem, st>>>(s.reps, c->qa, c->qnorm, qb.nQ, maxQ, s.Dp, s.Hkv, s.max_frames, n_visible,
+                                        q_group, scores);
   if (top_k > 0) {
     int n_cand = n_visible - c->cfg.window_frames;
     if (n_cand < 0) n_cand = 0;

@@ -160,7 +160,7 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   const int ctx_frames_max = cfg->max_topk + cfg->window_frames;
   const int maxQ = cfg->max_questions;
   CREATE_CUDA(cudaMalloc(&c->qa, (size_t)s.L * maxQ * s.Dp * sizeof(float)), "allocating question vectors");
-  CREATE_CUDA(cudaMalloc(&c->qnorm, (size_t)s.L * maxQ * sizeof(float)), "allocating question norms");
+  CREATE_CUDA(cudaMalloc(&c->qnorm, (size_t)s.L * maxQ * s.Hkv * sizeof(float)), "allocating question norms");
   CREATE_CUDA(cudaMalloc(&c->scores, (size_t)s.L * maxQ * s.max_frames * sizeof(float)), "allocating the score buffer");
   CREATE_CUDA(cudaMalloc(&c->ctx_tbl, (size_t)s.L * maxQ * (ctx_frames_max + 1) * sizeof(char*)), "allocating the context table");
   c->part_units = 2048;

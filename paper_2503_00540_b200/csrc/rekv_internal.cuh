@@ -75,7 +75,7 @@ struct rekv_ctx {
 
   // scratch (device)
   float* qa;                        // [L][max_questions][Dp] fp32 question vectors
-  float* qnorm;                     // [L][max_questions]
+  float* qnorm;                     // [L][max_questions][H_kv] partial sums of squares of the question vector
   float* scores;                    // [L][max_questions][max_frames]
   char** ctx_tbl;                   // [L][max_questions][max_topk + W] page pointers
   float* part_o;                    // split-KV partial outputs
