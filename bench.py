@@ -51,7 +51,7 @@ class ClockSampler:
     def start(self):
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
-                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                       "--format=csv,noheader,nounits", "-lms", "20"], stdout=self.f,
                                       stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
@@ -183,8 +183,6 @@ def run_cuda(args, w):
     n_total_steps = 2 * (K + Wu) + 4
     T0 = w["T"] - n_total_steps  # the stream ends at ~T frames after all appends
 
-    if args.debug:
-        rekv.lib().rekv_debug_set(args.debug)
     g = rekv.ReKV(w["L"], w["Hq"], w["Hkv"], w["D"], w["Nf"], w["T"] + 8, w["W"], max_q_tokens=w["Nq"],
                   max_topk=w["k"], max_questions=1, device=local, flags=rekv.FLAG_TIMING)
     kf = torch.empty((w["L"], w["Nf"], w["Hkv"], w["D"]), dtype=torch.bfloat16, device=dev)
@@ -337,11 +335,10 @@ def run_cuda(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--debug", type=int, default=0)
     ap.add_argument("--layers", type=int, default=None, help="profiling only: fewer layers than the workload")
     ap.add_argument("--frames", type=int, default=None, help="profiling only: a shorter stream")
     args = ap.parse_args()

@@ -40,8 +40,6 @@ struct TcParams {
   int per;          // (unit, frame) steps per CTA
   long long total;  // units * ncf
   float scale_log2;
-  int debug;
-  long long* trace;
 };
 
 struct UnitInfo {
@@ -158,7 +156,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   uint32_t ring = 0;    // K/V tiles moved so far (K and V of a frame are consecutive ring entries)
   uint32_t chunk_cnt[2] = {0u, 0u};  // token chunks processed so far, per row tile (barrier phases)
 
-  if (p.debug & 64) pos = end;
   while (pos < end) {
     const long long u = pos / p.ncf;
     const int f0 = (int)(pos - u * p.ncf);
@@ -206,13 +203,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
           const uint32_t dst = s_kv + b * tile_bytes;
           const char* src = kt + (long long)kv * 2 * half_bytes;
           if (elect_one()) {
-            if (p.debug & 2) {
-              mbar_arrive(bars.full(b));
-            } else {
-              mbar_expect_tx(bars.full(b), 2u * half_bytes);
-              bulk_g2s(dst, src, half_bytes, bars.full(b));
-              bulk_g2s(dst + half_stride, src + half_bytes, half_bytes, bars.full(b));
-            }
+            mbar_expect_tx(bars.full(b), 2u * half_bytes);
+            bulk_g2s(dst, src, half_bytes, bars.full(b));
+            bulk_g2s(dst + half_stride, src + half_bytes, half_bytes, bars.full(b));
           }
           __syncwarp();
         }
@@ -228,7 +221,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         const uint32_t half16 = half_stride >> 4;
         const int tiles = ui.tiles;
         bool ok = true;
-        const bool trm = (p.debug & 256) && blockIdx.x == 0 && lane == 0;
 #define REKV_DESC(lo) (((uint64_t)desc_hi << 32) | (uint64_t)(lo))
 #define REKV_ISSUE_S(T, I)                                                                                    \
   do {                                                                                                        \
@@ -243,12 +235,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
       const uint32_t idesc_ = idesc_bf16(128, N_, 0);                                                         \
       const uint32_t d_ = tmem + col_s(T);                                                                    \
       if (elect_one()) {                                                                                      \
-      if (!(p.debug & 16)) {                                                                                  \
       _Pragma("unroll") for (int kk = 0; kk < 4; ++kk)                                                        \
           mma_ss(d_, REKV_DESC(q_lo + 2 * kk), REKV_DESC(k_lo + 2 * kk), idesc_, kk > 0);                     \
       _Pragma("unroll") for (int kk = 0; kk < 4; ++kk)                                                        \
           mma_ss(d_, REKV_DESC(q_lo + (Q_TILE_BYTES / 32) + 2 * kk), REKV_DESC(k_lo + half16 + 2 * kk), idesc_, 1); \
-      }                                                                                                       \
       tc_commit(bars.s_full(T));                                                                              \
       if (part_ == cpf - 1 && (T) == tiles - 1) tc_commit(bars.empty(b_)); /* K tile no longer needed */      \
       }                                                                                                       \
@@ -261,15 +251,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     const uint32_t r_ = ring + 2 * fi_ + 1, b_ = r_ % KV_BUFS;                                                \
     const uint32_t tok0_ = part_ ? p.NA : 0, nk_ = (part_ ? p.NB : p.NA) >> 4;                                \
     if (part_ == 0 && (T) == 0) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                                 \
-    if (trm && (I) < 20) p.trace[((I) * 2 + (T)) * 4 + 0] = clock64();                                        \
-    if (ok && !(p.debug & 8)) ok = wait(bars.p_ready(T), (chunk_cnt[T] + (I)) & 1);                           \
-    if (trm && (I) < 20) p.trace[((I) * 2 + (T)) * 4 + 1] = clock64();                                        \
+    if (ok) ok = wait(bars.p_ready(T), (chunk_cnt[T] + (I)) & 1);                                             \
     if (ok) {                                                                                                 \
       tc_fence_after();                                                                                       \
       const uint32_t v_lo = ((s_kv + b_ * tile_bytes + tok0_ * 128u) >> 4) | lbo_v;                           \
       const uint32_t d_ = tmem + col_o(T), a_ = tmem + col_s(T);                                              \
       if (elect_one()) {                                                                                      \
-      if (!(p.debug & 32))                                                                                    \
       _Pragma("unroll") for (int kk = 0; kk < 8; ++kk)                                                        \
           if (kk < (int)nk_) mma_ts(d_, a_ + 8 * kk, REKV_DESC(v_lo + 128 * kk), idesc_pv, ((I) > 0) | (kk > 0)); \
       tc_commit(bars.pv_done(T));                                                                             \
@@ -282,14 +269,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         if (tiles == 2 && ok) REKV_ISSUE_S(1, 0);
         for (int i = 0; i < nchunks && ok; ++i) {
           REKV_ISSUE_PV(0, i);
-          if (trm && i < 20) p.trace[(i * 2 + 0) * 4 + 2] = clock64();
           if (i + 1 < nchunks && ok) REKV_ISSUE_S(0, i + 1);
-          if (trm && i < 20) p.trace[(i * 2 + 0) * 4 + 3] = clock64();
           if (tiles == 2 && ok) {
             REKV_ISSUE_PV(1, i);
-            if (trm && i < 20) p.trace[(i * 2 + 1) * 4 + 2] = clock64();
             if (i + 1 < nchunks && ok) REKV_ISSUE_S(1, i + 1);
-            if (trm && i < 20) p.trace[(i * 2 + 1) * 4 + 3] = clock64();
           }
         }
 #undef REKV_ISSUE_S
@@ -312,20 +295,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
           const int tok0 = part ? p.NA : 0, N = part ? p.NB : p.NA;
           const int nv = min(N, p.Nf - tok0);  // valid tokens of this chunk
           const int npc = N >> 4;
-          const bool tr = (p.debug & 256) && blockIdx.x == 0 && (warp == 2 || warp == 6) && lane == 0 && i < 40;
-          if (tr) p.trace[(1 + t) * 256 + i * 4 + 0] = clock64();
           if (!wait(bars.s_full(t), (chunk_cnt[t] + i) & 1)) {
             ok = false;
             break;
           }
           tc_fence_after();
-          if (tr) p.trace[(1 + t) * 256 + i * 4 + 1] = clock64();
-          if (p.debug & 1) {
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bars.p_ready(t));
-            continue;
-          }
           // Online softmax, one pass over S.  S is read from TMEM in groups of two 16-column pieces,
           // the next group's load in flight while the current one is processed.  A group whose
           // scaled maximum exceeds the maximum in use by more than the threshold (always the very
@@ -462,13 +436,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
           l_sum += (ps0 + ps1) + (ps2 + ps3);
           tmem_wait_st();
           tc_fence_before();
-          if (tr) p.trace[(1 + t) * 256 + i * 4 + 2] = clock64();
           __syncwarp();
           if (lane == 0) mbar_arrive(bars.p_ready(t));
-          if (tr) p.trace[(1 + t) * 256 + i * 4 + 3] = clock64();
         }
         // ---- output of this range: final rows, or a partial for the combine kernel ----
-        if (ok && wait(bars.pv_done(t), (chunk_cnt[t] + nchunks - 1) & 1) && !(p.debug & 128)) {
+        if (ok && wait(bars.pv_done(t), (chunk_cnt[t] + nchunks - 1) & 1)) {
           tc_fence_after();
           const int rr = ui.m0 + t * 128 + row;
           const bool valid = rr < ui.rows_q;
@@ -572,15 +544,6 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
 
 }  // namespace
 
-static int g_debug = 0;
-static long long* g_trace = nullptr;
-extern "C" void rekv_debug_set(int v) { g_debug = v; }
-extern "C" int rekv_debug_trace(long long* host, int n) {
-  if (!g_trace) return -1;
-  cudaDeviceSynchronize();
-  return (int)cudaMemcpy(host, g_trace, n * sizeof(long long), cudaMemcpyDeviceToHost);
-}
-
 cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
                                    void* out, cudaStream_t st, bool timed) {
   const StoreView& s = c->sv;
@@ -607,12 +570,6 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   p.ncf = ncf;
   p.layer0 = layer0;
   p.scale_log2 = 1.4426950408889634f / sqrtf(128.f);
-  p.debug = g_debug;
-  if (g_debug & 256) {
-    if (!g_trace) { cudaMalloc(&g_trace, 1024 * sizeof(long long)); }
-    cudaMemsetAsync(g_trace, 0, 1024 * sizeof(long long), st);
-  }
-  p.trace = g_trace;
   int MP = 0;
   for (int i = 0; i < qb.nQ; ++i) MP += ((qb.cu[i + 1] - qb.cu[i]) * s.G + 255) / 256;
   p.MP = MP;
