@@ -23,9 +23,20 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-# BASELINE configs[1]: Qwen2-7B-like decoder, 1-hour stream at 0.5 fps
-WORKLOAD = dict(name="7b_hbm_1800f", L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503,
-                off_scale=0.5)
+# The headline workload is BASELINE configs[1] (Qwen2-7B-like decoder, 1-hour stream at 0.5 fps, whole
+# cache in HBM).  The other full-size configurations can be timed with --workload; they are parity-test
+# cases, not the bench line.
+WORKLOADS = {
+    "7b_hbm_1800f": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503, off_scale=0.5,
+                         tail=0, nQ=1, appends_per_step=1),
+    "7b_offload_10800f": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=10800, W=8, k=64, Nq=32, seed=2503,
+                              off_scale=0.5, tail=64, nQ=1, appends_per_step=1),
+    "7b_stream_batch16": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=32, Nq=(24, 64), seed=2503,
+                              off_scale=0.5, tail=0, nQ=16, appends_per_step=10),
+    "72b_offload_1800f": dict(L=80, Hq=64, Hkv=8, D=128, Nf=196, T=1800, W=8, k=32, Nq=64, seed=2503,
+                              off_scale=0.5, tail=32, nQ=1, appends_per_step=1),
+}
+WORKLOAD = dict(WORKLOADS["7b_hbm_1800f"], name="7b_hbm_1800f")
 N_ROTATE = 8  # distinct questions rotated through the timed steps
 
 
@@ -84,18 +95,26 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def algorithmic_bytes(w):
-    """Bytes the method must move per question (all layers): representatives once, Q in / O out, the
-    (k + W) context frames' K and V once."""
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch from the committed ncu capture
+# (profiles/), scaled to the full workload by the layers processed; None where no capture exists.
+TRAFFIC_NCU = {}
+
+
+def algorithmic_bytes(w, sum_nq=None, nQ=1):
+    """Bytes the method must move per question batch (all layers): representatives once, Q in / O out,
+    every question's k retrieved frames' K and V once, the W window frames once."""
+    sum_nq = w["Nq"] if sum_nq is None else sum_nq
     page = w["Hkv"] * 2 * w["Nf"] * w["D"] * 2
     reps = w["L"] * w["T"] * w["Hkv"] * w["D"] * 4
-    qo = 2 * w["L"] * w["Nq"] * w["Hq"] * w["D"] * 2
-    kv = w["L"] * (w["k"] + w["W"]) * page
-    return dict(reps=reps, q_out=qo, kv=kv, total=reps + qo + kv, attend_kernel=kv + qo)
+    qo = 2 * w["L"] * sum_nq * w["Hq"] * w["D"] * 2
+    kv = w["L"] * (nQ * w["k"] + w["W"]) * page
+    kv_read = w["L"] * nQ * (w["k"] + w["W"]) * page  # what the attention kernel is asked to read
+    return dict(reps=reps, q_out=qo, kv=kv, total=reps + qo + kv, attend_kernel=kv_read + qo)
 
 
-def attention_flops(w):
-    return 4.0 * w["L"] * w["Nq"] * w["Hq"] * (w["k"] + w["W"]) * w["Nf"] * w["D"]
+def attention_flops(w, sum_nq=None):
+    sum_nq = w["Nq"] if sum_nq is None else sum_nq
+    return 4.0 * w["L"] * sum_nq * w["Hq"] * (w["k"] + w["W"]) * w["Nf"] * w["D"]
 
 
 # ------------------------------------------------------------------------------------------ CPU oracle arm
@@ -168,6 +187,23 @@ def run_reference(args, w):
 
 
 # ------------------------------------------------------------------------------------------ CUDA arm
+def pinned_h2d_gbs(dev, n_bytes=1 << 30, reps=5):
+    """Measured pinned host -> device copy bandwidth (the host-link peak of this machine)."""
+    h = torch.empty(n_bytes, dtype=torch.uint8).pin_memory()
+    d = torch.empty(n_bytes, dtype=torch.uint8, device=dev)
+    best = 1e30
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        d.copy_(h, non_blocking=True)
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    del h, d
+    return n_bytes / best / 1e6
+
+
 def run_cuda(args, w):
     import torch.distributed as dist
     from paper_2503_00540_b200 import rekv, synth
@@ -180,36 +216,53 @@ def run_cuda(args, w):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     K, Wu = args.steps, args.warmup
+    aps, nQ = w["appends_per_step"], w["nQ"]
     n_total_steps = 2 * (K + Wu) + 4
-    T0 = w["T"] - n_total_steps  # the stream ends at ~T frames after all appends
+    n_new = n_total_steps * aps
+    T0 = w["T"] - n_new  # the stream ends at ~T frames after all appends
+    if isinstance(w["Nq"], tuple):
+        lengths = synth.question_lengths(w["seed"], nQ, w["Nq"][0], w["Nq"][1])
+    else:
+        lengths = [w["Nq"]] * nQ
+    cu = [0]
+    for n in lengths:
+        cu.append(cu[-1] + n)
+    w["Nq_total"] = cu[-1]
 
-    g = rekv.ReKV(w["L"], w["Hq"], w["Hkv"], w["D"], w["Nf"], w["T"] + 8, w["W"], max_q_tokens=w["Nq"],
-                  max_topk=w["k"], max_questions=1, device=local, flags=rekv.FLAG_TIMING)
+    g = rekv.ReKV(w["L"], w["Hq"], w["Hkv"], w["D"], w["Nf"], w["T"] + 8, w["W"], hbm_tail_frames=w["tail"],
+                  max_q_tokens=cu[-1], max_topk=w["k"], max_questions=nQ, device=local, flags=rekv.FLAG_TIMING)
     kf = torch.empty((w["L"], w["Nf"], w["Hkv"], w["D"]), dtype=torch.bfloat16, device=dev)
     vf = torch.empty_like(kf)
     for f in range(T0):
         synth.frame(w["seed"], synth.K, f, w["L"], w["Nf"], w["Hkv"], w["D"], w["off_scale"], device=dev, out=kf)
         synth.frame(w["seed"], synth.V, f, w["L"], w["Nf"], w["Hkv"], w["D"], w["off_scale"], device=dev, out=vf)
         g.append_frame(kf, vf)
-    # the frames appended inside the timed steps, and the rotating questions, resident in HBM
-    n_new = n_total_steps
+    # the frames appended inside the timed steps (a ring of 16, content irrelevant to the timing) and the
+    # rotating question batches, resident in HBM
+    ring_n = min(16, n_new)
     new_k = [synth.frame(w["seed"], synth.K, T0 + i, w["L"], w["Nf"], w["Hkv"], w["D"], w["off_scale"], device=dev)
-             for i in range(n_new)]
+             for i in range(ring_n)]
     new_v = [synth.frame(w["seed"], synth.V, T0 + i, w["L"], w["Nf"], w["Hkv"], w["D"], w["off_scale"], device=dev)
-             for i in range(n_new)]
-    qs = [synth.question(w["seed"], i, w["L"], w["Nq"], w["Hq"], w["D"], device=dev) for i in range(N_ROTATE)]
-    cu = [0, w["Nq"]]
+             for i in range(ring_n)]
+    qs = [torch.cat([synth.question(w["seed"], r * nQ + i, w["L"], n, w["Hq"], w["D"], device=dev)
+                     for i, n in enumerate(lengths)], dim=1).contiguous() for r in range(N_ROTATE)]
     out = torch.empty_like(qs[0])
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream(dev)
     state = {"next": 0}
 
+    def appends(src_k, src_v):
+        nf = 0
+        for _ in range(aps):
+            j = state["next"]
+            state["next"] += 1
+            nf = g.append_frame(src_k[j % len(src_k)], src_v[j % len(src_v)])
+        return nf
+
     def step_device(i, ev=None):
-        j = state["next"]
-        state["next"] += 1
         if ev:
             ev[0].record(stream)
-        nf = g.append_frame(new_k[j], new_v[j])
+        nf = appends(new_k, new_v)
         if ev:
             ev[1].record(stream)
         g.question(qs[i % N_ROTATE], cu, w["k"], nf + 1, out=out)
@@ -226,7 +279,6 @@ def run_cuda(args, w):
     for i in range(Wu):
         step_device(i)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    att_us = []
     sampler = ClockSampler(local)
     barrier()
     sampler.start()
@@ -241,15 +293,18 @@ def run_cuda(args, w):
     launches = g.launch_count() - l0
     clocks = sampler.stop()
     total_ms = t_begin.elapsed_time(t_end)
-    q_us = [e[1].elapsed_time(e[2]) * 1e3 for e in evs]
-    a_us = [e[0].elapsed_time(e[1]) * 1e3 for e in evs]
+    q_us = [e[1].elapsed_time(e[2]) * 1e3 / nQ for e in evs]
+    a_us = [e[0].elapsed_time(e[1]) * 1e3 / aps for e in evs]
     g.check_status()
 
-    # attention-kernel duration (library-internal events), sampled over a few more questions
+    # attention-kernel duration (library-internal events on the launching stream) and bytes over the host link
+    att_us, link_bytes = [], 0
     for i in range(min(K, 8)):
         g.question(qs[i % N_ROTATE], cu, w["k"], g.stats().frames, out=out)
         torch.cuda.synchronize()
-        att_us.append(g.stats().last_attend_kernel_us)
+        st = g.stats()
+        att_us.append(st.last_attend_kernel_us)
+        link_bytes = st.last_link_bytes
 
     # ---- end to end: inputs in pinned host memory, result read back, every step ----
     hk = [t.cpu().pin_memory() for t in new_k[:2]]
@@ -259,11 +314,12 @@ def run_cuda(args, w):
     dq = torch.empty_like(qs[0])
 
     def step_e2e(i, ev=None):
-        j = state["next"]
-        state["next"] += 1
-        kf.copy_(hk[i % 2], non_blocking=True)
-        vf.copy_(hv[i % 2], non_blocking=True)
-        nf = g.append_frame(kf, vf)
+        nf = 0
+        for a in range(aps):
+            state["next"] += 1
+            kf.copy_(hk[(i + a) % 2], non_blocking=True)
+            vf.copy_(hv[(i + a) % 2], non_blocking=True)
+            nf = g.append_frame(kf, vf)
         if ev:
             ev[0].record(stream)
         dq.copy_(hq[i % N_ROTATE], non_blocking=True)
@@ -279,7 +335,7 @@ def run_cuda(args, w):
     for i in range(K):
         step_e2e(i, evs2[i])
     barrier()
-    e2e_us = [e[0].elapsed_time(e[1]) * 1e3 for e in evs2]
+    e2e_us = [e[0].elapsed_time(e[1]) * 1e3 / nQ for e in evs2]
     g.check_status()
 
     def mean(x):
@@ -293,34 +349,48 @@ def run_cuda(args, w):
 
     if rank == 0:
         peaks = measured_peaks()
-        ab = algorithmic_bytes(w)
-        fl = attention_flops(w)
-        achieved = ab["attend_kernel"] / (att_kernel_us * 1e-6) / 1e9
+        ab = algorithmic_bytes(w, cu[-1], nQ)
+        fl = attention_flops(w, cu[-1])
         line = {
             "metric": "question_latency_us", "value": q_lat, "unit": "us", "n_gpus": world, "steps": K, "warmup": Wu,
             "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w["name"], "layers": w["L"], "q_heads": w["Hq"], "kv_heads": w["Hkv"],
-                       "frames": w["T"], "tokens_per_frame": w["Nf"], "q_tokens": w["Nq"], "top_k": w["k"],
-                       "window": w["W"], "cache_gb": 2 * w["L"] * w["T"] * w["Nf"] * w["Hkv"] * w["D"] * 2 / 1e9,
-                       "l2": "inputs larger than L2: each question streams 0.93 GB, 8 questions rotate",
+                       "frames": w["T"], "tokens_per_frame": w["Nf"], "questions_per_batch": nQ,
+                       "q_tokens": lengths if nQ > 1 else lengths[0], "top_k": w["k"], "window": w["W"],
+                       "hbm_tail_frames": w["tail"],
+                       "cache_gb": 2 * w["L"] * w["T"] * w["Nf"] * w["Hkv"] * w["D"] * 2 / 1e9,
+                       "l2": f"inputs larger than L2: a question batch streams {ab['total'] / 1e9:.2f} GB, "
+                             f"{N_ROTATE} batches rotate",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "step": "append 1 frame + 1 question (retrieve, gather, attend; all layers)"},
-            "question": {"bytes": ab["total"], "gbs": ab["total"] / (q_lat * 1e-6) / 1e9,
-                         "hbm_frac": ab["total"] / (q_lat * 1e-6) / 1e9 / peaks["hbm_gbs"],
-                         "frames_scored_per_s": None, "questions_per_s_all_gpus": world * 1e6 / q_lat},
+                       "step": f"append {aps} frame(s) + {nQ} question(s) (retrieve, gather, attend; all layers)"},
+            "question": {"bytes_per_batch": ab["total"], "gbs": ab["total"] / (q_lat * nQ * 1e-6) / 1e9,
+                         "hbm_frac": ab["total"] / (q_lat * nQ * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                         "attention_tflops": fl / (q_lat * nQ * 1e-6) / 1e12,
+                         "questions_per_s_all_gpus": world * 1e6 / q_lat},
             "append_us": app_us,
-            "roofline": {"kernel": "attention (step 5)", "bound": "hbm", "achieved": achieved,
-                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                         "traffic": None, "peak_source": peaks["source"], "kernel_us": att_kernel_us,
-                         "tensor_tflops": fl / (att_kernel_us * 1e-6) / 1e12,
-                         "tensor_frac": fl / (att_kernel_us * 1e-6) / 1e12 / peaks["bf16_tflops"]},
             "e2e": {"value": e2e_lat, "unit": "us",
-                    "h2d_bytes_per_step": 2 * kf.numel() * 2 + dq.numel() * 2, "d2h_bytes_per_step": out.numel() * 2},
+                    "h2d_bytes_per_step": aps * 2 * kf.numel() * 2 + dq.numel() * 2,
+                    "d2h_bytes_per_step": out.numel() * 2},
             "gpu_launches": int(launches),
             "clocks": clocks,
         }
-        if not args.no_cpu_baseline and world == 1:
+        if w["tail"] == 0:
+            achieved = ab["attend_kernel"] / (att_kernel_us * 1e-6) / 1e9
+            line["roofline"] = {"kernel": "attend_tc5_kernel (step 5)", "bound": "hbm", "achieved": achieved,
+                                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                                "traffic": TRAFFIC_NCU.get(w["name"]), "peak_source": peaks["source"],
+                                "kernel_us": att_kernel_us,
+                                "tensor_tflops": fl / (att_kernel_us * 1e-6) / 1e12,
+                                "tensor_frac": fl / (att_kernel_us * 1e-6) / 1e12 / peaks["bf16_tflops"]}
+        else:
+            link = pinned_h2d_gbs(dev)
+            achieved = link_bytes / (q_lat * 1e-6) / 1e9
+            line["roofline"] = {"kernel": "page_table_pull_kernel (step 4, host tier)", "bound": "host_link",
+                                "achieved": achieved, "peak": link, "unit": "GB/s", "frac": achieved / link,
+                                "traffic": None, "peak_source": "pinned H2D copy measured in this run",
+                                "link_bytes_per_question": link_bytes}
+        if not args.no_cpu_baseline and world == 1 and w["name"] == "7b_hbm_1800f":
             arm = OracleArm(w, w["L"])
             dt, scaled = arm.run(0)
             line["cpu_baseline"] = {"value": scaled * 1e6, "unit": "us", "cores": arm.cores, "kind": "oracle",
@@ -339,11 +409,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="7b_hbm_1800f", choices=sorted(WORKLOADS))
     ap.add_argument("--layers", type=int, default=None, help="profiling only: fewer layers than the workload")
     ap.add_argument("--frames", type=int, default=None, help="profiling only: a shorter stream")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
-    w = dict(WORKLOAD)
+    w = dict(WORKLOADS[args.workload], name=args.workload)
     if args.layers or args.frames:
         w["L"] = args.layers or w["L"]
         w["T"] = args.frames or w["T"]
