@@ -161,6 +161,26 @@ const char* rekv_last_error(rekv_ctx* ctx);
 int rekv_get_reps(rekv_ctx* ctx, int layer, int n_frames, float* dev_out, void* stream);
 int rekv_get_page(rekv_ctx* ctx, int frame, int layer, void* k_out, void* v_out, void* stream);
 
+/* Scoring without allocation (the paper has no counterpart; this entry point exists for hosts that
+ * cannot let a library allocate device memory -- a serving engine that owns the whole GPU through its
+ * own pool, or a latency-critical thread that must not meet cudaMalloc's device synchronisation).
+ * Computes, for one layer, the cosine score of every frame representative against each of nQ question
+ * vectors, exactly as rekv_retrieve does (question vector = mean over the question's tokens and over
+ * the G query heads of each KV group; norms clamped at 1e-8), without a context and without calling
+ * cudaMalloc, cudaFree or any allocating routine: its intermediate lives in a 66 048-byte array that
+ * is part of the library image (held by every GPU that loads the library until the process exits).
+ *   q          device bf16 [sum_Nq][H_q][128], the layer's query rows, questions packed back to back
+ *   cu_q       HOST int32[nQ+1] prefix sums of the question lengths; 1 <= nQ <= 16
+ *   reps       device fp32 [n_frames][H_kv*128] frame representatives (e.g. from rekv_get_reps)
+ *   scores_out device fp32 [nQ][n_frames]
+ * Limits: head_dim == 128, H_kv <= 8 (H_kv*128 <= 1024), nQ <= 16; anything larger is rejected with
+ * REKV_ERR_ARG and a message (rekv_last_error(NULL)).  Runs on the CURRENT device, on `stream`.
+ * The first call on a device resolves the array's device address (cudaGetSymbolAddress); make that
+ * first call outside any stream capture.  All calls on a device share the array: each call rewrites
+ * it completely and leaves its contents behind, and calls whose kernels overlap on the GPU race. */
+int rekv_score_frames_static(const void* q, const int32_t* cu_q, int nQ, int n_q_heads, int n_kv_heads, int head_dim,
+                             const float* reps, int n_frames, float* scores_out, void* stream);
+
 /* Number of kernels this library has launched on the context since creation (for launch counting). */
 int64_t rekv_launch_count(rekv_ctx* ctx);
 

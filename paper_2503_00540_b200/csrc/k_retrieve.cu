@@ -263,3 +263,112 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
   c->launches += 2;
   return cudaGetLastError();
 }
+
+// ---------------------------------------------------------------------------------------------
+// rekv_score_frames_static: scoring without any allocation.
+//
+// Some hosts cannot let a library allocate device memory: a serving engine that has handed the whole
+// GPU to its own memory pool, or a latency-critical thread for which the implicit device
+// synchronisation of cudaMalloc/cudaFree is not acceptable.  For them this entry point runs the
+// question-vector and cosine-score kernels of one layer with their intermediate (the fp32 question
+// vectors and their partial squared norms) in a fixed array that is part of the library image, so
+// nothing is allocated, here or in any routine it calls.
+//
+// The array lives in every GPU context that loads the library, for the life of the process.  All
+// calls on a device share it: it is fully rewritten by each call (nothing in it has to start at
+// zero), it keeps the last call's contents afterwards, and two calls whose kernels overlap on the
+// GPU (different streams, no ordering between them) race on it.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int STATIC_MAX_QUESTIONS = 16;
+constexpr int STATIC_MAX_DP = 1024;                       // H_kv * 128
+constexpr int STATIC_QA_FLOATS = STATIC_MAX_QUESTIONS * STATIC_MAX_DP;
+constexpr int STATIC_QSQ_FLOATS = STATIC_MAX_QUESTIONS * 8;
+// 66 048 bytes: question vectors [16][1024] followed by partial squared norms [16][8]
+static __device__ __align__(256) float g_static_scratch[STATIC_QA_FLOATS + STATIC_QSQ_FLOATS];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+float* g_static_scratch_addr[STATIC_MAX_DEVICES] = {nullptr};  // device address of the array, per device
+
+}  // namespace
+
+extern "C" int rekv_score_frames_static(const void* q, const int32_t* cu_q, int nQ, int n_q_heads, int n_kv_heads,
+                                        int head_dim, const float* reps, int n_frames, float* scores_out, void* stream) {
+  if (!q || !cu_q || !reps || !scores_out) {
+    rekv_set_error(nullptr, "rekv_score_frames_static: null pointer argument");
+    return REKV_ERR_ARG;
+  }
+  if (head_dim != REKV_HEAD_DIM || n_kv_heads < 1 || n_kv_heads > 8 || n_q_heads < n_kv_heads ||
+      n_q_heads % n_kv_heads) {
+    rekv_set_error(nullptr, "rekv_score_frames_static: head_dim must be 128 and 1 <= H_kv <= 8 must divide H_q");
+    return REKV_ERR_ARG;
+  }
+  if (nQ < 1 || nQ > STATIC_MAX_QUESTIONS) {
+    rekv_set_error(nullptr, "rekv_score_frames_static: at most 16 questions per call (fixed scratch size)");
+    return REKV_ERR_ARG;
+  }
+  if (n_frames < 1) {
+    rekv_set_error(nullptr, "rekv_score_frames_static: no frames");
+    return REKV_ERR_EMPTY;
+  }
+  QBatch qb;
+  qb.nQ = nQ;
+  if (cu_q[0] != 0) {
+    rekv_set_error(nullptr, "rekv_score_frames_static: cu_q[0] must be 0");
+    return REKV_ERR_ARG;
+  }
+  for (int i = 0; i < nQ; ++i) {
+    if (cu_q[i + 1] <= cu_q[i]) {
+      rekv_set_error(nullptr, "rekv_score_frames_static: a question has no tokens");
+      return REKV_ERR_ARG;
+    }
+    qb.cu[i] = cu_q[i];
+  }
+  qb.cu[nQ] = qb.sumNq = cu_q[nQ];
+
+  // Set-up, once per device, with that device current: in host code the array's name is only a
+  // stand-in; the kernels need its device address, which the runtime resolves here.
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) {
+    rekv_set_error(nullptr, "rekv_score_frames_static: no current CUDA device (or ordinal >= 64)");
+    cudaGetLastError();
+    return REKV_ERR_CUDA;
+  }
+  if (!g_static_scratch_addr[dev]) {
+    float* ptr = nullptr;
+    e = cudaGetSymbolAddress((void**)&ptr, g_static_scratch);
+    if (e != cudaSuccess || !ptr) {
+      rekv_set_error(nullptr, "rekv_score_frames_static: cudaGetSymbolAddress failed for the scratch array");
+      cudaGetLastError();
+      return REKV_ERR_CUDA;
+    }
+    g_static_scratch_addr[dev] = ptr;
+  }
+  float* qa = g_static_scratch_addr[dev];
+  float* qsq = qa + STATIC_QA_FLOATS;
+
+  const int Dp = n_kv_heads * REKV_HEAD_DIM, G = n_q_heads / n_kv_heads;
+  cudaStream_t st = (cudaStream_t)stream;
+  qmean_kernel<<<dim3(nQ, 1, n_kv_heads), 256, 0, st>>>((const __nv_bfloat162*)q, qb, n_q_heads, n_kv_heads, G, qa, qsq,
+                                                         STATIC_MAX_QUESTIONS);
+  // the question vectors of one call fit in 64 KB of dynamic shared memory only in groups
+  int q_group = (int)((96 * 1024) / (Dp * sizeof(float)));
+  if (q_group > nQ) q_group = nQ;
+  e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+  if (e != cudaSuccess) {
+    rekv_set_error(nullptr, "rekv_score_frames_static: cannot raise the shared-memory limit of the score kernel");
+    return REKV_ERR_CUDA;
+  }
+  dim3 grid((n_frames + SCORE_FRAMES_PER_CTA - 1) / SCORE_FRAMES_PER_CTA, 1);
+  score_kernel<<<grid, 256, (size_t)q_group * Dp * sizeof(float), st>>>(reps, qa, qsq, nQ, STATIC_MAX_QUESTIONS, Dp,
+                                                                       n_kv_heads, n_frames, n_frames, q_group,
+                                                                       scores_out);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    rekv_set_error(nullptr, cudaGetErrorString(e));
+    return REKV_ERR_CUDA;
+  }
+  return REKV_OK;
+}

@@ -42,7 +42,7 @@ class rekv_stats_t(ctypes.Structure):
 
 EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", "rekv_gather", "rekv_attend",
            "rekv_stats", "rekv_check_status", "rekv_last_error", "rekv_get_reps", "rekv_get_page",
-           "rekv_launch_count")
+           "rekv_launch_count", "rekv_score_frames_static")
 
 _lib = None
 
@@ -66,6 +66,7 @@ def lib() -> ctypes.CDLL:
         L.rekv_last_error.restype = ctypes.c_char_p
         L.rekv_get_reps.argtypes = [vp, i32, i32, vp, vp]
         L.rekv_get_page.argtypes = [vp, i32, i32, vp, vp, vp]
+        L.rekv_score_frames_static.argtypes = [vp, ip, i32, i32, i32, i32, vp, i32, vp, vp]
         L.rekv_launch_count.argtypes = [vp]
         L.rekv_launch_count.restype = ctypes.c_int64
         for name in EXPORTS:
@@ -213,3 +214,21 @@ def kv_cache_bytes(n_layers: int, n_frames: int, tokens_per_frame: int, n_kv_hea
                    bytes_per_element: int = 2) -> int:
     """K/V bytes of a stream: 2 * L * T * M * H * D * bytes (the paper's cache-size expression)."""
     return 2 * n_layers * n_frames * tokens_per_frame * n_kv_heads * head_dim * bytes_per_element
+
+
+def score_frames_static(q: torch.Tensor, cu_q: Sequence[int], n_kv_heads: int, reps: torch.Tensor,
+                        out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Allocation-free scoring of one layer (see rekv_score_frames_static in include/rekv.h).
+
+    q: bf16 [sum_Nq][H_q][128]; reps: fp32 [n_frames][H_kv*128]; returns fp32 [nQ][n_frames].  The output
+    tensor is the caller's (pass `out` to keep this call itself free of allocations)."""
+    nQ = len(cu_q) - 1
+    if out is None:
+        out = torch.empty((nQ, reps.shape[0]), dtype=torch.float32, device=q.device)
+    with torch.cuda.device(q.device):
+        rc = lib().rekv_score_frames_static(_ptr(q, torch.bfloat16), _cu_array(cu_q), nQ, q.shape[1], n_kv_heads,
+                                            q.shape[2], _ptr(reps, torch.float32), reps.shape[0],
+                                            _ptr(out, torch.float32), torch.cuda.current_stream(q.device).cuda_stream)
+    if rc < 0:
+        raise RekvError(rc, (lib().rekv_last_error(None) or b"").decode())
+    return out
