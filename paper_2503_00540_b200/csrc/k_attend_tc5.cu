@@ -159,6 +159,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem_slot;
+  // everything above is independent of earlier kernels; the context table and Q are not
+  grid_dep_wait();
+  grid_dep_launch();
   auto col_o = [](int t) { return (uint32_t)t * 128u; };
   auto col_s = [](int t) { return 256u + (uint32_t)t * 128u; };
 
@@ -514,7 +517,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
 }
 
 // Merge the partials of the units that were cut by a CTA boundary.
-// grid = (units, 2 row tiles, 4 row quarters); 4 warps x 8 rows, a warp per row, float4 per lane.
+// grid = (units, 2 row tiles, 32 groups of 4 rows); a warp per row, float4 per lane: one short
+// dependent chain per warp, enough warps in flight to hide its latency.
 __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
   const long long u = blockIdx.x;
   const int t = blockIdx.y;
@@ -523,10 +527,11 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
   const UnitInfo ui = decode_unit(p, u);
   if (t >= ui.tiles) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int k8 = 0; k8 < 8; ++k8) {
-    const int r = blockIdx.z * 32 + warp * 8 + k8;
+  grid_dep_wait();
+  {
+    const int r = blockIdx.z * 4 + warp;
     const int rr = ui.m0 + t * 128 + r;
-    if (rr >= ui.rows_q) break;
+    if (rr >= ui.rows_q) return;
     float M = -INFINITY;
     for (long long c = c_first; c <= c_last; ++c) M = fmaxf(M, p.part_ml[(((c + u) * 2 + t) * 128 + r) * 2]);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -608,14 +613,16 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     attr_set = true;
   }
   if (timed) cudaEventRecord(c->ev_t0, st);
-  attend_tc5_kernel<<<(unsigned)grid, TC_THREADS, smem, st>>>(p);
+  cudaError_t e1 = rekv_launch_pdl(attend_tc5_kernel, dim3((unsigned)grid), dim3(TC_THREADS), smem, st, p);
+  if (e1 != cudaSuccess) return e1;
   if (timed) {
     cudaEventRecord(c->ev_t1, st);
     c->timing_valid = true;
   }
   c->launches += 1;
   if (p.per != ncf) {
-    combine_tc5_kernel<<<dim3((unsigned)units, 2, 4), 128, 0, st>>>(p);
+    cudaError_t e2 = rekv_launch_pdl(combine_tc5_kernel, dim3((unsigned)units, 2, 32), dim3(128), 0, st, p);
+    if (e2 != cudaSuccess) return e2;
     c->launches += 1;
   }
   return cudaGetLastError();

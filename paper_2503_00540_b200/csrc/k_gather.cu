@@ -5,6 +5,7 @@
 // pulled over the host link into an HBM staging page by the same kernel (zero-copy reads of the
 // mapped pinned arena, 16 bytes per load, many loads in flight).  A second kernel can write the
 // context out contiguously in plain [token][dim] layout.
+#include "ptx_helpers.cuh"
 #include "rekv_internal.cuh"
 
 namespace {
@@ -19,6 +20,8 @@ __global__ void __launch_bounds__(256) page_table_pull_kernel(StoreView s, const
                                                               unsigned long long* __restrict__ link_bytes) {
   const int j = blockIdx.x / parts, part = blockIdx.x % parts;
   const int qi = blockIdx.y, l = layer0 + blockIdx.z;
+  rekv_ptx::grid_dep_wait();
+  rekv_ptx::grid_dep_launch();
   int frame;
   if (j < k_eff)
     frame = idx[((long long)l * nQ + qi) * top_k + j];
@@ -94,9 +97,12 @@ cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int 
   if (ncf <= 0 || layer1 <= layer0) return cudaSuccess;
   const int parts = c->sv.tail > 0 ? PULL_PARTS_HOST : 1;
   dim3 grid(ncf * parts, nQ, layer1 - layer0);
+  c->launches += 1;
+  if (c->sv.tail == 0)
+    return rekv_launch_pdl(page_table_pull_kernel, grid, dim3(256), 0, st, c->sv, idx, nQ, top_k, k_eff, ncf, n_visible,
+                           layer0, frames_now, parts, c->ctx_tbl, c->status, c->link_bytes);
   page_table_pull_kernel<<<grid, 256, 0, st>>>(c->sv, idx, nQ, top_k, k_eff, ncf, n_visible, layer0, frames_now,
                                                parts, c->ctx_tbl, c->status, c->link_bytes);
-  c->launches += 1;
   return cudaGetLastError();
 }
 

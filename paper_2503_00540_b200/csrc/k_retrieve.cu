@@ -1,5 +1,6 @@
 // Steps 2-3: question vector, cosine scores against every frame representative (Eq. 2, tau = 1),
 // and the exact top-r selection, per layer and per question.
+#include "ptx_helpers.cuh"
 #include "rekv_internal.cuh"
 
 namespace {
@@ -18,10 +19,18 @@ __global__ void __launch_bounds__(256) qmean_kernel(const __nv_bfloat162* __rest
   float sx = 0.f, sy = 0.f;
   for (int n = n0 + slice; n < n1; n += 4) {
     const __nv_bfloat162* row = q + (((long long)l * qb.sumNq + n) * Hq + g * G) * 64 + d2;
-    for (int j = 0; j < G; ++j) {
-      float2 f = __bfloat1622float2(row[j * 64]);
-      sx += f.x;
-      sy += f.y;
+    for (int j0 = 0; j0 < G; j0 += 8) {  // up to eight independent loads in flight
+      __nv_bfloat162 v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (j0 + j < G) v[j] = row[(j0 + j) * 64];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (j0 + j < G) {
+          float2 f = __bfloat1622float2(v[j]);
+          sx += f.x;
+          sy += f.y;
+        }
     }
   }
   __shared__ float2 part[4][64];
@@ -57,6 +66,8 @@ __global__ void __launch_bounds__(256) score_kernel(const float* __restrict__ re
                                                     float* __restrict__ scores) {
   extern __shared__ float4 s_q[];  // [q_group][Dp/4]
   __shared__ float s_qn[REKV_MAX_QUESTIONS];
+  rekv_ptx::grid_dep_wait();
+  rekv_ptx::grid_dep_launch();
   const int l = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int f0 = blockIdx.x * SCORE_FRAMES_PER_CTA;
@@ -148,6 +159,8 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
   __shared__ int warp_gt[16], warp_eq[16];
   __shared__ int s_base_gt, s_base_eq;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  rekv_ptx::grid_dep_wait();
+  rekv_ptx::grid_dep_launch();
 
   for (int j = k_eff + threadIdx.x; j < top_k; j += blockDim.x) out[j] = -1;
   if (k_eff <= 0) return;
@@ -252,12 +265,15 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
     attr_set = true;
   }
   dim3 grid((n_visible + SCORE_FRAMES_PER_CTA - 1) / SCORE_FRAMES_PER_CTA, s.L);
-  score_kernel<<<grid, 256, smem, st>>>(s.reps, c->qa, c->qnorm, qb.nQ, maxQ, s.Dp, s.Hkv, s.max_frames, n_visible,
-                                        q_group, scores);
+  cudaError_t e1 = rekv_launch_pdl(score_kernel, grid, dim3(256), smem, st, s.reps, c->qa, c->qnorm, qb.nQ, maxQ, s.Dp,
+                                   s.Hkv, s.max_frames, n_visible, q_group, scores);
+  if (e1 != cudaSuccess) return e1;
   if (top_k > 0) {
     int n_cand = n_visible - c->cfg.window_frames;
     if (n_cand < 0) n_cand = 0;
-    topk_kernel<<<dim3(qb.nQ, s.L), 512, 0, st>>>(scores, qb.nQ, n_visible, n_cand, top_k, k_eff, idx_out);
+    cudaError_t e2 = rekv_launch_pdl(topk_kernel, dim3(qb.nQ, s.L), dim3(512), 0, st, scores, qb.nQ, n_visible, n_cand,
+                                     top_k, k_eff, idx_out);
+    if (e2 != cudaSuccess) return e2;
     c->launches += 1;
   }
   c->launches += 2;

@@ -289,13 +289,13 @@ int rekv_gather(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, int n_visibl
   DeviceGuard guard(c->device);
   cudaStream_t st = (cudaStream_t)stream;
   const StoreView& s = c->sv;
-  REKV_CUDA(c, cudaMemsetAsync(c->link_bytes, 0, sizeof(unsigned long long), st));
   if (s.tail == 0) {
     REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, k_eff, n_visible, 0, s.L, c->frames, st));
     c->gather_layerwise = false;
   } else {
     // host tier: the pulls run layer by layer on the side stream (behind every write-through that is
     // still in flight there); attention of layer l only waits for layer l's event
+    REKV_CUDA(c, cudaMemsetAsync(c->link_bytes, 0, sizeof(unsigned long long), st));
     REKV_CUDA(c, cudaEventRecord(c->ev_main, st));
     REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_main, 0));
     for (int l = 0; l < s.L; ++l) {

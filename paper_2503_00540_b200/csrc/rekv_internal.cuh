@@ -108,6 +108,24 @@ struct rekv_ctx {
 
 void rekv_set_error(rekv_ctx* ctx, const char* msg);
 
+// Launch with programmatic stream serialization: the kernel may begin (its prologue up to
+// grid_dep_wait()) while the previous kernel of the stream is still draining.
+template <typename... KArgs, typename... Args>
+inline cudaError_t rekv_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                   Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- kernel launchers (each returns the cudaError_t of its launches) -----------------------
 // k_append.cu
 cudaError_t rekv_launch_append(rekv_ctx* c, const void* k, const void* v, int frame, cudaStream_t st);
