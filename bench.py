@@ -49,7 +49,11 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs.
+
+    nvidia-smi needs a moment to start, so it is launched before the warm-up; mark_begin()/mark_end()
+    delimit the samples that fall inside the timed region (if the region is shorter than one sampling
+    period, the sample taken right after it is used)."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -58,6 +62,10 @@ class ClockSampler:
         self.gpu = gpu_index
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.p = None
+        self.begin = self.end = 0
+
+    def _lines(self):
+        return [r for r in open(self.f.name).read().splitlines() if r.strip()]
 
     def start(self):
         try:
@@ -67,18 +75,31 @@ class ClockSampler:
         except Exception:
             self.p = None
 
+    def mark_begin(self):
+        if self.p is None:
+            return
+        t0 = time.time()
+        while not self._lines() and time.time() - t0 < 3.0:  # wait for the first sample
+            time.sleep(0.02)
+        self.begin = len(self._lines())
+
+    def mark_end(self):
+        if self.p is None:
+            return
+        time.sleep(0.06)  # let the sample that covers the end of the region land
+        self.end = len(self._lines())
+
     def stop(self):
         if self.p is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
         self.p.terminate()
         try:
             self.p.wait(timeout=5)
         except Exception:
             self.p.kill()
-        self.f.flush()
-        rows = [r.split(",") for r in open(self.f.name).read().strip().splitlines() if r.strip()]
+        rows = [r.split(",") for r in self._lines()]
         os.unlink(self.f.name)
+        rows = rows[max(self.begin - 1, 0):max(self.end, self.begin + 1)]
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
@@ -187,6 +208,15 @@ def run_reference(args, w):
 
 
 # ------------------------------------------------------------------------------------------ CUDA arm
+def max_over_ranks(values, device, world):
+    """Every reported time is the maximum over the ranks (replicas run independently)."""
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
 def pinned_h2d_gbs(dev, n_bytes=1 << 30, reps=5):
     """Measured pinned host -> device copy bandwidth (the host-link peak of this machine)."""
     h = torch.empty(n_bytes, dtype=torch.uint8).pin_memory()
@@ -276,12 +306,13 @@ def run_cuda(args, w):
         torch.cuda.synchronize()
 
     # ---- device-resident timing ----
+    sampler = ClockSampler(local)
+    sampler.start()
     for i in range(Wu):
         step_device(i)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    sampler = ClockSampler(local)
     barrier()
-    sampler.start()
+    sampler.mark_begin()
     l0 = g.launch_count()
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
@@ -290,6 +321,7 @@ def run_cuda(args, w):
         step_device(i, evs[i])
     t_end.record(stream)
     barrier()
+    sampler.mark_end()
     launches = g.launch_count() - l0
     clocks = sampler.stop()
     total_ms = t_begin.elapsed_time(t_end)
@@ -341,11 +373,21 @@ def run_cuda(args, w):
     def mean(x):
         return sum(x) / len(x)
 
-    vals = torch.tensor([mean(q_us), total_ms / K, mean(e2e_us), mean(a_us), mean(att_us)], dtype=torch.float64,
-                        device=dev)
-    if world > 1:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    q_lat, ms_step, e2e_lat, app_us, att_kernel_us = vals.tolist()
+    # steps 2-3 alone (question vectors, scores, selection): frames scored per second
+    n_vis = g.stats().frames
+    ev_r = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    for i in range(3):
+        g.retrieve(qs[i % N_ROTATE], cu, w["k"], n_vis)
+    torch.cuda.synchronize()
+    ev_r[0].record(stream)
+    for i in range(10):
+        g.retrieve(qs[i % N_ROTATE], cu, w["k"], n_vis)
+    ev_r[1].record(stream)
+    torch.cuda.synchronize()
+    retrieve_us = ev_r[0].elapsed_time(ev_r[1]) * 1e3 / 10
+
+    q_lat, ms_step, e2e_lat, app_us, att_kernel_us, retrieve_us = max_over_ranks(
+        [mean(q_us), total_ms / K, mean(e2e_us), mean(a_us), mean(att_us), retrieve_us], dev, world)
 
     if rank == 0:
         peaks = measured_peaks()
@@ -367,6 +409,8 @@ def run_cuda(args, w):
             "question": {"bytes_per_batch": ab["total"], "gbs": ab["total"] / (q_lat * nQ * 1e-6) / 1e9,
                          "hbm_frac": ab["total"] / (q_lat * nQ * 1e-6) / 1e9 / peaks["hbm_gbs"],
                          "attention_tflops": fl / (q_lat * nQ * 1e-6) / 1e12,
+                         "retrieve_us_per_batch": retrieve_us,
+                         "frames_scored_per_s_all_gpus": world * w["L"] * n_vis * nQ / (retrieve_us * 1e-6),
                          "questions_per_s_all_gpus": world * 1e6 / q_lat},
             "append_us": app_us,
             "e2e": {"value": e2e_lat, "unit": "us",

@@ -52,8 +52,6 @@ enum {
 
 /* rekv_config.flags */
 enum {
-  REKV_FLAG_HOST_GATHER_COPY_ENGINE = 1u << 0, /* host tier: per-page cudaMemcpyAsync instead of the
-                                                  zero-copy gather kernel (needs a host sync on the indices) */
   REKV_FLAG_ATTEND_LEGACY_MMA = 1u << 1,        /* use the mma.sync attention kernel instead of tcgen05 */
   REKV_FLAG_TIMING = 1u << 2                    /* bracket the attention kernel with CUDA events on the caller's
                                                   stream; rekv_stats then reports its duration */

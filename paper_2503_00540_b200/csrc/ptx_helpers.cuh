@@ -99,13 +99,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 
-// two non-negative finite floats -> packed bf16x2 with integer arithmetic only (round half up): keeps
-// the conversion off the transcendental/conversion pipe, which the softmax exponentials saturate
-__device__ __forceinline__ uint32_t pack_bf16_int(float lo, float hi) {
-  const uint32_t a = __float_as_uint(lo) + 0x8000u, b = __float_as_uint(hi) + 0x8000u;
-  return __byte_perm(a, b, 0x7632);
-}
-
 // ---- 5th-generation tensor cores: tensor memory (TMEM) and tcgen05.mma -------------------------
 // TMEM address: bits 31..16 lane, bits 15..0 column (one column = 32 bits per lane).
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {  // whole warp

@@ -15,7 +15,6 @@ import torch
 from . import _build
 
 OK, ERR_ARG, ERR_FULL, ERR_EMPTY, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT, ERR_STATE = 0, -1, -2, -3, -4, -5, -6, -7
-FLAG_HOST_GATHER_COPY_ENGINE = 1 << 0
 FLAG_ATTEND_LEGACY_MMA = 1 << 1
 FLAG_TIMING = 1 << 2
 
