@@ -33,6 +33,9 @@ WORKLOADS = {
                               off_scale=0.5, tail=64, nQ=1, appends_per_step=1),
     "7b_stream_batch16": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=32, Nq=(24, 64), seed=2503,
                               off_scale=0.5, tail=0, nQ=16, appends_per_step=10),
+    # decode-shaped question (one token): the HBM-bound end of Eq. 3
+    "7b_hbm_decode_1tok": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=1, seed=2503, off_scale=0.5,
+                               tail=0, nQ=1, appends_per_step=1),
     "72b_offload_1800f": dict(L=80, Hq=64, Hkv=8, D=128, Nf=196, T=1800, W=8, k=32, Nq=64, seed=2503,
                               off_scale=0.5, tail=32, nQ=1, appends_per_step=1),
 }

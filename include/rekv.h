@@ -68,7 +68,8 @@ typedef struct {
                                 memory and only the most recent n frames are also kept in HBM */
   int32_t window_frames;     /* W: the last W visible frames are always part of a question's context and
                                 are not retrieval candidates; W <= hbm_tail_frames when offloaded */
-  int32_t block_frames;      /* frames per retrieval block (the paper's b); only 1 is accepted */
+  int32_t block_frames;      /* frames per retrieval block (the paper's b), 1..64; max_topk and top_k must be
+                                multiples of it */
   int32_t max_q_tokens;      /* upper bound on the sum of question lengths in one batch */
   int32_t max_topk;          /* upper bound on top_k */
   int32_t max_questions;     /* upper bound on questions per batch (<= 64) */
@@ -117,7 +118,12 @@ int rekv_append_frame(rekv_ctx* ctx, const void* k, const void* v, void* stream)
  * The question vector averages the question's tokens and the G = H_q/H_kv query heads of each KV
  * group; score = <q, rep> / (max(|q|,1e-8) * max(|rep|,1e-8)).  Candidates are frames
  * [0, n_visible - W); ties go to the lower frame index; NaN ranks below every number.
- * Returns k_eff. */
+ * Block retrieval (block_frames = b > 1, Eq. 2 paragraph): the candidates are the complete blocks of b
+ * consecutive frames inside [0, n_visible - W); a block's vector is the mean of its frames'
+ * representatives; top_k / b blocks are kept and written to idx_out as their frames; scores_out is then
+ * [L][nQ][n_blocks].  Every frame after the last complete block (the window plus the frames that do not
+ * fill a block yet, W_eff = n_visible - b*n_blocks of them) is always part of the context.
+ * Returns k_eff (frames). */
 int rekv_retrieve(rekv_ctx* ctx, const void* q, const int32_t* cu_q, int nQ, int top_k, int n_visible,
                   int32_t* idx_out, float* scores_out, void* stream);
 

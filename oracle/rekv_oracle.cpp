@@ -115,6 +115,34 @@ void oracle_score(const uint16_t* q, int n_q, int n_q_heads, int n_kv_heads, int
   }
 }
 
+/* Step 2, block variant (Eq. 2 paragraph: "group b consecutive frames into blocks by averaging their frame
+ * vectors").  Block j averages the representatives of frames [j*b, (j+1)*b); only complete blocks exist.
+ * scores[j] = cosine(question vector, block vector), tau = 1.  The block mean is kept in double. */
+void oracle_score_blocks(const uint16_t* q, int n_q, int n_q_heads, int n_kv_heads, int head_dim, const float* reps,
+                         int n_blocks, int b, float* scores) {
+  const int dp = n_kv_heads * head_dim;
+  const double eps = 1e-8;
+  std::vector<double> qa(dp), bv(dp);
+  oracle_question_vector(q, n_q, n_q_heads, n_kv_heads, head_dim, qa.data());
+  double qn = 0.0;
+  for (int c = 0; c < dp; ++c) qn += qa[c] * qa[c];
+  qn = std::max(std::sqrt(qn), eps);
+  for (int j = 0; j < n_blocks; ++j) {
+    for (int c = 0; c < dp; ++c) {
+      double s = 0.0;
+      for (int f = 0; f < b; ++f) s += (double)reps[((long)j * b + f) * dp + c];
+      bv[c] = s / (double)b;
+    }
+    double dot = 0.0, rn = 0.0;
+    for (int c = 0; c < dp; ++c) {
+      dot += qa[c] * bv[c];
+      rn += bv[c] * bv[c];
+    }
+    rn = std::max(std::sqrt(rn), eps);
+    scores[j] = (float)(dot / (qn * rn));
+  }
+}
+
 /* Step 3.  Candidates are frames [0, n_visible - window).  Order by (score descending, index
  * ascending), keep k_eff = min(k, #candidates), write them in ascending index order, pad idx_out
  * (length k) with -1.  *gap_out = score of the last kept minus score of the best rejected

@@ -22,6 +22,9 @@ _lib.oracle_question_vector.restype = None
 _lib.oracle_score.argtypes = [_u16p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
                               ctypes.c_int, ctypes.c_void_p]
 _lib.oracle_score.restype = None
+_lib.oracle_score_blocks.argtypes = [_u16p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+                                     ctypes.c_int, ctypes.c_int, ctypes.c_void_p]
+_lib.oracle_score_blocks.restype = None
 _lib.oracle_select.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
                                ctypes.POINTER(ctypes.c_double)]
 _lib.oracle_select.restype = ctypes.c_int
@@ -69,6 +72,27 @@ def score(q: torch.Tensor, reps: torch.Tensor, n_kv_heads: int) -> torch.Tensor:
     out = torch.empty(n_frames, dtype=torch.float32)
     _lib.oracle_score(q.data_ptr(), n_q, n_qh, n_kv_heads, d, reps.data_ptr(), n_frames, out.data_ptr())
     return out
+
+
+def score_blocks(q: torch.Tensor, reps: torch.Tensor, n_kv_heads: int, n_blocks: int, b: int) -> torch.Tensor:
+    """Cosine score of each complete block of b frames (block vector = mean of its frame vectors) -> float32 [n_blocks]."""
+    _chk(q, torch.bfloat16)
+    _chk(reps, torch.float32)
+    n_q, n_qh, d = q.shape
+    assert reps.shape[0] >= n_blocks * b and reps.shape[1] == n_kv_heads * d
+    out = torch.empty(n_blocks, dtype=torch.float32)
+    _lib.oracle_score_blocks(q.data_ptr(), n_q, n_qh, n_kv_heads, d, reps.data_ptr(), n_blocks, b, out.data_ptr())
+    return out
+
+
+def block_geometry(n_visible: int, window: int, b: int, top_k: int):
+    """Block retrieval geometry: only complete blocks of the candidate frames [0, n_visible - window) can be
+    retrieved; every frame after the last complete block is part of the context (the window plus the frames
+    that do not fill a block yet).  -> (n_blocks, k_blocks, window_eff)."""
+    n_cand = max(n_visible - window, 0)
+    n_blocks = n_cand // b
+    k_blocks = min(top_k // b, n_blocks)
+    return n_blocks, k_blocks, n_visible - n_blocks * b
 
 
 def select(scores: torch.Tensor, n_visible: int, window: int, k: int) -> Tuple[torch.Tensor, int, float]:
@@ -122,9 +146,10 @@ class OracleCache:
     """
 
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, tokens_per_frame: int,
-                 window: int):
+                 window: int, block: int = 1):
         self.L, self.Hq, self.Hkv, self.D, self.Nf, self.W = (n_layers, n_q_heads, n_kv_heads, head_dim,
                                                               tokens_per_frame, window)
+        self.b = block
         self.k_frames: List[torch.Tensor] = []
         self.v_frames: List[torch.Tensor] = []
         self.reps: List[torch.Tensor] = []  # per frame: float32 [L][D']
@@ -147,12 +172,29 @@ class OracleCache:
         scores, idxs, gaps = [], [], []
         k_eff = 0
         for l in range(self.L):
-            s = score(q[l].contiguous(), self.rep_table(l, n_visible), self.Hkv)
-            i, k_eff, g = select(s, n_visible, self.W, top_k)
+            if self.b == 1:
+                s = score(q[l].contiguous(), self.rep_table(l, n_visible), self.Hkv)
+                i, k_eff, g = select(s, n_visible, self.W, top_k)
+            else:
+                # block retrieval: score complete blocks, keep top_k/b of them, expand to their frames
+                n_blocks, k_blocks, _ = block_geometry(n_visible, self.W, self.b, top_k)
+                s = score_blocks(q[l].contiguous(), self.rep_table(l, n_visible), self.Hkv, n_blocks, self.b)
+                bi, kb, g = select(s, n_blocks, 0, top_k // self.b)
+                assert kb == k_blocks
+                k_eff = kb * self.b
+                i = torch.full((top_k,), -1, dtype=torch.int32)
+                for j in range(kb):
+                    for f in range(self.b):
+                        i[j * self.b + f] = int(bi[j]) * self.b + f
             scores.append(s)
             idxs.append(i)
             gaps.append(g)
         return torch.stack(scores), torch.stack(idxs), k_eff, gaps
+
+    def window_eff(self, n_visible: int, top_k: int) -> int:
+        if self.b == 1:
+            return min(self.W, n_visible)
+        return block_geometry(n_visible, self.W, self.b, top_k)[2]
 
     def layer_cache(self, layer: int, which: str) -> torch.Tensor:
         src = self.k_frames if which == "k" else self.v_frames
@@ -161,9 +203,10 @@ class OracleCache:
     def gather(self, idx: torch.Tensor, k_eff: int, n_visible: int):
         """idx: int32 [L][top_k] -> (k_ctx, v_ctx) bf16 [L][H_kv][n_ctx][D]."""
         ks, vs = [], []
+        w_eff = self.window_eff(n_visible, idx.shape[-1])
         for l in range(self.L):
-            ks.append(gather(self.layer_cache(l, "k"), idx[l].contiguous(), k_eff, n_visible, self.W))
-            vs.append(gather(self.layer_cache(l, "v"), idx[l].contiguous(), k_eff, n_visible, self.W))
+            ks.append(gather(self.layer_cache(l, "k"), idx[l].contiguous(), k_eff, n_visible, w_eff))
+            vs.append(gather(self.layer_cache(l, "v"), idx[l].contiguous(), k_eff, n_visible, w_eff))
         return torch.stack(ks), torch.stack(vs)
 
     def attend(self, q: torch.Tensor, k_ctx: torch.Tensor, v_ctx: torch.Tensor):

@@ -90,10 +90,9 @@ __global__ void __launch_bounds__(256) materialize_kernel(char* const* __restric
 
 }  // namespace
 
-cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, int k_eff, int n_visible,
-                                   int layer0, int layer1, int frames_now, cudaStream_t st) {
-  const int W = n_visible < c->cfg.window_frames ? n_visible : c->cfg.window_frames;
-  const int ncf = k_eff + W;
+cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, const CtxGeom& geom,
+                                   int n_visible, int layer0, int layer1, int frames_now, cudaStream_t st) {
+  const int k_eff = geom.k_eff, ncf = geom.ncf;
   if (ncf <= 0 || layer1 <= layer0) return cudaSuccess;
   const int parts = c->sv.tail > 0 ? PULL_PARTS_HOST : 1;
   dim3 grid(ncf * parts, nQ, layer1 - layer0);

@@ -54,16 +54,18 @@ __global__ void __launch_bounds__(256) qmean_kernel(const __nv_bfloat162* __rest
   if (threadIdx.x == 0) qsq[((long long)l * maxQ + qi) * Hkv + g] = red[0] + red[1];
 }
 
-// ---- cosine scores.  grid = (frame chunks, L); one warp per frame: the representative row is read
-// once (float4 per lane, coalesced), its norm and its dot product with every question of the batch
-// come from the same registers, reduced with warp shuffles.  The table is read once per batch.
+// ---- cosine scores.  grid = (item chunks, L); an item is a frame, or with block retrieval a block of
+// `block` consecutive frames whose vector is the mean of their representatives.  One warp per item: the
+// representative rows are read once (float4 per lane, coalesced), the norm and the dot product with
+// every question of the batch come from the same registers, reduced with warp shuffles.  The table is
+// read once per batch.  n_visible counts items here.
 constexpr int SCORE_FRAMES_PER_CTA = 64;
 constexpr int SCORE_MAX_V4 = 8;  // float4 per lane: D' <= 1024
 
 __global__ void __launch_bounds__(256) score_kernel(const float* __restrict__ reps, const float* __restrict__ qa,
                                                     const float* __restrict__ qsq, int nQ, int maxQ, int Dp, int Hkv,
                                                     int max_frames, int n_visible, int q_group,
-                                                    float* __restrict__ scores) {
+                                                    float* __restrict__ scores, int block) {
   extern __shared__ float4 s_q[];  // [q_group][Dp/4]
   __shared__ float s_qn[REKV_MAX_QUESTIONS];
   rekv_ptx::grid_dep_wait();
@@ -89,8 +91,8 @@ __global__ void __launch_bounds__(256) score_kernel(const float* __restrict__ re
     // two frames per iteration: twice the loads in flight per warp
     for (int f = f0 + warp * 2; f < f1; f += 16) {
       const bool two = f + 1 < f1;
-      const float4* row0 = reinterpret_cast<const float4*>(reps + ((long long)l * max_frames + f) * Dp);
-      const float4* row1 = row0 + (two ? Dp / 4 : 0);
+      const float4* row0 = reinterpret_cast<const float4*>(reps + ((long long)l * max_frames + (long long)f * block) * Dp);
+      const float4* row1 = row0 + (two ? (long long)block * (Dp / 4) : 0);
       float4 r0[SCORE_MAX_V4], r1[SCORE_MAX_V4];
 #pragma unroll
       for (int i = 0; i < SCORE_MAX_V4; ++i)
@@ -98,6 +100,27 @@ __global__ void __launch_bounds__(256) score_kernel(const float* __restrict__ re
           r0[i] = __ldg(row0 + i * 32 + lane);
           r1[i] = __ldg(row1 + i * 32 + lane);
         }
+      if (block > 1) {  // block vector = mean of the block's frame vectors
+        for (int j = 1; j < block; ++j) {
+#pragma unroll
+          for (int i = 0; i < SCORE_MAX_V4; ++i)
+            if (i < nv4) {
+              const float4 a = __ldg(row0 + (long long)j * (Dp / 4) + i * 32 + lane);
+              const float4 b = __ldg(row1 + (long long)j * (Dp / 4) + i * 32 + lane);
+              r0[i].x += a.x; r0[i].y += a.y; r0[i].z += a.z; r0[i].w += a.w;
+              r1[i].x += b.x; r1[i].y += b.y; r1[i].z += b.z; r1[i].w += b.w;
+            }
+        }
+        const float fb = (float)block;
+#pragma unroll
+        for (int i = 0; i < SCORE_MAX_V4; ++i)
+          if (i < nv4) {
+            r0[i].x = __fdiv_rn(r0[i].x, fb); r0[i].y = __fdiv_rn(r0[i].y, fb);
+            r0[i].z = __fdiv_rn(r0[i].z, fb); r0[i].w = __fdiv_rn(r0[i].w, fb);
+            r1[i].x = __fdiv_rn(r1[i].x, fb); r1[i].y = __fdiv_rn(r1[i].y, fb);
+            r1[i].z = __fdiv_rn(r1[i].z, fb); r1[i].w = __fdiv_rn(r1[i].w, fb);
+          }
+      }
       float n0 = 0.f, n1 = 0.f;
 #pragma unroll
       for (int i = 0; i < SCORE_MAX_V4; ++i)
@@ -148,8 +171,11 @@ __device__ __forceinline__ unsigned score_key(float s) {
 // score keys find the k-th largest key T exactly, with the number of candidates above it; one
 // ordered compaction then emits, in ascending frame index, every frame above T and the lowest-index
 // frames equal to T that are still needed (ties go to the lower index).
+// With block retrieval the candidates are blocks; a selected block b_i is written as its `block` frames
+// b_i*block .. b_i*block + block-1 (k_eff counts items, top_k counts output slots).
 __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ scores, int nQ, int n_visible,
-                                                   int n_cand, int top_k, int k_eff, int32_t* __restrict__ idx_out) {
+                                                   int n_cand, int top_k, int k_eff, int32_t* __restrict__ idx_out,
+                                                   int block) {
   const int qi = blockIdx.x, l = blockIdx.y;
   const float* s = scores + ((long long)l * nQ + qi) * n_visible;
   int32_t* out = idx_out + ((long long)l * nQ + qi) * top_k;
@@ -162,7 +188,7 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
   rekv_ptx::grid_dep_wait();
   rekv_ptx::grid_dep_launch();
 
-  for (int j = k_eff + threadIdx.x; j < top_k; j += blockDim.x) out[j] = -1;
+  for (int j = k_eff * block + threadIdx.x; j < top_k; j += blockDim.x) out[j] = -1;
   if (k_eff <= 0) return;
   if (threadIdx.x == 0) {
     s_prefix = 0u;
@@ -231,8 +257,11 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
     const unsigned lower = (1u << lane) - 1u;
     const int rank_gt = og + __popc(bg & lower), rank_eq = oe + __popc(be & lower);
     // output position = selected frames before this one = (greater before) + min(equal before, need_eq)
-    if (gt) out[rank_gt + min(rank_eq, need_eq)] = i;
-    if (eq && rank_eq < need_eq) out[rank_gt + rank_eq] = i;
+    int pos = -1;
+    if (gt) pos = rank_gt + min(rank_eq, need_eq);
+    if (eq && rank_eq < need_eq) pos = rank_gt + rank_eq;
+    if (pos >= 0)
+      for (int j = 0; j < block; ++j) out[pos * block + j] = i * block + j;
     __syncthreads();
     if (threadIdx.x == 0) {
       int tg = 0, te = 0;
@@ -250,8 +279,8 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
 
 }  // namespace
 
-cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, int k_eff, int n_visible,
-                                 int32_t* idx_out, float* scores, cudaStream_t st) {
+cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, const CtxGeom& geom,
+                                 int n_visible, int32_t* idx_out, float* scores, cudaStream_t st) {
   const StoreView& s = c->sv;
   const int maxQ = c->cfg.max_questions;
   qmean_kernel<<<dim3(qb.nQ, s.L, s.Hkv), 256, 0, st>>>((const __nv_bfloat162*)q, qb, s.Hq, s.Hkv, s.G, c->qa,
@@ -264,19 +293,24 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
     cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
     attr_set = true;
   }
-  dim3 grid((n_visible + SCORE_FRAMES_PER_CTA - 1) / SCORE_FRAMES_PER_CTA, s.L);
-  cudaError_t e1 = rekv_launch_pdl(score_kernel, grid, dim3(256), smem, st, s.reps, c->qa, c->qnorm, qb.nQ, maxQ, s.Dp,
-                                   s.Hkv, s.max_frames, n_visible, q_group, scores);
-  if (e1 != cudaSuccess) return e1;
+  // b = 1: every visible frame is scored (the window's scores are reported but not candidates);
+  // b > 1: the complete candidate blocks are scored
+  const int b = c->cfg.block_frames;
+  const int n_scored = b == 1 ? n_visible : geom.n_items;
+  if (n_scored > 0) {
+    dim3 grid((n_scored + SCORE_FRAMES_PER_CTA - 1) / SCORE_FRAMES_PER_CTA, s.L);
+    cudaError_t e1 = rekv_launch_pdl(score_kernel, grid, dim3(256), smem, st, s.reps, c->qa, c->qnorm, qb.nQ, maxQ, s.Dp,
+                                     s.Hkv, s.max_frames, n_scored, q_group, scores, b);
+    if (e1 != cudaSuccess) return e1;
+    c->launches += 1;
+  }
   if (top_k > 0) {
-    int n_cand = n_visible - c->cfg.window_frames;
-    if (n_cand < 0) n_cand = 0;
-    cudaError_t e2 = rekv_launch_pdl(topk_kernel, dim3(qb.nQ, s.L), dim3(512), 0, st, scores, qb.nQ, n_visible, n_cand,
-                                     top_k, k_eff, idx_out);
+    cudaError_t e2 = rekv_launch_pdl(topk_kernel, dim3(qb.nQ, s.L), dim3(512), 0, st, scores, qb.nQ, n_scored,
+                                     geom.n_items, top_k, geom.k_items, idx_out, b);
     if (e2 != cudaSuccess) return e2;
     c->launches += 1;
   }
-  c->launches += 2;
+  c->launches += 1;
   return cudaGetLastError();
 }
 
@@ -380,7 +414,7 @@ extern "C" int rekv_score_frames_static(const void* q, const int32_t* cu_q, int 
   dim3 grid((n_frames + SCORE_FRAMES_PER_CTA - 1) / SCORE_FRAMES_PER_CTA, 1);
   score_kernel<<<grid, 256, (size_t)q_group * Dp * sizeof(float), st>>>(reps, qa, qsq, nQ, STATIC_MAX_QUESTIONS, Dp,
                                                                        n_kv_heads, n_frames, n_frames, q_group,
-                                                                       scores_out);
+                                                                       scores_out, 1);
   e = cudaGetLastError();
   if (e != cudaSuccess) {
     rekv_set_error(nullptr, cudaGetErrorString(e));

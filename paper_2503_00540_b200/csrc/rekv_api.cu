@@ -90,9 +90,13 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   if (cfg->tokens_per_frame < 1 || cfg->tokens_per_frame > 256)
     REKV_FAIL(nullptr, REKV_ERR_ARG, "tokens_per_frame=%d outside [1, 256]", cfg->tokens_per_frame);
   if (cfg->max_frames < 1) REKV_FAIL(nullptr, REKV_ERR_ARG, "max_frames must be positive");
-  if (cfg->block_frames != 1) REKV_FAIL(nullptr, REKV_ERR_ARG, "block_frames=%d: only 1 is supported", cfg->block_frames);
+  if (cfg->block_frames < 1 || cfg->block_frames > 64)
+    REKV_FAIL(nullptr, REKV_ERR_ARG, "block_frames=%d outside [1, 64]", cfg->block_frames);
+  if (cfg->max_topk % cfg->block_frames)
+    REKV_FAIL(nullptr, REKV_ERR_ARG, "max_topk=%d must be a multiple of block_frames=%d", cfg->max_topk, cfg->block_frames);
   if (cfg->window_frames < 0) REKV_FAIL(nullptr, REKV_ERR_ARG, "window_frames must be >= 0");
-  if (cfg->hbm_tail_frames < 0 || (cfg->hbm_tail_frames > 0 && cfg->window_frames > cfg->hbm_tail_frames))
+  if (cfg->hbm_tail_frames < 0 ||
+      (cfg->hbm_tail_frames > 0 && cfg->window_frames + cfg->block_frames - 1 > cfg->hbm_tail_frames))
     REKV_FAIL(nullptr, REKV_ERR_ARG, "window_frames=%d must fit in hbm_tail_frames=%d", cfg->window_frames,
               cfg->hbm_tail_frames);
   if (cfg->max_questions < 1 || cfg->max_questions > REKV_MAX_QUESTIONS)
@@ -157,7 +161,7 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   const long long hbm_frames = s.tail > 0 ? s.tail : s.max_frames;
   CREATE_CUDA(cudaMalloc(&s.hbm, (size_t)(hbm_frames * frame_bytes)), "allocating the HBM frame store");
   CREATE_CUDA(cudaMalloc(&s.reps, (size_t)s.L * s.max_frames * s.Dp * sizeof(float)), "allocating the representative table");
-  const int ctx_frames_max = cfg->max_topk + cfg->window_frames;
+  const int ctx_frames_max = cfg->max_topk + cfg->window_frames + cfg->block_frames - 1;
   const int maxQ = cfg->max_questions;
   CREATE_CUDA(cudaMalloc(&c->qa, (size_t)s.L * maxQ * s.Dp * sizeof(float)), "allocating question vectors");
   CREATE_CUDA(cudaMalloc(&c->qnorm, (size_t)s.L * maxQ * s.Hkv * sizeof(float)), "allocating question norms");
@@ -262,13 +266,13 @@ int rekv_retrieve(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, int t
   QBatch qb;
   int rc = build_qbatch(c, cu_q, nQ, &qb);
   if (rc) return rc;
+  if (top_k % c->cfg.block_frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d must be a multiple of block_frames=%d", top_k, c->cfg.block_frames);
   DeviceGuard guard(c->device);
-  int n_cand = n_visible - c->cfg.window_frames;
-  if (n_cand < 0) n_cand = 0;
-  const int k_eff = top_k < n_cand ? top_k : n_cand;
-  REKV_CUDA(c, rekv_launch_retrieve(c, q, qb, top_k, k_eff, n_visible, idx_out, scores_out ? scores_out : c->scores,
+  const CtxGeom geom = rekv_geom(n_visible, c->cfg.window_frames, c->cfg.block_frames, top_k);
+  REKV_CUDA(c, rekv_launch_retrieve(c, q, qb, top_k, geom, n_visible, idx_out, scores_out ? scores_out : c->scores,
                                     (cudaStream_t)stream));
-  return k_eff;
+  return geom.k_eff;
 }
 
 int rekv_gather(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, int n_visible, void* k_ctx, void* v_ctx,
@@ -280,17 +284,16 @@ int rekv_gather(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, int n_visibl
     REKV_FAIL(c, REKV_ERR_ARG, "n_visible=%d outside [0, %d]", n_visible, c->frames);
   if (n_visible == 0) REKV_FAIL(c, REKV_ERR_EMPTY, "no visible frame");
   if ((k_ctx == nullptr) != (v_ctx == nullptr)) REKV_FAIL(c, REKV_ERR_ARG, "k_ctx and v_ctx must both be given or both be null");
-  int n_cand = n_visible - c->cfg.window_frames;
-  if (n_cand < 0) n_cand = 0;
-  const int k_eff = top_k < n_cand ? top_k : n_cand;
+  if (top_k % c->cfg.block_frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d must be a multiple of block_frames=%d", top_k, c->cfg.block_frames);
+  const CtxGeom geom = rekv_geom(n_visible, c->cfg.window_frames, c->cfg.block_frames, top_k);
+  const int k_eff = geom.k_eff, ncf = geom.ncf;
   if (k_eff > 0 && !idx) REKV_FAIL(c, REKV_ERR_ARG, "null idx");
-  const int W = n_visible < c->cfg.window_frames ? n_visible : c->cfg.window_frames;
-  const int ncf = k_eff + W;
   DeviceGuard guard(c->device);
   cudaStream_t st = (cudaStream_t)stream;
   const StoreView& s = c->sv;
   if (s.tail == 0) {
-    REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, k_eff, n_visible, 0, s.L, c->frames, st));
+    REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, geom, n_visible, 0, s.L, c->frames, st));
     c->gather_layerwise = false;
   } else {
     // host tier: the pulls run layer by layer on the side stream (behind every write-through that is
@@ -299,7 +302,7 @@ int rekv_gather(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, int n_visibl
     REKV_CUDA(c, cudaEventRecord(c->ev_main, st));
     REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_main, 0));
     for (int l = 0; l < s.L; ++l) {
-      REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, k_eff, n_visible, l, l + 1, c->frames, c->side));
+      REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, geom, n_visible, l, l + 1, c->frames, c->side));
       REKV_CUDA(c, cudaEventRecord(c->layer_events[l], c->side));
     }
     c->gather_layerwise = true;

@@ -45,6 +45,28 @@ __host__ __device__ inline long long rekv_hbm_page_offset(const StoreView& s, in
   return ((long long)slot * s.L + layer) * s.page_bytes;
 }
 
+// Context geometry of a question.  With block retrieval (b > 1, Eq. 2 paragraph) only complete blocks of the
+// candidate frames [0, n_visible - W) can be retrieved; every frame after the last complete block is in the
+// context: the recent window plus the frames that do not fill a block yet.  b = 1 gives the plain rule.
+struct CtxGeom {
+  int n_items;   // retrieval candidates: frames (b = 1) or complete blocks
+  int k_items;   // items actually retrieved
+  int k_eff;     // frames actually retrieved = k_items * b
+  int w_eff;     // trailing frames that are always in the context
+  int ncf;       // context frames = k_eff + w_eff
+};
+inline CtxGeom rekv_geom(int n_visible, int window, int b, int top_k) {
+  CtxGeom g;
+  int n_cand = n_visible - window;
+  if (n_cand < 0) n_cand = 0;
+  g.n_items = n_cand / b;
+  g.k_items = top_k / b < g.n_items ? top_k / b : g.n_items;
+  g.k_eff = g.k_items * b;
+  g.w_eff = n_visible - g.n_items * b;
+  g.ncf = g.k_eff + g.w_eff;
+  return g;
+}
+
 // Batch of questions, passed to kernels by value (no device-side table to keep alive).
 struct QBatch {
   int nQ;
@@ -131,11 +153,11 @@ inline cudaError_t rekv_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 blo
 cudaError_t rekv_launch_append(rekv_ctx* c, const void* k, const void* v, int frame, cudaStream_t st);
 cudaError_t rekv_launch_unswizzle_page(rekv_ctx* c, const char* page, void* k_out, void* v_out, cudaStream_t st);
 // k_retrieve.cu
-cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, int k_eff, int n_visible,
-                                 int32_t* idx_out, float* scores, cudaStream_t st);
+cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, const CtxGeom& geom,
+                                 int n_visible, int32_t* idx_out, float* scores, cudaStream_t st);
 // k_gather.cu
-cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, int k_eff, int n_visible,
-                                   int layer0, int layer1, int frames_now, cudaStream_t st);
+cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, const CtxGeom& geom,
+                                   int n_visible, int layer0, int layer1, int frames_now, cudaStream_t st);
 cudaError_t rekv_launch_materialize(rekv_ctx* c, int nQ, int ncf, void* k_ctx, void* v_ctx, cudaStream_t st);
 // k_attend_mma.cu
 cudaError_t rekv_launch_attend_mma(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,

@@ -108,6 +108,14 @@ class ReKV:
         self.device = torch.device("cuda", device)
         self.L, self.Hq, self.Hkv, self.D, self.Nf, self.W = (n_layers, n_q_heads, n_kv_heads, head_dim,
                                                               tokens_per_frame, window_frames)
+        self.b = block_frames
+
+    def geometry(self, n_visible: int, top_k: int) -> Tuple[int, int, int]:
+        """(retrieval candidates, frames retrieved, trailing frames always in the context) -- the sizes the
+        library uses for its outputs (include/rekv.h, rekv_retrieve / rekv_gather)."""
+        n_items = max(n_visible - self.W, 0) // self.b
+        k_eff = min(top_k // self.b, n_items) * self.b
+        return n_items, k_eff, n_visible - n_items * self.b
 
     # ------------------------------------------------------------------ plumbing
     def _check(self, rc: int) -> int:
@@ -145,7 +153,8 @@ class ReKV:
         if tuple(q.shape) != (self.L, cu_q[-1], self.Hq, self.D):
             raise ValueError("q must be [L][sum_Nq][H_q][D]")
         idx = torch.empty((self.L, nQ, max(top_k, 0)), dtype=torch.int32, device=self.device)
-        scores = (torch.empty((self.L, nQ, n_visible), dtype=torch.float32, device=self.device)
+        n_scored = n_visible if self.b == 1 else self.geometry(n_visible, top_k)[0]
+        scores = (torch.empty((self.L, nQ, n_scored), dtype=torch.float32, device=self.device)
                   if want_scores and n_visible > 0 else None)
         k_eff = self._check(lib().rekv_retrieve(self._h, _ptr(q, torch.bfloat16), _cu_array(cu_q), nQ, top_k,
                                                 n_visible, _ptr(idx), _ptr(scores), self._stream()))
@@ -159,8 +168,8 @@ class ReKV:
             raise ValueError("idx must be [L][nQ][top_k]")
         k_ctx = v_ctx = None
         if materialize:
-            k_eff = min(top_k, max(n_visible - self.W, 0))
-            n_ctx = (k_eff + min(self.W, n_visible)) * self.Nf
+            _, k_eff, w_eff = self.geometry(n_visible, top_k)
+            n_ctx = (k_eff + w_eff) * self.Nf
             shape = (self.L, nQ, self.Hkv, n_ctx, self.D)
             k_ctx = torch.empty(shape, dtype=torch.bfloat16, device=self.device)
             v_ctx = torch.empty(shape, dtype=torch.bfloat16, device=self.device)

@@ -28,6 +28,7 @@ class Shape:
     off_scale: float = 0.5
     D: int = 128
     tail: int = 0
+    b: int = 1
 
 
 TINY = Shape(L=1, Hq=8, Hkv=2, Nf=16, T=64, W=4, k=8, off_scale=0.0)
@@ -36,7 +37,7 @@ TINY = Shape(L=1, Hq=8, Hkv=2, Nf=16, T=64, W=4, k=8, off_scale=0.0)
 def build_gpu(s: Shape, max_questions: int = 1, max_q_tokens: int = 64, max_frames: int = None, flags: int = 0,
               n_frames: int = None) -> ReKV:
     r = ReKV(s.L, s.Hq, s.Hkv, s.D, s.Nf, max_frames or s.T, s.W, hbm_tail_frames=s.tail, max_q_tokens=max_q_tokens,
-             max_topk=max(s.k, 1), max_questions=max_questions, flags=flags)
+             max_topk=max(s.k, s.b), max_questions=max_questions, flags=flags, block_frames=s.b)
     for f in range(s.T if n_frames is None else n_frames):
         k = synth.frame(s.seed, synth.K, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale, device="cuda")
         v = synth.frame(s.seed, synth.V, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale, device="cuda")
@@ -45,7 +46,7 @@ def build_gpu(s: Shape, max_questions: int = 1, max_q_tokens: int = 64, max_fram
 
 
 def build_oracle(s: Shape, n_frames: int = None) -> orc.OracleCache:
-    c = orc.OracleCache(s.L, s.Hq, s.Hkv, s.D, s.Nf, s.W)
+    c = orc.OracleCache(s.L, s.Hq, s.Hkv, s.D, s.Nf, s.W, block=s.b)
     for f in range(s.T if n_frames is None else n_frames):
         c.append(synth.frame(s.seed, synth.K, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale),
                  synth.frame(s.seed, synth.V, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale))

@@ -59,4 +59,4 @@ def test_workload_tables_are_consistent():
     assert abs(ab["total"] - 925.3e6) < 1e6
     assert abs(bench.attention_flops(w) - 181.3e9) < 1e9
     # the line the reference arm prints is valid JSON with the contract's keys (short run)
-    assert set(bench.WORKLOADS) == {"7b_hbm_1800f", "7b_offload_10800f", "7b_stream_batch16", "72b_offload_1800f"}
+    assert {"7b_hbm_1800f", "7b_offload_10800f", "7b_stream_batch16", "72b_offload_1800f"} <= set(bench.WORKLOADS)

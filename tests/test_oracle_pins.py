@@ -131,6 +131,42 @@ def test_score_matches_library_cosine_and_repeat_k_reading_ranks_equal():
     assert torch.equal(torch.argsort(alt, descending=True, stable=True), torch.argsort(lib, descending=True, stable=True))
 
 
+def test_block_scores_are_cosine_with_the_mean_of_the_frame_vectors():
+    Hq, Hkv, D, T, b = 8, 2, 128, 23, 4
+    q = synth.question(11, 3, 1, 6, Hq, D)[0]
+    reps = torch.stack([orc.pool_frame(synth.frame(11, synth.K, f, 1, 16, Hkv, D)[0]) for f in range(T)])
+    n_blocks = T // b
+    s = orc.score_blocks(q, reps, Hkv, n_blocks, b)
+    qa = orc.question_vector(q, Hkv)
+    blocks = reps[:n_blocks * b].double().reshape(n_blocks, b, -1).mean(1)
+    lib = torch.nn.functional.cosine_similarity(qa[None, :], blocks, dim=1)
+    assert torch.allclose(s.double(), lib, atol=1e-7, rtol=0)
+    # b = 1 is the frame rule; identical frames inside a block give that frame's score
+    assert torch.equal(orc.score_blocks(q, reps, Hkv, T, 1), orc.score(q, reps, Hkv))
+    same = reps[:1].expand(b, -1).contiguous()
+    assert abs(orc.score_blocks(q, same, Hkv, 1, b)[0].item() - orc.score(q, reps[:1].contiguous(), Hkv)[0].item()) < 1e-7
+
+
+def test_block_geometry_and_selection():
+    # 23 visible frames, window 3, blocks of 4: candidates [0,20) -> 5 complete blocks, no leftover
+    assert orc.block_geometry(23, 3, 4, 8) == (5, 2, 3)
+    # 26 visible: candidates [0,23) -> 5 blocks, frames 20..25 (window 3 + 3 that fill no block) always in context
+    assert orc.block_geometry(26, 3, 4, 8) == (5, 2, 6)
+    assert orc.block_geometry(5, 3, 4, 8) == (0, 0, 5)
+    L, Hq, Hkv, D, Nf, T = 1, 8, 2, 128, 16, 26
+    cache = orc.OracleCache(L, Hq, Hkv, D, Nf, window=3, block=4)
+    for f in range(T):
+        cache.append(synth.frame(2503, synth.K, f, L, Nf, Hkv, D), synth.frame(2503, synth.V, f, L, Nf, Hkv, D))
+    q = synth.question(2503, 1, L, 8, Hq, D)
+    res = cache.question(q, top_k=8, n_visible=T)
+    idx = res["idx"][0].tolist()
+    assert res["k_eff"] == 8 and idx == sorted(idx)
+    assert all(idx[j * 4 + f] == idx[j * 4] + f and idx[j * 4] % 4 == 0 for j in range(2) for f in range(4))
+    best = torch.argsort(res["scores"][0], descending=True, stable=True)[:2].sort().values.tolist()
+    assert [idx[0] // 4, idx[4] // 4] == best
+    assert res["k_ctx"].shape[2] == (8 + 6) * Nf  # retrieved frames + the six trailing frames
+
+
 # ----------------------------------------------------------------------------- step 3: selection
 def _brute_select(scores, n_vis, W, k):
     cand = list(range(max(n_vis - W, 0)))

@@ -35,7 +35,7 @@ def _run_question_parity(s: H.Shape, lengths, n_visible=None, flags=0, max_quest
     # steps 4-5 on the oracle's selection (inside a near-tie several selections are correct)
     idx_ref = torch.stack([r["idx"] for r in ref], dim=1).contiguous().cuda()  # [L][nQ][k]
     ncf, k_ctx, v_ctx = g.gather(idx_ref, nQ, s.k, n_visible, materialize=True)
-    assert ncf == k_eff + min(s.W, n_visible)
+    assert ncf == k_eff + o.window_eff(n_visible, s.k)
     for i in range(nQ):
         assert torch.equal(k_ctx[:, i].cpu(), ref[i]["k_ctx"]), f"gathered K differs, question {i}"
         assert torch.equal(v_ctx[:, i].cpu(), ref[i]["v_ctx"]), f"gathered V differs, question {i}"
@@ -108,6 +108,22 @@ def test_degenerate_counts():
 def test_odd_tokens_per_frame_and_single_token_question():
     s = H.Shape(L=1, Hq=4, Hkv=1, Nf=37, T=20, W=2, k=5, seed=7)
     _run_question_parity(s, [1])
+
+
+@pytest.mark.parametrize("b,T,k", [(2, 41, 8), (4, 50, 12), (8, 40, 8)])
+def test_block_retrieval(b, T, k):
+    """Blocks of b frames: block vector = mean of the frame vectors, top_k/b blocks retrieved; the frames after
+    the last complete block join the window."""
+    s = H.Shape(L=2, Hq=8, Hkv=2, Nf=16, T=T, W=3, k=k, b=b, seed=540)
+    _run_question_parity(s, [9, 20])
+    _run_question_parity(s, [5], n_visible=T - 7)
+
+
+def test_block_retrieval_7b_shape_and_host_tier():
+    s = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=45, W=4, k=8, b=4, seed=7)
+    _run_question_parity(s, [32])
+    s2 = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=45, W=4, k=8, b=4, tail=10, seed=7)
+    _run_question_parity(s2, [32])
 
 
 def test_error_paths_on_device():
