@@ -148,6 +148,28 @@ int rekv_gather(rekv_ctx* ctx, const int32_t* idx, int nQ, int top_k, int n_visi
  * Returns 0, or REKV_ERR_STATE without a preceding gather. */
 int rekv_attend(rekv_ctx* ctx, const void* q, const int32_t* cu_q, int nQ, void* out, void* stream);
 
+/* Layer-sequential form of steps 2-5.  A decoder produces layer l+1's queries only from layer l's
+ * output, and the paper retrieves independently in every layer, so a model integrates the path one
+ * layer at a time: this call enqueues retrieve -> gather -> attend of ONE layer on `stream`.
+ *   layer     0 .. n_layers-1
+ *   q         device bf16 [sum_Nq][H_q][D]: that layer's query rows, questions packed back to back
+ *   cu_q, nQ, top_k, n_visible   as in rekv_retrieve
+ *   idx_out   device int32 [nQ][top_k] (nullable): the layer's selection, ascending, -1 past k_eff
+ *   out       device bf16 [sum_Nq][H_q][D]
+ * Same arithmetic, kernels and results as the all-layer calls restricted to that layer.  Nothing is
+ * allocated and the host is not synchronised; on a context whose cache is all in HBM the call may be
+ * captured into a CUDA graph (one graph per layer, replayed while the stored frames, n_visible and the
+ * buffers stay the same); an offloaded context uses the internal side stream and must not be captured.
+ * The context built for the layer stays valid for rekv_attend_layer until the next gather of that layer.
+ * Returns the number of context frames, or a negative error code. */
+int rekv_question_layer(rekv_ctx* ctx, int layer, const void* q, const int32_t* cu_q, int nQ, int top_k, int n_visible,
+                        int32_t* idx_out, void* out, void* stream);
+
+/* Step 5 of one layer over the context that layer's last rekv_question_layer (or rekv_gather) built:
+ * the decode steps that follow a question reuse its retrieved context with new query rows.
+ * q, out: device bf16 [sum_Nq][H_q][D]; nQ must equal the gathered batch.  Returns 0 or an error code. */
+int rekv_attend_layer(rekv_ctx* ctx, int layer, const void* q, const int32_t* cu_q, int nQ, void* out, void* stream);
+
 /* Fills *out with store accounting and the last call's counters. */
 int rekv_stats(rekv_ctx* ctx, rekv_stats_t* out);
 

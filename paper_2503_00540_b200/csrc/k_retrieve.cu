@@ -6,13 +6,13 @@
 namespace {
 
 // ---- question vector: mean over the question's tokens and over the G query heads of each KV group
-// grid = (nQ, L, H_kv); 256 threads = 4 token slices x 64 dim pairs: every load instruction of a warp
+// grid = (nQ, layers, H_kv), layer = layer0 + blockIdx.y; 256 threads = 4 token slices x 64 dim pairs: every load instruction of a warp
 // covers 128 contiguous bytes of one (token, head) row.  Writes the group's 128 dims of the question
 // vector and its partial sum of squares (the score kernel adds the H_kv partials).
 __global__ void __launch_bounds__(256) qmean_kernel(const __nv_bfloat162* __restrict__ q, QBatch qb, int Hq, int Hkv,
                                                     int G, float* __restrict__ qa, float* __restrict__ qsq,
-                                                    int maxQ) {
-  const int qi = blockIdx.x, l = blockIdx.y, g = blockIdx.z;
+                                                    int maxQ, int layer0) {
+  const int qi = blockIdx.x, l = layer0 + blockIdx.y, g = blockIdx.z;
   const int Dp = Hkv * 128;
   const int n0 = qb.cu[qi], n1 = qb.cu[qi + 1];
   const int d2 = threadIdx.x & 63, slice = threadIdx.x >> 6;
@@ -65,12 +65,12 @@ constexpr int SCORE_MAX_V4 = 8;  // float4 per lane: D' <= 1024
 __global__ void __launch_bounds__(256) score_kernel(const float* __restrict__ reps, const float* __restrict__ qa,
                                                     const float* __restrict__ qsq, int nQ, int maxQ, int Dp, int Hkv,
                                                     int max_frames, int n_visible, int q_group,
-                                                    float* __restrict__ scores, int block) {
+                                                    float* __restrict__ scores, int block, int layer0) {
   extern __shared__ float4 s_q[];  // [q_group][Dp/4]
   __shared__ float s_qn[REKV_MAX_QUESTIONS];
   rekv_ptx::grid_dep_wait();
   rekv_ptx::grid_dep_launch();
-  const int l = blockIdx.y;
+  const int l = layer0 + blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int f0 = blockIdx.x * SCORE_FRAMES_PER_CTA;
   const int f1 = min(f0 + SCORE_FRAMES_PER_CTA, n_visible);
@@ -175,8 +175,8 @@ __device__ __forceinline__ unsigned score_key(float s) {
 // b_i*block .. b_i*block + block-1 (k_eff counts items, top_k counts output slots).
 __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ scores, int nQ, int n_visible,
                                                    int n_cand, int top_k, int k_eff, int32_t* __restrict__ idx_out,
-                                                   int block) {
-  const int qi = blockIdx.x, l = blockIdx.y;
+                                                   int block, int layer0) {
+  const int qi = blockIdx.x, l = layer0 + blockIdx.y;
   const float* s = scores + ((long long)l * nQ + qi) * n_visible;
   int32_t* out = idx_out + ((long long)l * nQ + qi) * top_k;
   __shared__ unsigned hist[256];
@@ -280,11 +280,14 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
 }  // namespace
 
 cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, const CtxGeom& geom,
-                                 int n_visible, int32_t* idx_out, float* scores, cudaStream_t st) {
+                                 int n_visible, int layer0, int layer1, int32_t* idx_out, float* scores, cudaStream_t st) {
+  // q, idx_out and scores are indexed with the absolute layer by the kernels; a caller that holds one
+  // layer's rows only passes pointers moved back by layer0 layers
   const StoreView& s = c->sv;
   const int maxQ = c->cfg.max_questions;
-  qmean_kernel<<<dim3(qb.nQ, s.L, s.Hkv), 256, 0, st>>>((const __nv_bfloat162*)q, qb, s.Hq, s.Hkv, s.G, c->qa,
-                                                       c->qnorm, maxQ);
+  const int nl = layer1 - layer0;
+  qmean_kernel<<<dim3(qb.nQ, nl, s.Hkv), 256, 0, st>>>((const __nv_bfloat162*)q, qb, s.Hq, s.Hkv, s.G, c->qa,
+                                                      c->qnorm, maxQ, layer0);
   int q_group = (int)((96 * 1024) / (s.Dp * sizeof(float)));
   if (q_group > qb.nQ) q_group = qb.nQ;
   size_t smem = (size_t)q_group * s.Dp * sizeof(float);
@@ -298,15 +301,15 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
   const int b = c->cfg.block_frames;
   const int n_scored = b == 1 ? n_visible : geom.n_items;
   if (n_scored > 0) {
-    dim3 grid((n_scored + SCORE_FRAMES_PER_CTA - 1) / SCORE_FRAMES_PER_CTA, s.L);
+    dim3 grid((n_scored + SCORE_FRAMES_PER_CTA - 1) / SCORE_FRAMES_PER_CTA, nl);
     cudaError_t e1 = rekv_launch_pdl(score_kernel, grid, dim3(256), smem, st, s.reps, c->qa, c->qnorm, qb.nQ, maxQ, s.Dp,
-                                     s.Hkv, s.max_frames, n_scored, q_group, scores, b);
+                                     s.Hkv, s.max_frames, n_scored, q_group, scores, b, layer0);
     if (e1 != cudaSuccess) return e1;
     c->launches += 1;
   }
   if (top_k > 0) {
-    cudaError_t e2 = rekv_launch_pdl(topk_kernel, dim3(qb.nQ, s.L), dim3(512), 0, st, scores, qb.nQ, n_scored,
-                                     geom.n_items, top_k, geom.k_items, idx_out, b);
+    cudaError_t e2 = rekv_launch_pdl(topk_kernel, dim3(qb.nQ, nl), dim3(512), 0, st, scores, qb.nQ, n_scored,
+                                     geom.n_items, top_k, geom.k_items, idx_out, b, layer0);
     if (e2 != cudaSuccess) return e2;
     c->launches += 1;
   }
@@ -402,7 +405,7 @@ extern "C" int rekv_score_frames_static(const void* q, const int32_t* cu_q, int 
   const int Dp = n_kv_heads * REKV_HEAD_DIM, G = n_q_heads / n_kv_heads;
   cudaStream_t st = (cudaStream_t)stream;
   qmean_kernel<<<dim3(nQ, 1, n_kv_heads), 256, 0, st>>>((const __nv_bfloat162*)q, qb, n_q_heads, n_kv_heads, G, qa, qsq,
-                                                         STATIC_MAX_QUESTIONS);
+                                                         STATIC_MAX_QUESTIONS, 0);
   // the question vectors of one call fit in 64 KB of dynamic shared memory only in groups
   int q_group = (int)((96 * 1024) / (Dp * sizeof(float)));
   if (q_group > nQ) q_group = nQ;
@@ -414,7 +417,7 @@ extern "C" int rekv_score_frames_static(const void* q, const int32_t* cu_q, int 
   dim3 grid((n_frames + SCORE_FRAMES_PER_CTA - 1) / SCORE_FRAMES_PER_CTA, 1);
   score_kernel<<<grid, 256, (size_t)q_group * Dp * sizeof(float), st>>>(reps, qa, qsq, nQ, STATIC_MAX_QUESTIONS, Dp,
                                                                        n_kv_heads, n_frames, n_frames, q_group,
-                                                                       scores_out, 1);
+                                                                       scores_out, 1, 0);
   e = cudaGetLastError();
   if (e != cudaSuccess) {
     rekv_set_error(nullptr, cudaGetErrorString(e));

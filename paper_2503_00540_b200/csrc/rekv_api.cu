@@ -62,6 +62,7 @@ void free_ctx(rekv_ctx* c) {
   cudaFree(c->part_o);
   cudaFree(c->part_ml);
   cudaFree(c->status);
+  cudaFree(c->idx_own);
   cudaFree(c->link_bytes);
   for (char* a : c->host_arenas) cudaFreeHost(a);
   for (cudaEvent_t e : c->slot_events) cudaEventDestroy(e);
@@ -74,6 +75,31 @@ void free_ctx(rekv_ctx* c) {
   delete c;
 }
 
+// The kernels index q, out and idx with the absolute layer; a per-layer buffer is passed moved back
+// by `layer` layers (only the addresses inside the caller's buffer are ever formed by the kernels).
+template <typename T>
+T* layer_view(T* base, int layer, long long bytes_per_layer) {
+  return reinterpret_cast<T*>(reinterpret_cast<intptr_t>(base) - (intptr_t)layer * bytes_per_layer);
+}
+
+int attend_one_layer(rekv_ctx* c, int layer, const void* q, const QBatch& qb, void* out, cudaStream_t st) {
+  const StoreView& s = c->sv;
+  const long long row_bytes = (long long)s.Hq * REKV_HEAD_DIM * 2;
+  if (c->g_ncf == 0) {
+    REKV_CUDA(c, cudaMemsetAsync(out, 0, (size_t)(qb.sumNq * row_bytes), st));
+    return REKV_OK;
+  }
+  const bool legacy = (c->cfg.flags & REKV_FLAG_ATTEND_LEGACY_MMA) != 0;
+  auto launch = legacy ? rekv_launch_attend_mma : rekv_launch_attend_tc5;
+  REKV_CUDA(c, launch(c, layer_view(q, layer, qb.sumNq * row_bytes), qb, c->g_ncf, layer, layer + 1,
+                      layer_view(out, layer, qb.sumNq * row_bytes), st, false));
+  if (s.tail > 0) {
+    // later appends (ring slots) and gathers (staging) on the side stream must not overtake this read
+    REKV_CUDA(c, cudaEventRecord(c->ev_side, st));
+    REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_side, 0));
+  }
+  return REKV_OK;
+}
 }  // namespace
 
 extern "C" {
@@ -130,6 +156,7 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   c->ctx_tbl = nullptr;
   c->status = nullptr;
   c->link_bytes = nullptr;
+  c->idx_own = nullptr;
 
   StoreView& s = c->sv;
   s.L = cfg->n_layers;
@@ -172,6 +199,8 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   CREATE_CUDA(cudaMalloc(&c->part_ml, c->part_units * 128 * 2 * sizeof(float)), "allocating split-KV partials");
   CREATE_CUDA(cudaMalloc(&c->status, sizeof(int)), "allocating the status word");
   CREATE_CUDA(cudaMemset(c->status, 0, sizeof(int)), "clearing the status word");
+  CREATE_CUDA(cudaMalloc(&c->idx_own, (size_t)s.L * maxQ * (c->cfg.max_topk > 0 ? c->cfg.max_topk : 1) * sizeof(int32_t)),
+              "allocating the selection buffer");
   CREATE_CUDA(cudaMalloc(&c->link_bytes, sizeof(unsigned long long)), "allocating counters");
   CREATE_CUDA(cudaMemset(c->link_bytes, 0, sizeof(unsigned long long)), "clearing counters");
   CREATE_CUDA(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking), "creating the side stream");
@@ -270,7 +299,7 @@ int rekv_retrieve(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, int t
     REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d must be a multiple of block_frames=%d", top_k, c->cfg.block_frames);
   DeviceGuard guard(c->device);
   const CtxGeom geom = rekv_geom(n_visible, c->cfg.window_frames, c->cfg.block_frames, top_k);
-  REKV_CUDA(c, rekv_launch_retrieve(c, q, qb, top_k, geom, n_visible, idx_out, scores_out ? scores_out : c->scores,
+  REKV_CUDA(c, rekv_launch_retrieve(c, q, qb, top_k, geom, n_visible, 0, c->sv.L, idx_out, scores_out ? scores_out : c->scores,
                                     (cudaStream_t)stream));
   return geom.k_eff;
 }
@@ -312,6 +341,7 @@ int rekv_gather(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, int n_visibl
   c->g_ncf = ncf;
   c->g_keff = k_eff;
   c->g_nvis = n_visible;
+  c->g_topk = top_k;
   if (k_ctx) {
     if (c->gather_layerwise) REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[s.L - 1], 0));
     REKV_CUDA(c, rekv_launch_materialize(c, nQ, ncf, k_ctx, v_ctx, st));
@@ -348,6 +378,64 @@ int rekv_attend(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, void* o
     REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_side, 0));
   }
   return REKV_OK;
+}
+
+int rekv_question_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu_q, int nQ, int top_k, int n_visible,
+                        int32_t* idx_out, void* out, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (!q || !out) REKV_FAIL(c, REKV_ERR_ARG, "null q or out");
+  if (layer < 0 || layer >= c->sv.L) REKV_FAIL(c, REKV_ERR_ARG, "layer=%d outside [0, %d)", layer, c->sv.L);
+  if (top_k < 0 || top_k > c->cfg.max_topk) REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d outside [0, %d]", top_k, c->cfg.max_topk);
+  if (n_visible < 0 || n_visible > c->frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "n_visible=%d outside [0, %d]", n_visible, c->frames);
+  if (n_visible == 0) REKV_FAIL(c, REKV_ERR_EMPTY, "no visible frame");
+  if (top_k % c->cfg.block_frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d must be a multiple of block_frames=%d", top_k, c->cfg.block_frames);
+  QBatch qb;
+  int rc = build_qbatch(c, cu_q, nQ, &qb);
+  if (rc) return rc;
+  DeviceGuard guard(c->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const StoreView& s = c->sv;
+  const CtxGeom geom = rekv_geom(n_visible, c->cfg.window_frames, c->cfg.block_frames, top_k);
+  const long long row_bytes = (long long)s.Hq * REKV_HEAD_DIM * 2;
+  // the selection goes to the caller's buffer if there is one, else to the context's own
+  int32_t* idx = idx_out ? layer_view(idx_out, layer, (long long)nQ * top_k * 4) : c->idx_own;
+  REKV_CUDA(c, rekv_launch_retrieve(c, layer_view(q, layer, qb.sumNq * row_bytes), qb, top_k, geom, n_visible, layer,
+                                    layer + 1, idx, c->scores, st));
+  if (s.tail == 0) {
+    REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, geom, n_visible, layer, layer + 1, c->frames, st));
+  } else {
+    REKV_CUDA(c, cudaEventRecord(c->ev_main, st));
+    REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_main, 0));
+    REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, geom, n_visible, layer, layer + 1, c->frames, c->side));
+    REKV_CUDA(c, cudaEventRecord(c->layer_events[layer], c->side));
+    REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[layer], 0));
+  }
+  c->gathered = true;
+  c->gather_layerwise = s.tail > 0;
+  c->g_nQ = nQ;
+  c->g_ncf = geom.ncf;
+  c->g_keff = geom.k_eff;
+  c->g_nvis = n_visible;
+  c->g_topk = top_k;
+  rc = attend_one_layer(c, layer, q, qb, out, st);
+  return rc ? rc : geom.ncf;
+}
+
+int rekv_attend_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu_q, int nQ, void* out, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (!q || !out) REKV_FAIL(c, REKV_ERR_ARG, "null q or out");
+  if (layer < 0 || layer >= c->sv.L) REKV_FAIL(c, REKV_ERR_ARG, "layer=%d outside [0, %d)", layer, c->sv.L);
+  if (!c->gathered) REKV_FAIL(c, REKV_ERR_STATE, "rekv_attend_layer needs a preceding gather of the layer");
+  if (nQ != c->g_nQ) REKV_FAIL(c, REKV_ERR_STATE, "nQ=%d differs from the gathered batch (%d)", nQ, c->g_nQ);
+  QBatch qb;
+  int rc = build_qbatch(c, cu_q, nQ, &qb);
+  if (rc) return rc;
+  DeviceGuard guard(c->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (c->gather_layerwise) REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[layer], 0));
+  return attend_one_layer(c, layer, q, qb, out, st);
 }
 
 int rekv_stats(rekv_ctx* c, rekv_stats_t* out) {

@@ -105,11 +105,12 @@ struct rekv_ctx {
   size_t part_units;                // capacity in (unit) entries of 128 rows
   int* status;                      // device status word
   unsigned long long* link_bytes;   // device counter: bytes pulled over the host link
+  int32_t* idx_own;                 // [L][max_questions][max_topk]: selections of the layer-sequential calls
 
   // state of the last gather
   bool gathered;
   bool gather_layerwise;            // layer events are pending (offloaded context)
-  int g_nQ, g_ncf, g_keff, g_nvis;
+  int g_nQ, g_ncf, g_keff, g_nvis, g_topk;
 };
 
 #define REKV_FAIL(ctx, code, ...)                         \
@@ -154,7 +155,7 @@ cudaError_t rekv_launch_append(rekv_ctx* c, const void* k, const void* v, int fr
 cudaError_t rekv_launch_unswizzle_page(rekv_ctx* c, const char* page, void* k_out, void* v_out, cudaStream_t st);
 // k_retrieve.cu
 cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, const CtxGeom& geom,
-                                 int n_visible, int32_t* idx_out, float* scores, cudaStream_t st);
+                                 int n_visible, int layer0, int layer1, int32_t* idx_out, float* scores, cudaStream_t st);
 // k_gather.cu
 cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, const CtxGeom& geom,
                                    int n_visible, int layer0, int layer1, int frames_now, cudaStream_t st);

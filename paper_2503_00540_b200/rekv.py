@@ -41,7 +41,7 @@ class rekv_stats_t(ctypes.Structure):
 
 EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", "rekv_gather", "rekv_attend",
            "rekv_stats", "rekv_check_status", "rekv_last_error", "rekv_get_reps", "rekv_get_page",
-           "rekv_launch_count", "rekv_score_frames_static")
+           "rekv_launch_count", "rekv_score_frames_static", "rekv_question_layer", "rekv_attend_layer")
 
 _lib = None
 
@@ -59,6 +59,8 @@ def lib() -> ctypes.CDLL:
         L.rekv_retrieve.argtypes = [vp, vp, ip, i32, i32, i32, vp, vp, vp]
         L.rekv_gather.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
         L.rekv_attend.argtypes = [vp, vp, ip, i32, vp, vp]
+        L.rekv_question_layer.argtypes = [vp, i32, vp, ip, i32, i32, i32, vp, vp, vp]
+        L.rekv_attend_layer.argtypes = [vp, i32, vp, ip, i32, vp, vp]
         L.rekv_stats.argtypes = [vp, ctypes.POINTER(rekv_stats_t)]
         L.rekv_check_status.argtypes = [vp, vp]
         L.rekv_last_error.argtypes = [vp]
@@ -193,6 +195,33 @@ class ReKV:
             idx, _, _ = self.retrieve(q, cu_q, top_k, n_visible)
         self.gather(idx, nQ, top_k, n_visible)
         return self.attend(q, cu_q, out)
+
+    def question_layer(self, layer: int, q: torch.Tensor, cu_q: Sequence[int], top_k: int, n_visible: int,
+                       out: Optional[torch.Tensor] = None, idx: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """retrieve -> gather -> attend of one layer.  q: bf16 [sum_Nq][H_q][D] of that layer -> same shape.
+        idx (optional, int32 [nQ][top_k]) receives the layer's selection."""
+        nQ = len(cu_q) - 1
+        if tuple(q.shape) != (cu_q[-1], self.Hq, self.D):
+            raise ValueError("q must be [sum_Nq][H_q][D]")
+        if idx is not None and tuple(idx.shape) != (nQ, top_k):
+            raise ValueError("idx must be [nQ][top_k]")
+        if out is None:
+            out = torch.empty_like(q)
+        self._check(lib().rekv_question_layer(self._h, layer, _ptr(q, torch.bfloat16), _cu_array(cu_q), nQ, top_k,
+                                              n_visible, _ptr(idx, torch.int32), _ptr(out, torch.bfloat16),
+                                              self._stream()))
+        return out
+
+    def attend_layer(self, layer: int, q: torch.Tensor, cu_q: Sequence[int],
+                     out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Attention of one layer over the context its last question_layer (or gather) built."""
+        if tuple(q.shape) != (cu_q[-1], self.Hq, self.D):
+            raise ValueError("q must be [sum_Nq][H_q][D]")
+        if out is None:
+            out = torch.empty_like(q)
+        self._check(lib().rekv_attend_layer(self._h, layer, _ptr(q, torch.bfloat16), _cu_array(cu_q), len(cu_q) - 1,
+                                            _ptr(out, torch.bfloat16), self._stream()))
+        return out
 
     # ------------------------------------------------------------------ accounting and test helpers
     def stats(self) -> rekv_stats_t:
