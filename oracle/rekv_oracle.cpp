@@ -14,6 +14,10 @@
  *   3. keep the r most similar frames   (Eq. 2 paragraph, "r most relevant")
  *   4. the retrieved K/V, R, are brought together as the context
  *   5. O = Attn(Q, R_k, R_v)            (Eq. 3)
+ *   5'. the whole of Eq. 3: O = Attn(W_Q X, [R_k, W_K X], [R_v, W_V X]) -- the
+ *      question's (and generated tokens') own K/V follow the retrieved context,
+ *      causally; rotary position embedding with the retrieved tokens taken as
+ *      consecutive tokens                 (Eq. 3, "Positional Encoding")
  *
  * Readings where the paper is silent (each also listed in the design notes):
  *   - GQA: the G query heads of one KV group are averaged so that question
@@ -25,6 +29,12 @@
  *     ascending frame order (temporal order).
  *   - Attn = softmax(Q K^T / sqrt(D)) V, no mask (all context precedes the
  *     question), query head h reads KV head floor(h / G).
+ *
+ *   - Eq. 3 in full: the retrieved tokens take positions 0 .. n_ctx-1 in
+ *     context order, the tokens of X continue at n_ctx; a query of X sees all
+ *     of R and the tokens of X up to itself.  Rotary embedding pairs dimension
+ *     i with i + D/2 (angle = position * theta^(-2i/D)); rotated queries and
+ *     keys are rounded to bf16 once, as a bf16 model holds them.
  *
  * Arithmetic: bf16 inputs are widened exactly; every sum is a double; each
  * stored result is rounded once (to float, and for attention also to bf16).
@@ -222,6 +232,79 @@ void oracle_attend(const uint16_t* q, int n_q, int n_q_heads, int n_kv_heads, in
       const double p = logit[j] / z;
       if (probs) probs[row * n_ctx + j] = p;
       for (int d = 0; d < head_dim; ++d) acc[d] += p * bf16_to_double(vh[j * head_dim + d]);
+    }
+    for (int d = 0; d < head_dim; ++d) {
+      const float o = (float)acc[d];
+      out_f32[row * head_dim + d] = o;
+      if (out_bf16) out_bf16[row * head_dim + d] = float_to_bf16_rne(o);
+    }
+  }
+}
+
+/* Rotary position embedding (RoFormer) of one vector of D dims at integer position pos:
+ * pair i = (x[i], x[i + D/2]) is turned by the angle pos * theta^(-2i/D).  Doubles in and out. */
+void oracle_rope(const double* x, int head_dim, long pos, double theta, double* out) {
+  const int half = head_dim / 2;
+  for (int i = 0; i < half; ++i) {
+    const double angle = (double)pos * std::pow(theta, -2.0 * (double)i / (double)head_dim);
+    const double c = std::cos(angle), s = std::sin(angle);
+    out[i] = x[i] * c - x[i + half] * s;
+    out[i + half] = x[i + half] * c + x[i] * s;
+  }
+}
+
+/* Eq. 3 in full.  q: [n_q][n_q_heads][D] (the rows of X being computed); k_ctx, v_ctx:
+ * [n_kv_heads][n_ctx][D] (R, in context order); k_self, v_self: [n_self][n_kv_heads][D], the K/V of X
+ * token-major as the model emits them, n_self >= n_q: query row n is token n_self - n_q + n of X
+ * (n_self == n_q: the question itself; n_q == 1: a decode step after n_self - 1 earlier tokens).
+ * Row n sees every token of R and the tokens 0 .. n_self - n_q + n of X.  rope_theta > 0 applies the
+ * rotary embedding: R at positions 0 .. n_ctx-1, X at n_ctx + its token index; rotated vectors are
+ * rounded to bf16.  rope_theta == 0: no positional term.  Outputs as oracle_attend. */
+void oracle_attend_full(const uint16_t* q, int n_q, int n_q_heads, int n_kv_heads, int head_dim, const uint16_t* k_ctx,
+                        const uint16_t* v_ctx, long n_ctx, const uint16_t* k_self, const uint16_t* v_self, int n_self,
+                        double rope_theta, float* out_f32, uint16_t* out_bf16) {
+  const int G = n_q_heads / n_kv_heads;
+  const double scale = 1.0 / std::sqrt((double)head_dim);
+  const long rows = (long)n_q * n_q_heads;
+  auto load = [&](const uint16_t* src, long pos, std::vector<double>& dst) {
+    std::vector<double> raw(head_dim);
+    for (int d = 0; d < head_dim; ++d) raw[d] = bf16_to_double(src[d]);
+    if (rope_theta > 0.0) {
+      std::vector<double> rot(head_dim);
+      oracle_rope(raw.data(), head_dim, pos, rope_theta, rot.data());
+      for (int d = 0; d < head_dim; ++d) dst[d] = bf16_to_double(float_to_bf16_rne((float)rot[d]));
+    } else {
+      dst = raw;
+    }
+  };
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long row = 0; row < rows; ++row) {
+    const int n = (int)(row / n_q_heads), h = (int)(row % n_q_heads);
+    const int g = h / G;
+    const int x_tok = n_self - n_q + n;        // this row's token index inside X
+    const long n_seen = n_ctx + x_tok + 1;     // all of R, then X up to and including itself
+    std::vector<double> qd(head_dim), kd(head_dim), logit((size_t)n_seen), acc(head_dim, 0.0);
+    load(q + row * head_dim, n_ctx + x_tok, qd);
+    double m = -std::numeric_limits<double>::infinity();
+    for (long j = 0; j < n_seen; ++j) {
+      const uint16_t* kj = j < n_ctx ? k_ctx + ((long)g * n_ctx + j) * head_dim
+                                     : k_self + ((j - n_ctx) * n_kv_heads + g) * head_dim;
+      load(kj, j, kd);
+      double s = 0.0;
+      for (int d = 0; d < head_dim; ++d) s += qd[d] * kd[d];
+      logit[j] = s * scale;
+      m = std::max(m, logit[j]);
+    }
+    double z = 0.0;
+    for (long j = 0; j < n_seen; ++j) {
+      logit[j] = std::exp(logit[j] - m);
+      z += logit[j];
+    }
+    for (long j = 0; j < n_seen; ++j) {
+      const uint16_t* vj = j < n_ctx ? v_ctx + ((long)g * n_ctx + j) * head_dim
+                                     : v_self + ((j - n_ctx) * n_kv_heads + g) * head_dim;
+      const double p = logit[j] / z;
+      for (int d = 0; d < head_dim; ++d) acc[d] += p * bf16_to_double(vj[d]);
     }
     for (int d = 0; d < head_dim; ++d) {
       const float o = (float)acc[d];

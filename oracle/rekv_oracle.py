@@ -34,6 +34,12 @@ _lib.oracle_gather.restype = ctypes.c_int
 _lib.oracle_attend.argtypes = [_u16p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, _u16p, _u16p,
                                ctypes.c_long, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
 _lib.oracle_attend.restype = None
+_lib.oracle_rope.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_long, ctypes.c_double, ctypes.c_void_p]
+_lib.oracle_rope.restype = None
+_lib.oracle_attend_full.argtypes = [_u16p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, _u16p, _u16p,
+                                    ctypes.c_long, _u16p, _u16p, ctypes.c_int, ctypes.c_double, ctypes.c_void_p,
+                                    ctypes.c_void_p]
+_lib.oracle_attend_full.restype = None
 _lib.oracle_kv_cache_bytes.argtypes = [ctypes.c_int, ctypes.c_long, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                        ctypes.c_int]
 _lib.oracle_kv_cache_bytes.restype = ctypes.c_double
@@ -132,6 +138,31 @@ def attend(q: torch.Tensor, k_ctx: torch.Tensor, v_ctx: torch.Tensor, want_probs
     _lib.oracle_attend(q.data_ptr(), n_q, n_qh, n_kv, d, k_ctx.data_ptr(), v_ctx.data_ptr(), n_ctx, out.data_ptr(),
                        out_b.data_ptr(), probs.data_ptr() if want_probs else None)
     return out, out_b, probs
+
+
+def rope(x: torch.Tensor, pos: int, theta: float) -> torch.Tensor:
+    """Rotary embedding of one float64 vector [D] at position pos (pairs i, i + D/2)."""
+    _chk(x, torch.float64)
+    out = torch.empty_like(x)
+    _lib.oracle_rope(x.data_ptr(), x.shape[0], pos, theta, out.data_ptr())
+    return out
+
+
+def attend_full(q: torch.Tensor, k_ctx: torch.Tensor, v_ctx: torch.Tensor, k_self: torch.Tensor, v_self: torch.Tensor,
+                rope_theta: float = 0.0):
+    """The whole of Eq. 3.  q: bf16 [N_q][H_q][D]; k_ctx, v_ctx: bf16 [H_kv][n_ctx][D] (n_ctx may be 0);
+    k_self, v_self: bf16 [N_self][H_kv][D], N_self >= N_q.  -> (out float32, out bf16) [N_q][H_q][D]."""
+    for t in (q, k_ctx, v_ctx, k_self, v_self):
+        _chk(t, torch.bfloat16)
+    n_q, n_qh, d = q.shape
+    n_kv, n_ctx, _ = k_ctx.shape
+    n_self = k_self.shape[0]
+    assert n_self >= n_q and k_self.shape == v_self.shape == (n_self, n_kv, d)
+    out = torch.empty(n_q, n_qh, d, dtype=torch.float32)
+    out_b = torch.empty(n_q, n_qh, d, dtype=torch.bfloat16)
+    _lib.oracle_attend_full(q.data_ptr(), n_q, n_qh, n_kv, d, k_ctx.data_ptr(), v_ctx.data_ptr(), n_ctx,
+                            k_self.data_ptr(), v_self.data_ptr(), n_self, rope_theta, out.data_ptr(), out_b.data_ptr())
+    return out, out_b
 
 
 def kv_cache_bytes(n_layers: int, n_frames: int, tokens_per_frame: int, n_kv_heads: int, head_dim: int,

@@ -328,6 +328,130 @@ def test_attention_is_invariant_to_context_order():
     assert torch.allclose(a, b, atol=1e-6)
 
 
+# ----------------------------------------------------------------------------- Eq. 3 in full: X's own K/V, RoPE
+def _complex_rope(x: np.ndarray, pos: int, theta: float) -> np.ndarray:
+    """RoFormer's definition: (x_i + i x_{i+D/2}) * exp(i * pos * theta^(-2i/D)), an independent statement."""
+    d = x.shape[-1]
+    z = x[..., : d // 2] + 1j * x[..., d // 2:]
+    ang = pos * theta ** (-2.0 * np.arange(d // 2) / d)
+    z = z * np.exp(1j * ang)
+    return np.concatenate([z.real, z.imag], axis=-1)
+
+
+def test_rope_closed_forms():
+    g = torch.Generator().manual_seed(3)
+    x = torch.randn(128, dtype=torch.float64, generator=g)
+    theta = 1e6
+    assert torch.equal(orc.rope(x, 0, theta), x)                                   # position 0 is the identity
+    for pos in (1, 7, 196, 14111):
+        r = orc.rope(x, pos, theta)
+        assert abs(r.norm().item() - x.norm().item()) < 1e-12                      # a rotation keeps the norm
+        np.testing.assert_allclose(r.numpy(), _complex_rope(x.numpy(), pos, theta), rtol=0, atol=1e-9)
+    # rotations compose: R(a) R(b) = R(a + b); and the first pair turns by exactly pos radians
+    np.testing.assert_allclose(orc.rope(orc.rope(x, 5, theta), 11, theta).numpy(), orc.rope(x, 16, theta).numpy(),
+                               atol=1e-12)
+    e0 = torch.zeros(128, dtype=torch.float64)
+    e0[0] = 1.0
+    r = orc.rope(e0, 3, theta)
+    assert abs(r[0].item() - math.cos(3.0)) < 1e-15 and abs(r[64].item() - math.sin(3.0)) < 1e-15
+    # the dot product of a rotated query and key depends on the position difference only
+    y = torch.randn(128, dtype=torch.float64, generator=g)
+    d1 = torch.dot(orc.rope(x, 40, theta), orc.rope(y, 33, theta)).item()
+    d2 = torch.dot(orc.rope(x, 1007, theta), orc.rope(y, 1000, theta)).item()
+    assert abs(d1 - d2) < 1e-9
+
+
+def _sdpa_full(q, k_ctx, v_ctx, k_self, v_self, theta):
+    """torch's scaled_dot_product_attention in fp64 on [R, X] with an explicit mask, GQA by head repetition,
+    rotary embedding by the complex-number form, rotated vectors rounded to bf16."""
+    n_q, hq, d = q.shape
+    hkv, n_ctx, _ = k_ctx.shape
+    n_self = k_self.shape[0]
+    G = hq // hkv
+
+    def rot(x, pos):  # x: bf16 [..., D] at integer positions pos (broadcast on the leading dims)
+        xd = x.double().numpy()
+        if theta <= 0:
+            return torch.from_numpy(xd)
+        out = np.empty_like(xd)
+        for idx in np.ndindex(xd.shape[:-1]):
+            out[idx] = _complex_rope(xd[idx], int(pos[idx]), theta)
+        return torch.from_numpy(out).float().to(torch.bfloat16).double()
+
+    k_all = torch.cat([k_ctx.permute(1, 0, 2), k_self], dim=0)          # [n_ctx + n_self][hkv][d]
+    v_all = torch.cat([v_ctx.permute(1, 0, 2), v_self], dim=0).double()
+    n_all = n_ctx + n_self
+    pos_k = np.broadcast_to(np.arange(n_all)[:, None], (n_all, hkv))
+    pos_q = np.broadcast_to((n_ctx + n_self - n_q + np.arange(n_q))[:, None], (n_q, hq))
+    kr, qr = rot(k_all, pos_k), rot(q, pos_q)
+    kh = kr.permute(1, 0, 2).repeat_interleave(G, dim=0)                # [hq][n_all][d]
+    vh = v_all.permute(1, 0, 2).repeat_interleave(G, dim=0)
+    mask = torch.zeros(n_q, n_all, dtype=torch.bool)
+    for n in range(n_q):
+        mask[n, : n_ctx + n_self - n_q + n + 1] = True
+    o = torch.nn.functional.scaled_dot_product_attention(qr.permute(1, 0, 2), kh, vh, attn_mask=mask)
+    return o.permute(1, 0, 2)
+
+
+def _full_inputs(seed, n_q, n_self, n_ctx, hq=4, hkv=2, d=128):
+    g = torch.Generator().manual_seed(seed)
+    r = lambda *sh: bf16(torch.randn(*sh, generator=g))
+    return r(n_q, hq, d), r(hkv, n_ctx, d), r(hkv, n_ctx, d), r(n_self, hkv, d), r(n_self, hkv, d)
+
+
+@pytest.mark.parametrize("theta", [0.0, 1e6])
+def test_attend_full_matches_masked_sdpa(theta):
+    for seed, (n_q, n_self, n_ctx) in enumerate([(5, 5, 12), (1, 9, 7), (3, 8, 0), (6, 6, 40)]):
+        q, kc, vc, ks, vs = _full_inputs(seed, n_q, n_self, n_ctx)
+        out, out_b = orc.attend_full(q, kc, vc, ks, vs, theta)
+        ref = _sdpa_full(q, kc, vc, ks, vs, theta)
+        np.testing.assert_allclose(out.double().numpy(), ref.numpy(), rtol=0, atol=2e-6)
+        assert torch.equal(out_b, out.to(torch.bfloat16))
+
+
+def test_attend_full_reduces_to_the_special_cases():
+    q, kc, vc, ks, vs = _full_inputs(11, 4, 4, 10)
+    # no retrieved context, no positions: plain causal self-attention; its first row is the first token's value
+    empty = torch.empty(2, 0, 128, dtype=torch.bfloat16)
+    out, _ = orc.attend_full(q, empty, empty, ks, vs, 0.0)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        q.double().permute(1, 0, 2), ks.double().permute(1, 0, 2).repeat_interleave(2, dim=0),
+        vs.double().permute(1, 0, 2).repeat_interleave(2, dim=0), is_causal=True).permute(1, 0, 2)
+    np.testing.assert_allclose(out.double().numpy(), ref.numpy(), atol=2e-6)
+    for h in range(4):
+        assert torch.equal(out[0, h], vs[0, h // 2].float())
+    # the tokens of X that follow a query do not reach it
+    ks2, vs2 = ks.clone(), vs.clone()
+    ks2[3], vs2[3] = bf16(torch.ones(2, 128)), bf16(torch.full((2, 128), 5.0))
+    out2, _ = orc.attend_full(q, kc, vc, ks2, vs2, 1e6)
+    out1, _ = orc.attend_full(q, kc, vc, ks, vs, 1e6)
+    assert torch.equal(out2[:3], out1[:3]) and not torch.equal(out2[3], out1[3])
+    # a decode step (one query, X grown by one token) is the last row of the same computation done at once
+    for theta in (0.0, 1e6):
+        whole, _ = orc.attend_full(q, kc, vc, ks, vs, theta)
+        last, _ = orc.attend_full(q[3:].contiguous(), kc, vc, ks, vs, theta)
+        assert torch.equal(last[0], whole[3])
+    # values all ones -> output all ones, with or without positions
+    ones_c, ones_s = bf16(torch.ones(2, 10, 128)), bf16(torch.ones(4, 2, 128))
+    for theta in (0.0, 1e4):
+        o, _ = orc.attend_full(q, kc, ones_c, ks, ones_s, theta)
+        assert (o - 1).abs().max().item() < 1e-6
+
+
+def test_attend_full_positions_are_relative_and_ordered():
+    """With rotary embedding the retrieved tokens count as consecutive tokens: the result changes when two
+    context tokens swap places (it does not without positions), and a key far away in position that equals
+    the query direction scores as the rotation by the distance says."""
+    q, kc, vc, ks, vs = _full_inputs(5, 2, 2, 6)
+    perm = [1, 0, 2, 3, 4, 5]
+    a0, _ = orc.attend_full(q, kc, vc, ks, vs, 0.0)
+    b0, _ = orc.attend_full(q, kc[:, perm].contiguous(), vc[:, perm].contiguous(), ks, vs, 0.0)
+    np.testing.assert_allclose(a0.numpy(), b0.numpy(), atol=1e-6)
+    a1, _ = orc.attend_full(q, kc, vc, ks, vs, 1e6)
+    b1, _ = orc.attend_full(q, kc[:, perm].contiguous(), vc[:, perm].contiguous(), ks, vs, 1e6)
+    assert (a1 - b1).abs().max().item() > 1e-3
+
+
 # ----------------------------------------------------------------------------- input generator
 def test_synthetic_inputs_have_the_stated_distribution():
     k = synth.frame(2503, synth.K, 0, 2, 196, 4, 128, off_scale=0.0).float()
