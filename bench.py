@@ -36,6 +36,10 @@ WORKLOADS = {
     # decode-shaped question (one token): the HBM-bound end of Eq. 3
     "7b_hbm_decode_1tok": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=1, seed=2503, off_scale=0.5,
                                tail=0, nQ=1, appends_per_step=1),
+    # Eq. 3 in full: the question's own K/V (causal) after the retrieved context, rotary embedding with the
+    # retrieved tokens at consecutive positions (base 1e6, the paper's Qwen2-based models)
+    "7b_hbm_full_eq3_rope": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503,
+                                 off_scale=0.5, tail=0, nQ=1, appends_per_step=1, full=True, rope_theta=1e6),
     "72b_offload_1800f": dict(L=80, Hq=64, Hkv=8, D=128, Nf=196, T=1800, W=8, k=32, Nq=64, seed=2503,
                               off_scale=0.5, tail=32, nQ=1, appends_per_step=1),
 }
@@ -187,6 +191,8 @@ def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    if w.get("full"):
+        raise SystemExit("the CPU-oracle arm times steps 2-5 of the retrieval path; use a workload without full=True")
     Ls = 2
     arm = OracleArm(w, Ls)
     times = []
@@ -263,7 +269,8 @@ def run_cuda(args, w):
     w["Nq_total"] = cu[-1]
 
     g = rekv.ReKV(w["L"], w["Hq"], w["Hkv"], w["D"], w["Nf"], w["T"] + 8, w["W"], hbm_tail_frames=w["tail"],
-                  max_q_tokens=cu[-1], max_topk=w["k"], max_questions=nQ, device=local, flags=rekv.FLAG_TIMING)
+                  max_q_tokens=cu[-1], max_topk=w["k"], max_questions=nQ, device=local, flags=rekv.FLAG_TIMING,
+                  max_self_tokens=cu[-1] if w.get("full") else 0, rope_theta=w.get("rope_theta", 0.0))
     kf = torch.empty((w["L"], w["Nf"], w["Hkv"], w["D"]), dtype=torch.bfloat16, device=dev)
     vf = torch.empty_like(kf)
     for f in range(T0):
@@ -280,6 +287,19 @@ def run_cuda(args, w):
     qs = [torch.cat([synth.question(w["seed"], r * nQ + i, w["L"], n, w["Hq"], w["D"], device=dev)
                      for i, n in enumerate(lengths)], dim=1).contiguous() for r in range(N_ROTATE)]
     out = torch.empty_like(qs[0])
+    if w.get("full"):  # the questions' own K/V (N_s = N_q: the question itself), same lengths as the queries
+        ks_self = torch.cat([synth.frame(w["seed"], synth.K, 1_000_000 + i, w["L"], n, w["Hkv"], w["D"], 0.0, device=dev)
+                             for i, n in enumerate(lengths)], dim=1).contiguous()
+        vs_self = torch.cat([synth.frame(w["seed"], synth.V, 1_000_000 + i, w["L"], n, w["Hkv"], w["D"], 0.0, device=dev)
+                             for i, n in enumerate(lengths)], dim=1).contiguous()
+
+        def ask(qt, n_vis, out):
+            idx, _, _ = g.retrieve(qt, cu, w["k"], n_vis)
+            g.gather(idx, nQ, w["k"], n_vis)
+            return g.attend_full(qt, ks_self, vs_self, cu, cu, out=out)
+    else:
+        def ask(qt, n_vis, out):
+            return g.question(qt, cu, w["k"], n_vis, out=out)
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream(dev)
     state = {"next": 0}
@@ -298,7 +318,7 @@ def run_cuda(args, w):
         nf = appends(new_k, new_v)
         if ev:
             ev[1].record(stream)
-        g.question(qs[i % N_ROTATE], cu, w["k"], nf + 1, out=out)
+        ask(qs[i % N_ROTATE], nf + 1, out)
         if ev:
             ev[2].record(stream)
 
@@ -335,7 +355,7 @@ def run_cuda(args, w):
     # attention-kernel duration (library-internal events on the launching stream) and bytes over the host link
     att_us, link_bytes = [], 0
     for i in range(min(K, 8)):
-        g.question(qs[i % N_ROTATE], cu, w["k"], g.stats().frames, out=out)
+        ask(qs[i % N_ROTATE], g.stats().frames, out)
         torch.cuda.synchronize()
         st = g.stats()
         att_us.append(st.last_attend_kernel_us)
@@ -358,7 +378,7 @@ def run_cuda(args, w):
         if ev:
             ev[0].record(stream)
         dq.copy_(hq[i % N_ROTATE], non_blocking=True)
-        g.question(dq, cu, w["k"], nf + 1, out=out)
+        ask(dq, nf + 1, out)
         hout.copy_(out, non_blocking=True)
         if ev:
             ev[1].record(stream)

@@ -75,6 +75,11 @@ typedef struct {
   int32_t max_questions;     /* upper bound on questions per batch (<= 64) */
   int32_t device;            /* CUDA device ordinal */
   uint32_t flags;
+  int32_t max_self_tokens;   /* rekv_attend_full: upper bound on the summed lengths of the questions' own
+                                K/V (question plus generated tokens) in one batch; 0 = that call is not used
+                                and its workspaces are not allocated */
+  float rope_theta;          /* rekv_attend_full: base of the rotary position embedding (1e6 for the paper's
+                                Qwen2-based models); 0 = no positional term */
 } rekv_config;
 
 typedef struct {
@@ -147,6 +152,26 @@ int rekv_gather(rekv_ctx* ctx, const int32_t* idx, int nQ, int top_k, int n_visi
  * no mask (every context token precedes the question); bf16 operands, fp32 accumulation and softmax.
  * Returns 0, or REKV_ERR_STATE without a preceding gather. */
 int rekv_attend(rekv_ctx* ctx, const void* q, const int32_t* cu_q, int nQ, void* out, void* stream);
+
+/* Eq. 3 in full: O = Attn(W_Q X, [R_k, W_K X], [R_v, W_V X]).  The context of the preceding rekv_gather
+ * is followed by the K/V of X itself -- the question's tokens and the tokens generated so far -- which a
+ * query row sees causally.
+ *   q         device bf16 [L][sum_Nq][H_q][D]: the rows of X being computed
+ *   k_self, v_self   device bf16 [L][sum_Ns][H_kv][D]: K/V of all of X, token-major, questions packed back
+ *             to back (not stored by the library)
+ *   cu_q, cu_self    HOST int32 [nQ+1] prefix sums of N_q and N_s per question, 1 <= N_q <= N_s:
+ *             query row n of a question is token N_s - N_q + n of its X and sees all of R and the tokens
+ *             0 .. N_s - N_q + n of X.  N_s == N_q: the question itself; N_q == 1: one decode step
+ *   out       device bf16 [L][sum_Nq][H_q][D]
+ * With rope_theta > 0 the rotary embedding (pairs i, i + D/2; angle = position * theta^(-2i/D)) is applied
+ * to q and to every key, the retrieved tokens taken as consecutive tokens ("Positional Encoding"
+ * paragraph): context token j (context order: retrieved frames ascending, then the trailing frames) has
+ * position j, token s of X has position n_ctx + s.  q, k_self and the stored keys are given UN-rotated;
+ * rotated vectors are rounded to bf16.  The rotated copies of the context's keys are written to a
+ * workspace first (one extra pass over the context's K).
+ * Needs max_self_tokens > 0 at creation.  Returns 0 or an error code (REKV_ERR_STATE without a gather). */
+int rekv_attend_full(rekv_ctx* ctx, const void* q, const void* k_self, const void* v_self, const int32_t* cu_q,
+                     const int32_t* cu_self, int nQ, void* out, void* stream);
 
 /* Layer-sequential form of steps 2-5.  A decoder produces layer l+1's queries only from layer l's
  * output, and the paper retrieves independently in every layer, so a model integrates the path one

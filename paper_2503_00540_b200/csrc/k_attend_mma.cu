@@ -340,7 +340,8 @@ int choose_splits(long long base, int ncf, size_t cap_units) {
 }  // namespace
 
 cudaError_t rekv_launch_attend_mma(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
-                                   void* out, cudaStream_t st, bool timed) {
+                                   void* out, cudaStream_t st, bool timed, const AttendFullArgs* full) {
+  if (full) return cudaErrorNotSupported;  // Eq. 3 in full runs on the tcgen05 kernel only
   const StoreView& s = c->sv;
   AttParams p;
   p.q = (const __nv_bfloat16*)q;

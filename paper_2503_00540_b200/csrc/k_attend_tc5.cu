@@ -55,6 +55,10 @@ struct TcParams {
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
   char* const* tbl;
+  // Eq. 3 in full (FULL instantiation and the merge kernel only; null otherwise)
+  char* const* tbl_k;      // per context slot: rotated copy of the page's K tiles, or null = K from the page
+  const float* self_o;     // per output row: sum of p*v over the tokens of X the row sees, relative to self_ml[0]
+  const float* self_ml;    // per output row: (max, sum) of that part, log2 domain
   float* part_o;
   float* part_ml;
   int* status;
@@ -108,6 +112,7 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return r;
 }
 
+template <bool FULL>
 __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParams p) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -192,6 +197,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     const UnitInfo ui = decode_unit(p, u);
     const int nchunks = nfr * cpf;
     char* const* pages = p.tbl + ((long long)ui.l * p.qb.nQ + ui.qi) * p.ncf + f0;
+    char* const* pages_k = (FULL && p.tbl_k) ? p.tbl_k + ((long long)ui.l * p.qb.nQ + ui.qi) * p.ncf + f0 : nullptr;
     const bool whole_unit = (nfr == p.ncf);
 
     // ---- Q row tiles -> shared memory in the swizzled K-major operand layout -------------------
@@ -231,6 +237,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
           }
           const uint32_t dst = s_kv + b * tile_bytes;
           const char* src = kt + (long long)kv * 2 * half_bytes;
+          if (FULL && kv == 0 && pages_k) src = pages_k[fi] + (long long)ui.g * 2 * half_bytes;  // rotated K tiles
           if (elect_one()) {
             mbar_expect_tx(bars.full(b), 2u * half_bytes);
             bulk_g2s(dst, src, half_bytes, bars.full(b));
@@ -458,22 +465,47 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
           const bool valid = rr < ui.rows_q;
           const int n = rr / p.G, j = rr - n * p.G;
           if (whole_unit) {
-            const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-            uint4* dst = reinterpret_cast<uint4*>(p.out + ((ui.q_row0 + (valid ? n : 0)) * p.Hq + ui.g * p.G + (valid ? j : 0)) * 128);
+            float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+            const long long out_row = (ui.q_row0 + (valid ? n : 0)) * p.Hq + ui.g * p.G + (valid ? j : 0);
+            uint4* dst = reinterpret_cast<uint4*>(p.out + out_row * 128);
+            // Eq. 3 in full: the part over the tokens of X joins here, O = (O_c w_c + O_x w_x) / (l_c w_c + l_x w_x)
+            float w_x = 0.f;
+            const float4* o_x = nullptr;
+            if (FULL && p.self_o) {
+              const float m_x = p.self_ml[out_row * 2], l_x = p.self_ml[out_row * 2 + 1];
+              const float M = fmaxf(m_used, m_x);
+              const float w_c = ex2(m_used - M);
+              w_x = ex2(m_x - M);
+              const float den = l_sum * w_c + l_x * w_x;
+              inv = den > 0.f ? w_c / den : 0.f;
+              w_x = den > 0.f ? w_x / den : 0.f;
+              o_x = reinterpret_cast<const float4*>(p.self_o + out_row * 128);
+            }
+            const float mul = (FULL && o_x) ? 1.f : inv;  // the merged values below are final already
 #pragma unroll
             for (int pc = 0; pc < 8; ++pc) {
               uint32_t o[16];
               tmem_ld16(t_o + pc * 16, o);
               tmem_wait_ld16(o);
+              if (FULL && o_x) {
+#pragma unroll
+                for (int v4 = 0; v4 < 4; ++v4) {
+                  const float4 x = __ldg(o_x + pc * 4 + v4);
+                  o[4 * v4] = __float_as_uint(__uint_as_float(o[4 * v4]) * inv + x.x * w_x);
+                  o[4 * v4 + 1] = __float_as_uint(__uint_as_float(o[4 * v4 + 1]) * inv + x.y * w_x);
+                  o[4 * v4 + 2] = __float_as_uint(__uint_as_float(o[4 * v4 + 2]) * inv + x.z * w_x);
+                  o[4 * v4 + 3] = __float_as_uint(__uint_as_float(o[4 * v4 + 3]) * inv + x.w * w_x);
+                }
+              }
               uint4 a, b;
-              a.x = pack_bf16(__uint_as_float(o[0]) * inv, __uint_as_float(o[1]) * inv);
-              a.y = pack_bf16(__uint_as_float(o[2]) * inv, __uint_as_float(o[3]) * inv);
-              a.z = pack_bf16(__uint_as_float(o[4]) * inv, __uint_as_float(o[5]) * inv);
-              a.w = pack_bf16(__uint_as_float(o[6]) * inv, __uint_as_float(o[7]) * inv);
-              b.x = pack_bf16(__uint_as_float(o[8]) * inv, __uint_as_float(o[9]) * inv);
-              b.y = pack_bf16(__uint_as_float(o[10]) * inv, __uint_as_float(o[11]) * inv);
-              b.z = pack_bf16(__uint_as_float(o[12]) * inv, __uint_as_float(o[13]) * inv);
-              b.w = pack_bf16(__uint_as_float(o[14]) * inv, __uint_as_float(o[15]) * inv);
+              a.x = pack_bf16(__uint_as_float(o[0]) * mul, __uint_as_float(o[1]) * mul);
+              a.y = pack_bf16(__uint_as_float(o[2]) * mul, __uint_as_float(o[3]) * mul);
+              a.z = pack_bf16(__uint_as_float(o[4]) * mul, __uint_as_float(o[5]) * mul);
+              a.w = pack_bf16(__uint_as_float(o[6]) * mul, __uint_as_float(o[7]) * mul);
+              b.x = pack_bf16(__uint_as_float(o[8]) * mul, __uint_as_float(o[9]) * mul);
+              b.y = pack_bf16(__uint_as_float(o[10]) * mul, __uint_as_float(o[11]) * mul);
+              b.z = pack_bf16(__uint_as_float(o[12]) * mul, __uint_as_float(o[13]) * mul);
+              b.w = pack_bf16(__uint_as_float(o[14]) * mul, __uint_as_float(o[15]) * mul);
               if (valid) {
                 dst[pc * 2] = a;
                 dst[pc * 2 + 1] = b;
@@ -532,10 +564,18 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
     const int r = blockIdx.z * 4 + warp;
     const int rr = ui.m0 + t * 128 + r;
     if (rr >= ui.rows_q) return;
-    float M = -INFINITY;
+    const int n = rr / p.G, j = rr - n * p.G;
+    const long long out_row = (ui.q_row0 + n) * p.Hq + ui.g * p.G + j;
+    float M = p.self_o ? p.self_ml[out_row * 2] : -INFINITY;
     for (long long c = c_first; c <= c_last; ++c) M = fmaxf(M, p.part_ml[(((c + u) * 2 + t) * 128 + r) * 2]);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float den = 0.f;
+    if (p.self_o) {  // Eq. 3 in full: the part over the tokens of X is one more partial
+      const float w = ex2(p.self_ml[out_row * 2] - M);
+      const float4 o = *reinterpret_cast<const float4*>(p.self_o + out_row * 128 + lane * 4);
+      acc = make_float4(w * o.x, w * o.y, w * o.z, w * o.w);
+      den = w * p.self_ml[out_row * 2 + 1];
+    }
     for (long long c = c_first; c <= c_last; ++c) {
       const long long base = ((c + u) * 2 + t) * 128 + r;
       const float m = p.part_ml[base * 2], ls = p.part_ml[base * 2 + 1];
@@ -548,20 +588,22 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
       den += w * ls;
     }
     const float inv = den > 0.f ? 1.f / den : 0.f;
-    const int n = rr / p.G, j = rr - n * p.G;
     uint2 packed;
     packed.x = pack_bf16(acc.x * inv, acc.y * inv);
     packed.y = pack_bf16(acc.z * inv, acc.w * inv);
-    *reinterpret_cast<uint2*>(p.out + ((ui.q_row0 + n) * p.Hq + ui.g * p.G + j) * 128 + lane * 4) = packed;
+    *reinterpret_cast<uint2*>(p.out + out_row * 128 + lane * 4) = packed;
   }
 }
 
 }  // namespace
 
 cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
-                                   void* out, cudaStream_t st, bool timed) {
+                                   void* out, cudaStream_t st, bool timed, const AttendFullArgs* full) {
   const StoreView& s = c->sv;
   TcParams p;
+  p.tbl_k = full ? full->tbl_k : nullptr;
+  p.self_o = full ? full->self_o : nullptr;
+  p.self_ml = full ? full->self_ml : nullptr;
   p.q = (const __nv_bfloat16*)q;
   p.out = (__nv_bfloat16*)out;
   p.tbl = c->ctx_tbl;
@@ -608,12 +650,15 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   if (smem > 227 * 1024) return cudaErrorInvalidValue;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attend_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(attend_tc5_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(attend_tc5_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   if (timed) cudaEventRecord(c->ev_t0, st);
-  cudaError_t e1 = rekv_launch_pdl(attend_tc5_kernel, dim3((unsigned)grid), dim3(TC_THREADS), smem, st, p);
+  cudaError_t e1 = full ? rekv_launch_pdl(attend_tc5_kernel<true>, dim3((unsigned)grid), dim3(TC_THREADS), smem, st, p)
+                        : rekv_launch_pdl(attend_tc5_kernel<false>, dim3((unsigned)grid), dim3(TC_THREADS), smem, st, p);
   if (e1 != cudaSuccess) return e1;
   if (timed) {
     cudaEventRecord(c->ev_t1, st);

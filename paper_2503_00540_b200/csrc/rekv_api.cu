@@ -63,6 +63,12 @@ void free_ctx(rekv_ctx* c) {
   cudaFree(c->part_ml);
   cudaFree(c->status);
   cudaFree(c->idx_own);
+  cudaFree(c->self_o);
+  cudaFree(c->self_ml);
+  cudaFree(c->q_rot);
+  cudaFree(c->rope_tab);
+  cudaFree(c->k_rot);
+  cudaFree(c->tbl_k);
   cudaFree(c->link_bytes);
   for (char* a : c->host_arenas) cudaFreeHost(a);
   for (cudaEvent_t e : c->slot_events) cudaEventDestroy(e);
@@ -92,7 +98,7 @@ int attend_one_layer(rekv_ctx* c, int layer, const void* q, const QBatch& qb, vo
   const bool legacy = (c->cfg.flags & REKV_FLAG_ATTEND_LEGACY_MMA) != 0;
   auto launch = legacy ? rekv_launch_attend_mma : rekv_launch_attend_tc5;
   REKV_CUDA(c, launch(c, layer_view(q, layer, qb.sumNq * row_bytes), qb, c->g_ncf, layer, layer + 1,
-                      layer_view(out, layer, qb.sumNq * row_bytes), st, false));
+                      layer_view(out, layer, qb.sumNq * row_bytes), st, false, nullptr));
   if (s.tail > 0) {
     // later appends (ring slots) and gathers (staging) on the side stream must not overtake this read
     REKV_CUDA(c, cudaEventRecord(c->ev_side, st));
@@ -128,6 +134,8 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   if (cfg->max_questions < 1 || cfg->max_questions > REKV_MAX_QUESTIONS)
     REKV_FAIL(nullptr, REKV_ERR_ARG, "max_questions=%d outside [1, %d]", cfg->max_questions, REKV_MAX_QUESTIONS);
   if (cfg->max_q_tokens < 1 || cfg->max_topk < 0) REKV_FAIL(nullptr, REKV_ERR_ARG, "max_q_tokens / max_topk out of range");
+  if (cfg->max_self_tokens < 0 || !(cfg->rope_theta >= 0.f) || (cfg->rope_theta > 0.f && cfg->rope_theta < 1.f))
+    REKV_FAIL(nullptr, REKV_ERR_ARG, "max_self_tokens must be >= 0 and rope_theta 0 or >= 1");
 
   int n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0) {
@@ -157,6 +165,12 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   c->status = nullptr;
   c->link_bytes = nullptr;
   c->idx_own = nullptr;
+  c->self_o = c->self_ml = nullptr;
+  c->q_rot = nullptr;
+  c->rope_tab = nullptr;
+  c->k_rot = nullptr;
+  c->tbl_k = nullptr;
+  c->rope_positions = 0;
 
   StoreView& s = c->sv;
   s.L = cfg->n_layers;
@@ -201,6 +215,23 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   CREATE_CUDA(cudaMemset(c->status, 0, sizeof(int)), "clearing the status word");
   CREATE_CUDA(cudaMalloc(&c->idx_own, (size_t)s.L * maxQ * (c->cfg.max_topk > 0 ? c->cfg.max_topk : 1) * sizeof(int32_t)),
               "allocating the selection buffer");
+  c->ctx_frames_max = ctx_frames_max;
+  if (c->cfg.max_self_tokens > 0) {  // workspaces of rekv_attend_full
+    const size_t rows = (size_t)s.L * c->cfg.max_q_tokens * s.Hq;
+    CREATE_CUDA(cudaMalloc(&c->self_o, rows * 128 * sizeof(float)), "allocating the self-attention partials");
+    CREATE_CUDA(cudaMalloc(&c->self_ml, rows * 2 * sizeof(float)), "allocating the self-attention partials");
+    if (c->cfg.rope_theta > 0.f) {
+      c->rope_positions = ctx_frames_max * s.Nf + c->cfg.max_self_tokens;
+      CREATE_CUDA(cudaMalloc(&c->q_rot, rows * 128 * sizeof(__nv_bfloat16)), "allocating rotated queries");
+      CREATE_CUDA(cudaMalloc(&c->rope_tab, (size_t)c->rope_positions * 64 * sizeof(float2)), "allocating the rotary table");
+      CREATE_CUDA(cudaMalloc(&c->k_rot, (size_t)s.L * maxQ * ctx_frames_max * (s.page_bytes / 2)),
+                  "allocating rotated key tiles");
+      CREATE_CUDA(cudaMalloc(&c->tbl_k, (size_t)s.L * maxQ * (ctx_frames_max + 1) * sizeof(char*)),
+                  "allocating the rotated-key table");
+      CREATE_CUDA(rekv_launch_rope_table(c, 0), "building the rotary table");
+      CREATE_CUDA(cudaDeviceSynchronize(), "building the rotary table");
+    }
+  }
   CREATE_CUDA(cudaMalloc(&c->link_bytes, sizeof(unsigned long long)), "allocating counters");
   CREATE_CUDA(cudaMemset(c->link_bytes, 0, sizeof(unsigned long long)), "clearing counters");
   CREATE_CUDA(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking), "creating the side stream");
@@ -367,11 +398,11 @@ int rekv_attend(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, void* o
   const bool legacy = (c->cfg.flags & REKV_FLAG_ATTEND_LEGACY_MMA) != 0;
   auto launch = legacy ? rekv_launch_attend_mma : rekv_launch_attend_tc5;
   if (!c->gather_layerwise) {
-    REKV_CUDA(c, launch(c, q, qb, c->g_ncf, 0, s.L, out, st, (c->cfg.flags & REKV_FLAG_TIMING) != 0));
+    REKV_CUDA(c, launch(c, q, qb, c->g_ncf, 0, s.L, out, st, (c->cfg.flags & REKV_FLAG_TIMING) != 0, nullptr));
   } else {
     for (int l = 0; l < s.L; ++l) {
       REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[l], 0));
-      REKV_CUDA(c, launch(c, q, qb, c->g_ncf, l, l + 1, out, st, false));
+      REKV_CUDA(c, launch(c, q, qb, c->g_ncf, l, l + 1, out, st, false, nullptr));
     }
     // later appends (ring slots) and gathers (staging) on the side stream must not overtake this read
     REKV_CUDA(c, cudaEventRecord(c->ev_side, st));
@@ -436,6 +467,52 @@ int rekv_attend_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu_q
   cudaStream_t st = (cudaStream_t)stream;
   if (c->gather_layerwise) REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[layer], 0));
   return attend_one_layer(c, layer, q, qb, out, st);
+}
+
+int rekv_attend_full(rekv_ctx* c, const void* q, const void* k_self, const void* v_self, const int32_t* cu_q,
+                     const int32_t* cu_self, int nQ, void* out, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (!q || !k_self || !v_self || !out) REKV_FAIL(c, REKV_ERR_ARG, "null q, k_self, v_self or out");
+  if (c->cfg.max_self_tokens <= 0) REKV_FAIL(c, REKV_ERR_STATE, "the context was created with max_self_tokens == 0");
+  if (c->cfg.flags & REKV_FLAG_ATTEND_LEGACY_MMA)
+    REKV_FAIL(c, REKV_ERR_STATE, "rekv_attend_full runs on the tcgen05 attention kernel only");
+  if (!c->gathered) REKV_FAIL(c, REKV_ERR_STATE, "rekv_attend_full needs a preceding rekv_gather");
+  if (nQ != c->g_nQ) REKV_FAIL(c, REKV_ERR_STATE, "nQ=%d differs from the gathered batch (%d)", nQ, c->g_nQ);
+  QBatch qb, sb;
+  int rc = build_qbatch(c, cu_q, nQ, &qb);
+  if (rc) return rc;
+  if (!cu_self || cu_self[0] != 0) REKV_FAIL(c, REKV_ERR_ARG, "cu_self must start at 0");
+  sb.nQ = nQ;
+  for (int i = 0; i <= nQ; ++i) sb.cu[i] = cu_self[i];
+  sb.sumNq = cu_self[nQ];
+  for (int i = 0; i < nQ; ++i)
+    if (sb.cu[i + 1] - sb.cu[i] < qb.cu[i + 1] - qb.cu[i])
+      REKV_FAIL(c, REKV_ERR_ARG, "question %d: %d tokens of its own K/V for %d query rows", i, sb.cu[i + 1] - sb.cu[i],
+                qb.cu[i + 1] - qb.cu[i]);
+  if (sb.sumNq > c->cfg.max_self_tokens)
+    REKV_FAIL(c, REKV_ERR_ARG, "%d tokens of own K/V exceed max_self_tokens=%d", sb.sumNq, c->cfg.max_self_tokens);
+  DeviceGuard guard(c->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const StoreView& s = c->sv;
+  // an offloaded context: every layer's pages must have arrived before the keys are rotated
+  if (c->gather_layerwise) REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[s.L - 1], 0));
+  REKV_CUDA(c, rekv_launch_attend_full_prepare(c, q, k_self, v_self, qb, sb, c->g_ncf, st));
+  const bool rope = c->cfg.rope_theta > 0.f;
+  if (c->g_ncf == 0) {
+    REKV_CUDA(c, rekv_launch_self_finalize(c, qb, out, st));
+  } else {
+    AttendFullArgs fa;
+    fa.tbl_k = rope ? c->tbl_k : nullptr;
+    fa.self_o = c->self_o;
+    fa.self_ml = c->self_ml;
+    REKV_CUDA(c, rekv_launch_attend_tc5(c, rope ? (const void*)c->q_rot : q, qb, c->g_ncf, 0, s.L, out, st,
+                                        (c->cfg.flags & REKV_FLAG_TIMING) != 0, &fa));
+  }
+  if (c->gather_layerwise) {
+    REKV_CUDA(c, cudaEventRecord(c->ev_side, st));
+    REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_side, 0));
+  }
+  return REKV_OK;
 }
 
 int rekv_stats(rekv_ctx* c, rekv_stats_t* out) {

@@ -107,6 +107,16 @@ struct rekv_ctx {
   unsigned long long* link_bytes;   // device counter: bytes pulled over the host link
   int32_t* idx_own;                 // [L][max_questions][max_topk]: selections of the layer-sequential calls
 
+  // Eq. 3 in full (allocated when max_self_tokens > 0)
+  float* self_o;                    // [L][max_q_tokens][H_q][128]
+  float* self_ml;                   // [L][max_q_tokens][H_q][2]
+  __nv_bfloat16* q_rot;             // [L][max_q_tokens][H_q][128] rotated queries (rope_theta > 0)
+  float2* rope_tab;                 // [rope_positions][64] (cos, sin)
+  int rope_positions;
+  char* k_rot;                      // [L][max_questions][ctx frames][H_kv] rotated K tiles
+  char** tbl_k;                     // [L][max_questions][ctx frames]
+  int ctx_frames_max;
+
   // state of the last gather
   bool gathered;
   bool gather_layerwise;            // layer events are pending (offloaded context)
@@ -149,6 +159,13 @@ inline cudaError_t rekv_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 blo
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Extra inputs of the attention kernel for Eq. 3 in full.
+struct AttendFullArgs {
+  char* const* tbl_k;    // rotated K tiles per context slot (null without rotary embedding)
+  const float* self_o;   // [L][sum_Nq][H_q][128] partial numerators over the tokens of X
+  const float* self_ml;  // [L][sum_Nq][H_q][2] their (max, sum), log2 domain
+};
+
 // ---- kernel launchers (each returns the cudaError_t of its launches) -----------------------
 // k_append.cu
 cudaError_t rekv_launch_append(rekv_ctx* c, const void* k, const void* v, int frame, cudaStream_t st);
@@ -162,7 +179,12 @@ cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int 
 cudaError_t rekv_launch_materialize(rekv_ctx* c, int nQ, int ncf, void* k_ctx, void* v_ctx, cudaStream_t st);
 // k_attend_mma.cu
 cudaError_t rekv_launch_attend_mma(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
-                                   void* out, cudaStream_t st, bool timed);
+                                   void* out, cudaStream_t st, bool timed, const AttendFullArgs* full = nullptr);
 // k_attend_tc5.cu
 cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
-                                   void* out, cudaStream_t st, bool timed);
+                                   void* out, cudaStream_t st, bool timed, const AttendFullArgs* full = nullptr);
+// k_attend_full.cu: the pieces of Eq. 3 in full around the attention kernel
+cudaError_t rekv_launch_rope_table(rekv_ctx* c, cudaStream_t st);
+cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const void* k_self, const void* v_self,
+                                            const QBatch& qb, const QBatch& sb, int ncf, cudaStream_t st);
+cudaError_t rekv_launch_self_finalize(rekv_ctx* c, const QBatch& qb, void* out, cudaStream_t st);

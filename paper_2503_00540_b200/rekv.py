@@ -29,7 +29,7 @@ class rekv_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "tokens_per_frame", "max_frames", "hbm_tail_frames",
         "window_frames", "block_frames", "max_q_tokens", "max_topk", "max_questions", "device")] + [
-            ("flags", ctypes.c_uint32)]
+            ("flags", ctypes.c_uint32), ("max_self_tokens", ctypes.c_int32), ("rope_theta", ctypes.c_float)]
 
 
 class rekv_stats_t(ctypes.Structure):
@@ -41,7 +41,7 @@ class rekv_stats_t(ctypes.Structure):
 
 EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", "rekv_gather", "rekv_attend",
            "rekv_stats", "rekv_check_status", "rekv_last_error", "rekv_get_reps", "rekv_get_page",
-           "rekv_launch_count", "rekv_score_frames_static", "rekv_question_layer", "rekv_attend_layer")
+           "rekv_launch_count", "rekv_score_frames_static", "rekv_question_layer", "rekv_attend_layer", "rekv_attend_full")
 
 _lib = None
 
@@ -61,6 +61,7 @@ def lib() -> ctypes.CDLL:
         L.rekv_attend.argtypes = [vp, vp, ip, i32, vp, vp]
         L.rekv_question_layer.argtypes = [vp, i32, vp, ip, i32, i32, i32, vp, vp, vp]
         L.rekv_attend_layer.argtypes = [vp, i32, vp, ip, i32, vp, vp]
+        L.rekv_attend_full.argtypes = [vp, vp, vp, vp, ip, ip, i32, vp, vp]
         L.rekv_stats.argtypes = [vp, ctypes.POINTER(rekv_stats_t)]
         L.rekv_check_status.argtypes = [vp, vp]
         L.rekv_last_error.argtypes = [vp]
@@ -99,10 +100,10 @@ class ReKV:
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, tokens_per_frame: int,
                  max_frames: int, window_frames: int, hbm_tail_frames: int = 0, max_q_tokens: int = 64,
                  max_topk: int = 64, max_questions: int = 1, device: int = 0, flags: int = 0,
-                 block_frames: int = 1):
+                 block_frames: int = 1, max_self_tokens: int = 0, rope_theta: float = 0.0):
         self.cfg = rekv_config(n_layers, n_q_heads, n_kv_heads, head_dim, tokens_per_frame, max_frames,
                                hbm_tail_frames, window_frames, block_frames, max_q_tokens, max_topk, max_questions,
-                               device, flags)
+                               device, flags, max_self_tokens, rope_theta)
         self._h = ctypes.c_void_p()
         rc = lib().rekv_create(ctypes.byref(self.cfg), ctypes.byref(self._h))
         if rc != 0:
@@ -195,6 +196,21 @@ class ReKV:
             idx, _, _ = self.retrieve(q, cu_q, top_k, n_visible)
         self.gather(idx, nQ, top_k, n_visible)
         return self.attend(q, cu_q, out)
+
+    def attend_full(self, q: torch.Tensor, k_self: torch.Tensor, v_self: torch.Tensor, cu_q: Sequence[int],
+                    cu_self: Sequence[int], out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Eq. 3 in full over the gathered context followed by the questions' own K/V (causal).
+        q: bf16 [L][sum_Nq][H_q][D]; k_self, v_self: bf16 [L][sum_Ns][H_kv][D] -> bf16 like q."""
+        if tuple(q.shape) != (self.L, cu_q[-1], self.Hq, self.D):
+            raise ValueError("q must be [L][sum_Nq][H_q][D]")
+        if tuple(k_self.shape) != (self.L, cu_self[-1], self.Hkv, self.D) or k_self.shape != v_self.shape:
+            raise ValueError("k_self and v_self must be [L][sum_Ns][H_kv][D]")
+        if out is None:
+            out = torch.empty_like(q)
+        self._check(lib().rekv_attend_full(self._h, _ptr(q, torch.bfloat16), _ptr(k_self, torch.bfloat16),
+                                           _ptr(v_self, torch.bfloat16), _cu_array(cu_q), _cu_array(cu_self),
+                                           len(cu_q) - 1, _ptr(out, torch.bfloat16), self._stream()))
+        return out
 
     def question_layer(self, layer: int, q: torch.Tensor, cu_q: Sequence[int], top_k: int, n_visible: int,
                        out: Optional[torch.Tensor] = None, idx: Optional[torch.Tensor] = None) -> torch.Tensor:

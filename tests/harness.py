@@ -35,9 +35,9 @@ TINY = Shape(L=1, Hq=8, Hkv=2, Nf=16, T=64, W=4, k=8, off_scale=0.0)
 
 
 def build_gpu(s: Shape, max_questions: int = 1, max_q_tokens: int = 64, max_frames: int = None, flags: int = 0,
-              n_frames: int = None) -> ReKV:
+              n_frames: int = None, **extra) -> ReKV:
     r = ReKV(s.L, s.Hq, s.Hkv, s.D, s.Nf, max_frames or s.T, s.W, hbm_tail_frames=s.tail, max_q_tokens=max_q_tokens,
-             max_topk=max(s.k, s.b), max_questions=max_questions, flags=flags, block_frames=s.b)
+             max_topk=max(s.k, s.b), max_questions=max_questions, flags=flags, block_frames=s.b, **extra)
     for f in range(s.T if n_frames is None else n_frames):
         k = synth.frame(s.seed, synth.K, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale, device="cuda")
         v = synth.frame(s.seed, synth.V, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale, device="cuda")
@@ -51,6 +51,18 @@ def build_oracle(s: Shape, n_frames: int = None) -> orc.OracleCache:
         c.append(synth.frame(s.seed, synth.K, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale),
                  synth.frame(s.seed, synth.V, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale))
     return c
+
+
+def self_kv(s: Shape, lengths: List[int], device="cpu", first_id: int = 0):
+    """Seeded K/V of the questions' own tokens, packed [L][sum][H_kv][D], and their prefix sums."""
+    ks = [synth.frame(s.seed, synth.K, 1_000_000 + first_id + i, s.L, n, s.Hkv, s.D, 0.0, device=device)
+          for i, n in enumerate(lengths)]
+    vs = [synth.frame(s.seed, synth.V, 1_000_000 + first_id + i, s.L, n, s.Hkv, s.D, 0.0, device=device)
+          for i, n in enumerate(lengths)]
+    cu = [0]
+    for n in lengths:
+        cu.append(cu[-1] + n)
+    return torch.cat(ks, dim=1).contiguous(), torch.cat(vs, dim=1).contiguous(), cu
 
 
 def questions(s: Shape, lengths: List[int], device="cpu", first_id: int = 0):

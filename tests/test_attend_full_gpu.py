@@ -1,0 +1,133 @@
+"""Eq. 3 in full on the GPU (the questions' own K/V after the retrieved context, causal; rotary embedding with
+the retrieved tokens at consecutive positions) against the CPU oracle, through the C ABI."""
+import pytest
+import torch
+
+from oracle import rekv_oracle as orc
+from paper_2503_00540_b200 import rekv
+from tests import harness as H
+
+pytestmark = pytest.mark.gpu
+
+THETAS = [pytest.param(0.0, id="no_rope"), pytest.param(1e6, id="rope_1e6")]
+
+
+def _run(s: H.Shape, nq_lengths, ns_lengths, theta, n_visible=None, top_k=None):
+    n_visible = s.T if n_visible is None else n_visible
+    top_k = s.k if top_k is None else top_k
+    nQ = len(nq_lengths)
+    g = H.build_gpu(s, max_questions=nQ, max_q_tokens=sum(nq_lengths), max_self_tokens=sum(ns_lengths),
+                    rope_theta=theta)
+    o = H.build_oracle(s)
+    q, cu = H.questions(s, nq_lengths, device="cuda")
+    ks, vs, cus = H.self_kv(s, ns_lengths, device="cuda")
+    q_cpu, ks_cpu, vs_cpu = q.cpu(), ks.cpu(), vs.cpu()
+    # the context is the oracle's selection (inside a near-tie several selections are correct)
+    refs = [o.question(q_cpu[:, cu[i]:cu[i + 1]].contiguous(), top_k, n_visible) for i in range(nQ)]
+    idx = torch.stack([r["idx"] for r in refs], dim=1).contiguous().cuda()
+    g.gather(idx, nQ, top_k, n_visible)
+    out = g.attend_full(q, ks, vs, cu, cus)
+    g.check_status()
+    worst = 0.0
+    for i in range(nQ):
+        for l in range(s.L):
+            ref, _ = orc.attend_full(q_cpu[l, cu[i]:cu[i + 1]].contiguous(), refs[i]["k_ctx"][l].contiguous(),
+                                     refs[i]["v_ctx"][l].contiguous(), ks_cpu[l, cus[i]:cus[i + 1]].contiguous(),
+                                     vs_cpu[l, cus[i]:cus[i + 1]].contiguous(), theta)
+            H.assert_attention(out[l:l + 1, cu[i]:cu[i + 1]], ref[None], f"Eq. 3 in full, layer {l} question {i}")
+            worst = max(worst, (out[l, cu[i]:cu[i + 1]].float().cpu() - ref).abs().max().item())
+    # the plain call must differ (the self part matters) unless nothing of X is visible -- never the case
+    plain = g.attend(q, cu)
+    assert not torch.equal(plain, out)
+    g.close()
+    return worst
+
+
+@pytest.mark.parametrize("theta", THETAS)
+def test_tiny(theta):
+    _run(H.TINY, [16], [16], theta)
+
+
+@pytest.mark.parametrize("theta", THETAS)
+def test_7b_shape_question_prefill(theta):
+    """224 query rows per KV head (two row tiles), 196-token frames, units cut by CTA boundaries and whole."""
+    _run(H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=40, W=8, k=12), [32], [32], theta)
+
+
+@pytest.mark.parametrize("theta", THETAS)
+def test_batch_of_mixed_lengths_with_generated_tokens(theta):
+    """N_s > N_q: some tokens of X (earlier question tokens, generated tokens) precede the query rows."""
+    s = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=30, W=4, k=6, seed=540)
+    _run(s, [24, 64, 1, 5], [24, 80, 37, 9], theta)
+
+
+@pytest.mark.parametrize("theta", THETAS)
+def test_decode_step_with_a_long_own_history(theta):
+    """One query row per question, 150 tokens of own K/V (three 64-token tiles in the self kernel)."""
+    s = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=24, W=4, k=8, seed=7)
+    _run(s, [1, 1], [150, 65], theta)
+
+
+@pytest.mark.parametrize("theta", THETAS)
+def test_72b_head_shape(theta):
+    _run(H.Shape(L=1, Hq=64, Hkv=8, Nf=196, T=20, W=4, k=6, seed=7), [48], [48], theta)
+
+
+@pytest.mark.parametrize("theta", THETAS)
+def test_many_units_take_the_whole_unit_path(theta):
+    """Enough (layer, head, question) units that every unit is produced whole by one CTA."""
+    s = H.Shape(L=8, Hq=16, Hkv=8, Nf=64, T=12, W=2, k=4)
+    _run(s, [8] * 12, [8] * 12, theta)
+
+
+@pytest.mark.parametrize("theta", THETAS)
+def test_host_tier(theta):
+    s = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=40, W=4, k=8, tail=8)
+    _run(s, [16, 32], [16, 40], theta)
+
+
+def test_no_context_is_causal_self_attention():
+    """top_k = 0 and W = 0: nothing retrieved, the result is the causal attention of X over itself."""
+    s = H.Shape(L=2, Hq=8, Hkv=2, Nf=16, T=8, W=0, k=0)
+    for theta in (0.0, 1e4):
+        g = H.build_gpu(s, max_questions=2, max_q_tokens=40, max_self_tokens=40, rope_theta=theta)
+        q, cu = H.questions(s, [16, 24], device="cuda")
+        ks, vs, cus = H.self_kv(s, [16, 24], device="cuda")
+        idx = torch.empty((s.L, 2, 0), dtype=torch.int32, device="cuda")
+        assert g.gather(idx, 2, 0, s.T)[0] == 0
+        out = g.attend_full(q, ks, vs, cu, cus)
+        g.check_status()
+        empty = torch.empty(s.Hkv, 0, s.D, dtype=torch.bfloat16)
+        for i in range(2):
+            for l in range(s.L):
+                ref, _ = orc.attend_full(q[l, cu[i]:cu[i + 1]].cpu().contiguous(), empty, empty,
+                                         ks[l, cus[i]:cus[i + 1]].cpu().contiguous(),
+                                         vs[l, cus[i]:cus[i + 1]].cpu().contiguous(), theta)
+                H.assert_attention(out[l:l + 1, cu[i]:cu[i + 1]], ref[None], f"self only, layer {l} question {i}")
+        g.close()
+
+
+def test_argument_and_state_errors():
+    s = H.TINY
+    q, cu = H.questions(s, [16], device="cuda")
+    ks, vs, cus = H.self_kv(s, [16], device="cuda")
+    g0 = H.build_gpu(s, max_questions=1, max_q_tokens=16)  # created without the workspaces
+    idx, _, _ = g0.retrieve(q, cu, s.k, s.T)
+    g0.gather(idx, 1, s.k, s.T)
+    with pytest.raises(rekv.RekvError) as e:
+        g0.attend_full(q, ks, vs, cu, cus)
+    assert e.value.code == rekv.ERR_STATE
+    g0.close()
+    g = H.build_gpu(s, max_questions=1, max_q_tokens=16, max_self_tokens=16)
+    with pytest.raises(rekv.RekvError) as e:  # no gather yet
+        g.attend_full(q, ks, vs, cu, cus)
+    assert e.value.code == rekv.ERR_STATE
+    g.gather(idx, 1, s.k, s.T)
+    with pytest.raises(rekv.RekvError) as e:  # fewer own tokens than query rows
+        g.attend_full(q, ks[:, :8].contiguous(), vs[:, :8].contiguous(), cu, [0, 8])
+    assert e.value.code == rekv.ERR_ARG
+    ks2, vs2, cus2 = H.self_kv(s, [20], device="cuda")
+    with pytest.raises(rekv.RekvError) as e:  # more own tokens than the workspaces hold
+        g.attend_full(q, ks2, vs2, cu, cus2)
+    assert e.value.code == rekv.ERR_ARG
+    g.close()
