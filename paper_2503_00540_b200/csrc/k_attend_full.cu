@@ -25,19 +25,29 @@ __global__ void rope_table_kernel(float2* __restrict__ tab, int n_pos, double th
   tab[pos * 64 + i] = make_float2((float)c, (float)s);
 }
 
-// rotates the 8 pairs (lo[e], hi[e]) held as bf16 in two 16-byte chunks; cs: the pairs' (cos, sin)
-__device__ __forceinline__ void rotate_chunk(uint4& lo, uint4& hi, const float2* __restrict__ cs) {
+// rotates the 8 pairs (lo[e], hi[e]) held as bf16 in two 16-byte chunks; cs: the pairs' (cos, sin),
+// two pairs per float4
+__device__ __forceinline__ void rotate_chunk(uint4& lo, uint4& hi, const float4 (&cs)[4]) {
   uint32_t* l = reinterpret_cast<uint32_t*>(&lo);
   uint32_t* h = reinterpret_cast<uint32_t*>(&hi);
 #pragma unroll
   for (int w = 0; w < 4; ++w) {
-    const float2 c0 = __ldg(cs + 2 * w), c1 = __ldg(cs + 2 * w + 1);
     const float x0 = __uint_as_float(l[w] << 16), x1 = __uint_as_float(l[w] & 0xFFFF0000u);
     const float y0 = __uint_as_float(h[w] << 16), y1 = __uint_as_float(h[w] & 0xFFFF0000u);
     // (x, y) -> (x cos - y sin, y cos + x sin); each product rounded once into the sum
-    l[w] = pack_bf16(fmaf(x0, c0.x, -y0 * c0.y), fmaf(x1, c1.x, -y1 * c1.y));
-    h[w] = pack_bf16(fmaf(y0, c0.x, x0 * c0.y), fmaf(y1, c1.x, x1 * c1.y));
+    l[w] = pack_bf16(fmaf(x0, cs[w].x, -y0 * cs[w].y), fmaf(x1, cs[w].z, -y1 * cs[w].w));
+    h[w] = pack_bf16(fmaf(y0, cs[w].x, x0 * cs[w].y), fmaf(y1, cs[w].z, x1 * cs[w].w));
   }
+}
+__device__ __forceinline__ void load_cs(float4 (&cs)[4], const float2* __restrict__ tab_row8) {
+  const float4* t = reinterpret_cast<const float4*>(tab_row8);
+#pragma unroll
+  for (int w = 0; w < 4; ++w) cs[w] = __ldg(t + w);
+}
+__device__ __forceinline__ void rotate_chunk(uint4& lo, uint4& hi, const float2* __restrict__ tab_row8) {
+  float4 cs[4];
+  load_cs(cs, tab_row8);
+  rotate_chunk(lo, hi, cs);
 }
 
 // Position of query row n (global row index in the packed batch): n_ctx + (N_s - N_q) + local index.
@@ -79,16 +89,32 @@ __global__ void __launch_bounds__(256) rope_stage_kernel(char* const* __restrict
   const long long half_bytes = (long long)Nf * 128;
   char* dst = k_rot + e * Hkv * 2 * half_bytes;
   if (threadIdx.x == 0) tbl_k[e] = dst;
-  const int items = Hkv * Nf * 8;
-  for (int it = threadIdx.x; it < items; it += 256) {
-    const int c = it & 7, r = (it >> 3) % Nf, g = (it >> 3) / Nf;
+  // a thread takes (row, chunk) positions and walks the KV heads: the (cos, sin) of a position are loaded
+  // once for all heads, and four heads' chunks are in flight before the first rotation
+  constexpr int U = 4;
+  for (int rc = threadIdx.x; rc < Nf * 8; rc += 256) {
+    const int c = rc & 7, r = rc >> 3;
     const long long off = (long long)r * 128 + ((c ^ (r & 7)) << 4);
-    const char* src = page + (long long)g * 4 * half_bytes;  // the page holds K then V of each KV head
-    uint4 lo = *reinterpret_cast<const uint4*>(src + off), hi = *reinterpret_cast<const uint4*>(src + half_bytes + off);
-    rotate_chunk(lo, hi, tab + ((long long)slot * Nf + r) * 64 + c * 8);
-    char* d = dst + (long long)g * 2 * half_bytes;
-    *reinterpret_cast<uint4*>(d + off) = lo;
-    *reinterpret_cast<uint4*>(d + half_bytes + off) = hi;
+    float4 cs[4];
+    load_cs(cs, tab + ((long long)slot * Nf + r) * 64 + c * 8);
+    for (int g0 = 0; g0 < Hkv; g0 += U) {
+      uint4 lo[U], hi[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        if (g0 + u < Hkv) {
+          const char* src = page + (long long)(g0 + u) * 4 * half_bytes + off;  // the page holds K then V of each KV head
+          lo[u] = __ldcs(reinterpret_cast<const uint4*>(src));
+          hi[u] = __ldcs(reinterpret_cast<const uint4*>(src + half_bytes));
+        }
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        if (g0 + u < Hkv) {
+          rotate_chunk(lo[u], hi[u], cs);
+          char* d = dst + (long long)(g0 + u) * 2 * half_bytes + off;
+          *reinterpret_cast<uint4*>(d) = lo[u];
+          *reinterpret_cast<uint4*>(d + half_bytes) = hi[u];
+        }
+    }
   }
 }
 
@@ -236,17 +262,29 @@ cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const vo
     rope_q_kernel<<<grid, 256, 0, st>>>((const uint4*)q, (uint4*)c->q_rot, qb, sb, s.Hq, n_ctx_tokens, c->rope_tab);
     c->launches += 1;
     q_eff = c->q_rot;
-    if (ncf > 0) {
-      rope_stage_kernel<<<dim3(ncf, qb.nQ, s.L), 256, 0, st>>>(c->ctx_tbl, c->tbl_k, c->k_rot, qb.nQ, ncf, s.Hkv, s.Nf,
-                                                               c->rope_tab);
-      c->launches += 1;
-    }
   }
-  self_attend_kernel<<<dim3(s.Hq, qb.nQ, s.L), 256, 0, st>>>(q_eff, (const __nv_bfloat16*)k_self,
-                                                            (const __nv_bfloat16*)v_self, qb, sb, s.Hq, s.Hkv, s.G,
-                                                            n_ctx_tokens, rope ? c->rope_tab : nullptr,
-                                                            1.4426950408889634f / sqrtf(128.f), c->self_o, c->self_ml);
+  // the part over X (latency-bound) runs on the side stream beside the pass over the context's keys
+  // (bandwidth-bound); both are joined before the attention kernel
+  const bool fork = rope && ncf > 0;
+  cudaStream_t st_self = fork ? c->side : st;
+  cudaError_t e;
+  if (fork) {
+    if ((e = cudaEventRecord(c->ev_main, st)) != cudaSuccess) return e;
+    if ((e = cudaStreamWaitEvent(c->side, c->ev_main, 0)) != cudaSuccess) return e;
+  }
+  self_attend_kernel<<<dim3(s.Hq, qb.nQ, s.L), 256, 0, st_self>>>(q_eff, (const __nv_bfloat16*)k_self,
+                                                                 (const __nv_bfloat16*)v_self, qb, sb, s.Hq, s.Hkv, s.G,
+                                                                 n_ctx_tokens, rope ? c->rope_tab : nullptr,
+                                                                 1.4426950408889634f / sqrtf(128.f), c->self_o,
+                                                                 c->self_ml);
   c->launches += 1;
+  if (fork) {
+    if ((e = cudaEventRecord(c->ev_side, c->side)) != cudaSuccess) return e;
+    rope_stage_kernel<<<dim3(ncf, qb.nQ, s.L), 256, 0, st>>>(c->ctx_tbl, c->tbl_k, c->k_rot, qb.nQ, ncf, s.Hkv, s.Nf,
+                                                             c->rope_tab);
+    c->launches += 1;
+    if ((e = cudaStreamWaitEvent(st, c->ev_side, 0)) != cudaSuccess) return e;
+  }
   return cudaGetLastError();
 }
 
