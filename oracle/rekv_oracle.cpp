@@ -14,6 +14,9 @@
  *   3. keep the r most similar frames   (Eq. 2 paragraph, "r most relevant")
  *   4. the retrieved K/V, R, are brought together as the context
  *   5. O = Attn(Q, R_k, R_v)            (Eq. 3)
+ *   2'. external retrieval: the same cosine on embeddings from a CLIP-like
+ *      encoder, divided by the temperature tau; one selection for all layers
+ *                                         (Eq. 2, external-retrieval paragraph)
  *   5'. the whole of Eq. 3: O = Attn(W_Q X, [R_k, W_K X], [R_v, W_V X]) -- the
  *      question's (and generated tokens') own K/V follow the retrieved context,
  *      causally; rotary position embedding with the retrieved tokens taken as
@@ -122,6 +125,33 @@ void oracle_score(const uint16_t* q, int n_q, int n_q_heads, int n_kv_heads, int
     }
     rn = std::max(std::sqrt(rn), eps);
     scores[f] = (float)(dot / (qn * rn));
+  }
+}
+
+/* External retrieval (Eq. 2 with its temperature): Sim(v, q) = <v, q> / (tau |v| |q|) between the question's
+ * embedding q [dim] and frame embeddings embs [n_frames][dim] (floats, from a CLIP-like encoder outside this
+ * library); with b > 1 the vector of a block is the mean of its b frame vectors (kept in double) and
+ * n_items counts complete blocks.  Norms are clamped at 1e-8 as in the internal variant. */
+void oracle_score_external(const float* q, const float* embs, int dim, int n_items, int b, double tau,
+                           float* scores) {
+  const double eps = 1e-8;
+  double qn = 0.0;
+  for (int c = 0; c < dim; ++c) qn += (double)q[c] * (double)q[c];
+  qn = std::max(std::sqrt(qn), eps);
+  std::vector<double> v(dim);
+  for (int j = 0; j < n_items; ++j) {
+    for (int c = 0; c < dim; ++c) {
+      double s = 0.0;
+      for (int f = 0; f < b; ++f) s += (double)embs[((long)j * b + f) * dim + c];
+      v[c] = s / (double)b;
+    }
+    double dot = 0.0, vn = 0.0;
+    for (int c = 0; c < dim; ++c) {
+      dot += (double)q[c] * v[c];
+      vn += v[c] * v[c];
+    }
+    vn = std::max(std::sqrt(vn), eps);
+    scores[j] = (float)(dot / (tau * qn * vn));
   }
 }
 

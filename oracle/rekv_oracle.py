@@ -34,6 +34,9 @@ _lib.oracle_gather.restype = ctypes.c_int
 _lib.oracle_attend.argtypes = [_u16p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, _u16p, _u16p,
                                ctypes.c_long, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
 _lib.oracle_attend.restype = None
+_lib.oracle_score_external.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                       ctypes.c_double, ctypes.c_void_p]
+_lib.oracle_score_external.restype = None
 _lib.oracle_rope.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_long, ctypes.c_double, ctypes.c_void_p]
 _lib.oracle_rope.restype = None
 _lib.oracle_attend_full.argtypes = [_u16p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, _u16p, _u16p,
@@ -89,6 +92,37 @@ def score_blocks(q: torch.Tensor, reps: torch.Tensor, n_kv_heads: int, n_blocks:
     out = torch.empty(n_blocks, dtype=torch.float32)
     _lib.oracle_score_blocks(q.data_ptr(), n_q, n_qh, n_kv_heads, d, reps.data_ptr(), n_blocks, b, out.data_ptr())
     return out
+
+
+def score_external(q_emb: torch.Tensor, embs: torch.Tensor, tau: float, n_items: int = None, b: int = 1) -> torch.Tensor:
+    """Eq. 2 with its temperature on external embeddings.  q_emb: float32 [E]; embs: float32 [T][E];
+    n_items frames (b == 1) or complete blocks of b frames -> float32 [n_items]."""
+    _chk(q_emb, torch.float32)
+    _chk(embs, torch.float32)
+    n_items = embs.shape[0] // b if n_items is None else n_items
+    assert embs.shape[1] == q_emb.shape[0] and embs.shape[0] >= n_items * b
+    out = torch.empty(n_items, dtype=torch.float32)
+    _lib.oracle_score_external(q_emb.data_ptr(), embs.data_ptr(), q_emb.shape[0], n_items, b, tau, out.data_ptr())
+    return out
+
+
+def retrieve_external(q_emb: torch.Tensor, embs: torch.Tensor, tau: float, top_k: int, n_visible: int, window: int,
+                      b: int = 1):
+    """External retrieval of one question: one selection for all layers.
+    -> (scores float32, idx int32 [top_k] ascending frames padded with -1, k_eff, gap)."""
+    if b == 1:
+        s = score_external(q_emb, embs[:n_visible].contiguous(), tau)
+        i, k_eff, g = select(s, n_visible, window, top_k)
+        return s, i, k_eff, g
+    n_blocks, k_blocks, _ = block_geometry(n_visible, window, b, top_k)
+    s = score_external(q_emb, embs[:n_visible].contiguous(), tau, n_blocks, b)
+    bi, kb, g = select(s, n_blocks, 0, top_k // b)
+    assert kb == k_blocks
+    i = torch.full((top_k,), -1, dtype=torch.int32)
+    for j in range(kb):
+        for f in range(b):
+            i[j * b + f] = int(bi[j]) * b + f
+    return s, i, kb * b, g
 
 
 def block_geometry(n_visible: int, window: int, b: int, top_k: int):

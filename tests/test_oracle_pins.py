@@ -328,6 +328,52 @@ def test_attention_is_invariant_to_context_order():
     assert torch.allclose(a, b, atol=1e-6)
 
 
+# ----------------------------------------------------------------------------- external retrieval (Eq. 2 with tau)
+def test_external_scores_closed_forms_and_library_cosine():
+    g = torch.Generator().manual_seed(9)
+    E, T = 1152, 40
+    embs = torch.randn(T, E, generator=g)
+    q = torch.randn(E, generator=g)
+    embs[3] = 2.5 * q          # parallel -> 1 / tau
+    embs[4] = -0.5 * q         # antiparallel -> -1 / tau
+    embs[5] = 0.0
+    embs[5, 0], q0 = 1.0, q.clone()
+    q0[0] = 0.0                # orthogonal to frame 5
+    for tau in (1.0, 0.07, 3.0):
+        s = orc.score_external(q, embs, tau)
+        assert abs(s[3].item() - 1 / tau) < 1e-5 / tau and abs(s[4].item() + 1 / tau) < 1e-5 / tau
+        ref = torch.nn.functional.cosine_similarity(embs.double(), q.double()[None], dim=1) / tau
+        np.testing.assert_allclose(s.double().numpy(), ref.numpy(), rtol=0, atol=2e-7 / tau)
+        assert orc.score_external(q0, embs, tau)[5].item() == 0.0
+        # positive rescaling of the question or of a frame changes nothing; tau only rescales
+        np.testing.assert_allclose(orc.score_external(7 * q, embs, tau).numpy(), s.numpy(), atol=2e-6 / tau)
+        np.testing.assert_allclose((orc.score_external(q, embs, 1.0) / tau).numpy(), s.numpy(), rtol=1e-6, atol=1e-9)
+    # zero vectors are clamped, not NaN
+    assert orc.score_external(torch.zeros(E), embs, 1.0).abs().max().item() == 0.0
+
+
+def test_external_retrieval_selection_is_tau_invariant_and_blocks_average_frames():
+    g = torch.Generator().manual_seed(10)
+    E, T, W = 64, 50, 4
+    embs = torch.randn(T, E, generator=g)
+    q = torch.randn(E, generator=g)
+    s1, i1, k1, _ = orc.retrieve_external(q, embs, 1.0, 8, T, W)
+    s2, i2, k2, _ = orc.retrieve_external(q, embs, 0.05, 8, T, W)
+    assert torch.equal(i1, i2) and k1 == k2 == 8
+    brute = sorted(sorted(range(T - W), key=lambda f: (-s1[f].item(), f))[:8])
+    assert i1.tolist() == brute
+    assert all(f < T - W for f in i1.tolist())          # the window is not a candidate
+    # blocks: the vector of a block is the mean of its frame vectors
+    b = 4
+    sb, ib, kb, _ = orc.retrieve_external(q, embs, 0.5, 8, T, W, b)
+    n_blocks = (T - W) // b
+    means = embs[: n_blocks * b].view(n_blocks, b, E).double().mean(dim=1)
+    ref = torch.nn.functional.cosine_similarity(means, q.double()[None], dim=1) / 0.5
+    np.testing.assert_allclose(sb.double().numpy(), ref.numpy(), atol=1e-6)
+    top = sorted(sorted(range(n_blocks), key=lambda j: (-sb[j].item(), j))[:2])
+    assert ib.tolist() == [j * b + f for j in top for f in range(b)] and kb == 8
+
+
 # ----------------------------------------------------------------------------- Eq. 3 in full: X's own K/V, RoPE
 def _complex_rope(x: np.ndarray, pos: int, theta: float) -> np.ndarray:
     """RoFormer's definition: (x_i + i x_{i+D/2}) * exp(i * pos * theta^(-2i/D)), an independent statement."""
