@@ -40,6 +40,9 @@ WORKLOADS = {
     # retrieved tokens at consecutive positions (base 1e6, the paper's Qwen2-based models)
     "7b_hbm_full_eq3_rope": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503,
                                  off_scale=0.5, tail=0, nQ=1, appends_per_step=1, full=True, rope_theta=1e6),
+    # external retrieval (the paper's baseline retriever): SigLIP-sized frame embeddings, one selection for all layers
+    "7b_hbm_external_1152": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503,
+                                 off_scale=0.5, tail=0, nQ=1, appends_per_step=1, ext_dim=1152, tau=0.07),
     "72b_offload_1800f": dict(L=80, Hq=64, Hkv=8, D=128, Nf=196, T=1800, W=8, k=32, Nq=64, seed=2503,
                               off_scale=0.5, tail=32, nQ=1, appends_per_step=1),
 }
@@ -134,6 +137,8 @@ def algorithmic_bytes(w, sum_nq=None, nQ=1):
     sum_nq = w["Nq"] if sum_nq is None else sum_nq
     page = w["Hkv"] * 2 * w["Nf"] * w["D"] * 2
     reps = w["L"] * w["T"] * w["Hkv"] * w["D"] * 4
+    if w.get("ext_dim"):  # external retrieval reads the embedding table once, for all layers
+        reps = w["T"] * w["ext_dim"] * 4
     qo = 2 * w["L"] * sum_nq * w["Hq"] * w["D"] * 2
     kv = w["L"] * (nQ * w["k"] + w["W"]) * page
     kv_read = w["L"] * nQ * (w["k"] + w["W"]) * page  # what the attention kernel is asked to read
@@ -191,7 +196,7 @@ def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    if w.get("full"):
+    if w.get("full") or w.get("ext_dim"):
         raise SystemExit("the CPU-oracle arm times steps 2-5 of the retrieval path; use a workload without full=True")
     Ls = 2
     arm = OracleArm(w, Ls)
@@ -270,7 +275,8 @@ def run_cuda(args, w):
 
     g = rekv.ReKV(w["L"], w["Hq"], w["Hkv"], w["D"], w["Nf"], w["T"] + 8, w["W"], hbm_tail_frames=w["tail"],
                   max_q_tokens=cu[-1], max_topk=w["k"], max_questions=nQ, device=local, flags=rekv.FLAG_TIMING,
-                  max_self_tokens=cu[-1] if w.get("full") else 0, rope_theta=w.get("rope_theta", 0.0))
+                  max_self_tokens=cu[-1] if w.get("full") else 0, rope_theta=w.get("rope_theta", 0.0),
+                  ext_embed_dim=w.get("ext_dim", 0))
     kf = torch.empty((w["L"], w["Nf"], w["Hkv"], w["D"]), dtype=torch.bfloat16, device=dev)
     vf = torch.empty_like(kf)
     for f in range(T0):
@@ -297,6 +303,21 @@ def run_cuda(args, w):
             idx, _, _ = g.retrieve(qt, cu, w["k"], n_vis)
             g.gather(idx, nQ, w["k"], n_vis)
             return g.attend_full(qt, ks_self, vs_self, cu, cu, out=out)
+    elif w.get("ext_dim"):
+        # seeded stand-ins for the external encoder's embeddings (its weights are not in this repository)
+        gen = torch.Generator().manual_seed(w["seed"])
+        common = torch.randn(w["ext_dim"], generator=gen)
+        ext_frames = (torch.randn(w["T"] + 8, w["ext_dim"], generator=gen) + 0.7 * common).to(dev)
+        ext_q = [(torch.randn(nQ, w["ext_dim"], generator=gen) + 0.7 * common).to(dev) for _ in range(N_ROTATE)]
+        for f in range(T0):
+            g.set_frame_embedding(f, ext_frames[f])
+        ext_state = {"i": 0}
+
+        def ask(qt, n_vis, out):
+            ext_state["i"] += 1
+            idx, _, _ = g.retrieve_external(ext_q[ext_state["i"] % N_ROTATE], w["k"], n_vis, w["tau"])
+            g.gather(idx, nQ, w["k"], n_vis)
+            return g.attend(qt, cu, out)
     else:
         def ask(qt, n_vis, out):
             return g.question(qt, cu, w["k"], n_vis, out=out)
@@ -310,6 +331,8 @@ def run_cuda(args, w):
             j = state["next"]
             state["next"] += 1
             nf = g.append_frame(src_k[j % len(src_k)], src_v[j % len(src_v)])
+            if w.get("ext_dim"):
+                g.set_frame_embedding(nf, ext_frames[nf])
         return nf
 
     def step_device(i, ev=None):
@@ -375,6 +398,8 @@ def run_cuda(args, w):
             kf.copy_(hk[(i + a) % 2], non_blocking=True)
             vf.copy_(hv[(i + a) % 2], non_blocking=True)
             nf = g.append_frame(kf, vf)
+            if w.get("ext_dim"):
+                g.set_frame_embedding(nf, ext_frames[nf])
         if ev:
             ev[0].record(stream)
         dq.copy_(hq[i % N_ROTATE], non_blocking=True)
@@ -399,12 +424,18 @@ def run_cuda(args, w):
     # steps 2-3 alone (question vectors, scores, selection): frames scored per second
     n_vis = g.stats().frames
     ev_r = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    if w.get("ext_dim"):
+        def retrieve_only(i):
+            g.retrieve_external(ext_q[i % N_ROTATE], w["k"], n_vis, w["tau"])
+    else:
+        def retrieve_only(i):
+            g.retrieve(qs[i % N_ROTATE], cu, w["k"], n_vis)
     for i in range(3):
-        g.retrieve(qs[i % N_ROTATE], cu, w["k"], n_vis)
+        retrieve_only(i)
     torch.cuda.synchronize()
     ev_r[0].record(stream)
     for i in range(10):
-        g.retrieve(qs[i % N_ROTATE], cu, w["k"], n_vis)
+        retrieve_only(i)
     ev_r[1].record(stream)
     torch.cuda.synchronize()
     retrieve_us = ev_r[0].elapsed_time(ev_r[1]) * 1e3 / 10
@@ -470,7 +501,8 @@ def run_cuda(args, w):
                          "layer_sequential_mode": ("one CUDA graph replay per layer" if w["tail"] == 0
                                                    else "one eager call per layer"),
                          "retrieve_us_per_batch": retrieve_us,
-                         "frames_scored_per_s_all_gpus": world * w["L"] * n_vis * nQ / (retrieve_us * 1e-6),
+                         "frames_scored_per_s_all_gpus": (world * (1 if w.get("ext_dim") else w["L"]) * n_vis * nQ
+                                                          / (retrieve_us * 1e-6)),
                          "questions_per_s_all_gpus": world * 1e6 / q_lat},
             "append_us": app_us,
             "e2e": {"value": e2e_lat, "unit": "us",

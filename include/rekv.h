@@ -80,6 +80,9 @@ typedef struct {
                                 and its workspaces are not allocated */
   float rope_theta;          /* rekv_attend_full: base of the rotary position embedding (1e6 for the paper's
                                 Qwen2-based models); 0 = no positional term */
+  int32_t ext_embed_dim;     /* external retrieval: dimension of the frame / question embeddings of a CLIP-like
+                                encoder (1152 for the paper's SigLIP-SO400M); a multiple of 4, <= 2048; 0 = the
+                                embedding table is not allocated */
 } rekv_config;
 
 typedef struct {
@@ -172,6 +175,21 @@ int rekv_attend(rekv_ctx* ctx, const void* q, const int32_t* cu_q, int nQ, void*
  * Needs max_self_tokens > 0 at creation.  Returns 0 or an error code (REKV_ERR_STATE without a gather). */
 int rekv_attend_full(rekv_ctx* ctx, const void* q, const void* k_self, const void* v_self, const int32_t* cu_q,
                      const int32_t* cu_self, int nQ, void* out, void* stream);
+
+/* External retrieval (Eq. 2 with its temperature; the paper's baseline retriever).  The embeddings come from
+ * a CLIP-like encoder outside this library.  rekv_set_frame_embedding stores the embedding of an appended
+ * frame (device fp32 [ext_embed_dim], copied).  rekv_retrieve_external scores every visible frame -- or
+ * every complete block of block_frames frames, whose vector is the mean of its frames' embeddings --
+ *   Sim(v, q) = <v, q> / (tau |v| |q|)        (norms clamped at 1e-8)
+ * against each of nQ question embeddings (q_emb: device fp32 [nQ][ext_embed_dim]) and selects as
+ * rekv_retrieve does (candidates exclude the window, ties to the lower index, ascending output).  One
+ * selection serves all layers: idx_out, device int32 [L][nQ][top_k], receives it in every layer's block, so
+ * that rekv_gather takes it unchanged.  scores_out (nullable): device fp32 [nQ][n_scored], n_scored as in
+ * rekv_retrieve.  Needs ext_embed_dim > 0 and embeddings for all of [0, n_visible).  tau > 0.
+ * Returns k_eff or a negative error code. */
+int rekv_set_frame_embedding(rekv_ctx* ctx, int frame, const float* emb, void* stream);
+int rekv_retrieve_external(rekv_ctx* ctx, const float* q_emb, int nQ, int top_k, int n_visible, float tau,
+                           int32_t* idx_out, float* scores_out, void* stream);
 
 /* Layer-sequential form of steps 2-5.  A decoder produces layer l+1's queries only from layer l's
  * output, and the paper retrieves independently in every layer, so a model integrates the path one

@@ -277,6 +277,83 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
   (void)n_gt;
 }
 
+// ---- external retrieval (Eq. 2 with its temperature): cosine of each question embedding with every frame
+// embedding (or with the mean of a block's frame embeddings), divided by tau.  grid = ceil(items / 8), 256
+// threads, a warp per item: the item's vector is read once into registers (float4 per lane, coalesced) and
+// scored against every question of the batch, whose embeddings sit in shared memory in groups.
+constexpr int EXT_MAX_V4 = 16;  // float4 per lane: embedding dim <= 2048
+__global__ void __launch_bounds__(256) ext_score_kernel(const float* __restrict__ embs, const float* __restrict__ q,
+                                                        int nQ, int E, int n_items, int block, int q_group, float tau,
+                                                        float* __restrict__ scores) {
+  extern __shared__ float4 s_qe[];  // [q_group][E/4]
+  __shared__ float s_qn[REKV_MAX_QUESTIONS];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int item = blockIdx.x * 8 + warp;
+  const int e4 = E / 4;
+  const float eps = 1e-8f;
+  float4 r[EXT_MAX_V4];
+  float vn = 0.f;
+  if (item < n_items) {
+#pragma unroll
+    for (int i = 0; i < EXT_MAX_V4; ++i)
+      if (i * 32 + lane < e4) {
+        const float4* row = reinterpret_cast<const float4*>(embs + (long long)item * block * E) + i * 32 + lane;
+        float4 a = __ldg(row);
+        for (int j = 1; j < block; ++j) {  // block vector = mean of the block's frame vectors
+          const float4 b = __ldg(row + (long long)j * e4);
+          a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+        }
+        if (block > 1) {
+          const float fb = (float)block;
+          a.x = __fdiv_rn(a.x, fb); a.y = __fdiv_rn(a.y, fb); a.z = __fdiv_rn(a.z, fb); a.w = __fdiv_rn(a.w, fb);
+        }
+        r[i] = a;
+        vn += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+      }
+    for (int o = 16; o; o >>= 1) vn += __shfl_xor_sync(0xffffffffu, vn, o);
+    vn = fmaxf(__fsqrt_rn(vn), eps);
+  }
+  for (int qg0 = 0; qg0 < nQ; qg0 += q_group) {
+    const int qn = min(q_group, nQ - qg0);
+    __syncthreads();
+    const float4* src = reinterpret_cast<const float4*>(q + (long long)qg0 * E);
+    for (int i = threadIdx.x; i < qn * e4; i += 256) s_qe[i] = src[i];
+    __syncthreads();
+    for (int qi = warp; qi < qn; qi += 8) {  // the questions' norms
+      float sq = 0.f;
+      for (int i = lane; i < e4; i += 32) {
+        const float4 a = s_qe[qi * e4 + i];
+        sq += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+      }
+      for (int o = 16; o; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      if (lane == 0) s_qn[qi] = fmaxf(__fsqrt_rn(sq), eps);
+    }
+    __syncthreads();
+    if (item < n_items) {
+      for (int qi = 0; qi < qn; ++qi) {
+        float d = 0.f;
+#pragma unroll
+        for (int i = 0; i < EXT_MAX_V4; ++i)
+          if (i * 32 + lane < e4) {
+            const float4 a = s_qe[qi * e4 + i * 32 + lane];
+            d += r[i].x * a.x + r[i].y * a.y + r[i].z * a.z + r[i].w * a.w;
+          }
+        for (int o = 16; o; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+        if (lane == 0) scores[(long long)(qg0 + qi) * n_items + item] = __fdiv_rn(d, tau * s_qn[qi] * vn);
+      }
+    }
+  }
+}
+
+// the external selection is the same in every layer: copies layer 0's [nQ][top_k] block to the others
+__global__ void replicate_idx_kernel(int32_t* __restrict__ idx, int per_layer, int L) {
+  rekv_ptx::grid_dep_wait();
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= per_layer) return;
+  const int32_t v = idx[i];
+  for (int l = 1; l < L; ++l) idx[(long long)l * per_layer + i] = v;
+}
+
 }  // namespace
 
 cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, const CtxGeom& geom,
@@ -314,6 +391,39 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
     c->launches += 1;
   }
   c->launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t rekv_launch_retrieve_external(rekv_ctx* c, const float* q_emb, int nQ, int top_k, const CtxGeom& geom,
+                                          int n_visible, float tau, int32_t* idx_out, float* scores, cudaStream_t st) {
+  const StoreView& s = c->sv;
+  const int E = c->cfg.ext_embed_dim, b = c->cfg.block_frames;
+  const int n_scored = b == 1 ? n_visible : geom.n_items;
+  int q_group = (int)((96 * 1024) / (E * sizeof(float)));
+  if (q_group > nQ) q_group = nQ;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(ext_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  if (n_scored > 0) {
+    ext_score_kernel<<<(n_scored + 7) / 8, 256, (size_t)q_group * E * sizeof(float), st>>>(c->ext_emb, q_emb, nQ, E, n_scored,
+                                                                                         b, q_group, tau, scores);
+    c->launches += 1;
+  }
+  if (top_k > 0) {
+    cudaError_t e2 = rekv_launch_pdl(topk_kernel, dim3(nQ, 1), dim3(512), 0, st, (const float*)scores, nQ, n_scored,
+                                     geom.n_items, top_k, geom.k_items, idx_out, b, 0);
+    if (e2 != cudaSuccess) return e2;
+    const int per_layer = nQ * top_k;
+    if (s.L > 1) {
+      cudaError_t e3 = rekv_launch_pdl(replicate_idx_kernel, dim3((per_layer + 255) / 256), dim3(256), 0, st, idx_out,
+                                       per_layer, s.L);
+      if (e3 != cudaSuccess) return e3;
+    }
+    c->launches += 2;
+  }
   return cudaGetLastError();
 }
 

@@ -63,6 +63,7 @@ void free_ctx(rekv_ctx* c) {
   cudaFree(c->part_ml);
   cudaFree(c->status);
   cudaFree(c->idx_own);
+  cudaFree(c->ext_emb);
   cudaFree(c->self_o);
   cudaFree(c->self_ml);
   cudaFree(c->q_rot);
@@ -136,6 +137,8 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   if (cfg->max_q_tokens < 1 || cfg->max_topk < 0) REKV_FAIL(nullptr, REKV_ERR_ARG, "max_q_tokens / max_topk out of range");
   if (cfg->max_self_tokens < 0 || !(cfg->rope_theta >= 0.f) || (cfg->rope_theta > 0.f && cfg->rope_theta < 1.f))
     REKV_FAIL(nullptr, REKV_ERR_ARG, "max_self_tokens must be >= 0 and rope_theta 0 or >= 1");
+  if (cfg->ext_embed_dim < 0 || cfg->ext_embed_dim > 2048 || cfg->ext_embed_dim % 4)
+    REKV_FAIL(nullptr, REKV_ERR_ARG, "ext_embed_dim=%d must be a multiple of 4 in [0, 2048]", cfg->ext_embed_dim);
 
   int n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0) {
@@ -166,6 +169,8 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   c->link_bytes = nullptr;
   c->idx_own = nullptr;
   c->self_o = c->self_ml = nullptr;
+  c->ext_emb = nullptr;
+  c->ext_frames = 0;
   c->q_rot = nullptr;
   c->rope_tab = nullptr;
   c->k_rot = nullptr;
@@ -216,6 +221,9 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   CREATE_CUDA(cudaMalloc(&c->idx_own, (size_t)s.L * maxQ * (c->cfg.max_topk > 0 ? c->cfg.max_topk : 1) * sizeof(int32_t)),
               "allocating the selection buffer");
   c->ctx_frames_max = ctx_frames_max;
+  if (c->cfg.ext_embed_dim > 0)
+    CREATE_CUDA(cudaMalloc(&c->ext_emb, (size_t)s.max_frames * c->cfg.ext_embed_dim * sizeof(float)),
+                "allocating the embedding table");
   if (c->cfg.max_self_tokens > 0) {  // workspaces of rekv_attend_full
     const size_t rows = (size_t)s.L * c->cfg.max_q_tokens * s.Hq;
     CREATE_CUDA(cudaMalloc(&c->self_o, rows * 128 * sizeof(float)), "allocating the self-attention partials");
@@ -467,6 +475,42 @@ int rekv_attend_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu_q
   cudaStream_t st = (cudaStream_t)stream;
   if (c->gather_layerwise) REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[layer], 0));
   return attend_one_layer(c, layer, q, qb, out, st);
+}
+
+int rekv_set_frame_embedding(rekv_ctx* c, int frame, const float* emb, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (c->cfg.ext_embed_dim <= 0) REKV_FAIL(c, REKV_ERR_STATE, "the context was created with ext_embed_dim == 0");
+  if (!emb) REKV_FAIL(c, REKV_ERR_ARG, "null embedding");
+  if (frame < 0 || frame >= c->frames) REKV_FAIL(c, REKV_ERR_ARG, "frame=%d outside [0, %d)", frame, c->frames);
+  DeviceGuard guard(c->device);
+  const size_t bytes = (size_t)c->cfg.ext_embed_dim * sizeof(float);
+  REKV_CUDA(c, cudaMemcpyAsync(c->ext_emb + (size_t)frame * c->cfg.ext_embed_dim, emb, bytes, cudaMemcpyDeviceToDevice,
+                               (cudaStream_t)stream));
+  if (frame == c->ext_frames) c->ext_frames = frame + 1;  // embeddings are expected in frame order
+  return REKV_OK;
+}
+
+int rekv_retrieve_external(rekv_ctx* c, const float* q_emb, int nQ, int top_k, int n_visible, float tau,
+                           int32_t* idx_out, float* scores_out, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (c->cfg.ext_embed_dim <= 0) REKV_FAIL(c, REKV_ERR_STATE, "the context was created with ext_embed_dim == 0");
+  if (!q_emb) REKV_FAIL(c, REKV_ERR_ARG, "null q_emb");
+  if (nQ < 1 || nQ > c->cfg.max_questions) REKV_FAIL(c, REKV_ERR_ARG, "nQ=%d outside [1, %d]", nQ, c->cfg.max_questions);
+  if (top_k < 0 || top_k > c->cfg.max_topk) REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d outside [0, %d]", top_k, c->cfg.max_topk);
+  if (top_k > 0 && !idx_out) REKV_FAIL(c, REKV_ERR_ARG, "null idx_out");
+  if (!(tau > 0.f)) REKV_FAIL(c, REKV_ERR_ARG, "tau must be positive");
+  if (n_visible < 0 || n_visible > c->frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "n_visible=%d outside [0, %d]", n_visible, c->frames);
+  if (n_visible == 0) REKV_FAIL(c, REKV_ERR_EMPTY, "no visible frame");
+  if (n_visible > c->ext_frames)
+    REKV_FAIL(c, REKV_ERR_STATE, "embeddings are set for %d frames, %d are visible", c->ext_frames, n_visible);
+  if (top_k % c->cfg.block_frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d must be a multiple of block_frames=%d", top_k, c->cfg.block_frames);
+  DeviceGuard guard(c->device);
+  const CtxGeom geom = rekv_geom(n_visible, c->cfg.window_frames, c->cfg.block_frames, top_k);
+  REKV_CUDA(c, rekv_launch_retrieve_external(c, q_emb, nQ, top_k, geom, n_visible, tau, idx_out,
+                                             scores_out ? scores_out : c->scores, (cudaStream_t)stream));
+  return geom.k_eff;
 }
 
 int rekv_attend_full(rekv_ctx* c, const void* q, const void* k_self, const void* v_self, const int32_t* cu_q,

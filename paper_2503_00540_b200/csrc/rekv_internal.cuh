@@ -107,6 +107,10 @@ struct rekv_ctx {
   unsigned long long* link_bytes;   // device counter: bytes pulled over the host link
   int32_t* idx_own;                 // [L][max_questions][max_topk]: selections of the layer-sequential calls
 
+  // external retrieval (allocated when ext_embed_dim > 0)
+  float* ext_emb;                   // [max_frames][ext_embed_dim] frame embeddings
+  int ext_frames;                   // embeddings are set for frames [0, ext_frames)
+
   // Eq. 3 in full (allocated when max_self_tokens > 0)
   float* self_o;                    // [L][max_q_tokens][H_q][128]
   float* self_ml;                   // [L][max_q_tokens][H_q][2]
@@ -173,6 +177,8 @@ cudaError_t rekv_launch_unswizzle_page(rekv_ctx* c, const char* page, void* k_ou
 // k_retrieve.cu
 cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, const CtxGeom& geom,
                                  int n_visible, int layer0, int layer1, int32_t* idx_out, float* scores, cudaStream_t st);
+cudaError_t rekv_launch_retrieve_external(rekv_ctx* c, const float* q_emb, int nQ, int top_k, const CtxGeom& geom,
+                                          int n_visible, float tau, int32_t* idx_out, float* scores, cudaStream_t st);
 // k_gather.cu
 cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, const CtxGeom& geom,
                                    int n_visible, int layer0, int layer1, int frames_now, cudaStream_t st);

@@ -29,7 +29,8 @@ class rekv_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "tokens_per_frame", "max_frames", "hbm_tail_frames",
         "window_frames", "block_frames", "max_q_tokens", "max_topk", "max_questions", "device")] + [
-            ("flags", ctypes.c_uint32), ("max_self_tokens", ctypes.c_int32), ("rope_theta", ctypes.c_float)]
+            ("flags", ctypes.c_uint32), ("max_self_tokens", ctypes.c_int32), ("rope_theta", ctypes.c_float),
+            ("ext_embed_dim", ctypes.c_int32)]
 
 
 class rekv_stats_t(ctypes.Structure):
@@ -41,7 +42,8 @@ class rekv_stats_t(ctypes.Structure):
 
 EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", "rekv_gather", "rekv_attend",
            "rekv_stats", "rekv_check_status", "rekv_last_error", "rekv_get_reps", "rekv_get_page",
-           "rekv_launch_count", "rekv_score_frames_static", "rekv_question_layer", "rekv_attend_layer", "rekv_attend_full")
+           "rekv_launch_count", "rekv_score_frames_static", "rekv_question_layer", "rekv_attend_layer", "rekv_attend_full",
+           "rekv_set_frame_embedding", "rekv_retrieve_external")
 
 _lib = None
 
@@ -62,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.rekv_question_layer.argtypes = [vp, i32, vp, ip, i32, i32, i32, vp, vp, vp]
         L.rekv_attend_layer.argtypes = [vp, i32, vp, ip, i32, vp, vp]
         L.rekv_attend_full.argtypes = [vp, vp, vp, vp, ip, ip, i32, vp, vp]
+        L.rekv_set_frame_embedding.argtypes = [vp, i32, vp, vp]
+        L.rekv_retrieve_external.argtypes = [vp, vp, i32, i32, i32, ctypes.c_float, vp, vp, vp]
         L.rekv_stats.argtypes = [vp, ctypes.POINTER(rekv_stats_t)]
         L.rekv_check_status.argtypes = [vp, vp]
         L.rekv_last_error.argtypes = [vp]
@@ -100,10 +104,10 @@ class ReKV:
     def __init__(self, n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, tokens_per_frame: int,
                  max_frames: int, window_frames: int, hbm_tail_frames: int = 0, max_q_tokens: int = 64,
                  max_topk: int = 64, max_questions: int = 1, device: int = 0, flags: int = 0,
-                 block_frames: int = 1, max_self_tokens: int = 0, rope_theta: float = 0.0):
+                 block_frames: int = 1, max_self_tokens: int = 0, rope_theta: float = 0.0, ext_embed_dim: int = 0):
         self.cfg = rekv_config(n_layers, n_q_heads, n_kv_heads, head_dim, tokens_per_frame, max_frames,
                                hbm_tail_frames, window_frames, block_frames, max_q_tokens, max_topk, max_questions,
-                               device, flags, max_self_tokens, rope_theta)
+                               device, flags, max_self_tokens, rope_theta, ext_embed_dim)
         self._h = ctypes.c_void_p()
         rc = lib().rekv_create(ctypes.byref(self.cfg), ctypes.byref(self._h))
         if rc != 0:
@@ -196,6 +200,23 @@ class ReKV:
             idx, _, _ = self.retrieve(q, cu_q, top_k, n_visible)
         self.gather(idx, nQ, top_k, n_visible)
         return self.attend(q, cu_q, out)
+
+    def set_frame_embedding(self, frame: int, emb: torch.Tensor) -> None:
+        """emb: float32 [ext_embed_dim], the external encoder's embedding of an appended frame."""
+        self._check(lib().rekv_set_frame_embedding(self._h, frame, _ptr(emb, torch.float32), self._stream()))
+
+    def retrieve_external(self, q_emb: torch.Tensor, top_k: int, n_visible: int, tau: float,
+                          want_scores: bool = False) -> Tuple[torch.Tensor, int, Optional[torch.Tensor]]:
+        """q_emb: float32 [nQ][ext_embed_dim].  Returns (idx int32 [L][nQ][top_k], the same selection in every
+        layer; k_eff; scores float32 [nQ][n_scored] or None)."""
+        nQ = q_emb.shape[0]
+        idx = torch.empty((self.L, nQ, max(top_k, 0)), dtype=torch.int32, device=self.device)
+        n_scored = n_visible if self.b == 1 else self.geometry(n_visible, top_k)[0]
+        scores = (torch.empty((nQ, n_scored), dtype=torch.float32, device=self.device)
+                  if want_scores and n_visible > 0 else None)
+        k_eff = self._check(lib().rekv_retrieve_external(self._h, _ptr(q_emb, torch.float32), nQ, top_k, n_visible,
+                                                         tau, _ptr(idx), _ptr(scores), self._stream()))
+        return idx, k_eff, scores
 
     def attend_full(self, q: torch.Tensor, k_self: torch.Tensor, v_self: torch.Tensor, cu_q: Sequence[int],
                     cu_self: Sequence[int], out: Optional[torch.Tensor] = None) -> torch.Tensor:

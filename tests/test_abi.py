@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_config_struct_matches_header_layout():
-    assert ctypes.sizeof(rekv.rekv_config) == 16 * 4
+    assert ctypes.sizeof(rekv.rekv_config) == 17 * 4
     assert ctypes.sizeof(rekv.rekv_stats_t) == 7 * 8 + 2 * 4 + 8
 
 
@@ -49,6 +49,7 @@ def test_create_rejects_bad_shapes_before_touching_a_device():
         (dict(max_questions=65), "max_questions"),
         (dict(rope_theta=0.5), "rope_theta"),
         (dict(max_self_tokens=-1), "max_self_tokens"),
+        (dict(ext_embed_dim=1150), "ext_embed_dim"),
     ]:
         base = dict(n_layers=1, n_q_heads=8, n_kv_heads=2, head_dim=128, tokens_per_frame=16, max_frames=8,
                     window_frames=2)
