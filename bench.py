@@ -40,6 +40,10 @@ WORKLOADS = {
     # retrieved tokens at consecutive positions (base 1e6, the paper's Qwen2-based models)
     "7b_hbm_full_eq3_rope": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503,
                                  off_scale=0.5, tail=0, nQ=1, appends_per_step=1, full=True, rope_theta=1e6),
+    # Eq. 1, one step of stream encoding: the incoming frame's tokens attend the local window (the last W stored
+    # frames, nothing retrieved) and themselves causally, then the frame's K/V are appended
+    "7b_encode_frame_w8": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=0, Nq=196, seed=2503,
+                               off_scale=0.5, tail=0, nQ=1, appends_per_step=1, full=True, rope_theta=1e6),
     # external retrieval (the paper's baseline retriever): SigLIP-sized frame embeddings, one selection for all layers
     "7b_hbm_external_1152": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503,
                                  off_scale=0.5, tail=0, nQ=1, appends_per_step=1, ext_dim=1152, tau=0.07),
@@ -299,8 +303,10 @@ def run_cuda(args, w):
         vs_self = torch.cat([synth.frame(w["seed"], synth.V, 1_000_000 + i, w["L"], n, w["Hkv"], w["D"], 0.0, device=dev)
                              for i, n in enumerate(lengths)], dim=1).contiguous()
 
+        no_idx = torch.empty((w["L"], nQ, 0), dtype=torch.int32, device=dev)
+
         def ask(qt, n_vis, out):
-            idx, _, _ = g.retrieve(qt, cu, w["k"], n_vis)
+            idx = g.retrieve(qt, cu, w["k"], n_vis)[0] if w["k"] > 0 else no_idx
             g.gather(idx, nQ, w["k"], n_vis)
             return g.attend_full(qt, ks_self, vs_self, cu, cu, out=out)
     elif w.get("ext_dim"):
@@ -454,6 +460,12 @@ def run_cuda(args, w):
                 with torch.cuda.graph(gr, stream=cap):
                     g.question_layer(l, q_l[l], cu, w["k"], n_vis, out=out[l])
                 layer_calls.append(gr.replay)
+            # the same 28 calls as consecutive nodes of ONE graph: what a decoder captured whole (its own
+            # kernels between the layers) pays for the path, without a graph launch per layer
+            gr_all = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr_all, stream=cap):
+                for l in range(w["L"]):
+                    g.question_layer(l, q_l[l], cu, w["k"], n_vis, out=out[l])
         stream.wait_stream(cap)
     else:
         for l in range(w["L"]):
@@ -469,6 +481,17 @@ def run_cuda(args, w):
     ev_r[1].record(stream)
     torch.cuda.synchronize()
     layer_seq_us = ev_r[0].elapsed_time(ev_r[1]) * 1e3 / n_seq / nQ
+    layer_seq_one_graph_us = None
+    if w["tail"] == 0:
+        for i in range(2 + n_seq):
+            if i == 2:
+                torch.cuda.synchronize()
+                ev_r[0].record(stream)
+            q_l.copy_(qs[i % N_ROTATE])
+            gr_all.replay()
+        ev_r[1].record(stream)
+        torch.cuda.synchronize()
+        layer_seq_one_graph_us = ev_r[0].elapsed_time(ev_r[1]) * 1e3 / n_seq / nQ
     g.check_status()
 
     q_sorted = sorted(q_us)
@@ -498,6 +521,7 @@ def run_cuda(args, w):
                          "attention_tflops": fl / (q_lat * nQ * 1e-6) / 1e12,
                          "median_us": q_median, "min_us": q_min,
                          "layer_sequential_us": layer_seq_us,
+                         "layer_sequential_one_graph_us": layer_seq_one_graph_us,
                          "layer_sequential_mode": ("one CUDA graph replay per layer" if w["tail"] == 0
                                                    else "one eager call per layer"),
                          "retrieve_us_per_batch": retrieve_us,

@@ -566,8 +566,10 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
     if (rr >= ui.rows_q) return;
     const int n = rr / p.G, j = rr - n * p.G;
     const long long out_row = (ui.q_row0 + n) * p.Hq + ui.g * p.G + j;
+    // the parts' maxima: a lane per part (independent loads), then the warp's maximum
     float M = p.self_o ? p.self_ml[out_row * 2] : -INFINITY;
-    for (long long c = c_first; c <= c_last; ++c) M = fmaxf(M, p.part_ml[(((c + u) * 2 + t) * 128 + r) * 2]);
+    for (long long c = c_first + lane; c <= c_last; c += 32) M = fmaxf(M, p.part_ml[(((c + u) * 2 + t) * 128 + r) * 2]);
+    for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float den = 0.f;
     if (p.self_o) {  // Eq. 3 in full: the part over the tokens of X is one more partial
@@ -576,16 +578,28 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
       acc = make_float4(w * o.x, w * o.y, w * o.z, w * o.w);
       den = w * p.self_ml[out_row * 2 + 1];
     }
-    for (long long c = c_first; c <= c_last; ++c) {
-      const long long base = ((c + u) * 2 + t) * 128 + r;
-      const float m = p.part_ml[base * 2], ls = p.part_ml[base * 2 + 1];
-      const float w = ex2(m - M);
-      const float4 o = *reinterpret_cast<const float4*>(p.part_o + base * 128 + lane * 4);
-      acc.x += w * o.x;
-      acc.y += w * o.y;
-      acc.z += w * o.z;
-      acc.w += w * o.w;
-      den += w * ls;
+    // the numerators, four parts' rows in flight, added in part order
+    for (long long c0 = c_first; c0 <= c_last; c0 += 4) {
+      float4 o[4];
+      float m[4], ls[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (c0 + i <= c_last) {
+          const long long base = ((c0 + i + u) * 2 + t) * 128 + r;
+          m[i] = p.part_ml[base * 2];
+          ls[i] = p.part_ml[base * 2 + 1];
+          o[i] = *reinterpret_cast<const float4*>(p.part_o + base * 128 + lane * 4);
+        }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (c0 + i <= c_last) {
+          const float w = ex2(m[i] - M);
+          acc.x += w * o[i].x;
+          acc.y += w * o[i].y;
+          acc.z += w * o[i].z;
+          acc.w += w * o[i].w;
+          den += w * ls[i];
+        }
     }
     const float inv = den > 0.f ? 1.f / den : 0.f;
     uint2 packed;

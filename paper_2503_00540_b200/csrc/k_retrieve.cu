@@ -6,10 +6,12 @@
 namespace {
 
 // ---- question vector: mean over the question's tokens and over the G query heads of each KV group
-// grid = (nQ, layers, H_kv), layer = layer0 + blockIdx.y; 256 threads = 4 token slices x 64 dim pairs: every load instruction of a warp
+// grid = (nQ, layers, H_kv), layer = layer0 + blockIdx.y; 1024 threads = 16 token slices x 64 dim pairs (a short
+// question is two or three rounds of loads deep): every load instruction of a warp
 // covers 128 contiguous bytes of one (token, head) row.  Writes the group's 128 dims of the question
 // vector and its partial sum of squares (the score kernel adds the H_kv partials).
-__global__ void __launch_bounds__(256) qmean_kernel(const __nv_bfloat162* __restrict__ q, QBatch qb, int Hq, int Hkv,
+constexpr int QM_SLICES = 16;
+__global__ void __launch_bounds__(QM_SLICES * 64) qmean_kernel(const __nv_bfloat162* __restrict__ q, QBatch qb, int Hq, int Hkv,
                                                     int G, float* __restrict__ qa, float* __restrict__ qsq,
                                                     int maxQ, int layer0) {
   const int qi = blockIdx.x, l = layer0 + blockIdx.y, g = blockIdx.z;
@@ -17,7 +19,7 @@ __global__ void __launch_bounds__(256) qmean_kernel(const __nv_bfloat162* __rest
   const int n0 = qb.cu[qi], n1 = qb.cu[qi + 1];
   const int d2 = threadIdx.x & 63, slice = threadIdx.x >> 6;
   float sx = 0.f, sy = 0.f;
-  for (int n = n0 + slice; n < n1; n += 4) {
+  for (int n = n0 + slice; n < n1; n += QM_SLICES) {
     const __nv_bfloat162* row = q + (((long long)l * qb.sumNq + n) * Hq + g * G) * 64 + d2;
     for (int j0 = 0; j0 < G; j0 += 8) {  // up to eight independent loads in flight
       __nv_bfloat162 v[8];
@@ -33,14 +35,18 @@ __global__ void __launch_bounds__(256) qmean_kernel(const __nv_bfloat162* __rest
         }
     }
   }
-  __shared__ float2 part[4][64];
+  __shared__ float2 part[QM_SLICES][64];
   __shared__ float red[2];
   part[slice][d2] = make_float2(sx, sy);
   __syncthreads();
   if (threadIdx.x < 64) {
     const float inv = (float)((n1 - n0) * G);
-    float ax = (part[0][d2].x + part[1][d2].x) + (part[2][d2].x + part[3][d2].x);
-    float ay = (part[0][d2].y + part[1][d2].y) + (part[2][d2].y + part[3][d2].y);
+    float ax = 0.f, ay = 0.f;
+#pragma unroll
+    for (int i = 0; i < QM_SLICES; i += 4) {  // fixed order
+      ax += (part[i][d2].x + part[i + 1][d2].x) + (part[i + 2][d2].x + part[i + 3][d2].x);
+      ay += (part[i][d2].y + part[i + 1][d2].y) + (part[i + 2][d2].y + part[i + 3][d2].y);
+    }
     ax = __fdiv_rn(ax, inv);
     ay = __fdiv_rn(ay, inv);
     float* dst = qa + ((long long)l * maxQ + qi) * Dp + g * 128;
@@ -363,7 +369,7 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
   const StoreView& s = c->sv;
   const int maxQ = c->cfg.max_questions;
   const int nl = layer1 - layer0;
-  qmean_kernel<<<dim3(qb.nQ, nl, s.Hkv), 256, 0, st>>>((const __nv_bfloat162*)q, qb, s.Hq, s.Hkv, s.G, c->qa,
+  qmean_kernel<<<dim3(qb.nQ, nl, s.Hkv), QM_SLICES * 64, 0, st>>>((const __nv_bfloat162*)q, qb, s.Hq, s.Hkv, s.G, c->qa,
                                                       c->qnorm, maxQ, layer0);
   int q_group = (int)((96 * 1024) / (s.Dp * sizeof(float)));
   if (q_group > qb.nQ) q_group = qb.nQ;
@@ -514,7 +520,7 @@ extern "C" int rekv_score_frames_static(const void* q, const int32_t* cu_q, int 
 
   const int Dp = n_kv_heads * REKV_HEAD_DIM, G = n_q_heads / n_kv_heads;
   cudaStream_t st = (cudaStream_t)stream;
-  qmean_kernel<<<dim3(nQ, 1, n_kv_heads), 256, 0, st>>>((const __nv_bfloat162*)q, qb, n_q_heads, n_kv_heads, G, qa, qsq,
+  qmean_kernel<<<dim3(nQ, 1, n_kv_heads), QM_SLICES * 64, 0, st>>>((const __nv_bfloat162*)q, qb, n_q_heads, n_kv_heads, G, qa, qsq,
                                                          STATIC_MAX_QUESTIONS, 0);
   // the question vectors of one call fit in 64 KB of dynamic shared memory only in groups
   int q_group = (int)((96 * 1024) / (Dp * sizeof(float)));

@@ -131,3 +131,28 @@ def test_argument_and_state_errors():
         g.attend_full(q, ks2, vs2, cu, cus2)
     assert e.value.code == rekv.ERR_ARG
     g.close()
+
+
+@pytest.mark.parametrize("theta", THETAS)
+def test_stream_encoding_step_is_the_same_computation(theta):
+    """Eq. 1 (sliding-window encoding): O = Attn(W_Q X, [L_k, W_K X], [L_v, W_V X]) with L the local window of the
+    stored K/V and X the incoming chunk.  With nothing retrieved (top_k = 0) the context of rekv_gather is exactly
+    the last W frames, so the encode step of a new frame is rekv_gather + rekv_attend_full on the frame's own
+    Q/K/V, followed by rekv_append_frame."""
+    s = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=12, W=3, k=0, seed=540)
+    g = H.build_gpu(s, max_questions=1, max_q_tokens=s.Nf, max_self_tokens=s.Nf, rope_theta=theta, max_frames=s.T + 1)
+    o = H.build_oracle(s)
+    # the chunk X: one new frame's tokens (queries, keys, values as the decoder layer makes them)
+    q, cu = H.questions(s, [s.Nf], device="cuda", first_id=77)
+    kx, vx, cux = H.self_kv(s, [s.Nf], device="cuda", first_id=77)
+    idx = torch.empty((s.L, 1, 0), dtype=torch.int32, device="cuda")
+    assert g.gather(idx, 1, 0, s.T)[0] == s.W
+    out = g.attend_full(q, kx, vx, cu, cux)
+    g.check_status()
+    assert g.append_frame(kx, vx) == s.T  # the chunk's K/V join the store (same [L][N_f][H_kv][D] layout)
+    k_win, v_win = o.gather(torch.empty((s.L, 0), dtype=torch.int32), 0, s.T)
+    for l in range(s.L):
+        ref, _ = orc.attend_full(q[l].cpu().contiguous(), k_win[l].contiguous(), v_win[l].contiguous(),
+                                 kx[l].cpu().contiguous(), vx[l].cpu().contiguous(), theta)
+        H.assert_attention(out[l:l + 1], ref[None], f"encode step, layer {l}")
+    g.close()
