@@ -7,17 +7,12 @@
 // contiguous bulk copies (the store keeps them in the 128-byte-swizzled operand layout) and applied
 // to both row tiles.  Warp roles:
 //   warp 0      bulk copies of K/V tiles into a 3-deep shared-memory ring (one lane)
-//   warps 1,10  tcgen05.mma issue (one lane each) for row tile 0 / 1: S = Q K^T into TMEM, O += P V with
-//               P read from TMEM
+//   warp 1      tcgen05.mma issue (one lane): S = Q K^T into TMEM, O += P V with P read from TMEM
 //   warps 2-5   softmax of row tile 0: one thread per row (= TMEM lane), fp32, lazy rescaling of O
 //   warps 6-9   softmax of row tile 1 -- the two tiles alternate on the tensor core, so one tile's
 //               softmax overlaps the other's matrix products
-// TMEM (512 columns): O0 [0,128)  O1 [128,256)  and per row tile a 128-column region holding S (up to
-// 80 fp32 columns) and, beside it, P (bf16 pairs, up to 40 columns).  A frame of N_f tokens is
-// processed as token chunks of <= 80.  Because P does not overwrite S, a tile's softmax releases S as
-// soon as it has read it, and the next chunk's Q K^T is issued while that softmax is still computing
-// exponentials: the tensor core always has a product queued and the softmax chain carries no
-// matrix product.
+// TMEM (512 columns): O0 [0,128)  O1 [128,256)  S0/P0 [256,384)  S1/P1 [384,512); P (bf16) overwrites
+// the front of its S.  A frame of N_f tokens is processed as one or two token chunks of <= 128.
 // A range that does not cover a whole unit leaves (max, sum, O) partials for the combine kernel.
 // Every wait is bounded: on expiry the status word is set and the CTA leaves.
 #include "ptx_helpers.cuh"
@@ -25,30 +20,12 @@
 
 using namespace rekv_ptx;
 
-// Optional cycle-stamp tracing of CTA 0 (compile with -DREKV_TRACE; never part of the shipped library):
-// slot layout is [role][chunk][event]; rekv_trace_read copies the stamps out.
-#ifdef REKV_TRACE
-__device__ long long g_rekv_trace[4096];
-#define REKV_STAMP(role, i, ev)                                                                  \
-  do {                                                                                           \
-    if (blockIdx.x == 0 && lane == 0 && (i) < 64) g_rekv_trace[(role) * 1024 + (i) * 8 + (ev)] = clock64(); \
-  } while (0)
-extern "C" int rekv_trace_read(long long* host, int n) {
-  cudaDeviceSynchronize();
-  return (int)cudaMemcpyFromSymbol(host, g_rekv_trace, n * sizeof(long long));
-}
-#else
-#define REKV_STAMP(role, i, ev) do { } while (0)
-#endif
-
 namespace {
 
-constexpr int TC_THREADS = 352;
+constexpr int TC_THREADS = 320;
 constexpr int KV_BUFS = 3;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t Q_TILE_BYTES = 128 * 256;  // 128 rows x 128 dims bf16
-constexpr uint32_t P_COL = 80;                // P sits beside S inside a tile's 128-column region
-constexpr int MAX_PARTS = 4;                  // token chunks per frame (N_f <= 256)
 constexpr float RESCALE_THRESHOLD = 8.f;      // log2 units: O is rescaled only when the row max grows by > 2^8
 
 struct TcParams {
@@ -63,8 +40,7 @@ struct TcParams {
   float* part_ml;
   int* status;
   QBatch qb;
-  int Hq, Hkv, G, Nf, Npad, cpf, ncf, MP, layer0;
-  int part_tok0[MAX_PARTS], part_n[MAX_PARTS];  // token chunks of a frame: first token, tokens (multiple of 16, <= 80)
+  int Hq, Hkv, G, Nf, Npad, NA, NB, ncf, MP, layer0;
   int per;          // (unit, frame) steps per CTA
   long long total;  // units * ncf
   float scale_log2;
@@ -95,7 +71,7 @@ __device__ __forceinline__ UnitInfo decode_unit(const TcParams& p, long long u) 
   return ui;
 }
 
-// barrier slots after the K/V ring: full[b], empty[b], s_full[t], p_ready[t], pv_done[t], s_free[t]
+// barrier slots after the K/V ring: full[b], empty[b], s_full[t], p_ready[t], pv_done[t]
 struct Bars {
   uint32_t base;
   __device__ __forceinline__ uint32_t full(uint32_t b) const { return base + 8 * b; }
@@ -103,7 +79,6 @@ struct Bars {
   __device__ __forceinline__ uint32_t s_full(uint32_t t) const { return base + 8 * (2 * KV_BUFS + t); }
   __device__ __forceinline__ uint32_t p_ready(uint32_t t) const { return base + 8 * (2 * KV_BUFS + 2 + t); }
   __device__ __forceinline__ uint32_t pv_done(uint32_t t) const { return base + 8 * (2 * KV_BUFS + 4 + t); }
-  __device__ __forceinline__ uint32_t s_free(uint32_t t) const { return base + 8 * (2 * KV_BUFS + 6 + t); }
 };
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -124,7 +99,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   const uint32_t s_bar = s_kv + KV_BUFS * tile_bytes;
   Bars bars;
   bars.base = s_bar;
-  volatile uint32_t* s_tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + (s_bar - s_base) + 8 * (2 * KV_BUFS + 8));
+  volatile uint32_t* s_tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + (s_bar - s_base) + 8 * (2 * KV_BUFS + 6));
   volatile uint32_t* s_abort = s_tmem_slot + 1;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -144,13 +119,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   if (tid == 0) {
     for (int i = 0; i < KV_BUFS; ++i) {
       mbar_init(bars.full(i), 1);
-      mbar_init(bars.empty(i), 2);  // one release per row-tile issuer
+      mbar_init(bars.empty(i), 1);
     }
     for (int t = 0; t < 2; ++t) {
       mbar_init(bars.s_full(t), 1);
       mbar_init(bars.p_ready(t), 4);  // one arrival per softmax warp
       mbar_init(bars.pv_done(t), 1);
-      mbar_init(bars.s_free(t), 4);   // one arrival per softmax warp
     }
     *s_abort = 0;
     fence_barrier_init();
@@ -181,7 +155,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     return false;
   };
 
-  const int cpf = p.cpf;                            // token chunks per frame
+  const int cpf = p.NB > 0 ? 2 : 1;                 // token chunks per frame
   const uint32_t half_bytes = (uint32_t)p.Nf * 128u;
   const uint32_t idesc_pv = idesc_bf16(128, 128, 1);
 
@@ -201,7 +175,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     const bool whole_unit = (nfr == p.ncf);
 
     // ---- Q row tiles -> shared memory in the swizzled K-major operand layout -------------------
-    if (warp >= 2 && warp < 10) {
+    if (warp >= 2) {
       const int t = (warp - 2) >> 2;
       const int row = ((warp & 3) << 5) | lane;
       if (t < ui.tiles) {
@@ -247,101 +221,74 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         }
         if (stop || *s_abort) break;
       }
-    } else if (warp == 1 || warp == 10) {
-      // ================= MMA issuers: warp 1 for row tile 0, warp 10 for row tile 1 =================
-      // Warp-uniform code; one elected lane issues.  Descriptors are built once per chunk; per
-      // instruction only the 14-bit start-address field advances.  Per tile: the next chunk's
-      // S = Q K^T is issued as soon as the tile's softmax group has read the current S, then the current
-      // chunk's O += P V once P is ready.  Each issuer releases a K/V ring tile after its last use; a
-      // unit with a single row tile leaves tile 1's issuer only the releases.
-      const int t = warp == 1 ? 0 : 1;
-      const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);  // SBO = 1024 B, version, SWIZZLE_128B
-      const uint32_t lbo_v = ((half_stride >> 4) & 0x3FFFu) << 16;      // pitch of V's two 64-dim blocks
-      const uint32_t lbo_k = 1u << 16;                                  // unused for K-major operands
-      const uint32_t half16 = half_stride >> 4;
-      const bool active = t < ui.tiles;
-      bool ok = true;
+    } else if (warp == 1) {
+      // ================= MMA issuer =================
+      // Descriptors are built once; per instruction only the 14-bit start-address field advances.
+      {
+        const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);  // SBO = 1024 B, version, SWIZZLE_128B
+        const uint32_t lbo_v = ((half_stride >> 4) & 0x3FFFu) << 16;      // pitch of V's two 64-dim blocks
+        const uint32_t lbo_k = 1u << 16;                                  // unused for K-major operands
+        const uint32_t half16 = half_stride >> 4;
+        const int tiles = ui.tiles;
+        bool ok = true;
 #define REKV_DESC(lo) (((uint64_t)desc_hi << 32) | (uint64_t)(lo))
-      uint32_t k_buf = ring % KV_BUFS, k_use = ring / KV_BUFS;              // K tile of the S stream
-      uint32_t v_buf = (ring + 1) % KV_BUFS, v_use = (ring + 1) / KV_BUFS;  // V tile of the P V stream
-      int s_part = 0, v_part = 0;
-      const uint32_t q_lo = ((s_q + t * Q_TILE_BYTES) >> 4) | lbo_k;
-      const uint32_t d_s = tmem + col_s(t), d_o = tmem + col_o(t), a_p = tmem + col_s(t) + P_COL;
-      auto issue_s = [&]() {
-        if (s_part == 0) ok = wait(bars.full(k_buf), k_use & 1);
-        if (!ok) return;
-        tc_fence_after();
-        const uint32_t k_lo = ((s_kv + k_buf * tile_bytes + (uint32_t)p.part_tok0[s_part] * 128u) >> 4) | lbo_k;
-        const uint32_t idesc = idesc_bf16(128, (uint32_t)p.part_n[s_part], 0);
-        const bool last_part = s_part == cpf - 1;
-        if (elect_one()) {
-          if (active) {
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk) mma_ss(d_s, REKV_DESC(q_lo + 2 * kk), REKV_DESC(k_lo + 2 * kk), idesc, kk > 0);
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              mma_ss(d_s, REKV_DESC(q_lo + (Q_TILE_BYTES / 32) + 2 * kk), REKV_DESC(k_lo + half16 + 2 * kk), idesc, 1);
-            tc_commit(bars.s_full(t));
+#define REKV_ISSUE_S(T, I)                                                                                    \
+  do {                                                                                                        \
+    const int fi_ = (I) / cpf, part_ = (I) - fi_ * cpf;                                                       \
+    const uint32_t r_ = ring + 2 * fi_, b_ = r_ % KV_BUFS;                                                    \
+    const uint32_t tok0_ = part_ ? p.NA : 0, N_ = part_ ? p.NB : p.NA;                                        \
+    if (part_ == 0 && (T) == 0) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                                 \
+    if (ok) {                                                                                                 \
+      tc_fence_after();                                                                                       \
+      const uint32_t k_lo = ((s_kv + b_ * tile_bytes + tok0_ * 128u) >> 4) | lbo_k;                           \
+      const uint32_t q_lo = ((s_q + (T) * Q_TILE_BYTES) >> 4) | lbo_k;                                        \
+      const uint32_t idesc_ = idesc_bf16(128, N_, 0);                                                         \
+      const uint32_t d_ = tmem + col_s(T);                                                                    \
+      if (elect_one()) {                                                                                      \
+      _Pragma("unroll") for (int kk = 0; kk < 4; ++kk)                                                        \
+          mma_ss(d_, REKV_DESC(q_lo + 2 * kk), REKV_DESC(k_lo + 2 * kk), idesc_, kk > 0);                     \
+      _Pragma("unroll") for (int kk = 0; kk < 4; ++kk)                                                        \
+          mma_ss(d_, REKV_DESC(q_lo + (Q_TILE_BYTES / 32) + 2 * kk), REKV_DESC(k_lo + half16 + 2 * kk), idesc_, 1); \
+      tc_commit(bars.s_full(T));                                                                              \
+      if (part_ == cpf - 1 && (T) == tiles - 1) tc_commit(bars.empty(b_)); /* K tile no longer needed */      \
+      }                                                                                                       \
+      __syncwarp();                                                                                           \
+    }                                                                                                         \
+  } while (0)
+#define REKV_ISSUE_PV(T, I)                                                                                   \
+  do {                                                                                                        \
+    const int fi_ = (I) / cpf, part_ = (I) - fi_ * cpf;                                                       \
+    const uint32_t r_ = ring + 2 * fi_ + 1, b_ = r_ % KV_BUFS;                                                \
+    const uint32_t tok0_ = part_ ? p.NA : 0, nk_ = (part_ ? p.NB : p.NA) >> 4;                                \
+    if (part_ == 0 && (T) == 0) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                                 \
+    if (ok) ok = wait(bars.p_ready(T), (chunk_cnt[T] + (I)) & 1);                                             \
+    if (ok) {                                                                                                 \
+      tc_fence_after();                                                                                       \
+      const uint32_t v_lo = ((s_kv + b_ * tile_bytes + tok0_ * 128u) >> 4) | lbo_v;                           \
+      const uint32_t d_ = tmem + col_o(T), a_ = tmem + col_s(T);                                              \
+      if (elect_one()) {                                                                                      \
+      _Pragma("unroll") for (int kk = 0; kk < 8; ++kk)                                                        \
+          if (kk < (int)nk_) mma_ts(d_, a_ + 8 * kk, REKV_DESC(v_lo + 128 * kk), idesc_pv, ((I) > 0) | (kk > 0)); \
+      tc_commit(bars.pv_done(T));                                                                             \
+      if (part_ == cpf - 1 && (T) == tiles - 1) tc_commit(bars.empty(b_)); /* V tile no longer needed */      \
+      }                                                                                                       \
+      __syncwarp();                                                                                           \
+    }                                                                                                         \
+  } while (0)
+        REKV_ISSUE_S(0, 0);
+        if (tiles == 2 && ok) REKV_ISSUE_S(1, 0);
+        for (int i = 0; i < nchunks && ok; ++i) {
+          REKV_ISSUE_PV(0, i);
+          if (i + 1 < nchunks && ok) REKV_ISSUE_S(0, i + 1);
+          if (tiles == 2 && ok) {
+            REKV_ISSUE_PV(1, i);
+            if (i + 1 < nchunks && ok) REKV_ISSUE_S(1, i + 1);
           }
-          if (last_part) tc_commit(bars.empty(k_buf));  // this tile no longer needs the K tile
         }
-        __syncwarp();
-        if (last_part) {
-          s_part = 0;
-          k_buf += 2;
-          if (k_buf >= KV_BUFS) {
-            k_buf -= KV_BUFS;
-            ++k_use;
-          }
-        } else {
-          ++s_part;
-        }
-      };
-      auto issue_pv = [&](const int i) {
-        if (v_part == 0) ok = wait(bars.full(v_buf), v_use & 1);
-        if (ok && active) ok = wait(bars.p_ready(t), (chunk_cnt[t] + i) & 1);
-        if (!ok) return;
-        tc_fence_after();
-        const uint32_t v_lo = ((s_kv + v_buf * tile_bytes + (uint32_t)p.part_tok0[v_part] * 128u) >> 4) | lbo_v;
-        const int nk = p.part_n[v_part] >> 4;
-        const bool last_part = v_part == cpf - 1;
-        if (elect_one()) {
-          if (active) {
-#pragma unroll
-            for (int kk = 0; kk < 5; ++kk)
-              if (kk < nk) mma_ts(d_o, a_p + 8 * kk, REKV_DESC(v_lo + 128 * kk), idesc_pv, (i > 0) | (kk > 0));
-            tc_commit(bars.pv_done(t));
-          }
-          if (last_part) tc_commit(bars.empty(v_buf));  // this tile no longer needs the V tile
-        }
-        __syncwarp();
-        if (last_part) {
-          v_part = 0;
-          v_buf += 2;
-          if (v_buf >= KV_BUFS) {
-            v_buf -= KV_BUFS;
-            ++v_use;
-          }
-        } else {
-          ++v_part;
-        }
-      };
-      // Tile 1 starts about half a chunk after tile 0 (once tile 0's softmax has read its first S), so
-      // that the two tiles' exponential phases interleave instead of colliding on the same unit.
-      if (t == 1 && active) ok = wait(bars.s_free(0), chunk_cnt[0] & 1);
-      if (ok) issue_s();
-      for (int i = 0; i < nchunks && ok; ++i) {
-        if (t == 0) REKV_STAMP(0, i, 0);
-        if (i + 1 < nchunks) {
-          if (active) ok = wait(bars.s_free(t), (chunk_cnt[t] + i) & 1);
-          if (t == 0) REKV_STAMP(0, i, 1);
-          if (ok) issue_s();
-        }
-        if (t == 0) REKV_STAMP(0, i, 2);
-        if (ok) issue_pv(i);
-        if (t == 0) REKV_STAMP(0, i, 3);
-      }
+#undef REKV_ISSUE_S
+#undef REKV_ISSUE_PV
 #undef REKV_DESC
+      }
       __syncwarp();
     } else {
       // ================= softmax + output, one thread per row =================
@@ -355,108 +302,152 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         bool ok = true;
         for (int i = 0; i < nchunks && ok; ++i) {
           const int part = i % cpf;
-          const int tok0 = p.part_tok0[part], N = p.part_n[part];
+          const int tok0 = part ? p.NA : 0, N = part ? p.NB : p.NA;
           const int nv = min(N, p.Nf - tok0);  // valid tokens of this chunk
-          const int npc = N >> 4;              // 16-column pieces (<= 5)
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 0);
+          const int npc = N >> 4;
           if (!wait(bars.s_full(t), (chunk_cnt[t] + i) & 1)) {
             ok = false;
             break;
           }
           tc_fence_after();
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 1);
-          // read the whole S row chunk, then hand S back: the next chunk's Q K^T may overwrite it now
-          uint32_t sv[5][16];
-#pragma unroll
-          for (int pc = 0; pc < 5; ++pc)
-            if (pc < npc) tmem_ld16(t_s + pc * 16, sv[pc]);
-#pragma unroll
-          for (int pc = 0; pc < 5; ++pc)
-            if (pc < npc) tmem_wait_ld16(sv[pc]);
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bars.s_free(t));
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 2);
-          // row maximum over the valid tokens
+          // Online softmax, one pass over S.  S is read from TMEM in groups of two 16-column pieces,
+          // the next group's load in flight while the current one is processed.  A group whose
+          // scaled maximum exceeds the maximum in use by more than the threshold (always the very
+          // first group) raises it: P pieces already written for this chunk, this chunk's partial
+          // sums, the running sum and O are rescaled by 2^(m_old - m_new).  This is rare after the
+          // first chunk, so the common path has no second read of S and no rescaling.
           const float NEG_INF = -INFINITY;
-          float g0 = NEG_INF, g1 = NEG_INF, g2 = NEG_INF, g3 = NEG_INF;
-#pragma unroll
-          for (int pc = 0; pc < 5; ++pc)
-            if (pc < npc) {
-              if (pc * 16 + 16 > nv) {  // the frame's ragged end: mask the pad tokens
-#pragma unroll
-                for (int j = 0; j < 16; ++j)
-                  if (pc * 16 + j >= nv) sv[pc][j] = __float_as_uint(NEG_INF);
-              }
-              g0 = max3(g0, __uint_as_float(sv[pc][0]), __uint_as_float(sv[pc][1]));
-              g1 = max3(g1, __uint_as_float(sv[pc][2]), __uint_as_float(sv[pc][3]));
-              g2 = max3(g2, __uint_as_float(sv[pc][4]), __uint_as_float(sv[pc][5]));
-              g3 = max3(g3, __uint_as_float(sv[pc][6]), __uint_as_float(sv[pc][7]));
-              g0 = max3(g0, __uint_as_float(sv[pc][8]), __uint_as_float(sv[pc][9]));
-              g1 = max3(g1, __uint_as_float(sv[pc][10]), __uint_as_float(sv[pc][11]));
-              g2 = max3(g2, __uint_as_float(sv[pc][12]), __uint_as_float(sv[pc][13]));
-              g3 = max3(g3, __uint_as_float(sv[pc][14]), __uint_as_float(sv[pc][15]));
-            }
-          const float gm = fmaxf(fmaxf(g0, g1), fmaxf(g2, g3)) * p.scale_log2;
-          // lazy rescaling: the maximum in use is raised only when exceeded by more than the threshold
-          // (always on the first chunk); O and the running sum then shrink by 2^(old - new)
-          const bool need = gm > m_used + RESCALE_THRESHOLD;
-          const float alpha = need ? ex2(m_used - gm) : 1.f;
-          if (need) m_used = gm;
-          const bool any_need = __any_sync(0xffffffffu, need);
-          // P = 2^(S*scale - m) as bf16 pairs (S registers are reused), row sum in fp32
-          const float neg_m = -m_used;
           float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
+          auto do_group = [&](uint32_t (&a)[16], uint32_t (&b)[16], const int pc0) {
+            const bool has_b = pc0 + 1 < npc;
+            if (pc0 * 16 + 32 > nv) {  // the group that holds the frame's ragged end: mask the pad tokens
 #pragma unroll
-          for (int pc = 0; pc < 5; ++pc)
-            if (pc < npc) {
+              for (int j = 0; j < 16; ++j) {
+                if (pc0 * 16 + j >= nv) a[j] = __float_as_uint(NEG_INF);
+                if (pc0 * 16 + 16 + j >= nv) b[j] = __float_as_uint(NEG_INF);
+              }
+            }
+            float g0 = max3(__uint_as_float(a[0]), __uint_as_float(a[1]), __uint_as_float(a[2]));
+            float g1 = max3(__uint_as_float(a[3]), __uint_as_float(a[4]), __uint_as_float(a[5]));
+            float g2 = max3(__uint_as_float(a[6]), __uint_as_float(a[7]), __uint_as_float(a[8]));
+            float g3 = max3(__uint_as_float(a[9]), __uint_as_float(a[10]), __uint_as_float(a[11]));
+            g0 = max3(g0, __uint_as_float(a[12]), __uint_as_float(a[13]));
+            g1 = max3(g1, __uint_as_float(a[14]), __uint_as_float(a[15]));
+            if (has_b) {
+              g2 = max3(g2, __uint_as_float(b[0]), __uint_as_float(b[1]));
+              g3 = max3(g3, __uint_as_float(b[2]), __uint_as_float(b[3]));
+              g0 = max3(g0, __uint_as_float(b[4]), __uint_as_float(b[5]));
+              g1 = max3(g1, __uint_as_float(b[6]), __uint_as_float(b[7]));
+              g2 = max3(g2, __uint_as_float(b[8]), __uint_as_float(b[9]));
+              g3 = max3(g3, __uint_as_float(b[10]), __uint_as_float(b[11]));
+              g0 = max3(g0, __uint_as_float(b[12]), __uint_as_float(b[13]));
+              g1 = max3(g1, __uint_as_float(b[14]), __uint_as_float(b[15]));
+            }
+            const float gm = fmaxf(fmaxf(g0, g1), fmaxf(g2, g3)) * p.scale_log2;
+            const bool need = gm > m_used + RESCALE_THRESHOLD;
+            if (__any_sync(0xffffffffu, need)) {
+              const float alpha = need ? ex2(m_used - gm) : 1.f;  // 0 when nothing has been seen yet
+              if (need) m_used = gm;
+#pragma unroll 1
+              for (int q = 0; q < pc0; ++q) {  // P pieces of this chunk written under the old maximum
+                uint32_t w[8];
+                tmem_ld8(t_s + q * 8, w);
+                tmem_wait_ld8(w);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  const float lo = __uint_as_float(w[e] << 16) * alpha, hi = __uint_as_float(w[e] & 0xFFFF0000u) * alpha;
+                  w[e] = pack_bf16(lo, hi);
+                }
+                tmem_st8(t_s + q * 8, w);
+              }
+              l_sum *= alpha;
+              ps0 *= alpha;
+              ps1 *= alpha;
+              ps2 *= alpha;
+              ps3 *= alpha;
+              if (i > 0) {  // O holds earlier chunks; their P V is complete (this chunk's S came after it)
+#pragma unroll 1
+                for (int pc = 0; pc < 8; ++pc) {
+                  uint32_t o[16];
+                  tmem_ld16(t_o + pc * 16, o);
+                  tmem_wait_ld16(o);
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+                  tmem_st16(t_o + pc * 16, o);
+                }
+              }
+            }
+            const float neg_m = -m_used;
+            uint32_t pk[8];
+#pragma unroll
+            for (int jj = 0; jj < 8; jj += 2) {
+              const float p0 = ex2(fmaf(__uint_as_float(a[2 * jj]), p.scale_log2, neg_m));
+              const float p1 = ex2(fmaf(__uint_as_float(a[2 * jj + 1]), p.scale_log2, neg_m));
+              const float p2 = ex2(fmaf(__uint_as_float(a[2 * jj + 2]), p.scale_log2, neg_m));
+              const float p3 = ex2(fmaf(__uint_as_float(a[2 * jj + 3]), p.scale_log2, neg_m));
+              ps0 += p0;
+              ps1 += p1;
+              ps2 += p2;
+              ps3 += p3;
+              pk[jj] = pack_bf16(p0, p1);
+              pk[jj + 1] = pack_bf16(p2, p3);
+            }
+            tmem_st8(t_s + pc0 * 8, pk);
+            if (has_b) {
 #pragma unroll
               for (int jj = 0; jj < 8; jj += 2) {
-                const float p0 = ex2(fmaf(__uint_as_float(sv[pc][2 * jj]), p.scale_log2, neg_m));
-                const float p1 = ex2(fmaf(__uint_as_float(sv[pc][2 * jj + 1]), p.scale_log2, neg_m));
-                const float p2 = ex2(fmaf(__uint_as_float(sv[pc][2 * jj + 2]), p.scale_log2, neg_m));
-                const float p3 = ex2(fmaf(__uint_as_float(sv[pc][2 * jj + 3]), p.scale_log2, neg_m));
+                const float p0 = ex2(fmaf(__uint_as_float(b[2 * jj]), p.scale_log2, neg_m));
+                const float p1 = ex2(fmaf(__uint_as_float(b[2 * jj + 1]), p.scale_log2, neg_m));
+                const float p2 = ex2(fmaf(__uint_as_float(b[2 * jj + 2]), p.scale_log2, neg_m));
+                const float p3 = ex2(fmaf(__uint_as_float(b[2 * jj + 3]), p.scale_log2, neg_m));
                 ps0 += p0;
                 ps1 += p1;
                 ps2 += p2;
                 ps3 += p3;
-                sv[pc][jj] = pack_bf16(p0, p1);
-                sv[pc][jj + 1] = pack_bf16(p2, p3);
+                pk[jj] = pack_bf16(p0, p1);
+                pk[jj + 1] = pack_bf16(p2, p3);
               }
+              tmem_st8(t_s + (pc0 + 1) * 8, pk);
             }
-          l_sum = l_sum * alpha + (ps0 + ps1) + (ps2 + ps3);
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 3);
-          // the previous chunk's P V must be complete before P is overwritten or O is rescaled
-          if (i > 0) {
-            if (!wait(bars.pv_done(t), (chunk_cnt[t] + i - 1) & 1)) {
-              ok = false;
-              break;
+          };
+          {
+            uint32_t a0[16], a1[16], b0[16], b1[16];
+            tmem_ld16(t_s, a0);
+            if (npc > 1) {
+              tmem_ld16(t_s + 16, a1);
+              tmem_wait_ld16(a1);
             }
-            tc_fence_after();
-            if (any_need) {
-#pragma unroll 1
-              for (int pc = 0; pc < 8; ++pc) {
-                uint32_t o[16];
-                tmem_ld16(t_o + pc * 16, o);
-                tmem_wait_ld16(o);
+            tmem_wait_ld16(a0);
 #pragma unroll
-                for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-                tmem_st16(t_o + pc * 16, o);
+            for (int h = 0; h < 2; ++h) {
+              const int pa = 4 * h, pb = 4 * h + 2;
+              if (pa < npc) {
+                if (pb < npc) {  // next group in flight while this one is processed
+                  tmem_ld16(t_s + pb * 16, b0);
+                  if (pb + 1 < npc) tmem_ld16(t_s + (pb + 1) * 16, b1);
+                }
+                do_group(a0, a1, pa);
+                if (pb < npc) {
+                  if (pb + 1 < npc) tmem_wait_ld16(b1);
+                  tmem_wait_ld16(b0);
+                  if (pa + 4 < npc) {
+                    tmem_ld16(t_s + (pa + 4) * 16, a0);
+                    if (pa + 5 < npc) tmem_ld16(t_s + (pa + 5) * 16, a1);
+                  }
+                  do_group(b0, b1, pb);
+                  if (pa + 4 < npc) {
+                    if (pa + 5 < npc) tmem_wait_ld16(a1);
+                    tmem_wait_ld16(a0);
+                  }
+                }
               }
             }
           }
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 4);
-#pragma unroll
-          for (int pc = 0; pc < 5; ++pc)
-            if (pc < npc) {
-              const uint32_t pk[8] = {sv[pc][0], sv[pc][1], sv[pc][2], sv[pc][3], sv[pc][4], sv[pc][5], sv[pc][6], sv[pc][7]};
-              tmem_st8(t_s + P_COL + pc * 8, pk);
-            }
+          l_sum += (ps0 + ps1) + (ps2 + ps3);
           tmem_wait_st();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bars.p_ready(t));
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 5);
         }
         // ---- output of this range: final rows, or a partial for the combine kernel ----
         if (ok && wait(bars.pv_done(t), (chunk_cnt[t] + nchunks - 1) & 1)) {
@@ -630,17 +621,12 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   p.G = s.G;
   p.Nf = s.Nf;
   p.Npad = (s.Nf + 15) & ~15;
-  {  // token chunks of at most 80, as even as multiples of 16 allow (196 tokens -> 80 + 64 + 64)
-    const int units = p.Npad / 16;
-    p.cpf = (units + 4) / 5;
-    const int base = units / p.cpf, rem = units % p.cpf;
-    int tok = 0;
-    for (int i = 0; i < MAX_PARTS; ++i) {
-      const int n = i < p.cpf ? (base + (i < rem ? 1 : 0)) * 16 : 0;
-      p.part_tok0[i] = tok;
-      p.part_n[i] = n;
-      tok += n;
-    }
+  if (p.Npad <= 128) {  // token chunks of at most 128, two per frame beyond that (196 tokens -> 112 + 96)
+    p.NA = p.Npad;
+    p.NB = 0;
+  } else {
+    p.NA = ((p.Npad / 2) + 15) & ~15;
+    p.NB = p.Npad - p.NA;
   }
   p.ncf = ncf;
   p.layer0 = layer0;
@@ -660,7 +646,7 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     p.per = (int)((p.total + grid - 1) / grid);
     grid = (p.total + p.per - 1) / p.per;
   }
-  const size_t smem = 2 * Q_TILE_BYTES + (size_t)KV_BUFS * 2 * p.Npad * 128 + 8 * (2 * KV_BUFS + 8) + 16 + 1024;
+  const size_t smem = 2 * Q_TILE_BYTES + (size_t)KV_BUFS * 2 * p.Npad * 128 + 8 * (2 * KV_BUFS + 6) + 16 + 1024;
   if (smem > 227 * 1024) return cudaErrorInvalidValue;
   static bool attr_set = false;
   if (!attr_set) {
