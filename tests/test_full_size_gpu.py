@@ -42,7 +42,7 @@ def _oracle_layer(s: H.Shape, layer: int, n_frames: int) -> torch.Tensor:
     return reps
 
 
-def _sampled_parity(g: rekv.ReKV, s: H.Shape, lengths, layers, n_visible, first_qid=0):
+def _sampled_parity(g: rekv.ReKV, s: H.Shape, lengths, layers, n_visible, first_qid=0, widened=False):
     nQ = len(lengths)
     q_gpu, cu = H.questions(s, lengths, device="cuda", first_id=first_qid)
     q_cpu = q_gpu.cpu()
@@ -80,19 +80,60 @@ def _sampled_parity(g: rekv.ReKV, s: H.Shape, lengths, layers, n_visible, first_
             r = H.assert_attention(out[l, cu[i]:cu[i + 1]], o, f"attention l{l} q{i}")
             worst = tuple(max(a, b) for a, b in zip(worst, r))
     del k_ctx, v_ctx
+    if widened:
+        worst_full = _widened_rows(g, s, lengths, layers, n_visible, q_gpu, cu, idx, idx_mix, ref, k_eff, out)
+        return worst, worst_full
+    return worst
+
+
+def _widened_rows(g, s, lengths, layers, n_visible, q_gpu, cu, idx, idx_mix, ref, k_eff, out_plain):
+    """The rows built beyond the five steps, at the same full size: the layer-sequential calls against the
+    all-layer result, and Eq. 3 in full (own K/V, rotary embedding at consecutive positions) against the oracle
+    in the sampled layers, on the oracle's selection."""
+    nQ = len(lengths)
+    q_cpu = q_gpu.cpu()
+    # layer-sequential calls use the library's own selection: same indices, same attention where it is the oracle's
+    for l in layers:
+        idx_l = torch.empty((nQ, s.k), dtype=torch.int32, device="cuda")
+        out_l = g.question_layer(l, q_gpu[l], cu, s.k, n_visible, idx=idx_l)
+        assert torch.equal(idx_l, idx[l])
+        if torch.equal(idx[l], idx_mix[l]):
+            d = (out_l.float() - out_plain[l].float()).abs()
+            assert d.max().item() <= 4e-3, f"layer call differs from the all-layer call in layer {l}: {d.max().item()}"
+    g.check_status()
+    # Eq. 3 in full
+    ks, vs, cus = H.self_kv(s, lengths, device="cuda")
+    g.gather(idx_mix, nQ, s.k, n_visible)
+    out = g.attend_full(q_gpu, ks, vs, cu, cus)
+    g.check_status()
+    theta = float(g.cfg.rope_theta)
+    worst = (0.0, 0.0, 0.0)
+    for l in layers:
+        for i in range(nQ):
+            frames = ref[(l, i)][:k_eff].tolist() + list(range(n_visible - min(s.W, n_visible), n_visible))
+            ck = torch.stack([synth.frame(s.seed, synth.K, f, 1, s.Nf, s.Hkv, s.D, s.off_scale, layer0=l)[0] for f in frames])
+            cv = torch.stack([synth.frame(s.seed, synth.V, f, 1, s.Nf, s.Hkv, s.D, s.off_scale, layer0=l)[0] for f in frames])
+            sub = torch.arange(k_eff, dtype=torch.int32)
+            kc = orc.gather(ck.contiguous(), sub, k_eff, len(frames), min(s.W, n_visible))
+            vc = orc.gather(cv.contiguous(), sub, k_eff, len(frames), min(s.W, n_visible))
+            o, _ = orc.attend_full(q_cpu[l, cu[i]:cu[i + 1]].contiguous(), kc, vc, ks[l, cus[i]:cus[i + 1]].cpu().contiguous(),
+                                   vs[l, cus[i]:cus[i + 1]].cpu().contiguous(), theta)
+            r = H.assert_attention(out[l, cu[i]:cu[i + 1]], o, f"Eq. 3 in full l{l} q{i}")
+            worst = tuple(max(a, b) for a, b in zip(worst, r))
     return worst
 
 
 def test_config2_7b_hbm_resident_1800_frames():
     """28 layers, 28/4 heads, 1800 x 196-token frames (20.2 GB in HBM), question 32, window 8, top-k 64."""
     s = H.Shape(L=28, Hq=28, Hkv=4, Nf=196, T=1800, W=8, k=64, seed=2503)
-    g = rekv.ReKV(s.L, s.Hq, s.Hkv, s.D, s.Nf, s.T, s.W, max_q_tokens=32, max_topk=64, flags=rekv.FLAG_TIMING)
+    g = rekv.ReKV(s.L, s.Hq, s.Hkv, s.D, s.Nf, s.T, s.W, max_q_tokens=32, max_topk=64, flags=rekv.FLAG_TIMING,
+                  max_self_tokens=32, rope_theta=1e6)
     _fill(g, s, s.T)
     st = g.stats()
     assert st.kv_bytes_hbm == st.kv_bytes_logical == rekv.kv_cache_bytes(28, 1800, 196, 4, 128)
     assert round(st.kv_bytes_logical / 2**30, 1) == 18.8  # the appendix's worked value
-    worst = _sampled_parity(g, s, [32], layers=[0, 13, 27], n_visible=s.T)
-    print("config 2 attention max/mean/rel:", worst)
+    worst, worst_full = _sampled_parity(g, s, [32], layers=[0, 13, 27], n_visible=s.T, widened=True)
+    print("config 2 attention max/mean/rel:", worst, "Eq. 3 in full with rotary embedding:", worst_full)
     g.close()
 
 
