@@ -132,7 +132,7 @@ class ClockSampler:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch from the committed ncu capture
 # (profiles/), scaled to the full workload by the layers processed; None where no capture exists.
-TRAFFIC_NCU = {"7b_hbm_1800f": 857.0e6}
+TRAFFIC_NCU = {"7b_hbm_1800f": 857.0e6, "7b_hbm_decode_1tok": 825.0e6}
 
 
 def algorithmic_bytes(w, sum_nq=None, nQ=1):
@@ -537,7 +537,8 @@ def run_cuda(args, w):
         }
         if w["tail"] == 0:
             achieved = ab["attend_kernel"] / (att_kernel_us * 1e-6) / 1e9
-            line["roofline"] = {"kernel": "attend_tc5_kernel (step 5)", "bound": "hbm", "achieved": achieved,
+            line["roofline"] = {"kernel": ("attend_decode_kernel (step 5)" if max(lengths) * (w["Hq"] // w["Hkv"]) <= 16
+                                           else "attend_tc5_kernel (step 5)"), "bound": "hbm", "achieved": achieved,
                                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                                 "traffic": TRAFFIC_NCU.get(w["name"]), "peak_source": peaks["source"],
                                 "kernel_us": att_kernel_us,
