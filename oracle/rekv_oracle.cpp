@@ -344,6 +344,54 @@ void oracle_attend_full(const uint16_t* q, int n_q, int n_q_heads, int n_kv_head
   }
 }
 
+/* Quantised host tier (the paper's "Limitations and Future Work" names quantisation as the way to shrink the
+ * offloaded cache; no formula is given, this is the reading built here).  A page row -- the 128 dims of one
+ * token of one KV head, K or V -- is stored as 128 FP8 E4M3 codes (1 sign, 4 exponent bits with bias 7,
+ * 3 mantissa bits; largest finite value 448, subnormal step 2^-9, no infinities) and one float scale:
+ *   scale = amax / 448 (1 if the row is all zero), code = round-to-nearest-even(x / scale) saturated at +-448,
+ * and read back as bf16_rne(value(code) * scale).  oracle_e4m3_encode is that rounding for one float. */
+uint8_t oracle_e4m3_encode(float x) {
+  const uint8_t sign = std::signbit(x) ? 0x80 : 0x00;
+  double a = std::fabs((double)x);
+  if (!(a == a)) return (uint8_t)(sign | 0x7F);  // NaN
+  if (a >= 464.0) return (uint8_t)(sign | 0x7E); // beyond the midpoint above 448: saturates (so do 448..464)
+  if (a < std::ldexp(1.0, -6)) {                 // subnormal range: multiples of 2^-9
+    const double q = std::nearbyint(a * 512.0);  // ties to even (default rounding mode)
+    return (uint8_t)(sign | (uint8_t)q);         // q == 8 is the smallest normal, code 0x08
+  }
+  int e;
+  std::frexp(a, &e);                             // a = f * 2^e, f in [0.5, 1)
+  e -= 1;                                        // a = m * 2^e, m in [1, 2)
+  double m = std::nearbyint(std::ldexp(a, -e) * 8.0);  // 8..16
+  if (m == 16.0) {
+    m = 8.0;
+    e += 1;
+  }
+  if (e > 8 || (e == 8 && m > 14.0)) return (uint8_t)(sign | 0x7E);  // 448 = 1.75 * 2^8
+  return (uint8_t)(sign | ((uint8_t)(e + 7) << 3) | (uint8_t)(m - 8.0));
+}
+
+double oracle_e4m3_decode(uint8_t c) {
+  const int e = (c >> 3) & 0xF, m = c & 7;
+  const double v = e == 0 ? std::ldexp((double)m, -9) : std::ldexp(1.0 + m / 8.0, e - 7);
+  return (c & 0x80) ? -v : v;
+}
+
+/* rows x 128 bf16 in, the same shape out: each row through the quantised host tier and back. */
+void oracle_fp8_roundtrip(const uint16_t* x, long rows, int dim, uint16_t* out, float* scales /* nullable */) {
+  for (long r = 0; r < rows; ++r) {
+    float amax = 0.f;
+    for (int d = 0; d < dim; ++d) amax = std::max(amax, std::fabs((float)bf16_to_double(x[r * dim + d])));
+    const float scale = amax > 0.f ? amax / 448.0f : 1.0f;
+    if (scales) scales[r] = scale;
+    for (int d = 0; d < dim; ++d) {
+      const float v = (float)bf16_to_double(x[r * dim + d]);
+      const uint8_t c = oracle_e4m3_encode(v / scale);
+      out[r * dim + d] = float_to_bf16_rne((float)oracle_e4m3_decode(c) * scale);
+    }
+  }
+}
+
 /* Bytes of K/V cache for a stream: 2 (K and V) * L * T * M * H * D * bytes_per_element
  * (the appendix's cache-size expression; fp16/bf16 -> 2 bytes). */
 double oracle_kv_cache_bytes(int n_layers, long n_frames, int tokens_per_frame, int n_kv_heads, int head_dim,

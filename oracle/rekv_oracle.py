@@ -37,6 +37,12 @@ _lib.oracle_attend.restype = None
 _lib.oracle_score_external.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                        ctypes.c_double, ctypes.c_void_p]
 _lib.oracle_score_external.restype = None
+_lib.oracle_e4m3_encode.argtypes = [ctypes.c_float]
+_lib.oracle_e4m3_encode.restype = ctypes.c_uint8
+_lib.oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+_lib.oracle_e4m3_decode.restype = ctypes.c_double
+_lib.oracle_fp8_roundtrip.argtypes = [_u16p, ctypes.c_long, ctypes.c_int, _u16p, ctypes.c_void_p]
+_lib.oracle_fp8_roundtrip.restype = None
 _lib.oracle_rope.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_long, ctypes.c_double, ctypes.c_void_p]
 _lib.oracle_rope.restype = None
 _lib.oracle_attend_full.argtypes = [_u16p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, _u16p, _u16p,
@@ -172,6 +178,25 @@ def attend(q: torch.Tensor, k_ctx: torch.Tensor, v_ctx: torch.Tensor, want_probs
     _lib.oracle_attend(q.data_ptr(), n_q, n_qh, n_kv, d, k_ctx.data_ptr(), v_ctx.data_ptr(), n_ctx, out.data_ptr(),
                        out_b.data_ptr(), probs.data_ptr() if want_probs else None)
     return out, out_b, probs
+
+
+def e4m3_encode(x: float) -> int:
+    return int(_lib.oracle_e4m3_encode(x))
+
+
+def e4m3_decode(code: int) -> float:
+    return float(_lib.oracle_e4m3_decode(code))
+
+
+def fp8_roundtrip(x: torch.Tensor, want_scales: bool = False):
+    """x: bf16 [..., 128]: every row through the quantised host tier (E4M3 codes + one float scale) and back."""
+    _chk(x, torch.bfloat16)
+    d = x.shape[-1]
+    rows = x.numel() // d
+    out = torch.empty_like(x)
+    scales = torch.empty(rows, dtype=torch.float32) if want_scales else None
+    _lib.oracle_fp8_roundtrip(x.data_ptr(), rows, d, out.data_ptr(), scales.data_ptr() if want_scales else None)
+    return (out, scales) if want_scales else out
 
 
 def rope(x: torch.Tensor, pos: int, theta: float) -> torch.Tensor:

@@ -374,6 +374,53 @@ def test_external_retrieval_selection_is_tau_invariant_and_blocks_average_frames
     assert ib.tolist() == [j * b + f for j in top for f in range(b)] and kb == 8
 
 
+# ----------------------------------------------------------------------------- quantised host tier (FP8 E4M3)
+def test_e4m3_rounding_matches_the_format_and_the_library_conversion():
+    # every code decodes to the value the format defines, and encodes back to itself
+    for c in range(256):
+        if (c & 0x7F) == 0x7F:
+            continue  # NaN codes
+        v = orc.e4m3_decode(c)
+        e, m = (c >> 3) & 15, c & 7
+        ref = (m / 8 * 2.0 ** -6) if e == 0 else (1 + m / 8) * 2.0 ** (e - 7)
+        assert abs(v) == ref and (v < 0 or c < 128 or ref == 0)
+        if ref != 0:
+            assert orc.e4m3_encode(v) == c
+    assert orc.e4m3_decode(0x7E) == 448.0 and orc.e4m3_decode(0x08) == 2.0 ** -6 and orc.e4m3_decode(0x01) == 2.0 ** -9
+    # ties go to the even mantissa; beyond the largest value it saturates
+    assert orc.e4m3_decode(orc.e4m3_encode(1.0625)) == 1.0      # midway 1.0 / 1.125 -> even (1.0)
+    assert orc.e4m3_decode(orc.e4m3_encode(1.1875)) == 1.25     # midway 1.125 / 1.25 -> even (1.25)
+    assert orc.e4m3_decode(orc.e4m3_encode(2.0 ** -10)) == 0.0  # midway 0 / 2^-9 -> even (0)
+    assert orc.e4m3_decode(orc.e4m3_encode(3 * 2.0 ** -10)) == 2.0 ** -8
+    assert orc.e4m3_decode(orc.e4m3_encode(1e4)) == 448.0 and orc.e4m3_decode(orc.e4m3_encode(-460.0)) == -448.0
+    # the library's conversion (torch.float8_e4m3fn, round to nearest even) on a dense sweep of the finite range
+    g = torch.Generator().manual_seed(4)
+    x = torch.cat([torch.randn(20000, generator=g) * s for s in (1e-3, 0.02, 1.0, 30.0, 150.0)]).clamp(-448, 448)
+    lib = x.to(torch.float8_e4m3fn).float()
+    mine = torch.tensor([orc.e4m3_decode(orc.e4m3_encode(float(v))) for v in x.tolist()])
+    assert torch.equal(lib, mine)
+
+
+def test_fp8_roundtrip_of_page_rows():
+    g = torch.Generator().manual_seed(5)
+    x = bf16(torch.randn(64, 128, generator=g) * torch.logspace(-3, 2, 64)[:, None])
+    y, scales = orc.fp8_roundtrip(x, want_scales=True)
+    amax = x.float().abs().amax(dim=1)
+    assert torch.equal(scales, amax / 448.0)
+    # independent statement with the library's conversion
+    ref = ((x.float() / scales[:, None]).to(torch.float8_e4m3fn).float() * scales[:, None]).to(torch.bfloat16)
+    assert torch.equal(y, ref)
+    # the row's largest element survives exactly, every element within half a code step of its binade
+    idx = x.float().abs().argmax(dim=1)
+    assert torch.equal(y[torch.arange(64), idx], x[torch.arange(64), idx])
+    rel = ((y.float() - x.float()).abs() / amax[:, None]).max().item()
+    assert rel <= 16.0 / 448.0 + 2.0 ** -8     # half a code step of the top binade (32 / 2 of 448), plus the bf16 rounding
+    # an all-zero row stays zero (scale 1), and the operation is idempotent
+    z = bf16(torch.zeros(2, 128))
+    assert torch.equal(orc.fp8_roundtrip(z), z)
+    assert torch.equal(orc.fp8_roundtrip(y), y)
+
+
 # ----------------------------------------------------------------------------- Eq. 3 in full: X's own K/V, RoPE
 def _complex_rope(x: np.ndarray, pos: int, theta: float) -> np.ndarray:
     """RoFormer's definition: (x_i + i x_{i+D/2}) * exp(i * pos * theta^(-2i/D)), an independent statement."""
