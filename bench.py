@@ -49,6 +49,11 @@ WORKLOADS = {
                                  off_scale=0.5, tail=0, nQ=1, appends_per_step=1, ext_dim=1152, tau=0.07),
     "72b_offload_1800f": dict(L=80, Hq=64, Hkv=8, D=128, Nf=196, T=1800, W=8, k=32, Nq=64, seed=2503,
                               off_scale=0.5, tail=32, nQ=1, appends_per_step=1),
+    # the two offloaded configurations with the quantised host tier (FP8 E4M3 rows + scales cross the link)
+    "7b_offload_10800f_fp8": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=10800, W=8, k=64, Nq=32, seed=2503,
+                                  off_scale=0.5, tail=64, nQ=1, appends_per_step=1, host_fp8=True),
+    "72b_offload_1800f_fp8": dict(L=80, Hq=64, Hkv=8, D=128, Nf=196, T=1800, W=8, k=32, Nq=64, seed=2503,
+                                  off_scale=0.5, tail=32, nQ=1, appends_per_step=1, host_fp8=True),
 }
 WORKLOAD = dict(WORKLOADS["7b_hbm_1800f"], name="7b_hbm_1800f")
 N_ROTATE = 8  # distinct questions rotated through the timed steps
@@ -278,7 +283,8 @@ def run_cuda(args, w):
     w["Nq_total"] = cu[-1]
 
     g = rekv.ReKV(w["L"], w["Hq"], w["Hkv"], w["D"], w["Nf"], w["T"] + 8, w["W"], hbm_tail_frames=w["tail"],
-                  max_q_tokens=cu[-1], max_topk=w["k"], max_questions=nQ, device=local, flags=rekv.FLAG_TIMING,
+                  max_q_tokens=cu[-1], max_topk=w["k"], max_questions=nQ, device=local,
+                  flags=rekv.FLAG_TIMING | (rekv.FLAG_HOST_FP8 if w.get("host_fp8") else 0),
                   max_self_tokens=cu[-1] if w.get("full") else 0, rope_theta=w.get("rope_theta", 0.0),
                   ext_embed_dim=w.get("ext_dim", 0))
     kf = torch.empty((w["L"], w["Nf"], w["Hkv"], w["D"]), dtype=torch.bfloat16, device=dev)

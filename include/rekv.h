@@ -53,8 +53,14 @@ enum {
 /* rekv_config.flags */
 enum {
   REKV_FLAG_ATTEND_LEGACY_MMA = 1u << 1,        /* use the mma.sync attention kernel instead of tcgen05 */
-  REKV_FLAG_TIMING = 1u << 2                    /* bracket the attention kernel with CUDA events on the caller's
+  REKV_FLAG_TIMING = 1u << 2,                   /* bracket the attention kernel with CUDA events on the caller's
                                                   stream; rekv_stats then reports its duration */
+  REKV_FLAG_HOST_FP8 = 1u << 3                  /* offloaded contexts only: the pinned-host tier holds each page row
+                                                  (128 dims of one token of one KV head) as 128 FP8 E4M3 codes and
+                                                  one float scale = amax / 448; pages pulled from it come back as
+                                                  bf16(code * scale).  Halves the bytes that cross the host link and
+                                                  the host memory; frames still in the HBM tail stay exact.  (The
+                                                  paper names quantisation as future work; not part of its method.) */
 };
 
 typedef struct {

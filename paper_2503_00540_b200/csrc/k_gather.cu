@@ -5,12 +5,101 @@
 // pulled over the host link into an HBM staging page by the same kernel (zero-copy reads of the
 // mapped pinned arena, 16 bytes per load, many loads in flight).  A second kernel can write the
 // context out contiguously in plain [token][dim] layout.
+#include <cuda_fp8.h>
+
 #include "ptx_helpers.cuh"
 #include "rekv_internal.cuh"
 
 namespace {
 
 constexpr int PULL_PARTS_HOST = 8;  // CTAs per page when pages may have to cross the host link
+
+// ---- FP8 host tier -----------------------------------------------------------------------------
+// Groups of 16 codes [g0, g1) of one host page -> bf16 in the swizzled page layout at dst.  A group is 16
+// consecutive dims of one row: two 16-byte chunks of the destination.  The rows' scales are staged in
+// shared memory first (coalesced reads of the scale block instead of one small host read per thread).
+__device__ __forceinline__ void dequant_groups(const char* __restrict__ src, char* __restrict__ dst, int Hkv, int Nf,
+                                               long long g0, long long g1, float* s_scale) {
+  const float* scales = reinterpret_cast<const float*>(src + (long long)Hkv * 2 * Nf * 128);
+  const long long r0 = g0 >> 3, r1 = (g1 + 7) >> 3;  // rows (tile-major) touched by this range
+  for (long long r = r0 + threadIdx.x; r < r1; r += blockDim.x) s_scale[r - r0] = __ldcs(scales + r);
+  __syncthreads();
+  const uint4* s4 = reinterpret_cast<const uint4*>(src);
+  for (long long g = g0 + threadIdx.x; g < g1; g += blockDim.x) {
+    const uint4 codes = __ldcs(s4 + g);
+    const long long row = g >> 3;
+    const int k = (int)(g & 7);                 // dims [16k, 16k + 16)
+    const int tile = (int)(row / Nf), r = (int)(row - (long long)tile * Nf);
+    const float sc = s_scale[row - r0];
+    const unsigned char* cb = reinterpret_cast<const unsigned char*>(&codes);
+    uint32_t w[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const float lo = __half2float(__half(__nv_cvt_fp8_to_halfraw(cb[2 * e], __NV_E4M3))) * sc;
+      const float hi = __half2float(__half(__nv_cvt_fp8_to_halfraw(cb[2 * e + 1], __NV_E4M3))) * sc;
+      w[e] = rekv_ptx::pack_bf16(lo, hi);
+    }
+    char* base = dst + (long long)tile * Nf * 256 + (long long)(k >> 2) * Nf * 128 + (long long)r * 128;
+    const int c0 = (2 * k) & 7;
+    *reinterpret_cast<uint4*>(base + ((c0 ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+    *reinterpret_cast<uint4*>(base + (((c0 + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+  }
+}
+constexpr int DEQ_MAX_ROWS = 2048;  // rows of scales a CTA stages (H_kv * 2 * N_f <= 8 * 2 * 208 = 3328 per page, / parts)
+
+// grid = (layers, H_kv * 2 tiles): the ring slot's bf16 pages of one frame -> the frame's FP8 form.
+// Eight threads per row (16 dims each); the row maximum comes from three shuffles among them.
+__global__ void __launch_bounds__(256) quantize_frame_kernel(const char* __restrict__ pages, char* __restrict__ q8,
+                                                             long long page_bytes, long long host_page_bytes, int Hkv,
+                                                             int Nf) {
+  const int l = blockIdx.x, tile = blockIdx.y;
+  const char* page = pages + (long long)l * page_bytes + (long long)tile * Nf * 256;
+  char* out = q8 + (long long)l * host_page_bytes;
+  float* scales = reinterpret_cast<float*>(out + (long long)Hkv * 2 * Nf * 128);
+  const int k = threadIdx.x & 7;
+  for (int r0 = 0; r0 < Nf; r0 += 32) {
+    const int r = r0 + (threadIdx.x >> 3);
+    const bool valid = r < Nf;
+    uint4 a = make_uint4(0, 0, 0, 0), b = a;
+    if (valid) {
+      const char* base = page + (long long)(k >> 2) * Nf * 128 + (long long)r * 128;
+      const int c0 = (2 * k) & 7;
+      a = *reinterpret_cast<const uint4*>(base + ((c0 ^ (r & 7)) << 4));
+      b = *reinterpret_cast<const uint4*>(base + (((c0 + 1) ^ (r & 7)) << 4));
+    }
+    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    float v[16];
+    float amax = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      v[2 * e] = __uint_as_float(w[e] << 16);
+      v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+      amax = fmaxf(amax, fmaxf(fabsf(v[2 * e]), fabsf(v[2 * e + 1])));
+    }
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
+    const float sc = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+    uint4 codes;
+    unsigned char* cb = reinterpret_cast<unsigned char*>(&codes);
+#pragma unroll
+    for (int e = 0; e < 16; ++e) cb[e] = __nv_cvt_float_to_fp8(__fdiv_rn(v[e], sc), __NV_SATFINITE, __NV_E4M3);
+    if (valid) {
+      *reinterpret_cast<uint4*>(out + ((long long)tile * Nf + r) * 128 + k * 16) = codes;
+      if (k == 0) scales[(long long)tile * Nf + r] = sc;
+    }
+  }
+}
+
+// one host page -> one bf16 page (test helper path); grid = parts
+__global__ void __launch_bounds__(256) dequant_page_kernel(const char* __restrict__ src, char* __restrict__ dst, int Hkv,
+                                                           int Nf) {
+  __shared__ float s_scale[DEQ_MAX_ROWS];
+  const long long n16 = (long long)Hkv * 2 * Nf * 8;
+  const long long per = ((n16 + gridDim.x - 1) / gridDim.x + 7) & ~7ll;
+  const long long g0 = blockIdx.x * per, g1 = min(g0 + per, n16);
+  if (g0 < g1) dequant_groups(src, dst, Hkv, Nf, g0, g1, s_scale);
+}
 
 // grid = (ncf * parts, nQ, layer1 - layer0)
 __global__ void __launch_bounds__(256) page_table_pull_kernel(StoreView s, const int32_t* __restrict__ idx, int nQ,
@@ -44,11 +133,19 @@ __global__ void __launch_bounds__(256) page_table_pull_kernel(StoreView s, const
   }
   if (threadIdx.x == 0 && part == 0) {
     tbl[slot] = page;
-    if (pull) atomicAdd(link_bytes, (unsigned long long)s.page_bytes);
+    if (pull) atomicAdd(link_bytes, (unsigned long long)s.host_page_bytes);
   }
   if (!pull) return;
   const char* src = s.host_arenas[frame / s.frames_per_arena] +
-                    ((long long)(frame % s.frames_per_arena) * s.L + l) * s.page_bytes;
+                    ((long long)(frame % s.frames_per_arena) * s.L + l) * s.host_page_bytes;
+  if (s.host_fp8) {  // codes and scales cross the link; the staging page receives bf16
+    __shared__ float s_scale[DEQ_MAX_ROWS];
+    const long long g16 = (long long)s.Hkv * 2 * s.Nf * 8;
+    const long long gper = ((g16 + parts - 1) / parts + 7) & ~7ll;  // whole rows per part
+    const long long g0 = part * gper, g1 = min(g0 + gper, g16);
+    if (g0 < g1) dequant_groups(src, page, s.Hkv, s.Nf, g0, g1, s_scale);
+    return;
+  }
   const long long n16 = s.page_bytes >> 4;
   const long long per = (n16 + parts - 1) / parts;
   const long long i0 = part * per, i1 = min(i0 + per, n16);
@@ -102,6 +199,22 @@ cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int 
                            layer0, frames_now, parts, c->ctx_tbl, c->status, c->link_bytes);
   page_table_pull_kernel<<<grid, 256, 0, st>>>(c->sv, idx, nQ, top_k, k_eff, ncf, n_visible, layer0, frames_now,
                                                parts, c->ctx_tbl, c->status, c->link_bytes);
+  return cudaGetLastError();
+}
+
+cudaError_t rekv_launch_quantize_frame(rekv_ctx* c, int frame, cudaStream_t st) {
+  const StoreView& s = c->sv;
+  const int slot = frame % s.tail;
+  quantize_frame_kernel<<<dim3(s.L, s.Hkv * 2), 256, 0, st>>>(s.hbm + rekv_hbm_page_offset(s, frame, 0),
+                                                            s.q8_ring + (long long)slot * s.L * s.host_page_bytes,
+                                                            s.page_bytes, s.host_page_bytes, s.Hkv, s.Nf);
+  c->launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t rekv_launch_dequant_page(rekv_ctx* c, const char* host_page, char* dst_page, cudaStream_t st) {
+  dequant_page_kernel<<<8, 256, 0, st>>>(host_page, dst_page, c->sv.Hkv, c->sv.Nf);
+  c->launches += 1;
   return cudaGetLastError();
 }
 

@@ -53,6 +53,7 @@ void free_ctx(rekv_ctx* c) {
   cudaDeviceSynchronize();
   cudaFree(c->sv.hbm);
   cudaFree(c->sv.staging);
+  cudaFree(c->sv.q8_ring);
   cudaFree(c->sv.reps);
   cudaFree(c->d_host_arenas);
   cudaFree(c->qa);
@@ -187,8 +188,12 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   s.max_frames = cfg->max_frames;
   s.tail = cfg->hbm_tail_frames;
   s.page_bytes = (long long)s.Hkv * 2 * s.Nf * 256;
+  s.host_fp8 = (s.tail > 0 && (cfg->flags & REKV_FLAG_HOST_FP8)) ? 1 : 0;
+  // FP8 host tier: 128 codes + one float scale per page row, padded to a multiple of 16 bytes
+  s.host_page_bytes = s.host_fp8 ? (((long long)s.Hkv * 2 * s.Nf * (128 + 4) + 15) & ~15ll) : s.page_bytes;
   const long long frame_bytes = s.page_bytes * s.L;
-  s.frames_per_arena = (int)(ARENA_BYTES / frame_bytes);
+  const long long host_frame_bytes = s.host_page_bytes * s.L;
+  s.frames_per_arena = (int)(ARENA_BYTES / host_frame_bytes);
   if (s.frames_per_arena < 1) s.frames_per_arena = 1;
 
 #define CREATE_CUDA(call, what)                                                                              \
@@ -255,11 +260,11 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
       int fr = s.max_frames - a * s.frames_per_arena;
       if (fr > s.frames_per_arena) fr = s.frames_per_arena;
       char* p = nullptr;
-      cudaError_t e = cudaHostAlloc((void**)&p, (size_t)fr * frame_bytes, cudaHostAllocDefault);
+      cudaError_t e = cudaHostAlloc((void**)&p, (size_t)fr * host_frame_bytes, cudaHostAllocDefault);
       if (e != cudaSuccess) {
         cudaGetLastError();
         char b[256];
-        snprintf(b, sizeof(b), "pinning host arena %d of %d (%lld bytes): %s", a, n_arenas, fr * frame_bytes,
+        snprintf(b, sizeof(b), "pinning host arena %d of %d (%lld bytes): %s", a, n_arenas, fr * host_frame_bytes,
                  cudaGetErrorString(e));
         free_ctx(c);
         rekv_set_error(nullptr, b);
@@ -272,6 +277,8 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
                 "uploading the arena table");
     s.host_arenas = c->d_host_arenas;
     CREATE_CUDA(cudaMalloc(&s.staging, (size_t)s.L * maxQ * ctx_frames_max * s.page_bytes), "allocating gather staging");
+    if (s.host_fp8)
+      CREATE_CUDA(cudaMalloc(&s.q8_ring, (size_t)s.tail * host_frame_bytes), "allocating the quantised write-through ring");
     c->slot_events.resize(s.tail);
     c->slot_event_valid.assign(s.tail, 0);
     for (int i = 0; i < s.tail; ++i)
@@ -308,12 +315,16 @@ int rekv_append_frame(rekv_ctx* c, const void* k, const void* v, void* stream) {
   REKV_CUDA(c, rekv_launch_append(c, k, v, f, st));
   if (s.tail > 0) {
     const int slot = f % s.tail;
-    const long long frame_bytes = s.page_bytes * s.L;
-    char* dst = c->host_arenas[f / s.frames_per_arena] + (long long)(f % s.frames_per_arena) * frame_bytes;
+    const long long host_frame_bytes = s.host_page_bytes * s.L;
+    char* dst = c->host_arenas[f / s.frames_per_arena] + (long long)(f % s.frames_per_arena) * host_frame_bytes;
+    const char* src = s.hbm + rekv_hbm_page_offset(s, f, 0);
+    if (s.host_fp8) {  // the frame's FP8 form is made on the caller's stream and written through instead
+      REKV_CUDA(c, rekv_launch_quantize_frame(c, f, st));
+      src = s.q8_ring + (long long)slot * host_frame_bytes;
+    }
     REKV_CUDA(c, cudaEventRecord(c->ev_main, st));
     REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_main, 0));
-    REKV_CUDA(c, cudaMemcpyAsync(dst, s.hbm + rekv_hbm_page_offset(s, f, 0), (size_t)frame_bytes,
-                                 cudaMemcpyDeviceToHost, c->side));
+    REKV_CUDA(c, cudaMemcpyAsync(dst, src, (size_t)host_frame_bytes, cudaMemcpyDeviceToHost, c->side));
     REKV_CUDA(c, cudaEventRecord(c->slot_events[slot], c->side));
     c->slot_event_valid[slot] = 1;
     c->d2h_pending = true;
@@ -569,7 +580,7 @@ int rekv_stats(rekv_ctx* c, rekv_stats_t* out) {
   const long long frame_bytes = s.page_bytes * s.L;
   const long long resident = s.tail > 0 ? (c->frames < s.tail ? c->frames : s.tail) : c->frames;
   out->kv_bytes_hbm = resident * frame_bytes;
-  out->kv_bytes_host = s.tail > 0 ? (long long)c->frames * frame_bytes : 0;
+  out->kv_bytes_host = s.tail > 0 ? (long long)c->frames * s.host_page_bytes * s.L : 0;
   out->kv_bytes_logical = 2ll * s.L * c->frames * s.Nf * s.Hkv * REKV_HEAD_DIM * 2;
   out->rep_bytes = (long long)s.L * c->frames * s.Dp * (long long)sizeof(float);
   unsigned long long lb = 0;
@@ -628,7 +639,13 @@ int rekv_get_page(rekv_ctx* c, int frame, int layer, void* k_out, void* v_out, v
     // host-only page: read it zero-copy once its write-through has landed
     REKV_CUDA(c, cudaStreamSynchronize(c->side));
     page = c->host_arenas[frame / s.frames_per_arena] +
-           ((long long)(frame % s.frames_per_arena) * s.L + layer) * s.page_bytes;
+           ((long long)(frame % s.frames_per_arena) * s.L + layer) * s.host_page_bytes;
+    if (s.host_fp8) {  // back to bf16 in the first staging page (nothing else is in flight: test helper)
+      REKV_CUDA(c, cudaStreamSynchronize(st));
+      REKV_CUDA(c, rekv_launch_dequant_page(c, page, s.staging, st));
+      page = s.staging;
+      c->gathered = false;  // the staging page belonged to the last gather's context
+    }
   }
   REKV_CUDA(c, rekv_launch_unswizzle_page(c, page, k_out, v_out, st));
   return REKV_OK;

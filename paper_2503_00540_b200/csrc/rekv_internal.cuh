@@ -27,6 +27,9 @@
 //   element (row, dim): + row*128 + (((dim%64)/8) ^ (row&7))*16 + (dim%8)*2
 // Pages are frame-major: page(frame, layer) = base + (slot(frame)*L + layer) * page_bytes, so one
 // appended frame is one contiguous range (one D2H copy to the host tier).
+// FP8 host tier (REKV_FLAG_HOST_FP8): a host page holds, for the same (head, K/V) tiles, rows of 128 E4M3
+// codes in natural dim order -- tile(h, kv) at (h*2 + kv) * N_f*128, row r at + r*128 -- followed by one
+// float scale per row, scale[(h*2 + kv)*N_f + r], at H_kv*2*N_f*128; padded to a multiple of 16 bytes.
 // ---------------------------------------------------------------------------------------------
 struct StoreView {
   char* hbm;                   // HBM tier (all frames, or a ring of `tail` frames when offloaded)
@@ -34,6 +37,9 @@ struct StoreView {
   char* staging;               // HBM staging pages for host-tier gathers (offloaded only)
   float* reps;                 // [L][max_frames][D'] fp32
   long long page_bytes;
+  long long host_page_bytes;   // bytes of a page in the host tier (= page_bytes, or the FP8 form)
+  char* q8_ring;               // FP8 host tier: the quantised form of the ring's frames, source of the write-through
+  int host_fp8;                // the host tier holds FP8 E4M3 codes + one float scale per page row
   int L, Hq, Hkv, G, Nf, Dp;   // Dp = Hkv * 128
   int max_frames, tail, frames_per_arena;
 };
@@ -180,6 +186,8 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
 cudaError_t rekv_launch_retrieve_external(rekv_ctx* c, const float* q_emb, int nQ, int top_k, const CtxGeom& geom,
                                           int n_visible, float tau, int32_t* idx_out, float* scores, cudaStream_t st);
 // k_gather.cu
+cudaError_t rekv_launch_quantize_frame(rekv_ctx* c, int frame, cudaStream_t st);
+cudaError_t rekv_launch_dequant_page(rekv_ctx* c, const char* host_page, char* dst_page, cudaStream_t st);
 cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, const CtxGeom& geom,
                                    int n_visible, int layer0, int layer1, int frames_now, cudaStream_t st);
 cudaError_t rekv_launch_materialize(rekv_ctx* c, int nQ, int ncf, void* k_ctx, void* v_ctx, cudaStream_t st);
