@@ -488,6 +488,32 @@ def run_cuda(args, w):
     torch.cuda.synchronize()
     layer_seq_us = ev_r[0].elapsed_time(ev_r[1]) * 1e3 / n_seq / nQ
     layer_seq_one_graph_us = None
+    decode_layers_us = None
+    if w["tail"] == 0 and not w.get("full") and max(lengths) * (w["Hq"] // w["Hkv"]) > 16:
+        # generation after the question: every new token attends the same retrieved context, layer by layer
+        # (rekv_attend_layer, one query row per question), all layers of a token as consecutive nodes of one graph
+        cu1 = list(range(nQ + 1))
+        qd = [synth.question(w["seed"], 900 + r, w["L"], nQ, w["Hq"], w["D"], device=dev) for r in range(2)]
+        qd_buf, od_buf = qd[0].clone(), torch.empty_like(qd[0])
+        g.question(qs[0], cu, w["k"], n_vis, out=out)            # the context the tokens reuse
+        g.gather(g.retrieve(qs[0], cu, w["k"], n_vis)[0], nQ, w["k"], n_vis)
+        cap2 = torch.cuda.Stream(dev)
+        cap2.wait_stream(stream)
+        with torch.cuda.stream(cap2):
+            gr_dec = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr_dec, stream=cap2):
+                for l in range(w["L"]):
+                    g.attend_layer(l, qd_buf[l], cu1, out=od_buf[l])
+        stream.wait_stream(cap2)
+        for i in range(2 + 20):
+            if i == 2:
+                torch.cuda.synchronize()
+                ev_r[0].record(stream)
+            qd_buf.copy_(qd[i % 2])
+            gr_dec.replay()
+        ev_r[1].record(stream)
+        torch.cuda.synchronize()
+        decode_layers_us = ev_r[0].elapsed_time(ev_r[1]) * 1e3 / 20
     if w["tail"] == 0:
         for i in range(2 + n_seq):
             if i == 2:
@@ -528,6 +554,7 @@ def run_cuda(args, w):
                          "median_us": q_median, "min_us": q_min,
                          "layer_sequential_us": layer_seq_us,
                          "layer_sequential_one_graph_us": layer_seq_one_graph_us,
+                         "decode_token_layer_by_layer_us": decode_layers_us,
                          "layer_sequential_mode": ("one CUDA graph replay per layer" if w["tail"] == 0
                                                    else "one eager call per layer"),
                          "retrieve_us_per_batch": retrieve_us,
