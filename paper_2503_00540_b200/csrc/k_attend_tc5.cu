@@ -40,6 +40,7 @@ struct TcParams {
   const float* self_ml;    // per output row: (max, sum) of that part, log2 domain
   float* part_o;
   float* part_ml;
+  int* unit_cnt;     // per unit: parts finished so far (decode kernel: the last part merges; self-resetting)
   int* status;
   QBatch qb;
   int Hq, Hkv, G, Nf, Npad, NA, NB, ncf, MP, layer0;
@@ -827,12 +828,74 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) attend_decode_kernel(const TcP
         } else if (DEC_GUARD(((long long)blockIdx.x + u) * 2 < 2048, 5)) {
           const long long slot = ((long long)blockIdx.x + u) * 2;
           float* po = p.part_o + (slot * 128 + r) * 128 + d0;
-          *reinterpret_cast<float4*>(po) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-          *reinterpret_cast<float4*>(po + 4) = make_float4(acc[4], acc[5], acc[6], acc[7]);
+          __stcg(reinterpret_cast<float4*>(po), make_float4(acc[0], acc[1], acc[2], acc[3]));
+          __stcg(reinterpret_cast<float4*>(po + 4), make_float4(acc[4], acc[5], acc[6], acc[7]));
           if ((tid & 15) == 0) {
-            p.part_ml[(slot * 128 + r) * 2] = M;
-            p.part_ml[(slot * 128 + r) * 2 + 1] = den;
+            __stcg(p.part_ml + (slot * 128 + r) * 2, M);
+            __stcg(p.part_ml + (slot * 128 + r) * 2 + 1, den);
           }
+        }
+      }
+    }
+    if (!whole_unit && p.unit_cnt) {
+      // The range covered a part of the unit.  The CTA that finishes a unit's last part merges all of them
+      // (no further launch): parts are published with a fence, counted with an atomic, and the counter is
+      // left at zero for the next launch.
+      volatile int& s_last = *reinterpret_cast<volatile int*>(smem + ring_bytes + 24);  // beside the barriers
+      const long long c_first = (u * p.ncf) / p.per, c_last = ((u + 1) * p.ncf - 1) / p.per;
+      __threadfence();
+      __syncthreads();
+      if (tid == 0) {
+        const int prev = atomicAdd(p.unit_cnt + u, 1);
+        s_last = (prev == (int)(c_last - c_first)) ? 1 : 0;
+        if (s_last) p.unit_cnt[u] = 0;
+      }
+      __syncthreads();
+      if (s_last) {
+        __threadfence();
+        const int r = tid >> 4, d0 = (tid & 15) * 8;
+        if (r < ui.rows_q) {
+          const long long out_row = row_index(r);
+          float M = p.self_o ? p.self_ml[out_row * 2] : -INFINITY;
+          for (long long cc = c_first; cc <= c_last; ++cc) M = fmaxf(M, __ldcg(p.part_ml + (((cc + u) * 2) * 128 + r) * 2));
+          float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          float den = 0.f;
+          if (p.self_o) {  // Eq. 3 in full: the part over the tokens of X is one more part
+            const float wt = ex2(p.self_ml[out_row * 2] - M);
+            const float4 x = *reinterpret_cast<const float4*>(p.self_o + out_row * 128 + d0);
+            const float4 y = *reinterpret_cast<const float4*>(p.self_o + out_row * 128 + d0 + 4);
+            acc[0] = wt * x.x; acc[1] = wt * x.y; acc[2] = wt * x.z; acc[3] = wt * x.w;
+            acc[4] = wt * y.x; acc[5] = wt * y.y; acc[6] = wt * y.z; acc[7] = wt * y.w;
+            den = wt * p.self_ml[out_row * 2 + 1];
+          }
+          for (long long c0 = c_first; c0 <= c_last; c0 += 4) {  // four parts in flight, added in part order
+            float4 x[4], y[4];
+            float pm[4], pl[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              if (c0 + i <= c_last) {
+                const long long base = ((c0 + i + u) * 2) * 128 + r;
+                pm[i] = __ldcg(p.part_ml + base * 2);
+                pl[i] = __ldcg(p.part_ml + base * 2 + 1);
+                x[i] = __ldcg(reinterpret_cast<const float4*>(p.part_o + base * 128 + d0));
+                y[i] = __ldcg(reinterpret_cast<const float4*>(p.part_o + base * 128 + d0 + 4));
+              }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              if (c0 + i <= c_last) {
+                const float wt = ex2(pm[i] - M);
+                acc[0] += wt * x[i].x; acc[1] += wt * x[i].y; acc[2] += wt * x[i].z; acc[3] += wt * x[i].w;
+                acc[4] += wt * y[i].x; acc[5] += wt * y[i].y; acc[6] += wt * y[i].z; acc[7] += wt * y[i].w;
+                den += wt * pl[i];
+              }
+          }
+          const float inv = den > 0.f ? 1.f / den : 0.f;
+          uint4 o;
+          o.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+          o.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+          o.z = pack_bf16(acc[4] * inv, acc[5] * inv);
+          o.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+          *reinterpret_cast<uint4*>(p.out + out_row * 128 + d0) = o;
         }
       }
     }
@@ -927,6 +990,7 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   p.tbl = c->ctx_tbl;
   p.part_o = c->part_o;
   p.part_ml = c->part_ml;
+  p.unit_cnt = c->unit_cnt;
   p.status = c->status;
   p.qb = qb;
   p.Hq = s.Hq;
@@ -964,13 +1028,17 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   bool few_rows = true;
   for (int i = 0; i < qb.nQ; ++i) few_rows = few_rows && (qb.cu[i + 1] - qb.cu[i]) * s.G <= 16;
   const size_t smem_dec = std::max((size_t)4 * 2 * p.Npad * 128, (size_t)DEC_SCRATCH) + 64 + 1024;
-  if (few_rows && smem_dec <= 227 * 1024) {
+  if (few_rows && smem_dec <= 227 * 1024 && (size_t)units <= c->part_units) {
     static bool dec_attr_set = false;
     if (!dec_attr_set) {
       cudaError_t e = cudaFuncSetAttribute(attend_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
       if (e != cudaSuccess) return e;
       dec_attr_set = true;
     }
+    // A unit cut into a few parts is merged by the CTA that finishes its last part (no further launch); when a
+    // launch has few units and therefore many parts per unit (one layer at a time), the merge kernel's
+    // parallelism is worth its launch.
+    if ((ncf + p.per - 1) / p.per + 1 > 4) p.unit_cnt = nullptr;
     if (timed) cudaEventRecord(c->ev_t0, st);
     cudaError_t e1 = rekv_launch_pdl(attend_decode_kernel, dim3((unsigned)grid), dim3(DEC_THREADS), smem_dec, st, p);
     if (e1 != cudaSuccess) return e1;
@@ -979,7 +1047,7 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
       c->timing_valid = true;
     }
     c->launches += 1;
-    if (p.per != ncf) {
+    if (p.per != ncf && !p.unit_cnt) {
       cudaError_t e2 = rekv_launch_pdl(combine_tc5_kernel, dim3((unsigned)units, 2, 32), dim3(128), 0, st, p);
       if (e2 != cudaSuccess) return e2;
       c->launches += 1;

@@ -62,6 +62,7 @@ void free_ctx(rekv_ctx* c) {
   cudaFree(c->ctx_tbl);
   cudaFree(c->part_o);
   cudaFree(c->part_ml);
+  cudaFree(c->unit_cnt);
   cudaFree(c->status);
   cudaFree(c->idx_own);
   cudaFree(c->ext_emb);
@@ -165,6 +166,7 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   c->gather_layerwise = false;
   memset(&c->sv, 0, sizeof(c->sv));
   c->qa = c->qnorm = c->scores = c->part_o = c->part_ml = nullptr;
+  c->unit_cnt = nullptr;
   c->ctx_tbl = nullptr;
   c->status = nullptr;
   c->link_bytes = nullptr;
@@ -221,6 +223,8 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   c->part_units = 2048;
   CREATE_CUDA(cudaMalloc(&c->part_o, c->part_units * 128 * 128 * sizeof(float)), "allocating split-KV partials");
   CREATE_CUDA(cudaMalloc(&c->part_ml, c->part_units * 128 * 2 * sizeof(float)), "allocating split-KV partials");
+  CREATE_CUDA(cudaMalloc(&c->unit_cnt, c->part_units * sizeof(int)), "allocating split-KV counters");
+  CREATE_CUDA(cudaMemset(c->unit_cnt, 0, c->part_units * sizeof(int)), "clearing split-KV counters");
   CREATE_CUDA(cudaMalloc(&c->status, sizeof(int)), "allocating the status word");
   CREATE_CUDA(cudaMemset(c->status, 0, sizeof(int)), "clearing the status word");
   CREATE_CUDA(cudaMalloc(&c->idx_own, (size_t)s.L * maxQ * (c->cfg.max_topk > 0 ? c->cfg.max_topk : 1) * sizeof(int32_t)),
@@ -606,6 +610,7 @@ int rekv_check_status(rekv_ctx* c, void* stream) {
   REKV_CUDA(c, cudaMemcpy(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost));
   if (st != 0) {
     REKV_CUDA(c, cudaMemset(c->status, 0, sizeof(int)));
+    REKV_CUDA(c, cudaMemset(c->unit_cnt, 0, c->part_units * sizeof(int)));  // a kernel that gave up may have left counts
     if (st == REKV_ERR_TIMEOUT) REKV_FAIL(c, REKV_ERR_TIMEOUT, "a device-side wait expired");
     REKV_FAIL(c, st, "a kernel reported error %d (an index outside the visible frames?)", st);
   }

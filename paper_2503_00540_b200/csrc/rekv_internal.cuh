@@ -109,6 +109,7 @@ struct rekv_ctx {
   float* part_o;                    // split-KV partial outputs
   float* part_ml;                   // split-KV partial (max, sum)
   size_t part_units;                // capacity in (unit) entries of 128 rows
+  int* unit_cnt;                    // [part_units] parts finished per unit (zero between launches)
   int* status;                      // device status word
   unsigned long long* link_bytes;   // device counter: bytes pulled over the host link
   int32_t* idx_own;                 // [L][max_questions][max_topk]: selections of the layer-sequential calls
