@@ -1038,6 +1038,10 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     // A unit cut into a few parts is merged by the CTA that finishes its last part (no further launch); when a
     // launch has few units and therefore many parts per unit (one layer at a time), the merge kernel's
     // parallelism is worth its launch.
+    if (p.per < 4 && p.per != ncf) {  // a small launch (one layer): four frames per CTA amortise its fixed cost
+      p.per = ncf < 4 ? ncf : 4;
+      grid = (p.total + p.per - 1) / p.per;
+    }
     if ((ncf + p.per - 1) / p.per + 1 > 4) p.unit_cnt = nullptr;
     if (timed) cudaEventRecord(c->ev_t0, st);
     cudaError_t e1 = rekv_launch_pdl(attend_decode_kernel, dim3((unsigned)grid), dim3(DEC_THREADS), smem_dec, st, p);
