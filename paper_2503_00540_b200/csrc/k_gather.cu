@@ -57,36 +57,45 @@ __global__ void __launch_bounds__(256) quantize_frame_kernel(const char* __restr
   char* out = q8 + (long long)l * host_page_bytes;
   float* scales = reinterpret_cast<float*>(out + (long long)Hkv * 2 * Nf * 128);
   const int k = threadIdx.x & 7;
-  for (int r0 = 0; r0 < Nf; r0 += 32) {
-    const int r = r0 + (threadIdx.x >> 3);
-    const bool valid = r < Nf;
-    uint4 a = make_uint4(0, 0, 0, 0), b = a;
-    if (valid) {
-      const char* base = page + (long long)(k >> 2) * Nf * 128 + (long long)r * 128;
-      const int c0 = (2 * k) & 7;
-      a = *reinterpret_cast<const uint4*>(base + ((c0 ^ (r & 7)) << 4));
-      b = *reinterpret_cast<const uint4*>(base + (((c0 + 1) ^ (r & 7)) << 4));
-    }
-    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-    float v[16];
-    float amax = 0.f;
+  constexpr int U = 4;  // rows per thread in flight: all their loads are issued before the first reduction
+  for (int r0 = 0; r0 < Nf; r0 += 32 * U) {
+    uint4 a[U], b[U];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      v[2 * e] = __uint_as_float(w[e] << 16);
-      v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
-      amax = fmaxf(amax, fmaxf(fabsf(v[2 * e]), fabsf(v[2 * e + 1])));
+    for (int u = 0; u < U; ++u) {
+      const int r = r0 + u * 32 + (threadIdx.x >> 3);
+      a[u] = make_uint4(0, 0, 0, 0);
+      b[u] = a[u];
+      if (r < Nf) {
+        const char* base = page + (long long)(k >> 2) * Nf * 128 + (long long)r * 128;
+        const int c0 = (2 * k) & 7;
+        a[u] = __ldcs(reinterpret_cast<const uint4*>(base + ((c0 ^ (r & 7)) << 4)));
+        b[u] = __ldcs(reinterpret_cast<const uint4*>(base + (((c0 + 1) ^ (r & 7)) << 4)));
+      }
     }
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
-    const float sc = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
-    uint4 codes;
-    unsigned char* cb = reinterpret_cast<unsigned char*>(&codes);
 #pragma unroll
-    for (int e = 0; e < 16; ++e) cb[e] = __nv_cvt_float_to_fp8(__fdiv_rn(v[e], sc), __NV_SATFINITE, __NV_E4M3);
-    if (valid) {
-      *reinterpret_cast<uint4*>(out + ((long long)tile * Nf + r) * 128 + k * 16) = codes;
-      if (k == 0) scales[(long long)tile * Nf + r] = sc;
+    for (int u = 0; u < U; ++u) {
+      const int r = r0 + u * 32 + (threadIdx.x >> 3);
+      const uint32_t w[8] = {a[u].x, a[u].y, a[u].z, a[u].w, b[u].x, b[u].y, b[u].z, b[u].w};
+      float v[16];
+      float amax = 0.f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        v[2 * e] = __uint_as_float(w[e] << 16);
+        v[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+        amax = fmaxf(amax, fmaxf(fabsf(v[2 * e]), fabsf(v[2 * e + 1])));
+      }
+      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
+      const float sc = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+      uint4 codes;
+      unsigned char* cb = reinterpret_cast<unsigned char*>(&codes);
+#pragma unroll
+      for (int e = 0; e < 16; ++e) cb[e] = __nv_cvt_float_to_fp8(__fdiv_rn(v[e], sc), __NV_SATFINITE, __NV_E4M3);
+      if (r < Nf) {
+        *reinterpret_cast<uint4*>(out + ((long long)tile * Nf + r) * 128 + k * 16) = codes;
+        if (k == 0) scales[(long long)tile * Nf + r] = sc;
+      }
     }
   }
 }
