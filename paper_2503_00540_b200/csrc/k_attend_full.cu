@@ -8,6 +8,8 @@
 //     a partial (max, sum, numerator) per output row; the attention kernel's epilogue, or the merge
 //     kernel for units cut by a CTA boundary, joins it with the part over R.
 // Pairing of dimensions: i with i + 64 (head_dim 128), angle = position * theta^(-2i/128).
+#include <algorithm>
+
 #include "ptx_helpers.cuh"
 #include "rekv_internal.cuh"
 
@@ -118,11 +120,13 @@ __global__ void __launch_bounds__(256) rope_stage_kernel(char* const* __restrict
   }
 }
 
-// The softmax part over the tokens of X.  grid = (H_q, nQ, L), 256 threads; the CTA holds the KV head's
-// keys (rotated on the way in) and values of one 64-token tile of X in shared memory, a warp walks the
-// question's query rows of this head: lane s scores key s (and s + 32), the row's running (max, sum) and
-// its numerator (4 dims per lane) are combined across tiles through the output arrays (same warp, same
-// row, so no other thread touches them).  Writes self_o (unnormalised, relative to the max) and self_ml.
+// The softmax part over the tokens of X (causal), on the tensor cores with mma.sync m16n8k16.
+// grid = (128-row blocks of the longest question, H_q, L * nQ), 256 threads: a warp owns 16 query rows
+// (tokens of the question, one head) and walks X's keys in tiles of 64; the KV head's K (rotated on the
+// way in) and V tiles sit in shared memory in the pages' layout -- two 64-dim halves of [64 rows][128 B]
+// with the 16-byte chunks XOR-swizzled by (row & 7) -- so ldmatrix reads them without bank conflicts.
+// Row n of a question (token N_s - N_q + n of X) sees keys 0 .. N_s - N_q + n.  Writes, per output row,
+// the numerator (unnormalised, relative to the row maximum) and (max, sum), log2 domain.
 constexpr int SELF_TILE = 64;
 __global__ void __launch_bounds__(256) self_attend_kernel(const __nv_bfloat16* __restrict__ q,
                                                           const __nv_bfloat16* __restrict__ k_self,
@@ -130,96 +134,159 @@ __global__ void __launch_bounds__(256) self_attend_kernel(const __nv_bfloat16* _
                                                           int Hq, int Hkv, int G, int n_ctx_tokens,
                                                           const float2* __restrict__ tab, float scale_log2,
                                                           float* __restrict__ self_o, float* __restrict__ self_ml) {
-  __shared__ uint32_t s_k[SELF_TILE][65];  // bf16 pairs; the odd row pitch keeps lane-per-key reads conflict-free
-  __shared__ uint2 s_v[SELF_TILE][32];     // 4 bf16 per lane
-  __shared__ float s_q[8][128];
-  const int h = blockIdx.x, qi = blockIdx.y, l = blockIdx.z;
+  __shared__ __align__(128) unsigned char s_kv[2 * 2 * SELF_TILE * 128];  // K tile, V tile
+  const int rb = blockIdx.x, h = blockIdx.y;
+  const int l = blockIdx.z / qb.nQ, qi = blockIdx.z - l * qb.nQ;
   const int g = h / G;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int q0 = qb.cu[qi], nq = qb.cu[qi + 1] - q0;
   const int s0 = sb.cu[qi], ns = sb.cu[qi + 1] - s0;
-  for (int t0 = 0; t0 < ns; t0 += SELF_TILE) {
-    const int nt = min(SELF_TILE, ns - t0);
-    __syncthreads();
-    // keys: 8 threads per token, a 16-byte chunk of each half, rotated at position n_ctx + token
-    for (int it = threadIdx.x; it < nt * 8; it += 256) {
-      const int c = it & 7, s = it >> 3;
-      const uint4* src = reinterpret_cast<const uint4*>(k_self + (((long long)l * sb.sumNq + s0 + t0 + s) * Hkv + g) * 128);
-      uint4 lo = src[c], hi = src[8 + c];
-      if (tab) rotate_chunk(lo, hi, tab + (long long)(n_ctx_tokens + t0 + s) * 64 + c * 8);
-      const uint32_t* a = reinterpret_cast<const uint32_t*>(&lo);
-      const uint32_t* b = reinterpret_cast<const uint32_t*>(&hi);
+  if (rb * 128 >= nq) return;
+  const uint32_t sK = smem_u32(s_kv), sV = sK + 2 * SELF_TILE * 128;
+  constexpr uint32_t half_stride = SELF_TILE * 128;
+
+  // this thread's two rows (fragment layout of m16n8k16: rows lane/4 and lane/4 + 8 of the warp's 16)
+  const int n_lo = rb * 128 + warp * 16 + (lane >> 2), n_hi = n_lo + 8;
+  const bool v_lo = n_lo < nq, v_hi = n_hi < nq;
+  const long long row_lo = ((long long)l * qb.sumNq + q0 + (v_lo ? n_lo : 0)) * Hq + h;
+  const long long row_hi = ((long long)l * qb.sumNq + q0 + (v_hi ? n_hi : 0)) * Hq + h;
+  uint32_t qf[8][4];
+  {
+    const uint32_t* plo = reinterpret_cast<const uint32_t*>(q + row_lo * 128);
+    const uint32_t* phi = reinterpret_cast<const uint32_t*>(q + row_hi * 128);
 #pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        s_k[s][c * 4 + w] = a[w];
-        s_k[s][32 + c * 4 + w] = b[w];
+    for (int kb = 0; kb < 8; ++kb) {
+      const int w = kb * 8 + (lane & 3);
+      qf[kb][0] = v_lo ? __ldg(plo + w) : 0u;
+      qf[kb][1] = v_hi ? __ldg(phi + w) : 0u;
+      qf[kb][2] = v_lo ? __ldg(plo + w + 4) : 0u;
+      qf[kb][3] = v_hi ? __ldg(phi + w + 4) : 0u;
+    }
+  }
+  const int last_lo = ns - nq + n_lo, last_hi = ns - nq + n_hi;        // last key each row sees
+  const int last_cta = ns - nq + min(rb * 128 + 127, nq - 1);          // ... and the row block
+  const int last_warp = ns - nq + min(rb * 128 + warp * 16 + 15, nq - 1);
+  float oacc[16][4];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
+  float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+  const int lm = lane >> 3, lr = lane & 7;
+
+  for (int t0 = 0; t0 <= last_cta; t0 += SELF_TILE) {
+    __syncthreads();  // the previous tile has been read by every warp
+    // K and V rows t0 .. t0+63 of X (zero beyond N_s): 8 threads per row, chunk c of each half per thread
+    for (int it = tid; it < SELF_TILE * 8; it += 256) {
+      const int c = it & 7, r = it >> 3;
+      const int s = t0 + r;
+      uint4 klo = make_uint4(0, 0, 0, 0), khi = klo, vlo = klo, vhi = klo;
+      if (s < ns) {
+        const long long base = (((long long)l * sb.sumNq + s0 + s) * Hkv + g) * 16;  // 16-byte chunks
+        const uint4* ks = reinterpret_cast<const uint4*>(k_self) + base;
+        const uint4* vs = reinterpret_cast<const uint4*>(v_self) + base;
+        klo = __ldg(ks + c);
+        khi = __ldg(ks + 8 + c);
+        vlo = __ldg(vs + c);
+        vhi = __ldg(vs + 8 + c);
+        if (tab) rotate_chunk(klo, khi, tab + (long long)(n_ctx_tokens + s) * 64 + c * 8);
+      }
+      const uint32_t off = r * 128 + ((c ^ (r & 7)) << 4);
+      *reinterpret_cast<uint4*>(s_kv + off) = klo;
+      *reinterpret_cast<uint4*>(s_kv + half_stride + off) = khi;
+      *reinterpret_cast<uint4*>(s_kv + 2 * half_stride + off) = vlo;
+      *reinterpret_cast<uint4*>(s_kv + 3 * half_stride + off) = vhi;
+    }
+    __syncthreads();
+    if (t0 > last_warp) continue;  // nothing of this tile is visible to this warp's rows (warp-uniform)
+    float sacc[8][4];
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb) {
+      sacc[nb][0] = sacc[nb][1] = sacc[nb][2] = sacc[nb][3] = 0.f;
+      const int tok = nb * 8 + lr;
+#pragma unroll
+      for (int kp = 0; kp < 4; ++kp) {
+        const int c = kp * 4 + lm;
+        const uint32_t addr = sK + (c >> 3) * half_stride + tok * 128 + (((c & 7) ^ (tok & 7)) << 4);
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4(b0, b1, b2, b3, addr);
+        mma_bf16_16816(sacc[nb], qf[2 * kp], b0, b1);
+        mma_bf16_16816(sacc[nb], qf[2 * kp + 1], b2, b3);
       }
     }
-    for (int it = threadIdx.x; it < nt * 32; it += 256) {
-      const int s = it >> 5, d4 = it & 31;
-      s_v[s][d4] = *reinterpret_cast<const uint2*>(v_self + (((long long)l * sb.sumNq + s0 + t0 + s) * Hkv + g) * 128 + d4 * 4);
-    }
-    __syncthreads();
-    for (int n = warp; n < nq; n += 8) {
-      const int last = ns - nq + n;  // the last token of X this row sees
-      if (last < t0) continue;       // (warp-uniform)
-      const long long out_row = ((long long)l * qb.sumNq + q0 + n) * Hq + h;
-      __syncwarp();
-      {
-        const uint2 qv = *reinterpret_cast<const uint2*>(q + out_row * 128 + lane * 4);
-        s_q[warp][lane * 4] = __uint_as_float(qv.x << 16);
-        s_q[warp][lane * 4 + 1] = __uint_as_float(qv.x & 0xFFFF0000u);
-        s_q[warp][lane * 4 + 2] = __uint_as_float(qv.y << 16);
-        s_q[warp][lane * 4 + 3] = __uint_as_float(qv.y & 0xFFFF0000u);
-      }
-      __syncwarp();
-      float sc[2];
+    float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const int s = half * 32 + lane;
-        float a0 = 0.f, a1 = 0.f;
-        if (s < nt) {
-#pragma unroll 16
-          for (int w = 0; w < 64; ++w) {
-            const uint32_t kk = s_k[s][w];
-            a0 = fmaf(s_q[warp][2 * w], __uint_as_float(kk << 16), a0);
-            a1 = fmaf(s_q[warp][2 * w + 1], __uint_as_float(kk & 0xFFFF0000u), a1);
-          }
-        }
-        sc[half] = (s < nt && t0 + s <= last) ? (a0 + a1) * scale_log2 : -INFINITY;
+    for (int nb = 0; nb < 8; ++nb) {
+      const int col = t0 + nb * 8 + (lane & 3) * 2;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int key = col + (e & 1);
+        const int last = (e < 2) ? last_lo : last_hi;
+        sacc[nb][e] = key <= last ? sacc[nb][e] * scale_log2 : -INFINITY;  // causal (covers keys beyond N_s too)
       }
-      float m_t = fmaxf(sc[0], sc[1]);
-      for (int o = 16; o; o >>= 1) m_t = fmaxf(m_t, __shfl_xor_sync(0xffffffffu, m_t, o));
-      float m_old = -INFINITY, l_old = 0.f;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (t0 > 0) {
-        m_old = self_ml[out_row * 2];
-        l_old = self_ml[out_row * 2 + 1];
-        acc = *reinterpret_cast<const float4*>(self_o + out_row * 128 + lane * 4);
+      mx_lo = fmaxf(mx_lo, fmaxf(sacc[nb][0], sacc[nb][1]));
+      mx_hi = fmaxf(mx_hi, fmaxf(sacc[nb][2], sacc[nb][3]));
+    }
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+    // a row that sees nothing of this tile keeps its state (its maximum stays where it was)
+    const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+    const float a_lo = mn_lo == -INFINITY ? 1.f : ex2(m_lo - mn_lo), a_hi = mn_hi == -INFINITY ? 1.f : ex2(m_hi - mn_hi);
+    const float sub_lo = mn_lo == -INFINITY ? 0.f : mn_lo, sub_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
+    m_lo = mn_lo;
+    m_hi = mn_hi;
+    l_lo *= a_lo;
+    l_hi *= a_hi;
+#pragma unroll
+    for (int nd = 0; nd < 16; ++nd) {
+      oacc[nd][0] *= a_lo;
+      oacc[nd][1] *= a_lo;
+      oacc[nd][2] *= a_hi;
+      oacc[nd][3] *= a_hi;
+    }
+    uint32_t pf[8][2];
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb) {
+      const float p0 = ex2(sacc[nb][0] - sub_lo), p1 = ex2(sacc[nb][1] - sub_lo);
+      const float p2 = ex2(sacc[nb][2] - sub_hi), p3 = ex2(sacc[nb][3] - sub_hi);
+      l_lo += p0 + p1;
+      l_hi += p2 + p3;
+      pf[nb][0] = pack_bf16(p0, p1);
+      pf[nb][1] = pack_bf16(p2, p3);
+    }
+#pragma unroll
+    for (int kb = 0; kb < 4; ++kb) {
+      const uint32_t a[4] = {pf[2 * kb][0], pf[2 * kb][1], pf[2 * kb + 1][0], pf[2 * kb + 1][1]};
+      const int tok = kb * 16 + (lm & 1) * 8 + lr;
+#pragma unroll
+      for (int dp = 0; dp < 8; ++dp) {
+        const int c = dp * 2 + (lm >> 1);
+        const uint32_t addr = sV + (c >> 3) * half_stride + tok * 128 + (((c & 7) ^ (tok & 7)) << 4);
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4_trans(b0, b1, b2, b3, addr);
+        mma_bf16_16816(oacc[2 * dp], a, b0, b1);
+        mma_bf16_16816(oacc[2 * dp + 1], a, b2, b3);
       }
-      const float m_new = fmaxf(m_old, m_t);  // finite: the row sees at least one token of this or an earlier tile
-      const float w_old = ex2(m_old - m_new);
-      const float p0 = ex2(sc[0] - m_new), p1 = ex2(sc[1] - m_new);
-      float l_t = p0 + p1;
-      for (int o = 16; o; o >>= 1) l_t += __shfl_xor_sync(0xffffffffu, l_t, o);
-      acc.x *= w_old;
-      acc.y *= w_old;
-      acc.z *= w_old;
-      acc.w *= w_old;
-      const int n_seen = min(nt, last - t0 + 1);
-      for (int s = 0; s < n_seen; ++s) {
-        const float pv = __shfl_sync(0xffffffffu, s < 32 ? p0 : p1, s & 31);
-        const uint2 vv = s_v[s][lane];
-        acc.x = fmaf(pv, __uint_as_float(vv.x << 16), acc.x);
-        acc.y = fmaf(pv, __uint_as_float(vv.x & 0xFFFF0000u), acc.y);
-        acc.z = fmaf(pv, __uint_as_float(vv.y << 16), acc.z);
-        acc.w = fmaf(pv, __uint_as_float(vv.y & 0xFFFF0000u), acc.w);
-      }
-      *reinterpret_cast<float4*>(self_o + out_row * 128 + lane * 4) = acc;
-      if (lane == 0) {
-        self_ml[out_row * 2] = m_new;
-        self_ml[out_row * 2 + 1] = l_old * w_old + l_t;
-      }
+    }
+  }
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+#pragma unroll
+  for (int nd = 0; nd < 16; ++nd) {
+    const int d = nd * 8 + (lane & 3) * 2;
+    if (v_lo) *reinterpret_cast<float2*>(self_o + row_lo * 128 + d) = make_float2(oacc[nd][0], oacc[nd][1]);
+    if (v_hi) *reinterpret_cast<float2*>(self_o + row_hi * 128 + d) = make_float2(oacc[nd][2], oacc[nd][3]);
+  }
+  if ((lane & 3) == 0) {
+    if (v_lo) {
+      self_ml[row_lo * 2] = m_lo;
+      self_ml[row_lo * 2 + 1] = l_lo;
+    }
+    if (v_hi) {
+      self_ml[row_hi * 2] = m_hi;
+      self_ml[row_hi * 2 + 1] = l_hi;
     }
   }
 }
@@ -272,11 +339,11 @@ cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const vo
     if ((e = cudaEventRecord(c->ev_main, st)) != cudaSuccess) return e;
     if ((e = cudaStreamWaitEvent(c->side, c->ev_main, 0)) != cudaSuccess) return e;
   }
-  self_attend_kernel<<<dim3(s.Hq, qb.nQ, s.L), 256, 0, st_self>>>(q_eff, (const __nv_bfloat16*)k_self,
-                                                                 (const __nv_bfloat16*)v_self, qb, sb, s.Hq, s.Hkv, s.G,
-                                                                 n_ctx_tokens, rope ? c->rope_tab : nullptr,
-                                                                 1.4426950408889634f / sqrtf(128.f), c->self_o,
-                                                                 c->self_ml);
+  int max_nq = 1;
+  for (int i = 0; i < qb.nQ; ++i) max_nq = std::max(max_nq, qb.cu[i + 1] - qb.cu[i]);
+  self_attend_kernel<<<dim3((max_nq + 127) / 128, s.Hq, s.L * qb.nQ), 256, 0, st_self>>>(
+      q_eff, (const __nv_bfloat16*)k_self, (const __nv_bfloat16*)v_self, qb, sb, s.Hq, s.Hkv, s.G, n_ctx_tokens,
+      rope ? c->rope_tab : nullptr, 1.4426950408889634f / sqrtf(128.f), c->self_o, c->self_ml);
   c->launches += 1;
   if (fork) {
     if ((e = cudaEventRecord(c->ev_side, c->side)) != cudaSuccess) return e;
