@@ -160,7 +160,9 @@ int rekv_gather(rekv_ctx* ctx, const int32_t* idx, int nQ, int top_k, int n_visi
  * out: device bf16 [L][sum_Nq][H_q][D].  For every layer, question token n and query head h:
  * out = softmax(q . K_ctx^T / sqrt(D)) V_ctx over the gathered context of KV head floor(h/G);
  * no mask (every context token precedes the question); bf16 operands, fp32 accumulation and softmax.
- * Returns 0, or REKV_ERR_STATE without a preceding gather. */
+ * Returns 0, or REKV_ERR_STATE without a preceding gather.
+ * rekv_retrieve, rekv_gather (page-list mode) and rekv_attend allocate nothing and do not synchronise the host:
+ * on a context whose cache is all in HBM the three calls may be captured into one CUDA graph. */
 int rekv_attend(rekv_ctx* ctx, const void* q, const int32_t* cu_q, int nQ, void* out, void* stream);
 
 /* Eq. 3 in full: O = Attn(W_Q X, [R_k, W_K X], [R_v, W_V X]).  The context of the preceding rekv_gather

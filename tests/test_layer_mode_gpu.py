@@ -139,3 +139,31 @@ def test_layer_call_argument_errors():
         g2.attend_layer(0, q[0], cu)  # nothing gathered yet
     g.close()
     g2.close()
+
+
+def test_all_layer_question_replayed_from_one_cuda_graph():
+    """retrieve -> gather -> attend for all layers captured once (HBM-resident cache) and replayed after the query
+    buffer changed: same bits as the eager calls."""
+    s = H.Shape(L=3, Hq=28, Hkv=4, Nf=196, T=40, W=8, k=12)
+    g = H.build_gpu(s, max_questions=2, max_q_tokens=48)
+    q, cu = H.questions(s, [16, 32], device="cuda")
+    q2, _ = H.questions(s, [16, 32], device="cuda", first_id=11)
+    eager = g.question(q, cu, s.k, s.T).clone()
+    eager2 = g.question(q2, cu, s.k, s.T).clone()
+    qbuf, out = q.clone(), torch.zeros_like(q)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=side):
+            g.question(qbuf, cu, s.k, s.T, out=out)
+    torch.cuda.current_stream().wait_stream(side)
+    gr.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager)
+    qbuf.copy_(q2)
+    gr.replay()
+    torch.cuda.synchronize()
+    g.check_status()
+    assert torch.equal(out, eager2)
+    g.close()
