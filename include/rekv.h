@@ -200,6 +200,13 @@ int rekv_set_frame_embedding(rekv_ctx* ctx, int frame, const float* emb, void* s
 int rekv_retrieve_external(rekv_ctx* ctx, const float* q_emb, int nQ, int top_k, int n_visible, float tau,
                            int32_t* idx_out, float* scores_out, void* stream);
 
+/* Steps 2-5 in one call, for all layers: what rekv_retrieve, rekv_gather (page-list mode) and rekv_attend do
+ * in sequence on the library's own selection, with the same results.  idx_out (nullable): device int32
+ * [L][nQ][top_k].  On a cache that is all in HBM the selection kernel writes the context table itself (one
+ * launch fewer).  Returns the number of context frames, or a negative error code. */
+int rekv_question(rekv_ctx* ctx, const void* q, const int32_t* cu_q, int nQ, int top_k, int n_visible, int32_t* idx_out,
+                  void* out, void* stream);
+
 /* Layer-sequential form of steps 2-5.  A decoder produces layer l+1's queries only from layer l's
  * output, and the paper retrieves independently in every layer, so a model integrates the path one
  * layer at a time: this call enqueues retrieve -> gather -> attend of ONE layer on `stream`.

@@ -179,9 +179,29 @@ __device__ __forceinline__ unsigned score_key(float s) {
 // frames equal to T that are still needed (ties go to the lower index).
 // With block retrieval the candidates are blocks; a selected block b_i is written as its `block` frames
 // b_i*block .. b_i*block + block-1 (k_eff counts items, top_k counts output slots).
+// With tbl != null (cache all in HBM) the block also writes the context table of its (layer, question) -- the
+// selected frames' pages then the trailing frames' pages, as the gather kernel would -- so that no further
+// launch stands between the selection and the attention.
+struct TopkTable {
+  char** tbl;            // [L][nQ][ncf] page pointers, or null
+  char* hbm;
+  long long page_bytes;
+  int L, ncf, n_vis_frames;
+};
+__device__ __forceinline__ void topk_write_table(const TopkTable& t, const int32_t* out, int k_frames, int l, int qi,
+                                                 int nQ) {
+  if (!t.tbl) return;
+  __syncthreads();  // the block's writes of the selection are visible to all its threads
+  char** row = t.tbl + ((long long)l * nQ + qi) * t.ncf;
+  for (int j = threadIdx.x; j < t.ncf; j += blockDim.x) {
+    const int frame = j < k_frames ? out[j] : t.n_vis_frames - (t.ncf - k_frames) + (j - k_frames);
+    row[j] = t.hbm + ((long long)frame * t.L + l) * t.page_bytes;
+  }
+}
+
 __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ scores, int nQ, int n_visible,
                                                    int n_cand, int top_k, int k_eff, int32_t* __restrict__ idx_out,
-                                                   int block, int layer0) {
+                                                   int block, int layer0, TopkTable tt) {
   const int qi = blockIdx.x, l = layer0 + blockIdx.y;
   const float* s = scores + ((long long)l * nQ + qi) * n_visible;
   int32_t* out = idx_out + ((long long)l * nQ + qi) * top_k;
@@ -195,7 +215,10 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
   rekv_ptx::grid_dep_launch();
 
   for (int j = k_eff * block + threadIdx.x; j < top_k; j += blockDim.x) out[j] = -1;
-  if (k_eff <= 0) return;
+  if (k_eff <= 0) {
+    topk_write_table(tt, out, 0, l, qi, nQ);
+    return;
+  }
   if (threadIdx.x == 0) {
     s_prefix = 0u;
     s_krem = k_eff;
@@ -281,6 +304,7 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
     __syncthreads();
   }
   (void)n_gt;
+  topk_write_table(tt, out, k_eff * block, l, qi, nQ);
 }
 
 // ---- external retrieval (Eq. 2 with its temperature): cosine of each question embedding with every frame
@@ -363,7 +387,8 @@ __global__ void replicate_idx_kernel(int32_t* __restrict__ idx, int per_layer, i
 }  // namespace
 
 cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, const CtxGeom& geom,
-                                 int n_visible, int layer0, int layer1, int32_t* idx_out, float* scores, cudaStream_t st) {
+                                 int n_visible, int layer0, int layer1, int32_t* idx_out, float* scores, cudaStream_t st,
+                                 bool write_table) {
   // q, idx_out and scores are indexed with the absolute layer by the kernels; a caller that holds one
   // layer's rows only passes pointers moved back by layer0 layers
   const StoreView& s = c->sv;
@@ -391,8 +416,17 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
     c->launches += 1;
   }
   if (top_k > 0) {
+    TopkTable tt = {};
+    if (write_table) {  // HBM-resident cache: the context table comes out of the same launch
+      tt.tbl = c->ctx_tbl;
+      tt.hbm = s.hbm;
+      tt.page_bytes = s.page_bytes;
+      tt.L = s.L;
+      tt.ncf = geom.ncf;
+      tt.n_vis_frames = n_visible;
+    }
     cudaError_t e2 = rekv_launch_pdl(topk_kernel, dim3(qb.nQ, nl), dim3(512), 0, st, scores, qb.nQ, n_scored,
-                                     geom.n_items, top_k, geom.k_items, idx_out, b, layer0);
+                                     geom.n_items, top_k, geom.k_items, idx_out, b, layer0, tt);
     if (e2 != cudaSuccess) return e2;
     c->launches += 1;
   }
@@ -420,7 +454,7 @@ cudaError_t rekv_launch_retrieve_external(rekv_ctx* c, const float* q_emb, int n
   }
   if (top_k > 0) {
     cudaError_t e2 = rekv_launch_pdl(topk_kernel, dim3(nQ, 1), dim3(512), 0, st, (const float*)scores, nQ, n_scored,
-                                     geom.n_items, top_k, geom.k_items, idx_out, b, 0);
+                                     geom.n_items, top_k, geom.k_items, idx_out, b, 0, TopkTable{});
     if (e2 != cudaSuccess) return e2;
     const int per_layer = nQ * top_k;
     if (s.L > 1) {

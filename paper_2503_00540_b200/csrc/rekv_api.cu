@@ -434,6 +434,44 @@ int rekv_attend(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, void* o
   return REKV_OK;
 }
 
+int rekv_question(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, int top_k, int n_visible, int32_t* idx_out,
+                  void* out, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (!q || !out) REKV_FAIL(c, REKV_ERR_ARG, "null q or out");
+  int32_t* idx = idx_out ? idx_out : c->idx_own;
+  const StoreView& s = c->sv;
+  if (s.tail > 0 || top_k == 0) {  // offloaded cache (or nothing to select): the three calls as they are
+    int rc = rekv_retrieve(c, q, cu_q, nQ, top_k, n_visible, idx, nullptr, stream);
+    if (rc < 0) return rc;
+    const int ncf = rekv_gather(c, idx, nQ, top_k, n_visible, nullptr, nullptr, stream);
+    if (ncf < 0) return ncf;
+    rc = rekv_attend(c, q, cu_q, nQ, out, stream);
+    return rc < 0 ? rc : ncf;
+  }
+  if (top_k < 0 || top_k > c->cfg.max_topk) REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d outside [0, %d]", top_k, c->cfg.max_topk);
+  if (n_visible < 0 || n_visible > c->frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "n_visible=%d outside [0, %d]", n_visible, c->frames);
+  if (n_visible == 0) REKV_FAIL(c, REKV_ERR_EMPTY, "no visible frame");
+  if (top_k % c->cfg.block_frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d must be a multiple of block_frames=%d", top_k, c->cfg.block_frames);
+  QBatch qb;
+  int rc = build_qbatch(c, cu_q, nQ, &qb);
+  if (rc) return rc;
+  DeviceGuard guard(c->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const CtxGeom geom = rekv_geom(n_visible, c->cfg.window_frames, c->cfg.block_frames, top_k);
+  REKV_CUDA(c, rekv_launch_retrieve(c, q, qb, top_k, geom, n_visible, 0, s.L, idx, c->scores, st, true));
+  c->gathered = true;
+  c->gather_layerwise = false;
+  c->g_nQ = nQ;
+  c->g_ncf = geom.ncf;
+  c->g_keff = geom.k_eff;
+  c->g_nvis = n_visible;
+  c->g_topk = top_k;
+  rc = rekv_attend(c, q, cu_q, nQ, out, stream);
+  return rc < 0 ? rc : geom.ncf;
+}
+
 int rekv_question_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu_q, int nQ, int top_k, int n_visible,
                         int32_t* idx_out, void* out, void* stream) {
   if (!c) return REKV_ERR_ARG;
@@ -455,9 +493,12 @@ int rekv_question_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu
   const long long row_bytes = (long long)s.Hq * REKV_HEAD_DIM * 2;
   // the selection goes to the caller's buffer if there is one, else to the context's own
   int32_t* idx = idx_out ? layer_view(idx_out, layer, (long long)nQ * top_k * 4) : c->idx_own;
+  // cache all in HBM: the selection kernel writes the layer's context table itself (top_k > 0 launches it)
+  const bool fused_table = s.tail == 0 && top_k > 0;
   REKV_CUDA(c, rekv_launch_retrieve(c, layer_view(q, layer, qb.sumNq * row_bytes), qb, top_k, geom, n_visible, layer,
-                                    layer + 1, idx, c->scores, st));
-  if (s.tail == 0) {
+                                    layer + 1, idx, c->scores, st, fused_table));
+  if (fused_table) {
+  } else if (s.tail == 0) {
     REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, geom, n_visible, layer, layer + 1, c->frames, st));
   } else {
     REKV_CUDA(c, cudaEventRecord(c->ev_main, st));

@@ -183,7 +183,8 @@ cudaError_t rekv_launch_append(rekv_ctx* c, const void* k, const void* v, int fr
 cudaError_t rekv_launch_unswizzle_page(rekv_ctx* c, const char* page, void* k_out, void* v_out, cudaStream_t st);
 // k_retrieve.cu
 cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, const CtxGeom& geom,
-                                 int n_visible, int layer0, int layer1, int32_t* idx_out, float* scores, cudaStream_t st);
+                                 int n_visible, int layer0, int layer1, int32_t* idx_out, float* scores, cudaStream_t st,
+                                 bool write_table = false);
 cudaError_t rekv_launch_retrieve_external(rekv_ctx* c, const float* q_emb, int nQ, int top_k, const CtxGeom& geom,
                                           int n_visible, float tau, int32_t* idx_out, float* scores, cudaStream_t st);
 // k_gather.cu

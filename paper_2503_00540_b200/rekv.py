@@ -44,7 +44,7 @@ class rekv_stats_t(ctypes.Structure):
 EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", "rekv_gather", "rekv_attend",
            "rekv_stats", "rekv_check_status", "rekv_last_error", "rekv_get_reps", "rekv_get_page",
            "rekv_launch_count", "rekv_score_frames_static", "rekv_question_layer", "rekv_attend_layer", "rekv_attend_full",
-           "rekv_set_frame_embedding", "rekv_retrieve_external")
+           "rekv_set_frame_embedding", "rekv_retrieve_external", "rekv_question")
 
 _lib = None
 
@@ -63,6 +63,7 @@ def lib() -> ctypes.CDLL:
         L.rekv_gather.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
         L.rekv_attend.argtypes = [vp, vp, ip, i32, vp, vp]
         L.rekv_question_layer.argtypes = [vp, i32, vp, ip, i32, i32, i32, vp, vp, vp]
+        L.rekv_question.argtypes = [vp, vp, ip, i32, i32, i32, vp, vp, vp]
         L.rekv_attend_layer.argtypes = [vp, i32, vp, ip, i32, vp, vp]
         L.rekv_attend_full.argtypes = [vp, vp, vp, vp, ip, ip, i32, vp, vp]
         L.rekv_set_frame_embedding.argtypes = [vp, i32, vp, vp]
@@ -195,10 +196,17 @@ class ReKV:
 
     def question(self, q: torch.Tensor, cu_q: Sequence[int], top_k: int, n_visible: int,
                  out: Optional[torch.Tensor] = None, idx: Optional[torch.Tensor] = None) -> torch.Tensor:
-        """retrieve -> gather -> attend for a batch of questions (the calls a user makes, in order)."""
+        """Steps 2-5 for a batch of questions: rekv_question on the library's own selection, or gather + attend on
+        a selection the caller passes."""
         nQ = len(cu_q) - 1
         if idx is None:
-            idx, _, _ = self.retrieve(q, cu_q, top_k, n_visible)
+            if tuple(q.shape) != (self.L, cu_q[-1], self.Hq, self.D):
+                raise ValueError("q must be [L][sum_Nq][H_q][D]")
+            if out is None:
+                out = torch.empty_like(q)
+            self._check(lib().rekv_question(self._h, _ptr(q, torch.bfloat16), _cu_array(cu_q), nQ, top_k, n_visible,
+                                            None, _ptr(out, torch.bfloat16), self._stream()))
+            return out
         self.gather(idx, nQ, top_k, n_visible)
         return self.attend(q, cu_q, out)
 
