@@ -303,6 +303,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         const uint32_t t_o = tmem + lane_base + col_o(t);
         float m_used = -INFINITY, l_sum = 0.f;
         bool ok = true;
+        // a warp whose 32 rows all lie beyond the unit's rows (the ragged second tile) only keeps the barriers moving
+        const bool warp_idle = ui.m0 + t * 128 + ((warp & 3) << 5) >= ui.rows_q;
         for (int i = 0; i < nchunks && ok; ++i) {
           const int part = i % cpf;
           const int tok0 = part ? p.NA : 0, N = part ? p.NB : p.NA;
@@ -313,6 +315,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
             break;
           }
           tc_fence_after();
+          if (warp_idle) {  // no valid row in this warp's 32 lanes: their P and O rows are never read back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bars.p_ready(t));
+            continue;
+          }
           // Online softmax, one pass over S.  S is read from TMEM in groups of two 16-column pieces,
           // the next group's load in flight while the current one is processed.  A group whose
           // scaled maximum exceeds the maximum in use by more than the threshold (always the very
