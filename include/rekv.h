@@ -229,6 +229,14 @@ int rekv_question_layer(rekv_ctx* ctx, int layer, const void* q, const int32_t* 
  * q, out: device bf16 [sum_Nq][H_q][D]; nQ must equal the gathered batch.  Returns 0 or an error code. */
 int rekv_attend_layer(rekv_ctx* ctx, int layer, const void* q, const int32_t* cu_q, int nQ, void* out, void* stream);
 
+/* Disk tier.  rekv_save synchronises the device and writes the context's stream state -- configuration, frame
+ * count, representatives, frame embeddings, every page (host tier as it is held, plus the exact frames of the HBM
+ * tail) -- to `path`.  rekv_load creates a context on `device` from such a file, ready for further appends and
+ * questions: the stream can be encoded by one process and questioned by others.  Both return 0 or an error code
+ * (rekv_last_error(NULL) after a failed load). */
+int rekv_save(rekv_ctx* ctx, const char* path);
+int rekv_load(const char* path, int device, rekv_ctx** out);
+
 /* Fills *out with store accounting and the last call's counters. */
 int rekv_stats(rekv_ctx* ctx, rekv_stats_t* out);
 

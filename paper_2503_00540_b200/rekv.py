@@ -44,7 +44,8 @@ class rekv_stats_t(ctypes.Structure):
 EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", "rekv_gather", "rekv_attend",
            "rekv_stats", "rekv_check_status", "rekv_last_error", "rekv_get_reps", "rekv_get_page",
            "rekv_launch_count", "rekv_score_frames_static", "rekv_question_layer", "rekv_attend_layer", "rekv_attend_full",
-           "rekv_set_frame_embedding", "rekv_retrieve_external", "rekv_question")
+           "rekv_set_frame_embedding", "rekv_retrieve_external", "rekv_question",
+           "rekv_save", "rekv_load")
 
 _lib = None
 
@@ -64,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.rekv_attend.argtypes = [vp, vp, ip, i32, vp, vp]
         L.rekv_question_layer.argtypes = [vp, i32, vp, ip, i32, i32, i32, vp, vp, vp]
         L.rekv_question.argtypes = [vp, vp, ip, i32, i32, i32, vp, vp, vp]
+        L.rekv_save.argtypes = [vp, ctypes.c_char_p]
+        L.rekv_load.argtypes = [ctypes.c_char_p, i32, ctypes.POINTER(vp)]
         L.rekv_attend_layer.argtypes = [vp, i32, vp, ip, i32, vp, vp]
         L.rekv_attend_full.argtypes = [vp, vp, vp, vp, ip, ip, i32, vp, vp]
         L.rekv_set_frame_embedding.argtypes = [vp, i32, vp, vp]
@@ -118,6 +121,28 @@ class ReKV:
         self.L, self.Hq, self.Hkv, self.D, self.Nf, self.W = (n_layers, n_q_heads, n_kv_heads, head_dim,
                                                               tokens_per_frame, window_frames)
         self.b = block_frames
+
+    def save(self, path: str) -> None:
+        """Writes the stream state (representatives, embeddings, every page) to a file."""
+        self._check(lib().rekv_save(self._h, path.encode()))
+
+    @classmethod
+    def load(cls, path: str, device: int = 0) -> "ReKV":
+        """A context created from a file written by save(), ready for further appends and questions."""
+        h = ctypes.c_void_p()
+        rc = lib().rekv_load(path.encode(), device, ctypes.byref(h))
+        if rc != 0:
+            raise RekvError(rc, (lib().rekv_last_error(None) or b"").decode())
+        self = cls.__new__(cls)
+        self._h = h
+        self.device = torch.device("cuda", device)
+        cfg = rekv_config.from_buffer_copy(open(path, "rb").read(8 + ctypes.sizeof(rekv_config))[8:])
+        cfg.device = device
+        self.cfg = cfg
+        self.L, self.Hq, self.Hkv, self.D, self.Nf, self.W = (cfg.n_layers, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim,
+                                                              cfg.tokens_per_frame, cfg.window_frames)
+        self.b = cfg.block_frames
+        return self
 
     def geometry(self, n_visible: int, top_k: int) -> Tuple[int, int, int]:
         """(retrieval candidates, frames retrieved, trailing frames always in the context) -- the sizes the
