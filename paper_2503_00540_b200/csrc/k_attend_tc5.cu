@@ -22,6 +22,22 @@
 
 using namespace rekv_ptx;
 
+// Optional cycle-stamp tracing of CTA 0 (compile with -DREKV_TRACE; never part of the shipped library):
+// slot layout is [role][chunk][event]; rekv_trace_read copies the stamps out.
+#ifdef REKV_TRACE
+__device__ long long g_rekv_trace[8192];
+#define REKV_STAMP(role, i, ev)                                                                  \
+  do {                                                                                           \
+    if (blockIdx.x == 0 && lane == 0 && (i) < 64) g_rekv_trace[(role) * 1024 + (i) * 8 + (ev)] = clock64(); \
+  } while (0)
+extern "C" int rekv_trace_read(long long* host, int n) {
+  cudaDeviceSynchronize();
+  return (int)cudaMemcpyFromSymbol(host, g_rekv_trace, n * sizeof(long long));
+}
+#else
+#define REKV_STAMP(role, i, ev) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int TC_THREADS = 320;
@@ -281,11 +297,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         REKV_ISSUE_S(0, 0);
         if (tiles == 2 && ok) REKV_ISSUE_S(1, 0);
         for (int i = 0; i < nchunks && ok; ++i) {
+          REKV_STAMP(0, i, 0);
           REKV_ISSUE_PV(0, i);
+          REKV_STAMP(0, i, 1);
           if (i + 1 < nchunks && ok) REKV_ISSUE_S(0, i + 1);
+          REKV_STAMP(0, i, 2);
           if (tiles == 2 && ok) {
             REKV_ISSUE_PV(1, i);
+            REKV_STAMP(0, i, 3);
             if (i + 1 < nchunks && ok) REKV_ISSUE_S(1, i + 1);
+            REKV_STAMP(0, i, 4);
           }
         }
 #undef REKV_ISSUE_S
@@ -310,11 +331,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
           const int tok0 = part ? p.NA : 0, N = part ? p.NB : p.NA;
           const int nv = min(N, p.Nf - tok0);  // valid tokens of this chunk
           const int npc = N >> 4;
+          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 0);
           if (!wait(bars.s_full(t), (chunk_cnt[t] + i) & 1)) {
             ok = false;
             break;
           }
           tc_fence_after();
+          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 1);
           if (warp_idle) {  // no valid row in this warp's 32 lanes: their P and O rows are never read back
             tc_fence_before();
             __syncwarp();
@@ -429,6 +452,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
               tmem_wait_ld16(a1);
             }
             tmem_wait_ld16(a0);
+            if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 4);
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
               const int pa = 4 * h, pb = 4 * h + 2;
@@ -438,14 +462,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
                   if (pb + 1 < npc) tmem_ld16(t_s + (pb + 1) * 16, b1);
                 }
                 do_group(a0, a1, pa);
+                if ((warp & 3) == 2 && h == 0) REKV_STAMP(1 + t, i, 5);
                 if (pb < npc) {
                   if (pb + 1 < npc) tmem_wait_ld16(b1);
                   tmem_wait_ld16(b0);
+                  if ((warp & 3) == 2 && h == 0) REKV_STAMP(1 + t, i, 6);
                   if (pa + 4 < npc) {
                     tmem_ld16(t_s + (pa + 4) * 16, a0);
                     if (pa + 5 < npc) tmem_ld16(t_s + (pa + 5) * 16, a1);
                   }
                   do_group(b0, b1, pb);
+                  if ((warp & 3) == 2 && h == 0) REKV_STAMP(1 + t, i, 7);
                   if (pa + 4 < npc) {
                     if (pa + 5 < npc) tmem_wait_ld16(a1);
                     tmem_wait_ld16(a0);
@@ -455,10 +482,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
             }
           }
           l_sum += (ps0 + ps1) + (ps2 + ps3);
+          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 2);
           tmem_wait_st();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bars.p_ready(t));
+          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 3);
         }
         // ---- output of this range: final rows, or a partial for the combine kernel ----
         if (ok && wait(bars.pv_done(t), (chunk_cnt[t] + nchunks - 1) & 1)) {
