@@ -8,14 +8,21 @@
 // to both row tiles.  Warp roles:
 //   warp 0      bulk copies of K/V tiles into a 3-deep shared-memory ring (one lane)
 //   warp 1      tcgen05.mma issue (one lane): S = Q K^T into TMEM, O += P V with P read from TMEM
-//   warps 2-5   softmax of row tile 0: one thread per row (= TMEM lane), fp32, lazy rescaling of O
-//   warps 6-9   softmax of row tile 1 -- the two tiles alternate on the tensor core, so one tile's
+//               (warps 2, 3 idle: the service warps form one warpgroup and give their registers up)
+//   warps 4-7   softmax of row tile 0: one thread per row (= TMEM lane), fp32, lazy rescaling of O
+//   warps 8-11  softmax of row tile 1 -- the two tiles alternate on the tensor core, so one tile's
 //               softmax overlaps the other's matrix products
+// After set-up the service warpgroup shrinks to 72 registers per thread and the softmax warpgroups grow to
+// 216 (setmaxnreg), so that a softmax thread holds a whole S row chunk (up to 112 values) at once: one
+// TMEM load phase with wide loads, one wait, one maximum and one rescaling decision per chunk.  The chunk's
+// last 16-column piece, the only one that can hold a frame's pad tokens, always lands in the same registers,
+// so masking touches 16 values instead of being predicated over the whole chunk.
 // TMEM (512 columns): O0 [0,128)  O1 [128,256)  S0/P0 [256,384)  S1/P1 [384,512); P (bf16) overwrites
 // the front of its S.  A frame of N_f tokens is processed as one or two token chunks of <= 128.
 // A range that does not cover a whole unit leaves (max, sum, O) partials for the combine kernel.
 // Every wait is bounded: on expiry the status word is set and the CTA leaves.
 #include <algorithm>
+#include <type_traits>
 
 #include "ptx_helpers.cuh"
 #include "rekv_internal.cuh"
@@ -40,7 +47,9 @@ extern "C" int rekv_trace_read(long long* host, int n) {
 
 namespace {
 
-constexpr int TC_THREADS = 320;
+constexpr int TC_THREADS = 384;
+constexpr int SM_WARP0 = 4;                            // first softmax warp
+constexpr int REGS_SERVICE = 72, REGS_SOFTMAX = 216;   // 128 * service + 256 * softmax <= 384 * 168
 constexpr int KV_BUFS = 3;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t Q_TILE_BYTES = 128 * 256;  // 128 rows x 128 dims bf16
@@ -178,6 +187,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   const uint32_t half_bytes = (uint32_t)p.Nf * 128u;
   const uint32_t idesc_pv = idesc_bf16(128, 128, 1);
 
+  // The roles run the same range loop with the role as a compile-time constant, so that each side of the
+  // register reallocation below is compiled against its own register budget.
+  auto run = [&](auto role) {
+  constexpr bool SOFTMAX = decltype(role)::value;
   long long pos = (long long)blockIdx.x * p.per;
   const long long end = min(pos + (long long)p.per, p.total);
   uint32_t ring = 0;    // K/V tiles moved so far (K and V of a frame are consecutive ring entries)
@@ -194,8 +207,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     const bool whole_unit = (nfr == p.ncf);
 
     // ---- Q row tiles -> shared memory in the swizzled K-major operand layout -------------------
-    if (warp >= 2) {
-      const int t = (warp - 2) >> 2;
+    if (warp >= SM_WARP0) {
+      const int t = (warp - SM_WARP0) >> 2;
       const int row = ((warp & 3) << 5) | lane;
       if (t < ui.tiles) {
         const int rr = ui.m0 + t * 128 + row;
@@ -214,6 +227,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     }
     __syncthreads();
 
+    if constexpr (!SOFTMAX) {
     if (warp == 0) {
       // ================= copy producer =================
       // the whole warp walks the ring (uniform control flow); one elected lane issues the copies
@@ -314,9 +328,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
 #undef REKV_DESC
       }
       __syncwarp();
+    }
     } else {
       // ================= softmax + output, one thread per row =================
-      const int t = (warp - 2) >> 2;
+      const int t = (warp - SM_WARP0) >> 2;
       if (t < ui.tiles) {
         const uint32_t lane_base = (uint32_t)((warp & 3) << 5) << 16;
         const int row = ((warp & 3) << 5) | lane;
@@ -344,81 +359,86 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
             if (lane == 0) mbar_arrive(bars.p_ready(t));
             continue;
           }
-          // Online softmax, one pass over S.  S is read from TMEM in groups of two 16-column pieces,
-          // the next group's load in flight while the current one is processed.  A group whose
-          // scaled maximum exceeds the maximum in use by more than the threshold (always the very
-          // first group) raises it: P pieces already written for this chunk, this chunk's partial
-          // sums, the running sum and O are rescaled by 2^(m_old - m_new).  This is rare after the
-          // first chunk, so the common path has no second read of S and no rescaling.
+          // The whole S row chunk comes into registers in one load phase (up to seven 16-column pieces), so there
+          // is one wait, one row maximum and one rescaling decision per chunk.  Lazy rescaling: the maximum in
+          // use is raised only when this chunk exceeds it by more than the threshold (always on the first
+          // chunk); O and the running sum then shrink by 2^(old - new).
           const float NEG_INF = -INFINITY;
+          const int npm = npc - 1;  // pieces before the chunk's last one, which always sits in sv[7]
+          uint32_t sv[8][16];
+#pragma unroll
+          for (int pc = 0; pc < 7; ++pc) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) sv[pc][j] = 0u;
+          }
+          if (npm >= 4) {
+            tmem_ld64(t_s, sv[0], sv[1], sv[2], sv[3]);
+            if (npm >= 6) tmem_ld32(t_s + 64, sv[4], sv[5]);
+            if (npm == 5) tmem_ld16(t_s + 64, sv[4]);
+            if (npm == 7) tmem_ld16(t_s + 96, sv[6]);
+          } else {
+            if (npm >= 2) tmem_ld32(t_s, sv[0], sv[1]);
+            if (npm == 1) tmem_ld16(t_s, sv[0]);
+            if (npm == 3) tmem_ld16(t_s + 32, sv[2]);
+          }
+          tmem_ld16(t_s + npm * 16, sv[7]);
+          tmem_wait_ld_chunk(sv);
+          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 4);
+          {  // the frame's ragged end lies inside the last piece: its pad tokens leave the maximum and the sum
+            const int nvt = nv - npm * 16;
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (j >= nvt) sv[7][j] = __float_as_uint(NEG_INF);
+          }
+          float g0 = max3(__uint_as_float(sv[7][0]), __uint_as_float(sv[7][1]), __uint_as_float(sv[7][2]));
+          float g1 = max3(__uint_as_float(sv[7][3]), __uint_as_float(sv[7][4]), __uint_as_float(sv[7][5]));
+          float g2 = max3(__uint_as_float(sv[7][6]), __uint_as_float(sv[7][7]), __uint_as_float(sv[7][8]));
+          float g3 = max3(__uint_as_float(sv[7][9]), __uint_as_float(sv[7][10]), __uint_as_float(sv[7][11]));
+          g0 = max3(g0, __uint_as_float(sv[7][12]), __uint_as_float(sv[7][13]));
+          g1 = max3(g1, __uint_as_float(sv[7][14]), __uint_as_float(sv[7][15]));
+#pragma unroll
+          for (int pc = 0; pc < 7; ++pc)
+            if (pc < npm) {
+              g0 = max3(g0, __uint_as_float(sv[pc][0]), __uint_as_float(sv[pc][1]));
+              g1 = max3(g1, __uint_as_float(sv[pc][2]), __uint_as_float(sv[pc][3]));
+              g2 = max3(g2, __uint_as_float(sv[pc][4]), __uint_as_float(sv[pc][5]));
+              g3 = max3(g3, __uint_as_float(sv[pc][6]), __uint_as_float(sv[pc][7]));
+              g0 = max3(g0, __uint_as_float(sv[pc][8]), __uint_as_float(sv[pc][9]));
+              g1 = max3(g1, __uint_as_float(sv[pc][10]), __uint_as_float(sv[pc][11]));
+              g2 = max3(g2, __uint_as_float(sv[pc][12]), __uint_as_float(sv[pc][13]));
+              g3 = max3(g3, __uint_as_float(sv[pc][14]), __uint_as_float(sv[pc][15]));
+            }
+          const float gm = fmaxf(fmaxf(g0, g1), fmaxf(g2, g3)) * p.scale_log2;
+          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 6);
+          const bool need = gm > m_used + RESCALE_THRESHOLD;
+          if (__any_sync(0xffffffffu, need)) {
+            const float alpha = need ? ex2(m_used - gm) : 1.f;  // 0 when nothing has been seen yet
+            if (need) m_used = gm;
+            l_sum *= alpha;
+            if (i > 0) {  // O holds earlier chunks; their P V is complete (this chunk's S came after it)
+#pragma unroll 1
+              for (int pc = 0; pc < 8; ++pc) {
+                uint32_t o[16];
+                tmem_ld16(t_o + pc * 16, o);
+                tmem_wait_ld16(o);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+                tmem_st16(t_o + pc * 16, o);
+              }
+            }
+          }
+          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 5);
+          // P = 2^(S*scale - m) as bf16 pairs over the front of S, row sum in fp32
+          const float neg_m = -m_used;
           float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
-          auto do_group = [&](uint32_t (&a)[16], uint32_t (&b)[16], const int pc0) {
-            const bool has_b = pc0 + 1 < npc;
-            if (pc0 * 16 + 32 > nv) {  // the group that holds the frame's ragged end: mask the pad tokens
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                if (pc0 * 16 + j >= nv) a[j] = __float_as_uint(NEG_INF);
-                if (pc0 * 16 + 16 + j >= nv) b[j] = __float_as_uint(NEG_INF);
-              }
-            }
-            float g0 = max3(__uint_as_float(a[0]), __uint_as_float(a[1]), __uint_as_float(a[2]));
-            float g1 = max3(__uint_as_float(a[3]), __uint_as_float(a[4]), __uint_as_float(a[5]));
-            float g2 = max3(__uint_as_float(a[6]), __uint_as_float(a[7]), __uint_as_float(a[8]));
-            float g3 = max3(__uint_as_float(a[9]), __uint_as_float(a[10]), __uint_as_float(a[11]));
-            g0 = max3(g0, __uint_as_float(a[12]), __uint_as_float(a[13]));
-            g1 = max3(g1, __uint_as_float(a[14]), __uint_as_float(a[15]));
-            if (has_b) {
-              g2 = max3(g2, __uint_as_float(b[0]), __uint_as_float(b[1]));
-              g3 = max3(g3, __uint_as_float(b[2]), __uint_as_float(b[3]));
-              g0 = max3(g0, __uint_as_float(b[4]), __uint_as_float(b[5]));
-              g1 = max3(g1, __uint_as_float(b[6]), __uint_as_float(b[7]));
-              g2 = max3(g2, __uint_as_float(b[8]), __uint_as_float(b[9]));
-              g3 = max3(g3, __uint_as_float(b[10]), __uint_as_float(b[11]));
-              g0 = max3(g0, __uint_as_float(b[12]), __uint_as_float(b[13]));
-              g1 = max3(g1, __uint_as_float(b[14]), __uint_as_float(b[15]));
-            }
-            const float gm = fmaxf(fmaxf(g0, g1), fmaxf(g2, g3)) * p.scale_log2;
-            const bool need = gm > m_used + RESCALE_THRESHOLD;
-            if (__any_sync(0xffffffffu, need)) {
-              const float alpha = need ? ex2(m_used - gm) : 1.f;  // 0 when nothing has been seen yet
-              if (need) m_used = gm;
-#pragma unroll 1
-              for (int q = 0; q < pc0; ++q) {  // P pieces of this chunk written under the old maximum
-                uint32_t w[8];
-                tmem_ld8(t_s + q * 8, w);
-                tmem_wait_ld8(w);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  const float lo = __uint_as_float(w[e] << 16) * alpha, hi = __uint_as_float(w[e] & 0xFFFF0000u) * alpha;
-                  w[e] = pack_bf16(lo, hi);
-                }
-                tmem_st8(t_s + q * 8, w);
-              }
-              l_sum *= alpha;
-              ps0 *= alpha;
-              ps1 *= alpha;
-              ps2 *= alpha;
-              ps3 *= alpha;
-              if (i > 0) {  // O holds earlier chunks; their P V is complete (this chunk's S came after it)
-#pragma unroll 1
-                for (int pc = 0; pc < 8; ++pc) {
-                  uint32_t o[16];
-                  tmem_ld16(t_o + pc * 16, o);
-                  tmem_wait_ld16(o);
-#pragma unroll
-                  for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-                  tmem_st16(t_o + pc * 16, o);
-                }
-              }
-            }
-            const float neg_m = -m_used;
+          auto do_piece = [&](const uint32_t (&v)[16], const uint32_t col) {
             uint32_t pk[8];
 #pragma unroll
             for (int jj = 0; jj < 8; jj += 2) {
-              const float p0 = ex2(fmaf(__uint_as_float(a[2 * jj]), p.scale_log2, neg_m));
-              const float p1 = ex2(fmaf(__uint_as_float(a[2 * jj + 1]), p.scale_log2, neg_m));
-              const float p2 = ex2(fmaf(__uint_as_float(a[2 * jj + 2]), p.scale_log2, neg_m));
-              const float p3 = ex2(fmaf(__uint_as_float(a[2 * jj + 3]), p.scale_log2, neg_m));
+              const float p0 = ex2(fmaf(__uint_as_float(v[2 * jj]), p.scale_log2, neg_m));
+              const float p1 = ex2(fmaf(__uint_as_float(v[2 * jj + 1]), p.scale_log2, neg_m));
+              const float p2 = ex2(fmaf(__uint_as_float(v[2 * jj + 2]), p.scale_log2, neg_m));
+              const float p3 = ex2(fmaf(__uint_as_float(v[2 * jj + 3]), p.scale_log2, neg_m));
               ps0 += p0;
               ps1 += p1;
               ps2 += p2;
@@ -426,61 +446,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
               pk[jj] = pack_bf16(p0, p1);
               pk[jj + 1] = pack_bf16(p2, p3);
             }
-            tmem_st8(t_s + pc0 * 8, pk);
-            if (has_b) {
-#pragma unroll
-              for (int jj = 0; jj < 8; jj += 2) {
-                const float p0 = ex2(fmaf(__uint_as_float(b[2 * jj]), p.scale_log2, neg_m));
-                const float p1 = ex2(fmaf(__uint_as_float(b[2 * jj + 1]), p.scale_log2, neg_m));
-                const float p2 = ex2(fmaf(__uint_as_float(b[2 * jj + 2]), p.scale_log2, neg_m));
-                const float p3 = ex2(fmaf(__uint_as_float(b[2 * jj + 3]), p.scale_log2, neg_m));
-                ps0 += p0;
-                ps1 += p1;
-                ps2 += p2;
-                ps3 += p3;
-                pk[jj] = pack_bf16(p0, p1);
-                pk[jj + 1] = pack_bf16(p2, p3);
-              }
-              tmem_st8(t_s + (pc0 + 1) * 8, pk);
-            }
+            tmem_st8(t_s + col, pk);
           };
-          {
-            uint32_t a0[16], a1[16], b0[16], b1[16];
-            tmem_ld16(t_s, a0);
-            if (npc > 1) {
-              tmem_ld16(t_s + 16, a1);
-              tmem_wait_ld16(a1);
-            }
-            tmem_wait_ld16(a0);
-            if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 4);
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              const int pa = 4 * h, pb = 4 * h + 2;
-              if (pa < npc) {
-                if (pb < npc) {  // next group in flight while this one is processed
-                  tmem_ld16(t_s + pb * 16, b0);
-                  if (pb + 1 < npc) tmem_ld16(t_s + (pb + 1) * 16, b1);
-                }
-                do_group(a0, a1, pa);
-                if ((warp & 3) == 2 && h == 0) REKV_STAMP(1 + t, i, 5);
-                if (pb < npc) {
-                  if (pb + 1 < npc) tmem_wait_ld16(b1);
-                  tmem_wait_ld16(b0);
-                  if ((warp & 3) == 2 && h == 0) REKV_STAMP(1 + t, i, 6);
-                  if (pa + 4 < npc) {
-                    tmem_ld16(t_s + (pa + 4) * 16, a0);
-                    if (pa + 5 < npc) tmem_ld16(t_s + (pa + 5) * 16, a1);
-                  }
-                  do_group(b0, b1, pb);
-                  if ((warp & 3) == 2 && h == 0) REKV_STAMP(1 + t, i, 7);
-                  if (pa + 4 < npc) {
-                    if (pa + 5 < npc) tmem_wait_ld16(a1);
-                    tmem_wait_ld16(a0);
-                  }
-                }
-              }
-            }
-          }
+          for (int pc = 0; pc < 7; ++pc)
+            if (pc < npm) do_piece(sv[pc], pc * 8);
+          do_piece(sv[7], npm * 8);
           l_sum += (ps0 + ps1) + (ps2 + ps3);
           if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 2);
           tmem_wait_st();
@@ -573,6 +544,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     __syncthreads();
     tc_fence_after();
     if (*s_abort) break;
+  }
+
+  };
+  if (warp < SM_WARP0) {
+    reg_dealloc<REGS_SERVICE>();
+    run(std::false_type{});
+  } else {
+    reg_alloc<REGS_SOFTMAX>();
+    run(std::true_type{});
   }
 
   __syncthreads();
