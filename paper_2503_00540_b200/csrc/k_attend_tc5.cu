@@ -29,13 +29,16 @@
 
 using namespace rekv_ptx;
 
-// Optional cycle-stamp tracing of CTA 0 (compile with -DREKV_TRACE; never part of the shipped library):
+// Optional cycle-stamp tracing of one CTA (compile with -DREKV_TRACE [-DREKV_TRACE_CTA=n]; never part of the shipped library):
 // slot layout is [role][chunk][event]; rekv_trace_read copies the stamps out.
 #ifdef REKV_TRACE
+#ifndef REKV_TRACE_CTA
+#define REKV_TRACE_CTA 0
+#endif
 __device__ long long g_rekv_trace[8192];
 #define REKV_STAMP(role, i, ev)                                                                  \
   do {                                                                                           \
-    if (blockIdx.x == 0 && lane == 0 && (i) < 64) g_rekv_trace[(role) * 1024 + (i) * 8 + (ev)] = clock64(); \
+    if (blockIdx.x == REKV_TRACE_CTA && lane == 0 && (i) < 64) g_rekv_trace[(role) * 1024 + (i) * 8 + (ev)] = clock64(); \
   } while (0)
 extern "C" int rekv_trace_read(long long* host, int n) {
   cudaDeviceSynchronize();
@@ -53,6 +56,8 @@ constexpr int REGS_SERVICE = 72, REGS_SOFTMAX = 216;   // 128 * service + 256 * 
 constexpr int KV_BUFS = 3;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t Q_TILE_BYTES = 128 * 256;  // 128 rows x 128 dims bf16
+constexpr uint32_t STAGE_ROW_F32 = 144, STAGE_ROW_BF16 = 80;  // epilogue staging rows: a quarter row + 16 bytes (no bank conflicts)
+constexpr uint32_t STAGE_WARP_BYTES = 32 * STAGE_ROW_F32;
 constexpr float RESCALE_THRESHOLD = 8.f;      // log2 units: O is rescaled only when the row max grows by > 2^8
 
 struct TcParams {
@@ -131,6 +136,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   volatile uint32_t* s_abort = s_tmem_slot + 1;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (warp == 6) REKV_STAMP(3, 0, 0);
 
   // ---- one-time set-up -------------------------------------------------------------------------
   {  // zero the pad rows [Nf, Npad) of every ring tile half; the bulk copies never write them
@@ -167,7 +173,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   tc_fence_after();
   const uint32_t tmem = *s_tmem_slot;
   // everything above is independent of earlier kernels; the context table and Q are not
+  if (warp == 6) REKV_STAMP(3, 0, 1);
   grid_dep_wait();
+  if (warp == 6) REKV_STAMP(3, 0, 2);
   grid_dep_launch();
   auto col_o = [](int t) { return (uint32_t)t * 128u; };
   auto col_s = [](int t) { return 256u + (uint32_t)t * 128u; };
@@ -184,6 +192,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   };
 
   const int cpf = p.NB > 0 ? 2 : 1;                 // token chunks per frame
+  // Barrier of a range segment for every warp but the copy producer, which runs ahead into the next segment (it is
+  // held back by the ring's empty barriers only), so that K/V tiles are already on their way during an epilogue.
+  auto seg_sync = [&]() {
+    if (warp != 0) asm volatile("bar.sync 1, %0;" ::"n"(TC_THREADS - 32) : "memory");
+  };
   const uint32_t half_bytes = (uint32_t)p.Nf * 128u;
   const uint32_t idesc_pv = idesc_bf16(128, 128, 1);
 
@@ -196,6 +209,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   uint32_t ring = 0;    // K/V tiles moved so far (K and V of a frame are consecutive ring entries)
   uint32_t chunk_cnt[2] = {0u, 0u};  // token chunks processed so far, per row tile (barrier phases)
 
+  int seg = 0;  // range segments so far (tracing only)
   while (pos < end) {
     const long long u = pos / p.ncf;
     const int f0 = (int)(pos - u * p.ncf);
@@ -205,6 +219,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     char* const* pages = p.tbl + ((long long)ui.l * p.qb.nQ + ui.qi) * p.ncf + f0;
     char* const* pages_k = (FULL && p.tbl_k) ? p.tbl_k + ((long long)ui.l * p.qb.nQ + ui.qi) * p.ncf + f0 : nullptr;
     const bool whole_unit = (nfr == p.ncf);
+    if (warp == 6) REKV_STAMP(3, 1 + seg, 0);
 
     // ---- Q row tiles -> shared memory in the swizzled K-major operand layout -------------------
     if (warp >= SM_WARP0) {
@@ -217,15 +232,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         const uint4* src =
             reinterpret_cast<const uint4*>(p.q + ((ui.q_row0 + (valid ? n : 0)) * p.Hq + ui.g * p.G + (valid ? j : 0)) * 128);
         unsigned char* dst = smem + t * Q_TILE_BYTES + row * 128;
+        uint4 x[16];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          uint4 x = valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
-          *reinterpret_cast<uint4*>(dst + (c >> 3) * (Q_TILE_BYTES / 2) + (((c & 7) ^ (row & 7)) << 4)) = x;
-        }
+        for (int c = 0; c < 16; ++c) x[c] = valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+          *reinterpret_cast<uint4*>(dst + (c >> 3) * (Q_TILE_BYTES / 2) + (((c & 7) ^ (row & 7)) << 4)) = x[c];
       }
       fence_proxy_async();
     }
-    __syncthreads();
+    seg_sync();
+    if (warp == 6) REKV_STAMP(3, 1 + seg, 1);
 
     if constexpr (!SOFTMAX) {
     if (warp == 0) {
@@ -342,7 +359,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         // a warp whose 32 rows all lie beyond the unit's rows (the ragged second tile) only keeps the barriers moving
         const bool warp_idle = ui.m0 + t * 128 + ((warp & 3) << 5) >= ui.rows_q;
         for (int i = 0; i < nchunks && ok; ++i) {
-          const int part = i % cpf;
+          const int part = cpf == 2 ? (i & 1) : 0;
           const int tok0 = part ? p.NA : 0, N = part ? p.NB : p.NA;
           const int nv = min(N, p.Nf - tok0);  // valid tokens of this chunk
           const int npc = N >> 4;
@@ -463,13 +480,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         // ---- output of this range: final rows, or a partial for the combine kernel ----
         if (ok && wait(bars.pv_done(t), (chunk_cnt[t] + nchunks - 1) & 1)) {
           tc_fence_after();
+          if (warp == 6) REKV_STAMP(3, 1 + seg, 2);
           const int rr = ui.m0 + t * 128 + row;
           const bool valid = rr < ui.rows_q;
           const int n = rr / p.G, j = rr - n * p.G;
+          // Rows leave through this warp's staging rows in the tile's Q region (no product reads Q any more), a
+          // quarter of the 128 columns at a time, so that the global stores are contiguous per row instead of one
+          // 16-byte piece per lane in 32 different rows.
+          unsigned char* stage = smem + t * Q_TILE_BYTES + (warp & 3) * STAGE_WARP_BYTES;
+          const int rr0 = ui.m0 + t * 128 + ((warp & 3) << 5);  // first row of this warp
           if (whole_unit) {
             float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
             const long long out_row = (ui.q_row0 + (valid ? n : 0)) * p.Hq + ui.g * p.G + (valid ? j : 0);
-            uint4* dst = reinterpret_cast<uint4*>(p.out + out_row * 128);
             // Eq. 3 in full: the part over the tokens of X joins here, O = (O_c w_c + O_x w_x) / (l_c w_c + l_x w_x)
             float w_x = 0.f;
             const float4* o_x = nullptr;
@@ -483,50 +505,81 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
               w_x = den > 0.f ? w_x / den : 0.f;
               o_x = reinterpret_cast<const float4*>(p.self_o + out_row * 128);
             }
-            const float mul = (FULL && o_x) ? 1.f : inv;  // the merged values below are final already
+            // rows this lane stores: r = 8 k + (lane >> 2), 16 bytes (8 bf16) at chunk (lane & 3) of the quarter
+            __nv_bfloat16* dst_k[4];
 #pragma unroll
-            for (int pc = 0; pc < 8; ++pc) {
-              uint32_t o[16];
-              tmem_ld16(t_o + pc * 16, o);
-              tmem_wait_ld16(o);
-              if (FULL && o_x) {
+            for (int k = 0; k < 4; ++k) {
+              const int r2 = rr0 + 8 * k + (lane >> 2);
+              const int n2 = r2 / p.G, j2 = r2 - n2 * p.G;
+              dst_k[k] = r2 < ui.rows_q ? p.out + ((ui.q_row0 + n2) * p.Hq + ui.g * p.G + j2) * 128 + (lane & 3) * 8 : nullptr;
+            }
+#pragma unroll 1
+            for (int qd = 0; qd < 4; ++qd) {
+              uint32_t o[2][16];
+              tmem_ld16(t_o + qd * 32, o[0]);
+              tmem_ld16(t_o + qd * 32 + 16, o[1]);
+              tmem_wait_ld16(o[0]);
+              tmem_wait_ld16(o[1]);
 #pragma unroll
-                for (int v4 = 0; v4 < 4; ++v4) {
-                  const float4 x = __ldg(o_x + pc * 4 + v4);
-                  o[4 * v4] = __float_as_uint(__uint_as_float(o[4 * v4]) * inv + x.x * w_x);
-                  o[4 * v4 + 1] = __float_as_uint(__uint_as_float(o[4 * v4 + 1]) * inv + x.y * w_x);
-                  o[4 * v4 + 2] = __float_as_uint(__uint_as_float(o[4 * v4 + 2]) * inv + x.z * w_x);
-                  o[4 * v4 + 3] = __float_as_uint(__uint_as_float(o[4 * v4 + 3]) * inv + x.w * w_x);
+              for (int h = 0; h < 2; ++h) {
+                if (FULL && o_x) {
+#pragma unroll
+                  for (int v4 = 0; v4 < 4; ++v4) {
+                    const float4 x = __ldg(o_x + qd * 8 + h * 4 + v4);
+                    o[h][4 * v4] = __float_as_uint(__uint_as_float(o[h][4 * v4]) * inv + x.x * w_x);
+                    o[h][4 * v4 + 1] = __float_as_uint(__uint_as_float(o[h][4 * v4 + 1]) * inv + x.y * w_x);
+                    o[h][4 * v4 + 2] = __float_as_uint(__uint_as_float(o[h][4 * v4 + 2]) * inv + x.z * w_x);
+                    o[h][4 * v4 + 3] = __float_as_uint(__uint_as_float(o[h][4 * v4 + 3]) * inv + x.w * w_x);
+                  }
+                } else {
+#pragma unroll
+                  for (int e = 0; e < 16; ++e) o[h][e] = __float_as_uint(__uint_as_float(o[h][e]) * inv);
                 }
+                uint4 a, b;
+                a.x = pack_bf16(__uint_as_float(o[h][0]), __uint_as_float(o[h][1]));
+                a.y = pack_bf16(__uint_as_float(o[h][2]), __uint_as_float(o[h][3]));
+                a.z = pack_bf16(__uint_as_float(o[h][4]), __uint_as_float(o[h][5]));
+                a.w = pack_bf16(__uint_as_float(o[h][6]), __uint_as_float(o[h][7]));
+                b.x = pack_bf16(__uint_as_float(o[h][8]), __uint_as_float(o[h][9]));
+                b.y = pack_bf16(__uint_as_float(o[h][10]), __uint_as_float(o[h][11]));
+                b.z = pack_bf16(__uint_as_float(o[h][12]), __uint_as_float(o[h][13]));
+                b.w = pack_bf16(__uint_as_float(o[h][14]), __uint_as_float(o[h][15]));
+                *reinterpret_cast<uint4*>(stage + lane * STAGE_ROW_BF16 + h * 32) = a;
+                *reinterpret_cast<uint4*>(stage + lane * STAGE_ROW_BF16 + h * 32 + 16) = b;
               }
-              uint4 a, b;
-              a.x = pack_bf16(__uint_as_float(o[0]) * mul, __uint_as_float(o[1]) * mul);
-              a.y = pack_bf16(__uint_as_float(o[2]) * mul, __uint_as_float(o[3]) * mul);
-              a.z = pack_bf16(__uint_as_float(o[4]) * mul, __uint_as_float(o[5]) * mul);
-              a.w = pack_bf16(__uint_as_float(o[6]) * mul, __uint_as_float(o[7]) * mul);
-              b.x = pack_bf16(__uint_as_float(o[8]) * mul, __uint_as_float(o[9]) * mul);
-              b.y = pack_bf16(__uint_as_float(o[10]) * mul, __uint_as_float(o[11]) * mul);
-              b.z = pack_bf16(__uint_as_float(o[12]) * mul, __uint_as_float(o[13]) * mul);
-              b.w = pack_bf16(__uint_as_float(o[14]) * mul, __uint_as_float(o[15]) * mul);
-              if (valid) {
-                dst[pc * 2] = a;
-                dst[pc * 2 + 1] = b;
+              __syncwarp();
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const uint4 x = *reinterpret_cast<const uint4*>(stage + (8 * k + (lane >> 2)) * STAGE_ROW_BF16 + (lane & 3) * 16);
+                if (dst_k[k]) *reinterpret_cast<uint4*>(dst_k[k] + qd * 32) = x;
               }
+              __syncwarp();
             }
           } else {
             const long long slot = ((long long)blockIdx.x + u) * 2 + t;
-            float4* po = reinterpret_cast<float4*>(p.part_o + (slot * 128 + row) * 128);
+            // rows this lane stores: r = 4 k + (lane >> 3), 16 bytes (4 floats) at chunk (lane & 7) of the quarter
+            float* po = p.part_o + ((slot * 128 + ((warp & 3) << 5) + (lane >> 3)) * 128 + (lane & 7) * 4);
+            const int nrows = ui.rows_q - rr0;  // valid rows of this warp (may exceed 32)
+#pragma unroll 1
+            for (int qd = 0; qd < 4; ++qd) {
+              uint32_t o[2][16];
+              tmem_ld16(t_o + qd * 32, o[0]);
+              tmem_ld16(t_o + qd * 32 + 16, o[1]);
+              tmem_wait_ld16(o[0]);
+              tmem_wait_ld16(o[1]);
 #pragma unroll
-            for (int pc = 0; pc < 8; ++pc) {
-              uint32_t o[16];
-              tmem_ld16(t_o + pc * 16, o);
-              tmem_wait_ld16(o);
-              if (valid) {
+              for (int h = 0; h < 2; ++h)
 #pragma unroll
                 for (int v4 = 0; v4 < 4; ++v4)
-                  po[pc * 4 + v4] = make_float4(__uint_as_float(o[4 * v4]), __uint_as_float(o[4 * v4 + 1]),
-                                                __uint_as_float(o[4 * v4 + 2]), __uint_as_float(o[4 * v4 + 3]));
+                  *reinterpret_cast<uint4*>(stage + lane * STAGE_ROW_F32 + h * 64 + v4 * 16) =
+                      make_uint4(o[h][4 * v4], o[h][4 * v4 + 1], o[h][4 * v4 + 2], o[h][4 * v4 + 3]);
+              __syncwarp();
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const uint4 x = *reinterpret_cast<const uint4*>(stage + (4 * k + (lane >> 3)) * STAGE_ROW_F32 + (lane & 7) * 16);
+                if (4 * k + (lane >> 3) < nrows) *reinterpret_cast<uint4*>(po + (long long)k * 4 * 128 + qd * 32) = x;
               }
+              __syncwarp();
             }
             if (valid) {
               p.part_ml[(slot * 128 + row) * 2] = m_used;
@@ -541,8 +594,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     if (ui.tiles == 2) chunk_cnt[1] += nchunks;
     pos += nfr;
     tc_fence_before();
-    __syncthreads();
+    seg_sync();
     tc_fence_after();
+    if (warp == 6) REKV_STAMP(3, 1 + seg, 3);
+    ++seg;
     if (*s_abort) break;
   }
 
@@ -555,6 +610,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     run(std::true_type{});
   }
 
+  if (warp == 6) REKV_STAMP(3, 0, 3);
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
 }
