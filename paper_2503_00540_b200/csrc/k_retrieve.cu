@@ -65,21 +65,21 @@ __global__ void __launch_bounds__(QM_SLICES * 64) qmean_kernel(const __nv_bfloat
 // representative rows are read once (float4 per lane, coalesced), the norm and the dot product with
 // every question of the batch come from the same registers, reduced with warp shuffles.  The table is
 // read once per batch.  n_visible counts items here.
-constexpr int SCORE_FRAMES_PER_CTA = 64;
-constexpr int SCORE_MAX_V4 = 8;  // float4 per lane: D' <= 1024
-
-__global__ void __launch_bounds__(256) score_kernel(const float* __restrict__ reps, const float* __restrict__ qa,
-                                                    const float* __restrict__ qsq, int nQ, int maxQ, int Dp, int Hkv,
-                                                    int max_frames, int n_visible, int q_group,
-                                                    float* __restrict__ scores, int block, int layer0) {
+// SCORE_MAX_V4 = float4 per lane (4: D' <= 512, 8: D' <= 1024); fpc = frames per CTA (a multiple of 16), chosen by
+// the launcher so that the whole grid is resident at once (no second, mostly empty wave).
+template <int SCORE_MAX_V4>
+__global__ void __launch_bounds__(256, SCORE_MAX_V4 <= 4 ? 4 : 2)
+    score_kernel(const float* __restrict__ reps, const float* __restrict__ qa, const float* __restrict__ qsq, int nQ,
+                 int maxQ, int Dp, int Hkv, int max_frames, int n_visible, int q_group, float* __restrict__ scores,
+                 int block, int layer0, int fpc) {
   extern __shared__ float4 s_q[];  // [q_group][Dp/4]
   __shared__ float s_qn[REKV_MAX_QUESTIONS];
   rekv_ptx::grid_dep_wait();
   rekv_ptx::grid_dep_launch();
   const int l = layer0 + blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int f0 = blockIdx.x * SCORE_FRAMES_PER_CTA;
-  const int f1 = min(f0 + SCORE_FRAMES_PER_CTA, n_visible);
+  const int f0 = blockIdx.x * fpc;
+  const int f1 = min(f0 + fpc, n_visible);
   const int nv4 = Dp / 128;  // float4 per lane
   const float eps = 1e-8f;
   if (threadIdx.x < nQ) {
@@ -219,6 +219,15 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
     topk_write_table(tt, out, 0, l, qi, nQ);
     return;
   }
+  // up to TK_CACHE * 512 candidates keep their keys in registers: one read of the scores instead of five
+  constexpr int TK_CACHE = 4;
+  const bool cached = n_cand <= TK_CACHE * 512;
+  unsigned kc[TK_CACHE];
+#pragma unroll
+  for (int j = 0; j < TK_CACHE; ++j) {
+    const int i = j * 512 + threadIdx.x;
+    kc[j] = (cached && i < n_cand) ? score_key(s[i]) : 0u;
+  }
   if (threadIdx.x == 0) {
     s_prefix = 0u;
     s_krem = k_eff;
@@ -231,9 +240,15 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
     __syncthreads();
     const unsigned prefix = s_prefix;
     const unsigned mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
-    for (int i = threadIdx.x; i < n_cand; i += blockDim.x) {
-      const unsigned key = score_key(s[i]);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    if (cached) {
+#pragma unroll
+      for (int j = 0; j < TK_CACHE; ++j)
+        if (j * 512 + (int)threadIdx.x < n_cand && (kc[j] & mask) == prefix) atomicAdd(&hist[(kc[j] >> shift) & 255u], 1u);
+    } else {
+      for (int i = threadIdx.x; i < n_cand; i += blockDim.x) {
+        const unsigned key = score_key(s[i]);
+        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      }
     }
     __syncthreads();
     if (warp == 0) {
@@ -268,9 +283,9 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
   const unsigned thr = s_prefix;  // key of the k_eff-th largest score
   const int need_eq = s_krem;     // how many candidates equal to it are selected (lowest indices first)
   const int n_gt = k_eff - need_eq;
-  for (int i0 = 0; i0 < n_cand; i0 += blockDim.x) {
+  auto emit = [&](const int i0, const unsigned key_in) {
     const int i = i0 + threadIdx.x;
-    const unsigned key = i < n_cand ? score_key(s[i]) : 0u;
+    const unsigned key = i < n_cand ? key_in : 0u;
     const bool gt = i < n_cand && key > thr, eq = i < n_cand && key == thr;
     const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
     if (lane == 0) {
@@ -302,6 +317,16 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
       s_base_eq += te;
     }
     __syncthreads();
+  };
+  if (cached) {
+#pragma unroll
+    for (int j = 0; j < TK_CACHE; ++j)
+      if (j * 512 < n_cand) emit(j * 512, kc[j]);
+  } else {
+    for (int i0 = 0; i0 < n_cand; i0 += blockDim.x) {
+      const int i = i0 + threadIdx.x;
+      emit(i0, i < n_cand ? score_key(s[i]) : 0u);
+    }
   }
   (void)n_gt;
   topk_write_table(tt, out, k_eff * block, l, qi, nQ);
@@ -384,6 +409,45 @@ __global__ void replicate_idx_kernel(int32_t* __restrict__ idx, int per_layer, i
   for (int l = 1; l < L; ++l) idx[(long long)l * per_layer + i] = v;
 }
 
+// Launch of the score kernel over frames [0, n_scored) of nl layers.  Frames per CTA grow until the grid fits the
+// device in one wave at the kernel's occupancy.
+template <int V4>
+cudaError_t launch_score_v4(bool pdl, cudaStream_t st, size_t smem, int nl, int n_scored, const float* reps, const float* qa,
+                            const float* qsq, int nQ, int maxQ, int Dp, int Hkv, int max_frames, int q_group, float* scores,
+                            int block, int layer0) {
+  static int sms = 0;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(score_kernel<V4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+    if (e != cudaSuccess) return e;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    attr_set = true;
+  }
+  int occ = 1;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, score_kernel<V4>, 256, smem) != cudaSuccess || occ < 1) occ = 1;
+  int per_layer = (sms * occ) / nl;
+  if (per_layer < 1) per_layer = 1;
+  int fpc = ((n_scored + per_layer - 1) / per_layer + 15) & ~15;
+  if (fpc < 16) fpc = 16;
+  dim3 grid((n_scored + fpc - 1) / fpc, nl);
+  if (pdl)
+    return rekv_launch_pdl(score_kernel<V4>, grid, dim3(256), smem, st, reps, qa, qsq, nQ, maxQ, Dp, Hkv, max_frames,
+                           n_scored, q_group, scores, block, layer0, fpc);
+  score_kernel<V4><<<grid, 256, smem, st>>>(reps, qa, qsq, nQ, maxQ, Dp, Hkv, max_frames, n_scored, q_group, scores, block,
+                                            layer0, fpc);
+  return cudaGetLastError();
+}
+cudaError_t launch_score(bool pdl, cudaStream_t st, size_t smem, int nl, int n_scored, const float* reps, const float* qa,
+                         const float* qsq, int nQ, int maxQ, int Dp, int Hkv, int max_frames, int q_group, float* scores,
+                         int block, int layer0) {
+  return Dp <= 512 ? launch_score_v4<4>(pdl, st, smem, nl, n_scored, reps, qa, qsq, nQ, maxQ, Dp, Hkv, max_frames, q_group,
+                                        scores, block, layer0)
+                   : launch_score_v4<8>(pdl, st, smem, nl, n_scored, reps, qa, qsq, nQ, maxQ, Dp, Hkv, max_frames, q_group,
+                                        scores, block, layer0);
+}
+
 }  // namespace
 
 cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, int top_k, const CtxGeom& geom,
@@ -399,19 +463,13 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
   int q_group = (int)((96 * 1024) / (s.Dp * sizeof(float)));
   if (q_group > qb.nQ) q_group = qb.nQ;
   size_t smem = (size_t)q_group * s.Dp * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-    attr_set = true;
-  }
   // b = 1: every visible frame is scored (the window's scores are reported but not candidates);
   // b > 1: the complete candidate blocks are scored
   const int b = c->cfg.block_frames;
   const int n_scored = b == 1 ? n_visible : geom.n_items;
   if (n_scored > 0) {
-    dim3 grid((n_scored + SCORE_FRAMES_PER_CTA - 1) / SCORE_FRAMES_PER_CTA, nl);
-    cudaError_t e1 = rekv_launch_pdl(score_kernel, grid, dim3(256), smem, st, s.reps, c->qa, c->qnorm, qb.nQ, maxQ, s.Dp,
-                                     s.Hkv, s.max_frames, n_scored, q_group, scores, b, layer0);
+    cudaError_t e1 = launch_score(true, st, smem, nl, n_scored, s.reps, c->qa, c->qnorm, qb.nQ, maxQ, s.Dp, s.Hkv,
+                                  s.max_frames, q_group, scores, b, layer0);
     if (e1 != cudaSuccess) return e1;
     c->launches += 1;
   }
@@ -559,16 +617,8 @@ extern "C" int rekv_score_frames_static(const void* q, const int32_t* cu_q, int 
   // the question vectors of one call fit in 64 KB of dynamic shared memory only in groups
   int q_group = (int)((96 * 1024) / (Dp * sizeof(float)));
   if (q_group > nQ) q_group = nQ;
-  e = cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-  if (e != cudaSuccess) {
-    rekv_set_error(nullptr, "rekv_score_frames_static: cannot raise the shared-memory limit of the score kernel");
-    return REKV_ERR_CUDA;
-  }
-  dim3 grid((n_frames + SCORE_FRAMES_PER_CTA - 1) / SCORE_FRAMES_PER_CTA, 1);
-  score_kernel<<<grid, 256, (size_t)q_group * Dp * sizeof(float), st>>>(reps, qa, qsq, nQ, STATIC_MAX_QUESTIONS, Dp,
-                                                                       n_kv_heads, n_frames, n_frames, q_group,
-                                                                       scores_out, 1, 0);
-  e = cudaGetLastError();
+  e = launch_score(false, st, (size_t)q_group * Dp * sizeof(float), 1, n_frames, reps, qa, qsq, nQ, STATIC_MAX_QUESTIONS, Dp,
+                   n_kv_heads, n_frames, q_group, scores_out, 1, 0);
   if (e != cudaSuccess) {
     rekv_set_error(nullptr, cudaGetErrorString(e));
     return REKV_ERR_CUDA;
