@@ -284,7 +284,7 @@ def run_cuda(args, w):
 
     g = rekv.ReKV(w["L"], w["Hq"], w["Hkv"], w["D"], w["Nf"], w["T"] + 8, w["W"], hbm_tail_frames=w["tail"],
                   max_q_tokens=cu[-1], max_topk=w["k"], max_questions=nQ, device=local,
-                  flags=rekv.FLAG_TIMING | (rekv.FLAG_HOST_FP8 if w.get("host_fp8") else 0),
+                  flags=(rekv.FLAG_HOST_FP8 if w.get("host_fp8") else 0),
                   max_self_tokens=cu[-1] if w.get("full") else 0, rope_theta=w.get("rope_theta", 0.0),
                   ext_embed_dim=w.get("ext_dim", 0))
     kf = torch.empty((w["L"], w["Nf"], w["Hkv"], w["D"]), dtype=torch.bfloat16, device=dev)
@@ -388,13 +388,16 @@ def run_cuda(args, w):
     g.check_status()
 
     # attention-kernel duration (library-internal events on the launching stream) and bytes over the host link
+    # (the event records stand between the attention kernel and its neighbours, so they are on only here)
     att_us, link_bytes = [], 0
+    g.set_timing(True)
     for i in range(min(K, 8)):
         ask(qs[i % N_ROTATE], g.stats().frames, out)
         torch.cuda.synchronize()
         st = g.stats()
         att_us.append(st.last_attend_kernel_us)
         link_bytes = st.last_link_bytes
+    g.set_timing(False)
 
     # ---- end to end: inputs in pinned host memory, result read back, every step ----
     hk = [t.cpu().pin_memory() for t in new_k[:2]]

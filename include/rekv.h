@@ -240,6 +240,12 @@ int rekv_load(const char* path, int device, rekv_ctx** out);
 /* Fills *out with store accounting and the last call's counters. */
 int rekv_stats(rekv_ctx* ctx, rekv_stats_t* out);
 
+/* Switches REKV_FLAG_TIMING on (enable != 0) or off for the calls that follow.  The two event records around
+ * the attention kernel stand between it and its neighbours in the stream, so a timed question is a few
+ * microseconds slower than an untimed one (its kernels no longer overlap each other's prologues): measure the
+ * kernel with the flag on and the question with it off.  Host-side only; returns REKV_OK. */
+int rekv_set_timing(rekv_ctx* ctx, int enable);
+
 /* Reads (and clears) the device status word after synchronising `stream`: 0, or REKV_ERR_TIMEOUT
  * if a bounded device-side wait gave up since the last check. */
 int rekv_check_status(rekv_ctx* ctx, void* stream);

@@ -642,6 +642,17 @@ int rekv_stats(rekv_ctx* c, rekv_stats_t* out) {
   return REKV_OK;
 }
 
+int rekv_set_timing(rekv_ctx* c, int enable) {
+  if (!c) return REKV_ERR_ARG;
+  if (enable) {
+    c->cfg.flags |= REKV_FLAG_TIMING;
+  } else {
+    c->cfg.flags &= ~(uint32_t)REKV_FLAG_TIMING;
+    c->timing_valid = false;
+  }
+  return REKV_OK;
+}
+
 int rekv_check_status(rekv_ctx* c, void* stream) {
   if (!c) return REKV_ERR_ARG;
   DeviceGuard guard(c->device);

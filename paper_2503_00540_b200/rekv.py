@@ -45,7 +45,7 @@ EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", 
            "rekv_stats", "rekv_check_status", "rekv_last_error", "rekv_get_reps", "rekv_get_page",
            "rekv_launch_count", "rekv_score_frames_static", "rekv_question_layer", "rekv_attend_layer", "rekv_attend_full",
            "rekv_set_frame_embedding", "rekv_retrieve_external", "rekv_question",
-           "rekv_save", "rekv_load")
+           "rekv_save", "rekv_load", "rekv_set_timing")
 
 _lib = None
 
@@ -73,6 +73,7 @@ def lib() -> ctypes.CDLL:
         L.rekv_retrieve_external.argtypes = [vp, vp, i32, i32, i32, ctypes.c_float, vp, vp, vp]
         L.rekv_stats.argtypes = [vp, ctypes.POINTER(rekv_stats_t)]
         L.rekv_check_status.argtypes = [vp, vp]
+        L.rekv_set_timing.argtypes = [vp, i32]
         L.rekv_last_error.argtypes = [vp]
         L.rekv_last_error.restype = ctypes.c_char_p
         L.rekv_get_reps.argtypes = [vp, i32, i32, vp, vp]
@@ -302,6 +303,10 @@ class ReKV:
 
     def check_status(self) -> None:
         self._check(lib().rekv_check_status(self._h, self._stream()))
+
+    def set_timing(self, enable: bool) -> None:
+        """Event records around the attention kernel on or off for the calls that follow (see rekv_set_timing)."""
+        self._check(lib().rekv_set_timing(self._h, 1 if enable else 0))
 
     def launch_count(self) -> int:
         return int(lib().rekv_launch_count(self._h))

@@ -89,6 +89,28 @@ def test_question_in_the_past_sees_only_visible_frames():
     _run_question_parity(s, [16], n_visible=37)
 
 
+def test_timing_switch_reports_the_kernel_and_leaves_results_alone():
+    """rekv_set_timing: with the event records on, the attention kernel's duration is reported; off, it is not;
+    the output bits are the same either way."""
+    s = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=80, W=8, k=16, seed=7)
+    g = H.build_gpu(s, max_q_tokens=32)
+    q, cu = H.questions(s, [32], device="cuda")
+    out_plain = g.question(q, cu, s.k, s.T).clone()
+    torch.cuda.synchronize()
+    assert g.stats().last_attend_kernel_us == 0.0
+    g.set_timing(True)
+    out_timed = g.question(q, cu, s.k, s.T).clone()
+    torch.cuda.synchronize()
+    assert g.stats().last_attend_kernel_us > 0.0
+    g.set_timing(False)
+    out_again = g.question(q, cu, s.k, s.T).clone()
+    torch.cuda.synchronize()
+    assert g.stats().last_attend_kernel_us == 0.0
+    assert torch.equal(out_plain, out_timed) and torch.equal(out_plain, out_again)
+    g.check_status()
+    g.close()
+
+
 def test_degenerate_counts():
     # k larger than the candidates -> every visible frame is attended; fewer frames than the window
     s = H.Shape(L=1, Hq=8, Hkv=2, Nf=16, T=10, W=4, k=32, off_scale=0.0)
