@@ -134,6 +134,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   bars.base = s_bar;
   volatile uint32_t* s_tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + (s_bar - s_base) + 8 * (2 * KV_BUFS + 6));
   volatile uint32_t* s_abort = s_tmem_slot + 1;
+  volatile uint32_t* s_stop = s_tmem_slot + 2;  // the abort flag as one thread saw it between two segment barriers
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (warp == 6) REKV_STAMP(3, 0, 0);
@@ -161,6 +162,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
       mbar_init(bars.pv_done(t), 1);
     }
     *s_abort = 0;
+    *s_stop = 0;
     fence_barrier_init();
   }
   if (warp == 0) {
@@ -598,7 +600,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     tc_fence_after();
     if (warp == 6) REKV_STAMP(3, 1 + seg, 3);
     ++seg;
-    if (*s_abort) break;
+    // The copy producer is outside the segment barriers and may raise the abort flag at any moment; the other warps
+    // must all leave together (one that left alone would never reach the next segment barrier), so they act on one
+    // thread's reading of the flag, taken between two barriers.
+    if (warp == 0) {
+      if (*s_abort) break;
+    } else {
+      if (warp == 1 && lane == 0 && *s_abort) *s_stop = 1;
+      seg_sync();
+      if (*s_stop) break;
+    }
   }
 
   };
