@@ -36,6 +36,9 @@ WORKLOADS = {
     # decode-shaped question (one token): the HBM-bound end of Eq. 3
     "7b_hbm_decode_1tok": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=1, seed=2503, off_scale=0.5,
                                tail=0, nQ=1, appends_per_step=1),
+    # a short question (10 tokens = 70 rows per KV head): one row tile per unit, run as two half-streams
+    "7b_hbm_short_q10": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=10, seed=2503, off_scale=0.5,
+                             tail=0, nQ=1, appends_per_step=1),
     # Eq. 3 in full: the question's own K/V (causal) after the retrieved context, rotary embedding with the
     # retrieved tokens at consecutive positions (base 1e6, the paper's Qwen2-based models)
     "7b_hbm_full_eq3_rope": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503,

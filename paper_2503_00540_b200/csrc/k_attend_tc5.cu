@@ -20,6 +20,10 @@
 // TMEM (512 columns): O0 [0,128)  O1 [128,256)  S0/P0 [256,384)  S1/P1 [384,512); P (bf16) overwrites
 // the front of its S.  A frame of N_f tokens is processed as one or two token chunks of <= 128.
 // A range that does not cover a whole unit leaves (max, sum, O) partials for the combine kernel.
+// A unit with a single row tile (at most 128 rows: short questions, the remainder of long ones) would leave the
+// tensor core idle during its softmax; it runs as two half-streams instead -- both tile slots work on the same rows,
+// the token chunks of the context dealt to them alternately, each with its own (max, sum, O) -- and the combine
+// kernel joins the two partials like those of any cut unit.
 // Every wait is bounded: on expiry the status word is set and the CTA leaves.
 #include <algorithm>
 #include <type_traits>
@@ -75,12 +79,18 @@ struct TcParams {
   QBatch qb;
   int Hq, Hkv, G, Nf, Npad, NA, NB, ncf, MP, layer0;
   int per;          // (unit, frame) steps per CTA
+  // A unit with one row tile has no second tile to overlap with; it is run as two half-streams on the two tile
+  // slots instead -- the same rows, the frame's token chunks dealt alternately -- whose (max, sum, O) partials the
+  // merge kernel joins.  n_split = questions whose last unit is such a unit (0 = off).
+  int n_split;
   long long total;  // units * ncf
   float scale_log2;
 };
 
 struct UnitInfo {
   int l, g, qi, m0, rows_q, tiles;
+  int split;   // one row tile, run as two half-streams
+  int srank;   // its rank among the launch's split units (partial slots when units are not cut)
   long long q_row0;
 };
 
@@ -90,16 +100,20 @@ __device__ __forceinline__ UnitInfo decode_unit(const TcParams& p, long long u) 
   long long r = u / p.MP;
   ui.g = (int)(r % p.Hkv);
   ui.l = p.layer0 + (int)(r / p.Hkv);
-  int qi = 0, mp = mpg;
+  int qi = 0, mp = mpg, before = 0;  // before = earlier questions whose last unit has one row tile
   for (; qi < p.qb.nQ - 1; ++qi) {
-    int t = ((p.qb.cu[qi + 1] - p.qb.cu[qi]) * p.G + 255) / 256;
+    const int rows = (p.qb.cu[qi + 1] - p.qb.cu[qi]) * p.G;
+    int t = (rows + 255) / 256;
     if (mp < t) break;
     mp -= t;
+    before += ((rows - 1) & 255) < 128;
   }
   ui.qi = qi;
   ui.rows_q = (p.qb.cu[qi + 1] - p.qb.cu[qi]) * p.G;
   ui.m0 = mp * 256;
   ui.tiles = (ui.rows_q - ui.m0 > 128) ? 2 : 1;
+  ui.split = p.n_split > 0 && ui.tiles == 1;
+  ui.srank = ((ui.l - p.layer0) * p.Hkv + ui.g) * p.n_split + before;
   ui.q_row0 = (long long)ui.l * p.qb.sumNq + p.qb.cu[qi];
   return ui;
 }
@@ -120,7 +134,9 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return r;
 }
 
-template <bool FULL>
+// FULL: Eq. 3 in full (rotated K tiles, the part over X joins in the epilogue).  SPLIT: the launch has units with a
+// single row tile, which run as two half-streams (compiled out otherwise: the common loop stays as it was).
+template <bool FULL, bool SPLIT>
 __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParams p) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -218,17 +234,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     const int nfr = (int)min((long long)(p.ncf - f0), end - pos);
     const UnitInfo ui = decode_unit(p, u);
     const int nchunks = nfr * cpf;
+    const bool split = SPLIT && ui.split != 0;
+    const int vtiles = split ? 2 : ui.tiles;  // tile slots in use
+    // chunks per tile slot and a slot's j-th chunk among the segment's: every chunk for both tiles, or alternately
+    const int nch0 = split ? (nchunks + 1) >> 1 : nchunks, nch1 = split ? nchunks >> 1 : nchunks;
+    auto chunk_of = [&](int T, int j) { return split ? 2 * j + T : j; };
     char* const* pages = p.tbl + ((long long)ui.l * p.qb.nQ + ui.qi) * p.ncf + f0;
     char* const* pages_k = (FULL && p.tbl_k) ? p.tbl_k + ((long long)ui.l * p.qb.nQ + ui.qi) * p.ncf + f0 : nullptr;
-    const bool whole_unit = (nfr == p.ncf);
+    const bool whole_unit = (nfr == p.ncf) && !split;
     if (warp == 6) REKV_STAMP(3, 1 + seg, 0);
 
     // ---- Q row tiles -> shared memory in the swizzled K-major operand layout -------------------
     if (warp >= SM_WARP0) {
       const int t = (warp - SM_WARP0) >> 2;
       const int row = ((warp & 3) << 5) | lane;
-      if (t < ui.tiles) {
-        const int rr = ui.m0 + t * 128 + row;
+      if (t < vtiles) {
+        const int rr = ui.m0 + (split ? 0 : t) * 128 + row;
         const bool valid = rr < ui.rows_q;
         const int n = rr / p.G, j = rr - n * p.G;
         const uint4* src =
@@ -281,7 +302,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         const uint32_t lbo_v = ((half_stride >> 4) & 0x3FFFu) << 16;      // pitch of V's two 64-dim blocks
         const uint32_t lbo_k = 1u << 16;                                  // unused for K-major operands
         const uint32_t half16 = half_stride >> 4;
-        const int tiles = ui.tiles;
+        const int tiles = vtiles;
         bool ok = true;
 #define REKV_DESC(lo) (((uint64_t)desc_hi << 32) | (uint64_t)(lo))
 #define REKV_ISSUE_S(T, I)                                                                                    \
@@ -289,7 +310,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     const int fi_ = (I) / cpf, part_ = (I) - fi_ * cpf;                                                       \
     const uint32_t r_ = ring + 2 * fi_, b_ = r_ % KV_BUFS;                                                    \
     const uint32_t tok0_ = part_ ? p.NA : 0, N_ = part_ ? p.NB : p.NA;                                        \
-    if (part_ == 0 && (T) == 0) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                                 \
+    if (part_ == 0 && ((T) == 0 || split)) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                      \
     if (ok) {                                                                                                 \
       tc_fence_after();                                                                                       \
       const uint32_t k_lo = ((s_kv + b_ * tile_bytes + tok0_ * 128u) >> 4) | lbo_k;                           \
@@ -302,44 +323,44 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
       _Pragma("unroll") for (int kk = 0; kk < 4; ++kk)                                                        \
           mma_ss(d_, REKV_DESC(q_lo + (Q_TILE_BYTES / 32) + 2 * kk), REKV_DESC(k_lo + half16 + 2 * kk), idesc_, 1); \
       tc_commit(bars.s_full(T));                                                                              \
-      if (part_ == cpf - 1 && (T) == tiles - 1) tc_commit(bars.empty(b_)); /* K tile no longer needed */      \
+      if (part_ == cpf - 1 && ((T) == tiles - 1 || split)) tc_commit(bars.empty(b_)); /* K tile done */       \
       }                                                                                                       \
       __syncwarp();                                                                                           \
     }                                                                                                         \
   } while (0)
-#define REKV_ISSUE_PV(T, I)                                                                                   \
+#define REKV_ISSUE_PV(T, I, J)                                                                                \
   do {                                                                                                        \
     const int fi_ = (I) / cpf, part_ = (I) - fi_ * cpf;                                                       \
     const uint32_t r_ = ring + 2 * fi_ + 1, b_ = r_ % KV_BUFS;                                                \
     const uint32_t tok0_ = part_ ? p.NA : 0, nk_ = (part_ ? p.NB : p.NA) >> 4;                                \
-    if (part_ == 0 && (T) == 0) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                                 \
-    if (ok) ok = wait(bars.p_ready(T), (chunk_cnt[T] + (I)) & 1);                                             \
+    if (part_ == 0 && ((T) == 0 || split)) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                      \
+    if (ok) ok = wait(bars.p_ready(T), (chunk_cnt[T] + (J)) & 1);                                             \
     if (ok) {                                                                                                 \
       tc_fence_after();                                                                                       \
       const uint32_t v_lo = ((s_kv + b_ * tile_bytes + tok0_ * 128u) >> 4) | lbo_v;                           \
       const uint32_t d_ = tmem + col_o(T), a_ = tmem + col_s(T);                                              \
       if (elect_one()) {                                                                                      \
       _Pragma("unroll") for (int kk = 0; kk < 8; ++kk)                                                        \
-          if (kk < (int)nk_) mma_ts(d_, a_ + 8 * kk, REKV_DESC(v_lo + 128 * kk), idesc_pv, ((I) > 0) | (kk > 0)); \
+          if (kk < (int)nk_) mma_ts(d_, a_ + 8 * kk, REKV_DESC(v_lo + 128 * kk), idesc_pv, ((J) > 0) | (kk > 0)); \
       tc_commit(bars.pv_done(T));                                                                             \
-      if (part_ == cpf - 1 && (T) == tiles - 1) tc_commit(bars.empty(b_)); /* V tile no longer needed */      \
+      if (part_ == cpf - 1 && ((T) == tiles - 1 || split)) tc_commit(bars.empty(b_)); /* V tile done */       \
       }                                                                                                       \
       __syncwarp();                                                                                           \
     }                                                                                                         \
   } while (0)
         REKV_ISSUE_S(0, 0);
-        if (tiles == 2 && ok) REKV_ISSUE_S(1, 0);
-        for (int i = 0; i < nchunks && ok; ++i) {
-          REKV_STAMP(0, i, 0);
-          REKV_ISSUE_PV(0, i);
-          REKV_STAMP(0, i, 1);
-          if (i + 1 < nchunks && ok) REKV_ISSUE_S(0, i + 1);
-          REKV_STAMP(0, i, 2);
-          if (tiles == 2 && ok) {
-            REKV_ISSUE_PV(1, i);
-            REKV_STAMP(0, i, 3);
-            if (i + 1 < nchunks && ok) REKV_ISSUE_S(1, i + 1);
-            REKV_STAMP(0, i, 4);
+        if (tiles == 2 && ok && chunk_of(1, 0) < nchunks) REKV_ISSUE_S(1, chunk_of(1, 0));
+        for (int j = 0; j < nch0 && ok; ++j) {
+          REKV_STAMP(0, j, 0);
+          REKV_ISSUE_PV(0, chunk_of(0, j), j);
+          REKV_STAMP(0, j, 1);
+          if (chunk_of(0, j + 1) < nchunks && ok) REKV_ISSUE_S(0, chunk_of(0, j + 1));
+          REKV_STAMP(0, j, 2);
+          if (tiles == 2 && ok && chunk_of(1, j) < nchunks) {
+            REKV_ISSUE_PV(1, chunk_of(1, j), j);
+            REKV_STAMP(0, j, 3);
+            if (chunk_of(1, j + 1) < nchunks && ok) REKV_ISSUE_S(1, chunk_of(1, j + 1));
+            REKV_STAMP(0, j, 4);
           }
         }
 #undef REKV_ISSUE_S
@@ -351,7 +372,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     } else {
       // ================= softmax + output, one thread per row =================
       const int t = (warp - SM_WARP0) >> 2;
-      if (t < ui.tiles) {
+      if (t < vtiles) {
+        const int rt = split ? 0 : t;              // the row tile this slot works on
+        const int nch = t ? nch1 : nch0;           // its chunks in this segment
         const uint32_t lane_base = (uint32_t)((warp & 3) << 5) << 16;
         const int row = ((warp & 3) << 5) | lane;
         const uint32_t t_s = tmem + lane_base + col_s(t);
@@ -359,9 +382,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         float m_used = -INFINITY, l_sum = 0.f;
         bool ok = true;
         // a warp whose 32 rows all lie beyond the unit's rows (the ragged second tile) only keeps the barriers moving
-        const bool warp_idle = ui.m0 + t * 128 + ((warp & 3) << 5) >= ui.rows_q;
-        for (int i = 0; i < nchunks && ok; ++i) {
-          const int part = cpf == 2 ? (i & 1) : 0;
+        const bool warp_idle = ui.m0 + rt * 128 + ((warp & 3) << 5) >= ui.rows_q;
+        for (int i = 0; i < nch && ok; ++i) {  // i counts this slot's chunks
+          const int part = cpf == 2 ? (chunk_of(t, i) & 1) : 0;
           const int tok0 = part ? p.NA : 0, N = part ? p.NB : p.NA;
           const int nv = min(N, p.Nf - tok0);  // valid tokens of this chunk
           const int npc = N >> 4;
@@ -480,17 +503,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
           if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 3);
         }
         // ---- output of this range: final rows, or a partial for the combine kernel ----
-        if (ok && wait(bars.pv_done(t), (chunk_cnt[t] + nchunks - 1) & 1)) {
+        if (ok && (nch == 0 || wait(bars.pv_done(t), (chunk_cnt[t] + nch - 1) & 1))) {
           tc_fence_after();
           if (warp == 6) REKV_STAMP(3, 1 + seg, 2);
-          const int rr = ui.m0 + t * 128 + row;
+          const int rr = ui.m0 + rt * 128 + row;
           const bool valid = rr < ui.rows_q;
           const int n = rr / p.G, j = rr - n * p.G;
           // Rows leave through this warp's staging rows in the tile's Q region (no product reads Q any more), a
           // quarter of the 128 columns at a time, so that the global stores are contiguous per row instead of one
           // 16-byte piece per lane in 32 different rows.
           unsigned char* stage = smem + t * Q_TILE_BYTES + (warp & 3) * STAGE_WARP_BYTES;
-          const int rr0 = ui.m0 + t * 128 + ((warp & 3) << 5);  // first row of this warp
+          const int rr0 = ui.m0 + rt * 128 + ((warp & 3) << 5);  // first row of this warp
           if (whole_unit) {
             float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
             const long long out_row = (ui.q_row0 + (valid ? n : 0)) * p.Hq + ui.g * p.G + (valid ? j : 0);
@@ -558,7 +581,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
               __syncwarp();
             }
           } else {
-            const long long slot = ((long long)blockIdx.x + u) * 2 + t;
+            const long long slot = (p.per == p.ncf ? (long long)ui.srank : (long long)blockIdx.x + u) * 2 + t;
             // rows this lane stores: r = 4 k + (lane >> 3), 16 bytes (4 floats) at chunk (lane & 7) of the quarter
             float* po = p.part_o + ((slot * 128 + ((warp & 3) << 5) + (lane >> 3)) * 128 + (lane & 7) * 4);
             const int nrows = ui.rows_q - rr0;  // valid rows of this warp (may exceed 32)
@@ -569,6 +592,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
               tmem_ld16(t_o + qd * 32 + 16, o[1]);
               tmem_wait_ld16(o[0]);
               tmem_wait_ld16(o[1]);
+              if (nch == 0) {  // a half-stream without a chunk in this segment: the neutral partial (-inf, 0, 0)
+#pragma unroll
+                for (int e = 0; e < 16; ++e) o[0][e] = o[1][e] = 0u;
+              }
 #pragma unroll
               for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -592,8 +619,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
       }
     }
     ring += 2 * nfr;
-    chunk_cnt[0] += nchunks;
-    if (ui.tiles == 2) chunk_cnt[1] += nchunks;
+    chunk_cnt[0] += nch0;
+    if (vtiles == 2) chunk_cnt[1] += nch1;
     pos += nfr;
     tc_fence_before();
     seg_sync();
@@ -1006,9 +1033,17 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
   const long long u = blockIdx.x;
   const int t = blockIdx.y;
   const long long c_first = (u * p.ncf) / p.per, c_last = ((u + 1) * p.ncf - 1) / p.per;
-  if (c_first == c_last) return;  // the unit was produced whole by one CTA
   const UnitInfo ui = decode_unit(p, u);
+  if (c_first == c_last && !ui.split) return;  // the unit was produced whole by one CTA
   if (t >= ui.tiles) return;
+  // parts of this (unit, row tile): one per CTA that worked on the unit -- two per CTA, the half-streams, for a
+  // unit with one row tile -- each in its partial slot
+  const int n_parts = (int)(c_last - c_first + 1) * (ui.split ? 2 : 1);
+  auto slot_of = [&](int k) -> long long {
+    const long long c = c_first + (ui.split ? k >> 1 : k);
+    const long long base = p.per == p.ncf ? (long long)ui.srank : c + u;
+    return base * 2 + (ui.split ? (k & 1) : t);
+  };
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   grid_dep_wait();
   {
@@ -1019,7 +1054,7 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
     const long long out_row = (ui.q_row0 + n) * p.Hq + ui.g * p.G + j;
     // the parts' maxima: a lane per part (independent loads), then the warp's maximum
     float M = p.self_o ? p.self_ml[out_row * 2] : -INFINITY;
-    for (long long c = c_first + lane; c <= c_last; c += 32) M = fmaxf(M, p.part_ml[(((c + u) * 2 + t) * 128 + r) * 2]);
+    for (int k = lane; k < n_parts; k += 32) M = fmaxf(M, p.part_ml[(slot_of(k) * 128 + r) * 2]);
     for (int o = 16; o; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float den = 0.f;
@@ -1030,20 +1065,20 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
       den = w * p.self_ml[out_row * 2 + 1];
     }
     // the numerators, four parts' rows in flight, added in part order
-    for (long long c0 = c_first; c0 <= c_last; c0 += 4) {
+    for (int k0 = 0; k0 < n_parts; k0 += 4) {
       float4 o[4];
       float m[4], ls[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i)
-        if (c0 + i <= c_last) {
-          const long long base = ((c0 + i + u) * 2 + t) * 128 + r;
+        if (k0 + i < n_parts) {
+          const long long base = slot_of(k0 + i) * 128 + r;
           m[i] = p.part_ml[base * 2];
           ls[i] = p.part_ml[base * 2 + 1];
           o[i] = *reinterpret_cast<const float4*>(p.part_o + base * 128 + lane * 4);
         }
 #pragma unroll
       for (int i = 0; i < 4; ++i)
-        if (c0 + i <= c_last) {
+        if (k0 + i < n_parts) {
           const float w = ex2(m[i] - M);
           acc.x += w * o[i].x;
           acc.y += w * o[i].y;
@@ -1091,6 +1126,7 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   }
   p.ncf = ncf;
   p.layer0 = layer0;
+  p.n_split = 0;
   p.scale_log2 = 1.4426950408889634f / sqrtf(128.f);
   int MP = 0;
   for (int i = 0; i < qb.nQ; ++i) MP += ((qb.cu[i + 1] - qb.cu[i]) * s.G + 255) / 256;
@@ -1142,26 +1178,39 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     }
     return cudaGetLastError();
   }
+  // units with a single row tile run as two half-streams whose partials the merge kernel joins; when units are
+  // not cut, those partials need two slots per such unit
+  {
+    int n_split = 0;
+    for (int i = 0; i < qb.nQ; ++i) n_split += (((qb.cu[i + 1] - qb.cu[i]) * s.G - 1) & 255) < 128;
+    if (p.per == ncf && (size_t)(layer1 - layer0) * s.Hkv * n_split * 2 > c->part_units) n_split = 0;
+    p.n_split = n_split;
+  }
   const size_t smem = 2 * Q_TILE_BYTES + (size_t)KV_BUFS * 2 * p.Npad * 128 + 8 * (2 * KV_BUFS + 6) + 16 + 1024;
   if (smem > 227 * 1024) return cudaErrorInvalidValue;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attend_tc5_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(attend_tc5_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attend_tc5_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      e = cudaFuncSetAttribute(attend_tc5_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(attend_tc5_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(attend_tc5_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   if (timed) cudaEventRecord(c->ev_t0, st);
-  cudaError_t e1 = full ? rekv_launch_pdl(attend_tc5_kernel<true>, dim3((unsigned)grid), dim3(TC_THREADS), smem, st, p)
-                        : rekv_launch_pdl(attend_tc5_kernel<false>, dim3((unsigned)grid), dim3(TC_THREADS), smem, st, p);
+  auto kernel = full ? (p.n_split > 0 ? attend_tc5_kernel<true, true> : attend_tc5_kernel<true, false>)
+                     : (p.n_split > 0 ? attend_tc5_kernel<false, true> : attend_tc5_kernel<false, false>);
+  cudaError_t e1 = rekv_launch_pdl(kernel, dim3((unsigned)grid), dim3(TC_THREADS), smem, st, p);
   if (e1 != cudaSuccess) return e1;
   if (timed) {
     cudaEventRecord(c->ev_t1, st);
     c->timing_valid = true;
   }
   c->launches += 1;
-  if (p.per != ncf) {
+  if (p.per != ncf || p.n_split > 0) {
     cudaError_t e2 = rekv_launch_pdl(combine_tc5_kernel, dim3((unsigned)units, 2, 32), dim3(128), 0, st, p);
     if (e2 != cudaSuccess) return e2;
     c->launches += 1;

@@ -1,5 +1,6 @@
 // The C ABI of librekv: context life cycle, argument checks, stream/event plumbing.
 // Every step of the path runs in the kernels of the k_*.cu files; this file only launches them.
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -220,7 +221,9 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   CREATE_CUDA(cudaMalloc(&c->qnorm, (size_t)s.L * maxQ * s.Hkv * sizeof(float)), "allocating question norms");
   CREATE_CUDA(cudaMalloc(&c->scores, (size_t)s.L * maxQ * s.max_frames * sizeof(float)), "allocating the score buffer");
   CREATE_CUDA(cudaMalloc(&c->ctx_tbl, (size_t)s.L * maxQ * (ctx_frames_max + 1) * sizeof(char*)), "allocating the context table");
-  c->part_units = 2048;
+  // 2048 slots cover every launch whose units are cut at CTA boundaries; launches of many whole units park two
+  // half-stream partials per unit with a single row tile (at most one per layer, KV head and question), up to a cap
+  c->part_units = std::min<size_t>(8192, std::max<size_t>(2048, (size_t)2 * s.L * s.Hkv * maxQ + 16));
   CREATE_CUDA(cudaMalloc(&c->part_o, c->part_units * 128 * 128 * sizeof(float)), "allocating split-KV partials");
   CREATE_CUDA(cudaMalloc(&c->part_ml, c->part_units * 128 * 2 * sizeof(float)), "allocating split-KV partials");
   CREATE_CUDA(cudaMalloc(&c->unit_cnt, c->part_units * sizeof(int)), "allocating split-KV counters");

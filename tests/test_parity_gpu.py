@@ -84,6 +84,20 @@ def test_72b_head_shape(flags):
     _run_question_parity(s, [64], flags=flags)
 
 
+def test_many_short_questions_whole_units_as_half_streams():
+    """640 units of one row tile each (more than four per SM, so no unit is cut at a CTA boundary): every unit runs
+    as two half-streams whose partials the merge kernel joins, with partial slots counted per such unit."""
+    s = H.Shape(L=4, Hq=16, Hkv=8, Nf=33, T=12, W=2, k=4, seed=540)
+    lengths = [9 + (7 * i) % 32 for i in range(20)]  # 18..80 rows per KV head
+    _run_question_parity(s, lengths, max_questions=20)
+
+
+def test_short_question_cut_at_cta_boundaries():
+    """One 10-token question at the 7B head shape: 70 rows = one row tile per unit, units cut at CTA boundaries."""
+    s = H.Shape(L=3, Hq=28, Hkv=4, Nf=196, T=30, W=4, k=12, seed=7)
+    _run_question_parity(s, [10])
+
+
 def test_question_in_the_past_sees_only_visible_frames():
     s = H.Shape(L=1, Hq=8, Hkv=2, Nf=16, T=64, W=4, k=8, off_scale=0.0)
     _run_question_parity(s, [16], n_visible=37)
