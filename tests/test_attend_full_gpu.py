@@ -81,6 +81,15 @@ def test_many_units_take_the_whole_unit_path(theta):
 
 
 @pytest.mark.parametrize("theta", THETAS)
+def test_many_short_questions_half_streams(theta):
+    """640 uncut units of one row tile each: two half-streams per unit, joined with the part over X by the merge
+    kernel."""
+    s = H.Shape(L=4, Hq=16, Hkv=8, Nf=33, T=12, W=2, k=4, seed=540)
+    nq = [9 + (7 * i) % 32 for i in range(20)]
+    _run(s, nq, [n + (i % 3) for i, n in enumerate(nq)], theta)
+
+
+@pytest.mark.parametrize("theta", THETAS)
 def test_host_tier(theta):
     s = H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=40, W=4, k=8, tail=8)
     _run(s, [16, 32], [16, 40], theta)
