@@ -39,6 +39,11 @@ WORKLOADS = {
     # a short question (10 tokens = 70 rows per KV head): one row tile per unit, run as two half-streams
     "7b_hbm_short_q10": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=10, seed=2503, off_scale=0.5,
                              tail=0, nQ=1, appends_per_step=1),
+    # block retrieval (Eq. 2 paragraph, b = 8): 8 blocks of 8 consecutive frames instead of 64 frames
+    "7b_hbm_block8": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503, off_scale=0.5,
+                          tail=0, nQ=1, appends_per_step=1, b=8),
+    "7b_offload_10800f_block8": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=10800, W=8, k=64, Nq=32, seed=2503,
+                                     off_scale=0.5, tail=64, nQ=1, appends_per_step=1, b=8),
     # Eq. 3 in full: the question's own K/V (causal) after the retrieved context, rotary embedding with the
     # retrieved tokens at consecutive positions (base 1e6, the paper's Qwen2-based models)
     "7b_hbm_full_eq3_rope": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503,
@@ -289,7 +294,7 @@ def run_cuda(args, w):
                   max_q_tokens=cu[-1], max_topk=w["k"], max_questions=nQ, device=local,
                   flags=(rekv.FLAG_HOST_FP8 if w.get("host_fp8") else 0),
                   max_self_tokens=cu[-1] if w.get("full") else 0, rope_theta=w.get("rope_theta", 0.0),
-                  ext_embed_dim=w.get("ext_dim", 0))
+                  ext_embed_dim=w.get("ext_dim", 0), block_frames=w.get("b", 1))
     kf = torch.empty((w["L"], w["Nf"], w["Hkv"], w["D"]), dtype=torch.bfloat16, device=dev)
     vf = torch.empty_like(kf)
     for f in range(T0):
