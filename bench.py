@@ -414,8 +414,14 @@ def run_cuda(args, w):
     hout = torch.empty(out.shape, dtype=out.dtype).pin_memory()
     dq = torch.empty_like(qs[0])
 
+    # The headline metric is the question's latency, so `e2e` is the question end to end: its queries copied from
+    # pinned host memory, steps 2-5, the output copied back (ev[1] .. ev[2]); the bytes declared for it are the
+    # bytes copied inside that region.  The whole step -- the frame's K/V copied from pinned host memory and
+    # appended first (ev[0] .. ev[2]) -- is reported beside it with its own byte count.
     def step_e2e(i, ev=None):
         nf = 0
+        if ev:
+            ev[0].record(stream)
         for a in range(aps):
             state["next"] += 1
             kf.copy_(hk[(i + a) % 2], non_blocking=True)
@@ -424,21 +430,22 @@ def run_cuda(args, w):
             if w.get("ext_dim"):
                 g.set_frame_embedding(nf, ext_frames[nf])
         if ev:
-            ev[0].record(stream)
+            ev[1].record(stream)
         dq.copy_(hq[i % N_ROTATE], non_blocking=True)
         ask(dq, nf + 1, out)
         hout.copy_(out, non_blocking=True)
         if ev:
-            ev[1].record(stream)
+            ev[2].record(stream)
 
     for i in range(Wu):
         step_e2e(i)
-    evs2 = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K)]
+    evs2 = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
     barrier()
     for i in range(K):
         step_e2e(i, evs2[i])
     barrier()
-    e2e_us = [e[0].elapsed_time(e[1]) * 1e3 / nQ for e in evs2]
+    e2e_us = [e[1].elapsed_time(e[2]) * 1e3 / nQ for e in evs2]
+    e2e_step_us = [e[0].elapsed_time(e[2]) * 1e3 for e in evs2]
     g.check_status()
 
     def mean(x):
@@ -538,9 +545,9 @@ def run_cuda(args, w):
     g.check_status()
 
     q_sorted = sorted(q_us)
-    q_lat, ms_step, e2e_lat, app_us, att_kernel_us, retrieve_us, layer_seq_us, q_median, q_min = max_over_ranks(
+    q_lat, ms_step, e2e_lat, app_us, att_kernel_us, retrieve_us, layer_seq_us, q_median, q_min, e2e_step = max_over_ranks(
         [mean(q_us), total_ms / K, mean(e2e_us), mean(a_us), mean(att_us), retrieve_us, layer_seq_us,
-         q_sorted[len(q_sorted) // 2], q_sorted[0]], dev, world)
+         q_sorted[len(q_sorted) // 2], q_sorted[0], mean(e2e_step_us)], dev, world)
 
     if rank == 0:
         peaks = measured_peaks()
@@ -574,8 +581,12 @@ def run_cuda(args, w):
                          "questions_per_s_all_gpus": world * 1e6 / q_lat},
             "append_us": app_us,
             "e2e": {"value": e2e_lat, "unit": "us",
-                    "h2d_bytes_per_step": aps * 2 * kf.numel() * 2 + dq.numel() * 2,
-                    "d2h_bytes_per_step": out.numel() * 2},
+                    "h2d_bytes_per_step": dq.numel() * 2,
+                    "d2h_bytes_per_step": out.numel() * 2,
+                    "region": "per question: queries H2D from pinned memory, steps 2-5, output D2H",
+                    "whole_step_us": e2e_step,
+                    "whole_step_h2d_bytes": aps * 2 * kf.numel() * 2 + dq.numel() * 2,
+                    "whole_step_region": f"{aps} frame(s) K/V H2D + append, then the question batch as above"},
             "gpu_launches": int(launches),
             "clocks": clocks,
         }
@@ -609,6 +620,41 @@ def run_cuda(args, w):
         dist.destroy_process_group()
 
 
+def rank_plumbing_check(args):
+    """Only the rank plumbing of the replicas-only N > 1 run, on CPU with the gloo backend: rendezvous from the
+    launcher's environment, barrier, maximum over the ranks of a per-rank time.  Rank 0 prints one JSON line.
+    The CPU tests use it to run the `--gpus N` launcher without a GPU."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    worst = max_over_ranks([100.0 + rank, 5.0 - rank], torch.device("cpu"), world)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"plumbing_check": True, "n_gpus": world, "max_over_ranks": worst}))
+
+
+def launch_replicas(args):
+    """`--gpus N` without a launcher's environment: start the N replica processes here, one per device, the way
+    the N > 1 run is specified (torch.distributed.run on one node, rendezvous on 127.0.0.1).  The replicas are
+    independent; the process group only carries the barriers and the maximum over the ranks."""
+    import socket
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")            # the communicator's set-up lines, kept off stdout
+    env.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
+    return subprocess.call(cmd, env=env)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -619,7 +665,13 @@ def main():
     ap.add_argument("--workload", default="7b_hbm_1800f", choices=sorted(WORKLOADS))
     ap.add_argument("--layers", type=int, default=None, help="profiling only: fewer layers than the workload")
     ap.add_argument("--frames", type=int, default=None, help="profiling only: a shorter stream")
+    ap.add_argument("--plumbing-check", action="store_true",
+                    help="run only the rank plumbing (gloo, CPU): what the CPU tests use to exercise --gpus N")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and (args.impl == "cuda" or args.plumbing_check):
+        sys.exit(launch_replicas(args))
+    if args.plumbing_check:
+        return rank_plumbing_check(args)
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     w = dict(WORKLOADS[args.workload], name=args.workload)
     if args.layers or args.frames:

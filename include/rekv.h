@@ -52,7 +52,6 @@ enum {
 
 /* rekv_config.flags */
 enum {
-  REKV_FLAG_ATTEND_LEGACY_MMA = 1u << 1,        /* use the mma.sync attention kernel instead of tcgen05 */
   REKV_FLAG_TIMING = 1u << 2,                   /* bracket the attention kernel with CUDA events on the caller's
                                                   stream; rekv_stats then reports its duration */
   REKV_FLAG_HOST_FP8 = 1u << 3                  /* offloaded contexts only: the pinned-host tier holds each page row
@@ -237,6 +236,17 @@ int rekv_attend_layer(rekv_ctx* ctx, int layer, const void* q, const int32_t* cu
 int rekv_save(rekv_ctx* ctx, const char* path);
 int rekv_load(const char* path, int device, rekv_ctx** out);
 
+/* Output geometry of a question that sees n_visible frames and asks for top_k: how the library sizes what
+ * rekv_retrieve and rekv_gather write (readings of the Eq. 2 paragraph: the last W visible frames are never
+ * candidates; with block retrieval only complete blocks are).  Host-side only, no device work.
+ *   n_scored   items scored per (layer, question): candidate blocks when block_frames > 1, else -- the score
+ *              array then covers every visible frame -- n_visible
+ *   k_eff      frames actually retrieved, min(top_k, candidates) rounded to whole blocks
+ *   w_eff      trailing frames that are always in the context; context frames = k_eff + w_eff
+ * Any of the three output pointers may be NULL.  Returns 0, or REKV_ERR_ARG on a negative argument or a
+ * top_k that is not a multiple of block_frames. */
+int rekv_geometry(rekv_ctx* ctx, int n_visible, int top_k, int32_t* n_scored, int32_t* k_eff, int32_t* w_eff);
+
 /* Fills *out with store accounting and the last call's counters. */
 int rekv_stats(rekv_ctx* ctx, rekv_stats_t* out);
 
@@ -249,6 +259,17 @@ int rekv_set_timing(rekv_ctx* ctx, int enable);
 /* Reads (and clears) the device status word after synchronising `stream`: 0, or REKV_ERR_TIMEOUT
  * if a bounded device-side wait gave up since the last check. */
 int rekv_check_status(rekv_ctx* ctx, void* stream);
+
+/* TEST-ONLY.  The kernels' device-side waits (on a copy, a matrix product, another warp) are bounded: when a
+ * wait runs out of iterations the kernel writes REKV_ERR_TIMEOUT to the status word, releases what it holds
+ * and returns, and the context stays usable.  This call makes that path reachable without a fault:
+ *   iterations       limit of every bounded wait of the attention kernels launched from now on (0 = the
+ *                    built-in limit, about a third of a second)
+ *   skip_copy_entry  >= 0: the copy producer of the attention kernel's first CTA leaves out the K/V tile copy
+ *                    with this sequence number, so that the wait for it expires with nothing in flight; -1 = off
+ * The affected launches produce no valid output; rekv_check_status then returns REKV_ERR_TIMEOUT once.
+ * Host-side only; returns REKV_OK. */
+int rekv_test_set_wait_limit(rekv_ctx* ctx, unsigned iterations, int skip_copy_entry);
 
 /* Message of the last failure on this context (or of the last failed rekv_create when ctx is NULL).
  * The pointer stays valid until the next failing call. */

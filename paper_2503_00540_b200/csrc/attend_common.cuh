@@ -21,7 +21,12 @@ struct TcParams {
   int* unit_cnt;     // per unit: parts finished so far (decode kernel: the last part merges; self-resetting)
   int* status;
   QBatch qb;
-  int Hq, Hkv, G, Nf, Npad, NA, NB, ncf, MP, layer0;
+  int Hq, Hkv, G, Nf, Npad, ncf, MP, layer0;
+  int Ns;           // tensor-core kernel: rows a frame takes in the token stream, N_f rounded up to a multiple of 8
+  // test-only knobs (0 = off): iteration limit of the bounded waits, and the ring entry whose copy the
+  // producer of CTA 0 leaves out so that a wait runs out with nothing in flight
+  unsigned wait_limit;
+  int skip_copy_entry;
   int per;          // (unit, frame) steps per CTA
   // A unit with one row tile has no second tile to overlap with; it is run as two half-streams on the two tile
   // slots instead -- the same rows, the frame's token chunks dealt alternately -- whose (max, sum, O) partials the

@@ -58,6 +58,8 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) attend_decode_kernel(const TcP
   long long pos = (long long)blockIdx.x * p.per;
   const long long end = min(pos + (long long)p.per, p.total);
   uint32_t cnt = 0;  // frames consumed so far by this CTA: stage = cnt & 1, phase = (cnt >> 1) & 1
+  uint32_t issued = 0;  // thread 0: frames whose copies have been issued (sequence numbers [0, issued))
+  const uint32_t wait_limit = p.wait_limit ? p.wait_limit : (1u << 22);
   bool ok = true;
 
   while (pos < end && ok) {
@@ -74,6 +76,8 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) attend_decode_kernel(const TcP
       const char* ks = pages_k ? pages_k[i] + (long long)ui.g * 2 * half_bytes : kt;
       const uint32_t bar = bar0 + 8 * st;
       const uint32_t dst = s_base + st * 2u * tile_bytes;
+      issued = cnt + i + 1;
+      if (p.skip_copy_entry >= 0 && blockIdx.x == 0 && (int)(cnt + i) == p.skip_copy_entry) return;  // test-only
       if (!DEC_GUARD(pages[i] != nullptr && (reinterpret_cast<uintptr_t>(kt) & 15) == 0 &&
                      (reinterpret_cast<uintptr_t>(ks) & 15) == 0 && (half_bytes & 15) == 0, 1)) return;
       if (!DEC_GUARD(dst + 2u * tile_bytes <= s_base + ring_bytes && (dst & 15) == 0 && (half_stride & 15) == 0, 2)) return;
@@ -115,7 +119,7 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) attend_decode_kernel(const TcP
     for (int i = 0; i < nfr; ++i) {
       const uint32_t st = (cnt + i) & 1;
       bool got = false;
-      for (uint32_t it = 0; it < (1u << 22); ++it) {
+      for (uint32_t it = 0; it < wait_limit; ++it) {
         if (mbar_try_wait(bar0 + 8 * st, ((cnt + i) >> 1) & 1)) {
           got = true;
           break;
@@ -211,12 +215,13 @@ __global__ void __launch_bounds__(DEC_THREADS, 1) attend_decode_kernel(const TcP
       if (ok && tid == 0 && i + 2 < nfr) issue(i + 2);
     }
     if (!ok) {
-      // a copy never completed: record it and give copies still in flight a bounded chance to land
+      // a copy never completed: record it and give the copies still in flight -- the last two frames issued, one
+      // per stage -- a bounded chance to land before the CTA's shared memory is given up
       if (tid == 0) {
         atomicExch(p.status, REKV_ERR_TIMEOUT);
-        for (int stg = 0; stg < 2; ++stg)
-          for (uint32_t it = 0; it < (1u << 16); ++it)
-            if (mbar_try_wait(bar0 + 8 * stg, 0) || mbar_try_wait(bar0 + 8 * stg, 1)) break;
+        for (uint32_t e = issued > 2 ? issued - 2 : 0; e < issued; ++e)
+          for (uint32_t it = 0; it < wait_limit && !mbar_try_wait(bar0 + 8 * (e & 1), (e >> 1) & 1); ++it)
+            __nanosleep(64);
       }
       __syncthreads();
       break;

@@ -3,22 +3,27 @@
 //
 // One CTA per SM, persistent over a contiguous range of (unit, context frame) steps ("stream-K"):
 // a unit is (layer, kv head, question, pair of 128-row tiles), a row being (question token, query
-// head of the KV group).  Each context frame's K and V head tiles are brought in once with
-// contiguous bulk copies (the store keeps them in the 128-byte-swizzled operand layout) and applied
-// to both row tiles.  Warp roles:
-//   warp 0      bulk copies of K/V tiles into a 3-deep shared-memory ring (one lane)
+// head of the KV group).  Eq. 3 without a positional term does not depend on the order or grouping of the
+// context tokens, so the frames of a range are taken as ONE token stream and cut into dense chunks of 128
+// tokens that run across frame boundaries: every matrix product has the full width, and a 196-token frame
+// costs 1.56 chunk phases instead of two.  In the stream a frame takes N_s = N_f rounded up to a multiple
+// of 8 rows, so that a token's row in a chunk tile has the swizzle phase (row & 7) it has in its page: a
+// chunk tile is then assembled in shared memory by contiguous bulk copies (the tail of one page's tile
+// half, the head of the next), with no layout change in HBM.  The N_s - N_f gap rows between two frames
+// and the rows after the range's last token are zeroed in shared memory and their logits masked.
+// Warp roles:
+//   warp 0      assembles K/V chunk tiles in a 5-deep shared-memory ring (bulk copies, one lane)
 //   warp 1      tcgen05.mma issue (one lane): S = Q K^T into TMEM, O += P V with P read from TMEM
 //               (warps 2, 3 idle: the service warps form one warpgroup and give their registers up)
 //   warps 4-7   softmax of row tile 0: one thread per row (= TMEM lane), fp32, lazy rescaling of O
 //   warps 8-11  softmax of row tile 1 -- the two tiles alternate on the tensor core, so one tile's
 //               softmax overlaps the other's matrix products
-// After set-up the service warpgroup shrinks to 72 registers per thread and the softmax warpgroups grow to
-// 216 (setmaxnreg), so that a softmax thread holds a whole S row chunk (up to 112 values) at once: one
-// TMEM load phase with wide loads, one wait, one maximum and one rescaling decision per chunk.  The chunk's
-// last 16-column piece, the only one that can hold a frame's pad tokens, always lands in the same registers,
-// so masking touches 16 values instead of being predicated over the whole chunk.
+// After set-up the service warpgroup shrinks to 88 registers per thread and the softmax warpgroups grow to
+// 208 (setmaxnreg), so that a softmax thread holds a whole S row chunk (128 values) at once: one TMEM load
+// instruction, one wait, one maximum and one rescaling decision per chunk, and two TMEM stores for P.  Columns
+// without a token are masked piece by piece (16 columns) behind a warp-uniform test of the piece's mask bits.
 // TMEM (512 columns): O0 [0,128)  O1 [128,256)  S0/P0 [256,384)  S1/P1 [384,512); P (bf16) overwrites
-// the front of its S.  A frame of N_f tokens is processed as one or two token chunks of <= 128.
+// the front of its S.
 // A range that does not cover a whole unit leaves (max, sum, O) partials for the combine kernel.
 // A unit with a single row tile (at most 128 rows: short questions, the remainder of long ones) would leave the
 // tensor core idle during its softmax; it runs as two half-streams instead -- both tile slots work on the same rows,
@@ -33,36 +38,27 @@
 using namespace rekv_ptx;
 using namespace rekv_att;
 
-// Optional cycle-stamp tracing of one CTA (compile with -DREKV_TRACE [-DREKV_TRACE_CTA=n]; never part of the shipped library):
-// slot layout is [role][chunk][event]; rekv_trace_read copies the stamps out.
-#ifdef REKV_TRACE
-#ifndef REKV_TRACE_CTA
-#define REKV_TRACE_CTA 0
-#endif
-__device__ long long g_rekv_trace[8192];
-#define REKV_STAMP(role, i, ev)                                                                  \
-  do {                                                                                           \
-    if (blockIdx.x == REKV_TRACE_CTA && lane == 0 && (i) < 64) g_rekv_trace[(role) * 1024 + (i) * 8 + (ev)] = clock64(); \
-  } while (0)
-extern "C" int rekv_trace_read(long long* host, int n) {
-  cudaDeviceSynchronize();
-  return (int)cudaMemcpyFromSymbol(host, g_rekv_trace, n * sizeof(long long));
-}
-#else
-#define REKV_STAMP(role, i, ev) do { } while (0)
-#endif
-
 namespace {
 
 constexpr int TC_THREADS = 384;
 constexpr int SM_WARP0 = 4;                            // first softmax warp
-constexpr int REGS_SERVICE = 72, REGS_SOFTMAX = 216;   // 128 * service + 256 * softmax <= 384 * 168
-constexpr int KV_BUFS = 3;
+constexpr int REGS_SERVICE = 88, REGS_SOFTMAX = 208;   // 128 * service + 256 * softmax <= 384 * 168
+constexpr int KV_BUFS = 5;
+constexpr int CHUNK = 128;                             // tokens (stream rows) per chunk
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t Q_TILE_BYTES = 128 * 256;  // 128 rows x 128 dims bf16
+constexpr uint32_t HALF_BYTES = CHUNK * 128;  // one 64-dim half of a chunk tile
+constexpr uint32_t TILE_BYTES = 2 * HALF_BYTES;
 constexpr uint32_t STAGE_ROW_F32 = 144, STAGE_ROW_BF16 = 80;  // epilogue staging rows: a quarter row + 16 bytes (no bank conflicts)
 constexpr uint32_t STAGE_WARP_BYTES = 32 * STAGE_ROW_F32;
-constexpr float RESCALE_THRESHOLD = 8.f;      // log2 units: O is rescaled only when the row max grows by > 2^8
+constexpr float RESCALE_SUM_LIMIT = 1.152921504606846976e18f;  // 2^60: a chunk's row sum beyond it raises the reference maximum
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+// P is cut (not rounded) to bf16: a value with mantissa m in [1, 2) loses u * 2^-7 / m of itself, u uniform in [0, 1).
+// The mantissa of 2^x is log-uniform, E[1/m] = 1 / (2 ln 2), so the mean loss is 0.7213 * 2^-8 of the value, and scaling
+// by 1 + 0.7213 * 2^-8 beforehand makes the cut value right on average (its spread equals that of rounding to
+// nearest).  log2 of that factor, and its inverse for the row sum:
+constexpr float TRUNC_GAIN_LOG2 = 0.0040592f;
+constexpr float TRUNC_GAIN_INV = 0.99719028f;
 
 // barrier slots after the K/V ring: full[b], empty[b], s_full[t], p_ready[t], pv_done[t]
 struct Bars {
@@ -87,11 +83,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const uint32_t s_base = smem_u32(smem);
-  const uint32_t tile_bytes = 2u * p.Npad * 128u;   // one K (or V) head tile: two 64-dim halves
-  const uint32_t half_stride = p.Npad * 128u;
   const uint32_t s_q = s_base;                       // two Q row tiles
-  const uint32_t s_kv = s_base + 2 * Q_TILE_BYTES;   // ring of KV_BUFS tiles
-  const uint32_t s_bar = s_kv + KV_BUFS * tile_bytes;
+  const uint32_t s_kv = s_base + 2 * Q_TILE_BYTES;   // ring of KV_BUFS chunk tiles
+  const uint32_t s_bar = s_kv + KV_BUFS * TILE_BYTES;
   Bars bars;
   bars.base = s_bar;
   volatile uint32_t* s_tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + (s_bar - s_base) + 8 * (2 * KV_BUFS + 6));
@@ -99,20 +93,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   volatile uint32_t* s_stop = s_tmem_slot + 2;  // the abort flag as one thread saw it between two segment barriers
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (warp == 6) REKV_STAMP(3, 0, 0);
 
   // ---- one-time set-up -------------------------------------------------------------------------
-  {  // zero the pad rows [Nf, Npad) of every ring tile half; the bulk copies never write them
-    const int pad_rows = p.Npad - p.Nf;
-    const int n16 = KV_BUFS * 2 * pad_rows * 8;
-    for (int i = tid; i < n16; i += TC_THREADS) {
-      int c = i & 7;
-      int r = (i >> 3) % pad_rows;
-      int hh = (i >> 3) / pad_rows;  // (buffer, half)
-      *reinterpret_cast<uint4*>(smem + 2 * Q_TILE_BYTES + (hh >> 1) * tile_bytes + (hh & 1) * half_stride +
-                                (p.Nf + r) * 128 + c * 16) = make_uint4(0, 0, 0, 0);
-    }
-  }
   if (tid == 0) {
     for (int i = 0; i < KV_BUFS; ++i) {
       mbar_init(bars.full(i), 1);
@@ -137,15 +119,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   tc_fence_after();
   const uint32_t tmem = *s_tmem_slot;
   // everything above is independent of earlier kernels; the context table and Q are not
-  if (warp == 6) REKV_STAMP(3, 0, 1);
   grid_dep_wait();
-  if (warp == 6) REKV_STAMP(3, 0, 2);
   grid_dep_launch();
   auto col_o = [](int t) { return (uint32_t)t * 128u; };
   auto col_s = [](int t) { return 256u + (uint32_t)t * 128u; };
 
+  const uint32_t wait_limit = p.wait_limit ? p.wait_limit : WAIT_LIMIT;
   auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
-    for (uint32_t it = 0; it < (1u << 22); ++it) {
+    for (uint32_t it = 0; it < wait_limit; ++it) {
       if (mbar_try_wait(bar, parity)) return true;
       if (*s_abort) return false;
       if (it > 2048) __nanosleep(64);
@@ -155,13 +136,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     return false;
   };
 
-  const int cpf = p.NB > 0 ? 2 : 1;                 // token chunks per frame
   // Barrier of a range segment for every warp but the copy producer, which runs ahead into the next segment (it is
   // held back by the ring's empty barriers only), so that K/V tiles are already on their way during an epilogue.
   auto seg_sync = [&]() {
     if (warp != 0) asm volatile("bar.sync 1, %0;" ::"n"(TC_THREADS - 32) : "memory");
   };
-  const uint32_t half_bytes = (uint32_t)p.Nf * 128u;
+  const uint32_t page_half_bytes = (uint32_t)p.Nf * 128u;   // one 64-dim half of a head tile in a page
   const uint32_t idesc_pv = idesc_bf16(128, 128, 1);
 
   // The roles run the same range loop with the role as a compile-time constant, so that each side of the
@@ -170,25 +150,27 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   constexpr bool SOFTMAX = decltype(role)::value;
   long long pos = (long long)blockIdx.x * p.per;
   const long long end = min(pos + (long long)p.per, p.total);
-  uint32_t ring = 0;    // K/V tiles moved so far (K and V of a frame are consecutive ring entries)
+  uint32_t ring = 0;    // chunk tiles moved so far (K and V of a chunk are consecutive ring entries)
+  uint32_t ring_issued = 0;  // copy producer: ring entries whose copies have been issued
   uint32_t chunk_cnt[2] = {0u, 0u};  // token chunks processed so far, per row tile (barrier phases)
 
-  int seg = 0;  // range segments so far (tracing only)
   while (pos < end) {
     const long long u = pos / p.ncf;
     const int f0 = (int)(pos - u * p.ncf);
     const int nfr = (int)min((long long)(p.ncf - f0), end - pos);
     const UnitInfo ui = decode_unit(p, u);
-    const int nchunks = nfr * cpf;
+    // the segment's token stream: frame i at rows [i N_s, i N_s + N_f); the last frame's gap rows are cut off
+    const int Lrows = (nfr - 1) * p.Ns + p.Nf;
+    const int nchunks = (Lrows + CHUNK - 1) / CHUNK;
     const bool split = SPLIT && ui.split != 0;
     const int vtiles = split ? 2 : ui.tiles;  // tile slots in use
     // chunks per tile slot and a slot's j-th chunk among the segment's: every chunk for both tiles, or alternately
     const int nch0 = split ? (nchunks + 1) >> 1 : nchunks, nch1 = split ? nchunks >> 1 : nchunks;
     auto chunk_of = [&](int T, int j) { return split ? 2 * j + T : j; };
+    auto chunk_n = [&](int I) { return (min(CHUNK, Lrows - I * CHUNK) + 15) & ~15; };  // columns of chunk I's products
     char* const* pages = p.tbl + ((long long)ui.l * p.qb.nQ + ui.qi) * p.ncf + f0;
     char* const* pages_k = (FULL && p.tbl_k) ? p.tbl_k + ((long long)ui.l * p.qb.nQ + ui.qi) * p.ncf + f0 : nullptr;
     const bool whole_unit = (nfr == p.ncf) && !split;
-    if (warp == 6) REKV_STAMP(3, 1 + seg, 0);
 
     // ---- Q row tiles -> shared memory in the swizzled K-major operand layout -------------------
     if (warp >= SM_WARP0) {
@@ -211,55 +193,93 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
       fence_proxy_async();
     }
     seg_sync();
-    if (warp == 6) REKV_STAMP(3, 1 + seg, 1);
 
     if constexpr (!SOFTMAX) {
     if (warp == 0) {
       // ================= copy producer =================
-      // the whole warp walks the ring (uniform control flow); one elected lane issues the copies
-      for (int fi = 0; fi < nfr; ++fi) {
-        const char* kt = pages[fi] + (long long)(ui.g * 2) * p.Nf * 256;
-        bool stop = false;
+      // the whole warp walks the ring (uniform control flow).  Per chunk tile: the rows no page covers (gap rows
+      // between frames, the rows after the stream's end up to the products' width) are zeroed by all lanes, then one
+      // elected lane issues the copies -- per frame that overlaps the chunk and per 64-dim half one contiguous piece.
+      const long long head_off = (long long)(ui.g * 2) * p.Nf * 256;   // this KV head's K tile inside a page
+      bool stop = false;
+      for (int I = 0; I < nchunks && !stop; ++I) {
+        const int row0 = I * CHUNK;
+        const int nrows = min(CHUNK, Lrows - row0);     // stream rows of this chunk
+        const int N = (nrows + 15) & ~15;
+        const int fi0 = row0 / p.Ns, fi1 = (row0 + nrows - 1) / p.Ns;
+        const int pos0 = row0 - fi0 * p.Ns;             // the chunk's first row inside frame fi0
+        uint32_t bytes = 0;
+        for (int fi = fi0; fi <= fi1; ++fi) {
+          const int ta = max(0, row0 - fi * p.Ns), tb = min(p.Nf, row0 + nrows - fi * p.Ns);
+          if (tb > ta) bytes += 2u * (uint32_t)(tb - ta) * 128u;
+        }
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
-          const uint32_t r = ring + 2 * fi + kv;
+          const uint32_t r = ring + 2 * I + kv;
           const uint32_t b = r % KV_BUFS, use = r / KV_BUFS;
           if (use > 0 && !wait(bars.empty(b), (use - 1) & 1)) {
             stop = true;
             break;
           }
-          const uint32_t dst = s_kv + b * tile_bytes;
-          const char* src = kt + (long long)kv * 2 * half_bytes;
-          if (FULL && kv == 0 && pages_k) src = pages_k[fi] + (long long)ui.g * 2 * half_bytes;  // rotated K tiles
-          if (elect_one()) {
-            mbar_expect_tx(bars.full(b), 2u * half_bytes);
-            bulk_g2s(dst, src, half_bytes, bars.full(b));
-            bulk_g2s(dst + half_stride, src + half_bytes, half_bytes, bars.full(b));
+          const uint32_t dst = s_kv + b * TILE_BYTES;
+          {  // rows without a token
+            int x = pos0 + lane;
+            for (int rr = lane; rr < N; rr += 32, x += 32) {
+              if (p.Ns >= CHUNK) {
+                if (x >= p.Ns) x -= p.Ns;
+              } else {
+                x %= p.Ns;
+              }
+              if (rr >= nrows || x >= p.Nf) {
+                unsigned char* row_ptr = smem + (dst - s_base) + rr * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                  *reinterpret_cast<uint4*>(row_ptr + c * 16) = make_uint4(0, 0, 0, 0);
+                  *reinterpret_cast<uint4*>(row_ptr + HALF_BYTES + c * 16) = make_uint4(0, 0, 0, 0);
+                }
+              }
+            }
+            fence_proxy_async();
+            __syncwarp();
           }
+          const bool skip = p.skip_copy_entry >= 0 && blockIdx.x == 0 && (int)r == p.skip_copy_entry;  // test-only
+          if (elect_one() && !skip) {
+            mbar_expect_tx(bars.full(b), bytes);
+            for (int fi = fi0; fi <= fi1; ++fi) {
+              const int ta = max(0, row0 - fi * p.Ns), tb = min(p.Nf, row0 + nrows - fi * p.Ns);
+              if (tb <= ta) continue;
+              const char* src = pages[fi] + head_off + (long long)kv * 2 * page_half_bytes;
+              if (FULL && kv == 0 && pages_k) src = pages_k[fi] + (long long)ui.g * 2 * page_half_bytes;  // rotated K tiles
+              const uint32_t d = dst + (uint32_t)(fi * p.Ns + ta - row0) * 128u;
+              const uint32_t nb = (uint32_t)(tb - ta) * 128u;
+              bulk_g2s(d, src + (long long)ta * 128, nb, bars.full(b));
+              bulk_g2s(d + HALF_BYTES, src + page_half_bytes + (long long)ta * 128, nb, bars.full(b));
+            }
+          }
+          ring_issued = r + 1;
           __syncwarp();
         }
-        if (stop || *s_abort) break;
+        if (*s_abort) stop = true;
       }
     } else if (warp == 1) {
       // ================= MMA issuer =================
       // Descriptors are built once; per instruction only the 14-bit start-address field advances.
       {
         const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);  // SBO = 1024 B, version, SWIZZLE_128B
-        const uint32_t lbo_v = ((half_stride >> 4) & 0x3FFFu) << 16;      // pitch of V's two 64-dim blocks
+        const uint32_t lbo_v = ((HALF_BYTES >> 4) & 0x3FFFu) << 16;       // pitch of V's two 64-dim blocks
         const uint32_t lbo_k = 1u << 16;                                  // unused for K-major operands
-        const uint32_t half16 = half_stride >> 4;
+        const uint32_t half16 = HALF_BYTES >> 4;
         const int tiles = vtiles;
         bool ok = true;
 #define REKV_DESC(lo) (((uint64_t)desc_hi << 32) | (uint64_t)(lo))
 #define REKV_ISSUE_S(T, I)                                                                                    \
   do {                                                                                                        \
-    const int fi_ = (I) / cpf, part_ = (I) - fi_ * cpf;                                                       \
-    const uint32_t r_ = ring + 2 * fi_, b_ = r_ % KV_BUFS;                                                    \
-    const uint32_t tok0_ = part_ ? p.NA : 0, N_ = part_ ? p.NB : p.NA;                                        \
-    if (part_ == 0 && ((T) == 0 || split)) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                      \
+    const uint32_t r_ = ring + 2 * (I), b_ = r_ % KV_BUFS;                                                    \
+    const uint32_t N_ = (uint32_t)chunk_n(I);                                                                 \
+    if ((T) == 0 || split) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                                      \
     if (ok) {                                                                                                 \
       tc_fence_after();                                                                                       \
-      const uint32_t k_lo = ((s_kv + b_ * tile_bytes + tok0_ * 128u) >> 4) | lbo_k;                           \
+      const uint32_t k_lo = ((s_kv + b_ * TILE_BYTES) >> 4) | lbo_k;                                          \
       const uint32_t q_lo = ((s_q + (T) * Q_TILE_BYTES) >> 4) | lbo_k;                                        \
       const uint32_t idesc_ = idesc_bf16(128, N_, 0);                                                         \
       const uint32_t d_ = tmem + col_s(T);                                                                    \
@@ -269,27 +289,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
       _Pragma("unroll") for (int kk = 0; kk < 4; ++kk)                                                        \
           mma_ss(d_, REKV_DESC(q_lo + (Q_TILE_BYTES / 32) + 2 * kk), REKV_DESC(k_lo + half16 + 2 * kk), idesc_, 1); \
       tc_commit(bars.s_full(T));                                                                              \
-      if (part_ == cpf - 1 && ((T) == tiles - 1 || split)) tc_commit(bars.empty(b_)); /* K tile done */       \
+      if ((T) == tiles - 1 || split) tc_commit(bars.empty(b_)); /* K tile done */                             \
       }                                                                                                       \
       __syncwarp();                                                                                           \
     }                                                                                                         \
   } while (0)
 #define REKV_ISSUE_PV(T, I, J)                                                                                \
   do {                                                                                                        \
-    const int fi_ = (I) / cpf, part_ = (I) - fi_ * cpf;                                                       \
-    const uint32_t r_ = ring + 2 * fi_ + 1, b_ = r_ % KV_BUFS;                                                \
-    const uint32_t tok0_ = part_ ? p.NA : 0, nk_ = (part_ ? p.NB : p.NA) >> 4;                                \
-    if (part_ == 0 && ((T) == 0 || split)) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                      \
+    const uint32_t r_ = ring + 2 * (I) + 1, b_ = r_ % KV_BUFS;                                                \
+    const uint32_t nk_ = (uint32_t)chunk_n(I) >> 4;                                                           \
+    if ((T) == 0 || split) ok = wait(bars.full(b_), (r_ / KV_BUFS) & 1);                                      \
     if (ok) ok = wait(bars.p_ready(T), (chunk_cnt[T] + (J)) & 1);                                             \
     if (ok) {                                                                                                 \
       tc_fence_after();                                                                                       \
-      const uint32_t v_lo = ((s_kv + b_ * tile_bytes + tok0_ * 128u) >> 4) | lbo_v;                           \
+      const uint32_t v_lo = ((s_kv + b_ * TILE_BYTES) >> 4) | lbo_v;                                          \
       const uint32_t d_ = tmem + col_o(T), a_ = tmem + col_s(T);                                              \
       if (elect_one()) {                                                                                      \
       _Pragma("unroll") for (int kk = 0; kk < 8; ++kk)                                                        \
           if (kk < (int)nk_) mma_ts(d_, a_ + 8 * kk, REKV_DESC(v_lo + 128 * kk), idesc_pv, ((J) > 0) | (kk > 0)); \
       tc_commit(bars.pv_done(T));                                                                             \
-      if (part_ == cpf - 1 && ((T) == tiles - 1 || split)) tc_commit(bars.empty(b_)); /* V tile done */       \
+      if ((T) == tiles - 1 || split) tc_commit(bars.empty(b_)); /* V tile done */                             \
       }                                                                                                       \
       __syncwarp();                                                                                           \
     }                                                                                                         \
@@ -297,16 +316,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         REKV_ISSUE_S(0, 0);
         if (tiles == 2 && ok && chunk_of(1, 0) < nchunks) REKV_ISSUE_S(1, chunk_of(1, 0));
         for (int j = 0; j < nch0 && ok; ++j) {
-          REKV_STAMP(0, j, 0);
           REKV_ISSUE_PV(0, chunk_of(0, j), j);
-          REKV_STAMP(0, j, 1);
           if (chunk_of(0, j + 1) < nchunks && ok) REKV_ISSUE_S(0, chunk_of(0, j + 1));
-          REKV_STAMP(0, j, 2);
           if (tiles == 2 && ok && chunk_of(1, j) < nchunks) {
             REKV_ISSUE_PV(1, chunk_of(1, j), j);
-            REKV_STAMP(0, j, 3);
             if (chunk_of(1, j + 1) < nchunks && ok) REKV_ISSUE_S(1, chunk_of(1, j + 1));
-            REKV_STAMP(0, j, 4);
           }
         }
 #undef REKV_ISSUE_S
@@ -330,77 +344,145 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         // a warp whose 32 rows all lie beyond the unit's rows (the ragged second tile) only keeps the barriers moving
         const bool warp_idle = ui.m0 + rt * 128 + ((warp & 3) << 5) >= ui.rows_q;
         for (int i = 0; i < nch && ok; ++i) {  // i counts this slot's chunks
-          const int part = cpf == 2 ? (chunk_of(t, i) & 1) : 0;
-          const int tok0 = part ? p.NA : 0, N = part ? p.NB : p.NA;
-          const int nv = min(N, p.Nf - tok0);  // valid tokens of this chunk
-          const int npc = N >> 4;
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 0);
+          // ---- the chunk's shape, worked out while its S is still being computed ----
+          const int I = chunk_of(t, i);
+          const int row0 = I * CHUNK;
+          const int nrows = min(CHUNK, Lrows - row0);
+          // columns without a token, a bit per column (warp-uniform): a lane looks at columns lane, lane + 32, ...
+          unsigned long long mw_lo, mw_hi;
+          {
+            const int pos0 = row0 % p.Ns;
+            uint32_t mw[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const int col = lane + 32 * k;
+              int x = pos0 + col;
+              if (p.Ns >= CHUNK) {
+                if (x >= p.Ns) x -= p.Ns;
+              } else {
+                x %= p.Ns;
+              }
+              mw[k] = __ballot_sync(0xffffffffu, col >= nrows || x >= p.Nf);
+            }
+            mw_lo = (unsigned long long)mw[0] | ((unsigned long long)mw[1] << 32);
+            mw_hi = (unsigned long long)mw[2] | ((unsigned long long)mw[3] << 32);
+          }
+          // -1: nothing to mask; 0..7: the only piece with masked columns, and its bits; 8: several pieces
+          int mask_pc = -1;
+          uint32_t mask_bits = 0;
+#pragma unroll
+          for (int pc = 0; pc < 8; ++pc) {
+            const uint32_t m16 = (uint32_t)(((pc & 4) ? mw_hi : mw_lo) >> ((pc & 3) * 16)) & 0xFFFFu;
+            if (m16) {
+              mask_pc = mask_pc < 0 ? pc : 8;
+              mask_bits = m16;
+            }
+          }
           if (!wait(bars.s_full(t), (chunk_cnt[t] + i) & 1)) {
             ok = false;
             break;
           }
           tc_fence_after();
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 1);
           if (warp_idle) {  // no valid row in this warp's 32 lanes: their P and O rows are never read back
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bars.p_ready(t));
             continue;
           }
-          // The whole S row chunk comes into registers in one load phase (up to seven 16-column pieces), so there
-          // is one wait, one row maximum and one rescaling decision per chunk.  Lazy rescaling: the maximum in
-          // use is raised only when this chunk exceeds it by more than the threshold (always on the first
-          // chunk); O and the running sum then shrink by 2^(old - new).
+          // The whole S row chunk comes into registers with ONE TMEM load instruction (a warp's tcgen05.ld/st
+          // instructions run one after the other at about 90 cycles each, whatever their width), so there is one
+          // wait, one row maximum and one rescaling decision per chunk.  Columns without a token -- a frame
+          // boundary's gap, the stream's end, the columns beyond the products' width, which hold stale values -- are
+          // masked piece by piece behind a warp-uniform test, so that only the piece that has some pays for it.
+          // Lazy rescaling: the maximum in use is raised only when this chunk exceeds it by more than the threshold
+          // (always on the first chunk); O and the running sum then shrink by 2^(old - new).
           const float NEG_INF = -INFINITY;
-          const int npm = npc - 1;  // pieces before the chunk's last one, which always sits in sv[7]
-          uint32_t sv[8][16];
+          uint32_t sv[128];
+          tmem_ld128(t_s, sv);
+          tmem_wait_ld128(sv);
+          if (mask_pc >= 0) {
+            auto mask16 = [&](uint32_t* v, uint32_t m16) {
 #pragma unroll
-          for (int pc = 0; pc < 7; ++pc) {
+              for (int j = 0; j < 16; ++j)
+                if ((m16 >> j) & 1u) v[j] = __float_as_uint(NEG_INF);
+            };
+            switch (mask_pc) {  // the one piece that has masked columns (warp-uniform)
+              case 0: mask16(sv, mask_bits); break;
+              case 1: mask16(sv + 16, mask_bits); break;
+              case 2: mask16(sv + 32, mask_bits); break;
+              case 3: mask16(sv + 48, mask_bits); break;
+              case 4: mask16(sv + 64, mask_bits); break;
+              case 5: mask16(sv + 80, mask_bits); break;
+              case 6: mask16(sv + 96, mask_bits); break;
+              case 7: mask16(sv + 112, mask_bits); break;
+              default:  // several pieces (N_f < 128, or the stream's last chunk): every piece tested
 #pragma unroll
-            for (int j = 0; j < 16; ++j) sv[pc][j] = 0u;
-          }
-          if (npm >= 4) {
-            tmem_ld64(t_s, sv[0], sv[1], sv[2], sv[3]);
-            if (npm >= 6) tmem_ld32(t_s + 64, sv[4], sv[5]);
-            if (npm == 5) tmem_ld16(t_s + 64, sv[4]);
-            if (npm == 7) tmem_ld16(t_s + 96, sv[6]);
-          } else {
-            if (npm >= 2) tmem_ld32(t_s, sv[0], sv[1]);
-            if (npm == 1) tmem_ld16(t_s, sv[0]);
-            if (npm == 3) tmem_ld16(t_s + 32, sv[2]);
-          }
-          tmem_ld16(t_s + npm * 16, sv[7]);
-          tmem_wait_ld_chunk(sv);
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 4);
-          {  // the frame's ragged end lies inside the last piece: its pad tokens leave the maximum and the sum
-            const int nvt = nv - npm * 16;
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (j >= nvt) sv[7][j] = __float_as_uint(NEG_INF);
-          }
-          float g0 = max3(__uint_as_float(sv[7][0]), __uint_as_float(sv[7][1]), __uint_as_float(sv[7][2]));
-          float g1 = max3(__uint_as_float(sv[7][3]), __uint_as_float(sv[7][4]), __uint_as_float(sv[7][5]));
-          float g2 = max3(__uint_as_float(sv[7][6]), __uint_as_float(sv[7][7]), __uint_as_float(sv[7][8]));
-          float g3 = max3(__uint_as_float(sv[7][9]), __uint_as_float(sv[7][10]), __uint_as_float(sv[7][11]));
-          g0 = max3(g0, __uint_as_float(sv[7][12]), __uint_as_float(sv[7][13]));
-          g1 = max3(g1, __uint_as_float(sv[7][14]), __uint_as_float(sv[7][15]));
-#pragma unroll
-          for (int pc = 0; pc < 7; ++pc)
-            if (pc < npm) {
-              g0 = max3(g0, __uint_as_float(sv[pc][0]), __uint_as_float(sv[pc][1]));
-              g1 = max3(g1, __uint_as_float(sv[pc][2]), __uint_as_float(sv[pc][3]));
-              g2 = max3(g2, __uint_as_float(sv[pc][4]), __uint_as_float(sv[pc][5]));
-              g3 = max3(g3, __uint_as_float(sv[pc][6]), __uint_as_float(sv[pc][7]));
-              g0 = max3(g0, __uint_as_float(sv[pc][8]), __uint_as_float(sv[pc][9]));
-              g1 = max3(g1, __uint_as_float(sv[pc][10]), __uint_as_float(sv[pc][11]));
-              g2 = max3(g2, __uint_as_float(sv[pc][12]), __uint_as_float(sv[pc][13]));
-              g3 = max3(g3, __uint_as_float(sv[pc][14]), __uint_as_float(sv[pc][15]));
+                for (int pc = 0; pc < 8; ++pc) {
+                  const uint32_t m16 = (uint32_t)(((pc & 4) ? mw_hi : mw_lo) >> ((pc & 3) * 16)) & 0xFFFFu;
+                  if (m16) mask16(sv + 16 * pc, m16);
+                }
+                break;
             }
-          const float gm = fmaxf(fmaxf(g0, g1), fmaxf(g2, g3)) * p.scale_log2;
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 6);
-          const bool need = gm > m_used + RESCALE_THRESHOLD;
+          }
+          auto row_max = [&]() -> float {  // of the chunk's logits, in log2 units
+            float gmx[8];
+#pragma unroll
+            for (int a8 = 0; a8 < 8; ++a8)
+              gmx[a8] = max3(__uint_as_float(sv[a8]), __uint_as_float(sv[8 + a8]), __uint_as_float(sv[16 + a8]));
+#pragma unroll
+            for (int c = 24; c + 16 <= 128; c += 16)
+#pragma unroll
+              for (int a8 = 0; a8 < 8; ++a8)
+                gmx[a8] = max3(gmx[a8], __uint_as_float(sv[c + a8]), __uint_as_float(sv[c + 8 + a8]));
+#pragma unroll
+            for (int a8 = 0; a8 < 8; ++a8) gmx[a8] = fmaxf(gmx[a8], __uint_as_float(sv[120 + a8]));
+            return max3(max3(gmx[0], gmx[1], gmx[2]), max3(gmx[3], gmx[4], gmx[5]), fmaxf(gmx[6], gmx[7])) * p.scale_log2;
+          };
+          // P = 2^(S*scale - m) as bf16 pairs over the front of S (two stores of 32 columns); returns the row sum.
+          // The conversion instruction shares the transcendental unit with ex2 (a quarter-rate pipe: 8 cycles per
+          // ex2 and 4 per packed pair and warp), which made that pipe the busiest part of the SM; so P is cut to
+          // bf16 by taking the upper halves (one byte permute per pair) of 2^(x - m) * (1 + TRUNC_GAIN), the factor
+          // that makes the cut value equal to 2^(x - m) on average over the mantissa -- folded into the exponent,
+          // and taken out of the row sum once at the end of the range.  All 128 columns are done whatever the
+          // chunk's width (masked columns give exactly 0): one straight run of code lets the compiler keep the
+          // transcendental unit fed.
+          auto exp_pass = [&]() -> float {
+            const float neg_m = TRUNC_GAIN_LOG2 - m_used;
+            float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+              uint32_t pk[32];
+#pragma unroll
+              for (int jj = 0; jj < 32; jj += 2) {
+                const uint32_t* v = sv + 64 * hf;
+                const float p0 = ex2(fmaf(__uint_as_float(v[2 * jj]), p.scale_log2, neg_m));
+                const float p1 = ex2(fmaf(__uint_as_float(v[2 * jj + 1]), p.scale_log2, neg_m));
+                const float p2 = ex2(fmaf(__uint_as_float(v[2 * jj + 2]), p.scale_log2, neg_m));
+                const float p3 = ex2(fmaf(__uint_as_float(v[2 * jj + 3]), p.scale_log2, neg_m));
+                ps0 += p0;
+                ps1 += p1;
+                ps2 += p2;
+                ps3 += p3;
+                pk[jj] = __byte_perm(__float_as_uint(p0), __float_as_uint(p1), 0x7632);
+                pk[jj + 1] = __byte_perm(__float_as_uint(p2), __float_as_uint(p3), 0x7632);
+              }
+              tmem_st32(t_s + 32 * hf, pk);
+            }
+            return (ps0 + ps1) + (ps2 + ps3);
+          };
+          // The reference value m of the exponentials is the row maximum of the range's FIRST chunk.  Later chunks
+          // do not look for their maximum at all (128 min/max instructions per row cost about 400 cycles a chunk):
+          // a softmax does not depend on m, which only has to keep 2^(x - m) inside the fp32 range, and values far
+          // above 1 lose nothing in fp32 sums or in bf16's 8 exponent bits.  So the exponentials are taken with the m
+          // in use, and only if a row's sum leaves [0, 2^60) -- a logit more than 60 octaves above m, or an overflow
+          // -- does the warp find the true maximum, shrink O and the running sum by 2^(old - new), and repeat the
+          // pass from the registers (the P stores of the first pass are simply overwritten).
+          if (i == 0) m_used = row_max();
+          float cs = exp_pass();
+          const bool need = !(cs < RESCALE_SUM_LIMIT);
           if (__any_sync(0xffffffffu, need)) {
-            const float alpha = need ? ex2(m_used - gm) : 1.f;  // 0 when nothing has been seen yet
+            const float gm = row_max();
+            const float alpha = need ? ex2(m_used - gm) : 1.f;
             if (need) m_used = gm;
             l_sum *= alpha;
             if (i > 0) {  // O holds earlier chunks; their P V is complete (this chunk's S came after it)
@@ -414,44 +496,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
                 tmem_st16(t_o + pc * 16, o);
               }
             }
+            cs = exp_pass();
           }
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 5);
-          // P = 2^(S*scale - m) as bf16 pairs over the front of S, row sum in fp32
-          const float neg_m = -m_used;
-          float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
-          auto do_piece = [&](const uint32_t (&v)[16], const uint32_t col) {
-            uint32_t pk[8];
-#pragma unroll
-            for (int jj = 0; jj < 8; jj += 2) {
-              const float p0 = ex2(fmaf(__uint_as_float(v[2 * jj]), p.scale_log2, neg_m));
-              const float p1 = ex2(fmaf(__uint_as_float(v[2 * jj + 1]), p.scale_log2, neg_m));
-              const float p2 = ex2(fmaf(__uint_as_float(v[2 * jj + 2]), p.scale_log2, neg_m));
-              const float p3 = ex2(fmaf(__uint_as_float(v[2 * jj + 3]), p.scale_log2, neg_m));
-              ps0 += p0;
-              ps1 += p1;
-              ps2 += p2;
-              ps3 += p3;
-              pk[jj] = pack_bf16(p0, p1);
-              pk[jj + 1] = pack_bf16(p2, p3);
-            }
-            tmem_st8(t_s + col, pk);
-          };
-#pragma unroll
-          for (int pc = 0; pc < 7; ++pc)
-            if (pc < npm) do_piece(sv[pc], pc * 8);
-          do_piece(sv[7], npm * 8);
-          l_sum += (ps0 + ps1) + (ps2 + ps3);
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 2);
+          l_sum += cs;
           tmem_wait_st();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bars.p_ready(t));
-          if ((warp & 3) == 2) REKV_STAMP(1 + t, i, 3);
         }
+        l_sum *= TRUNC_GAIN_INV;  // the row sum was taken over the scaled values
         // ---- output of this range: final rows, or a partial for the combine kernel ----
         if (ok && (nch == 0 || wait(bars.pv_done(t), (chunk_cnt[t] + nch - 1) & 1))) {
           tc_fence_after();
-          if (warp == 6) REKV_STAMP(3, 1 + seg, 2);
           const int rr = ui.m0 + rt * 128 + row;
           const bool valid = rr < ui.rows_q;
           const int n = rr / p.G, j = rr - n * p.G;
@@ -530,7 +586,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
             const long long slot = (p.per == p.ncf ? (long long)ui.srank : (long long)blockIdx.x + u) * 2 + t;
             // rows this lane stores: r = 4 k + (lane >> 3), 16 bytes (4 floats) at chunk (lane & 7) of the quarter
             float* po = p.part_o + ((slot * 128 + ((warp & 3) << 5) + (lane >> 3)) * 128 + (lane & 7) * 4);
-            const int nrows = ui.rows_q - rr0;  // valid rows of this warp (may exceed 32)
+            const int nrows_w = ui.rows_q - rr0;  // valid rows of this warp (may exceed 32)
 #pragma unroll 1
             for (int qd = 0; qd < 4; ++qd) {
               uint32_t o[2][16];
@@ -552,7 +608,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
 #pragma unroll
               for (int k = 0; k < 8; ++k) {
                 const uint4 x = *reinterpret_cast<const uint4*>(stage + (4 * k + (lane >> 3)) * STAGE_ROW_F32 + (lane & 7) * 16);
-                if (4 * k + (lane >> 3) < nrows) *reinterpret_cast<uint4*>(po + (long long)k * 4 * 128 + qd * 32) = x;
+                if (4 * k + (lane >> 3) < nrows_w) *reinterpret_cast<uint4*>(po + (long long)k * 4 * 128 + qd * 32) = x;
               }
               __syncwarp();
             }
@@ -564,15 +620,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         }
       }
     }
-    ring += 2 * nfr;
+    ring += 2 * nchunks;
     chunk_cnt[0] += nch0;
     if (vtiles == 2) chunk_cnt[1] += nch1;
     pos += nfr;
     tc_fence_before();
     seg_sync();
     tc_fence_after();
-    if (warp == 6) REKV_STAMP(3, 1 + seg, 3);
-    ++seg;
     // The copy producer is outside the segment barriers and may raise the abort flag at any moment; the other warps
     // must all leave together (one that left alone would never reach the next segment barrier), so they act on one
     // thread's reading of the flag, taken between two barriers.
@@ -582,6 +636,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
       if (warp == 1 && lane == 0 && *s_abort) *s_stop = 1;
       seg_sync();
       if (*s_stop) break;
+    }
+  }
+  if constexpr (!SOFTMAX) {
+    // A CTA that gives up must not return while copies into its shared memory are still on their way: the producer
+    // waits (bounded) for the tiles it has issued and nobody consumed -- at most the ring's depth.
+    if (warp == 0 && *s_abort) {
+      const uint32_t issued = ring_issued;
+      for (uint32_t r = issued > KV_BUFS ? issued - KV_BUFS : 0; r < issued; ++r)
+        for (uint32_t it = 0; it < wait_limit && !mbar_try_wait(bars.full(r % KV_BUFS), (r / KV_BUFS) & 1); ++it)
+          __nanosleep(64);
     }
   }
 
@@ -594,7 +658,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     run(std::true_type{});
   }
 
-  if (warp == 6) REKV_STAMP(3, 0, 3);
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, TMEM_COLS);
 }
@@ -621,13 +684,9 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   p.G = s.G;
   p.Nf = s.Nf;
   p.Npad = (s.Nf + 15) & ~15;
-  if (p.Npad <= 128) {  // token chunks of at most 128, two per frame beyond that (196 tokens -> 112 + 96)
-    p.NA = p.Npad;
-    p.NB = 0;
-  } else {
-    p.NA = ((p.Npad / 2) + 15) & ~15;
-    p.NB = p.Npad - p.NA;
-  }
+  p.Ns = (s.Nf + 7) & ~7;
+  p.wait_limit = c->test_wait_limit;
+  p.skip_copy_entry = c->test_skip_copy_entry;
   p.ncf = ncf;
   p.layer0 = layer0;
   p.n_split = 0;
@@ -637,7 +696,7 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   p.MP = MP;
   const long long units = (long long)(layer1 - layer0) * s.Hkv * MP;
   p.total = units * ncf;
-  const int n_sm = 148;
+  const int n_sm = rekv_sm_count();
   long long grid;
   if (units >= 4 * n_sm || (size_t)(n_sm + units) * 2 > c->part_units) {
     grid = units;  // enough units to fill the machine: one whole unit per CTA, no partials
@@ -653,12 +712,11 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   for (int i = 0; i < qb.nQ; ++i) few_rows = few_rows && (qb.cu[i + 1] - qb.cu[i]) * s.G <= 16;
   const size_t smem_dec = std::max((size_t)4 * 2 * p.Npad * 128, (size_t)DEC_SCRATCH) + 64 + 1024;
   if (few_rows && smem_dec <= 227 * 1024 && (size_t)units <= c->part_units) {
-    static bool dec_attr_set = false;
-    if (!dec_attr_set) {
-      cudaError_t e = cudaFuncSetAttribute(attend_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-      if (e != cudaSuccess) return e;
-      dec_attr_set = true;
-    }
+    static PerDeviceOnce dec_attr;
+    cudaError_t e = dec_attr.run([] {
+      return cudaFuncSetAttribute(attend_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    });
+    if (e != cudaSuccess) return e;
     // A unit cut into a few parts is merged by the CTA that finishes its last part (no further launch); when a
     // launch has few units and therefore many parts per unit (one layer at a time), the merge kernel's
     // parallelism is worth its launch.
@@ -690,10 +748,11 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     if (p.per == ncf && (size_t)(layer1 - layer0) * s.Hkv * n_split * 2 > c->part_units) n_split = 0;
     p.n_split = n_split;
   }
-  const size_t smem = 2 * Q_TILE_BYTES + (size_t)KV_BUFS * 2 * p.Npad * 128 + 8 * (2 * KV_BUFS + 6) + 16 + 1024;
-  if (smem > 227 * 1024) return cudaErrorInvalidValue;
-  static bool attr_set = false;
-  if (!attr_set) {
+  const size_t smem = 2 * Q_TILE_BYTES + (size_t)KV_BUFS * TILE_BYTES + 8 * (2 * KV_BUFS + 6) + 16 + 1024;
+  static_assert(2 * Q_TILE_BYTES + KV_BUFS * TILE_BYTES + 8 * (2 * KV_BUFS + 6) + 16 + 1024 <= 227 * 1024,
+                "shared-memory plan of the attention kernel");
+  static PerDeviceOnce attr;
+  cudaError_t ea = attr.run([] {
     cudaError_t e = cudaFuncSetAttribute(attend_tc5_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(attend_tc5_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
@@ -701,9 +760,9 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
       e = cudaFuncSetAttribute(attend_tc5_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(attend_tc5_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+    return e;
+  });
+  if (ea != cudaSuccess) return ea;
   if (timed) cudaEventRecord(c->ev_t0, st);
   auto kernel = full ? (p.n_split > 0 ? attend_tc5_kernel<true, true> : attend_tc5_kernel<true, false>)
                      : (p.n_split > 0 ? attend_tc5_kernel<false, true> : attend_tc5_kernel<false, false>);

@@ -415,16 +415,12 @@ template <int V4>
 cudaError_t launch_score_v4(bool pdl, cudaStream_t st, size_t smem, int nl, int n_scored, const float* reps, const float* qa,
                             const float* qsq, int nQ, int maxQ, int Dp, int Hkv, int max_frames, int q_group, float* scores,
                             int block, int layer0) {
-  static int sms = 0;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(score_kernel<V4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-    if (e != cudaSuccess) return e;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    attr_set = true;
-  }
+  static PerDeviceOnce attr;
+  cudaError_t ea = attr.run([] {
+    return cudaFuncSetAttribute(score_kernel<V4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+  });
+  if (ea != cudaSuccess) return ea;
+  const int sms = rekv_sm_count();
   int occ = 1;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, score_kernel<V4>, 256, smem) != cudaSuccess || occ < 1) occ = 1;
   int per_layer = (sms * occ) / nl;
@@ -499,12 +495,11 @@ cudaError_t rekv_launch_retrieve_external(rekv_ctx* c, const float* q_emb, int n
   const int n_scored = b == 1 ? n_visible : geom.n_items;
   int q_group = (int)((96 * 1024) / (E * sizeof(float)));
   if (q_group > nQ) q_group = nQ;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(ext_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceOnce attr;
+  cudaError_t ea = attr.run([] {
+    return cudaFuncSetAttribute(ext_score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+  });
+  if (ea != cudaSuccess) return ea;
   if (n_scored > 0) {
     ext_score_kernel<<<(n_scored + 7) / 8, 256, (size_t)q_group * E * sizeof(float), st>>>(c->ext_emb, q_emb, nQ, E, n_scored,
                                                                                          b, q_group, tau, scores);

@@ -99,9 +99,7 @@ int attend_one_layer(rekv_ctx* c, int layer, const void* q, const QBatch& qb, vo
     REKV_CUDA(c, cudaMemsetAsync(out, 0, (size_t)(qb.sumNq * row_bytes), st));
     return REKV_OK;
   }
-  const bool legacy = (c->cfg.flags & REKV_FLAG_ATTEND_LEGACY_MMA) != 0;
-  auto launch = legacy ? rekv_launch_attend_mma : rekv_launch_attend_tc5;
-  REKV_CUDA(c, launch(c, layer_view(q, layer, qb.sumNq * row_bytes), qb, c->g_ncf, layer, layer + 1,
+  REKV_CUDA(c, rekv_launch_attend_tc5(c, layer_view(q, layer, qb.sumNq * row_bytes), qb, c->g_ncf, layer, layer + 1,
                       layer_view(out, layer, qb.sumNq * row_bytes), st, false, nullptr));
   if (s.tail > 0) {
     // later appends (ring slots) and gathers (staging) on the side stream must not overtake this read
@@ -180,6 +178,8 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   c->k_rot = nullptr;
   c->tbl_k = nullptr;
   c->rope_positions = 0;
+  c->test_wait_limit = 0;
+  c->test_skip_copy_entry = -1;
 
   StoreView& s = c->sv;
   s.L = cfg->n_layers;
@@ -421,8 +421,7 @@ int rekv_attend(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, void* o
     REKV_CUDA(c, cudaMemsetAsync(out, 0, (size_t)s.L * qb.sumNq * s.Hq * REKV_HEAD_DIM * 2, st));
     return REKV_OK;
   }
-  const bool legacy = (c->cfg.flags & REKV_FLAG_ATTEND_LEGACY_MMA) != 0;
-  auto launch = legacy ? rekv_launch_attend_mma : rekv_launch_attend_tc5;
+  auto launch = rekv_launch_attend_tc5;
   if (!c->gather_layerwise) {
     REKV_CUDA(c, launch(c, q, qb, c->g_ncf, 0, s.L, out, st, (c->cfg.flags & REKV_FLAG_TIMING) != 0, nullptr));
   } else {
@@ -577,8 +576,6 @@ int rekv_attend_full(rekv_ctx* c, const void* q, const void* k_self, const void*
   if (!c) return REKV_ERR_ARG;
   if (!q || !k_self || !v_self || !out) REKV_FAIL(c, REKV_ERR_ARG, "null q, k_self, v_self or out");
   if (c->cfg.max_self_tokens <= 0) REKV_FAIL(c, REKV_ERR_STATE, "the context was created with max_self_tokens == 0");
-  if (c->cfg.flags & REKV_FLAG_ATTEND_LEGACY_MMA)
-    REKV_FAIL(c, REKV_ERR_STATE, "rekv_attend_full runs on the tcgen05 attention kernel only");
   if (!c->gathered) REKV_FAIL(c, REKV_ERR_STATE, "rekv_attend_full needs a preceding rekv_gather");
   if (nQ != c->g_nQ) REKV_FAIL(c, REKV_ERR_STATE, "nQ=%d differs from the gathered batch (%d)", nQ, c->g_nQ);
   QBatch qb, sb;
@@ -618,6 +615,18 @@ int rekv_attend_full(rekv_ctx* c, const void* q, const void* k_self, const void*
   return REKV_OK;
 }
 
+int rekv_geometry(rekv_ctx* c, int n_visible, int top_k, int32_t* n_scored, int32_t* k_eff, int32_t* w_eff) {
+  if (!c) return REKV_ERR_ARG;
+  if (n_visible < 0 || top_k < 0) REKV_FAIL(c, REKV_ERR_ARG, "n_visible and top_k must be >= 0");
+  if (top_k % c->cfg.block_frames)
+    REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d must be a multiple of block_frames=%d", top_k, c->cfg.block_frames);
+  const CtxGeom g = rekv_geom(n_visible, c->cfg.window_frames, c->cfg.block_frames, top_k);
+  if (n_scored) *n_scored = c->cfg.block_frames == 1 ? n_visible : g.n_items;
+  if (k_eff) *k_eff = g.k_eff;
+  if (w_eff) *w_eff = g.w_eff;
+  return REKV_OK;
+}
+
 int rekv_stats(rekv_ctx* c, rekv_stats_t* out) {
   if (!c || !out) return REKV_ERR_ARG;
   DeviceGuard guard(c->device);
@@ -653,6 +662,13 @@ int rekv_set_timing(rekv_ctx* c, int enable) {
     c->cfg.flags &= ~(uint32_t)REKV_FLAG_TIMING;
     c->timing_valid = false;
   }
+  return REKV_OK;
+}
+
+int rekv_test_set_wait_limit(rekv_ctx* c, unsigned iterations, int skip_copy_entry) {
+  if (!c) return REKV_ERR_ARG;
+  c->test_wait_limit = iterations;
+  c->test_skip_copy_entry = skip_copy_entry;
   return REKV_OK;
 }
 

@@ -128,6 +128,10 @@ struct rekv_ctx {
   char** tbl_k;                     // [L][max_questions][ctx frames]
   int ctx_frames_max;
 
+  // test-only knobs of the bounded device-side waits (rekv_test_set_wait_limit); 0 / -1 = off
+  unsigned test_wait_limit;
+  int test_skip_copy_entry;
+
   // state of the last gather
   bool gathered;
   bool gather_layerwise;            // layer events are pending (offloaded context)
@@ -151,6 +155,37 @@ struct rekv_ctx {
   } while (0)
 
 void rekv_set_error(rekv_ctx* ctx, const char* msg);
+
+// Launch state that belongs to one device: a function attribute (the dynamic shared-memory limit) is set on the
+// function of the CURRENT device only, so "already set" is kept per device ordinal, and the SM count is asked of
+// each device once.  A context created on a second device of the same process gets its own settings.
+constexpr int REKV_MAX_DEVICES = 64;
+struct PerDeviceOnce {
+  bool done[REKV_MAX_DEVICES] = {};
+  // runs set() unless it has succeeded before on the current device
+  template <typename F>
+  cudaError_t run(F&& set) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const bool known = dev >= 0 && dev < REKV_MAX_DEVICES;
+    if (known && done[dev]) return cudaSuccess;
+    e = set();
+    if (e == cudaSuccess && known) done[dev] = true;
+    return e;
+  }
+};
+inline int rekv_sm_count() {  // of the current device
+  static int sms[REKV_MAX_DEVICES] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+  const bool known = dev >= 0 && dev < REKV_MAX_DEVICES;
+  if (known && sms[dev] > 0) return sms[dev];
+  int n = 0;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 1;
+  if (known) sms[dev] = n;
+  return n;
+}
 
 // Launch with programmatic stream serialization: the kernel may begin (its prologue up to
 // grid_dep_wait()) while the previous kernel of the stream is still draining.
@@ -193,9 +228,6 @@ cudaError_t rekv_launch_dequant_page(rekv_ctx* c, const char* host_page, char* d
 cudaError_t rekv_launch_page_table(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, const CtxGeom& geom,
                                    int n_visible, int layer0, int layer1, int frames_now, cudaStream_t st);
 cudaError_t rekv_launch_materialize(rekv_ctx* c, int nQ, int ncf, void* k_ctx, void* v_ctx, cudaStream_t st);
-// k_attend_mma.cu
-cudaError_t rekv_launch_attend_mma(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
-                                   void* out, cudaStream_t st, bool timed, const AttendFullArgs* full = nullptr);
 // k_attend_tc5.cu
 cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb, int ncf, int layer0, int layer1,
                                    void* out, cudaStream_t st, bool timed, const AttendFullArgs* full = nullptr);

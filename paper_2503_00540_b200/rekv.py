@@ -15,7 +15,6 @@ import torch
 from . import _build
 
 OK, ERR_ARG, ERR_FULL, ERR_EMPTY, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT, ERR_STATE = 0, -1, -2, -3, -4, -5, -6, -7
-FLAG_ATTEND_LEGACY_MMA = 1 << 1
 FLAG_TIMING = 1 << 2
 FLAG_HOST_FP8 = 1 << 3
 
@@ -45,7 +44,8 @@ EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", 
            "rekv_stats", "rekv_check_status", "rekv_last_error", "rekv_get_reps", "rekv_get_page",
            "rekv_launch_count", "rekv_score_frames_static", "rekv_question_layer", "rekv_attend_layer", "rekv_attend_full",
            "rekv_set_frame_embedding", "rekv_retrieve_external", "rekv_question",
-           "rekv_save", "rekv_load", "rekv_set_timing")
+           "rekv_save", "rekv_load", "rekv_set_timing", "rekv_geometry",
+           "rekv_test_set_wait_limit")
 
 _lib = None
 
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.rekv_stats.argtypes = [vp, ctypes.POINTER(rekv_stats_t)]
         L.rekv_check_status.argtypes = [vp, vp]
         L.rekv_set_timing.argtypes = [vp, i32]
+        L.rekv_test_set_wait_limit.argtypes = [vp, ctypes.c_uint, i32]
+        L.rekv_geometry.argtypes = [vp, i32, i32, ip, ip, ip]
         L.rekv_last_error.argtypes = [vp]
         L.rekv_last_error.restype = ctypes.c_char_p
         L.rekv_get_reps.argtypes = [vp, i32, i32, vp, vp]
@@ -146,11 +148,11 @@ class ReKV:
         return self
 
     def geometry(self, n_visible: int, top_k: int) -> Tuple[int, int, int]:
-        """(retrieval candidates, frames retrieved, trailing frames always in the context) -- the sizes the
-        library uses for its outputs (include/rekv.h, rekv_retrieve / rekv_gather)."""
-        n_items = max(n_visible - self.W, 0) // self.b
-        k_eff = min(top_k // self.b, n_items) * self.b
-        return n_items, k_eff, n_visible - n_items * self.b
+        """(items scored per question, frames retrieved, trailing frames always in the context) as
+        rekv_geometry reports them: the sizes of what retrieve and gather write."""
+        n, k, w = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+        self._check(lib().rekv_geometry(self._h, n_visible, top_k, ctypes.byref(n), ctypes.byref(k), ctypes.byref(w)))
+        return n.value, k.value, w.value
 
     # ------------------------------------------------------------------ plumbing
     def _check(self, rc: int) -> int:
@@ -188,7 +190,7 @@ class ReKV:
         if tuple(q.shape) != (self.L, cu_q[-1], self.Hq, self.D):
             raise ValueError("q must be [L][sum_Nq][H_q][D]")
         idx = torch.empty((self.L, nQ, max(top_k, 0)), dtype=torch.int32, device=self.device)
-        n_scored = n_visible if self.b == 1 else self.geometry(n_visible, top_k)[0]
+        n_scored = self.geometry(n_visible, top_k)[0]
         scores = (torch.empty((self.L, nQ, n_scored), dtype=torch.float32, device=self.device)
                   if want_scores and n_visible > 0 else None)
         k_eff = self._check(lib().rekv_retrieve(self._h, _ptr(q, torch.bfloat16), _cu_array(cu_q), nQ, top_k,
@@ -246,7 +248,7 @@ class ReKV:
         layer; k_eff; scores float32 [nQ][n_scored] or None)."""
         nQ = q_emb.shape[0]
         idx = torch.empty((self.L, nQ, max(top_k, 0)), dtype=torch.int32, device=self.device)
-        n_scored = n_visible if self.b == 1 else self.geometry(n_visible, top_k)[0]
+        n_scored = self.geometry(n_visible, top_k)[0]
         scores = (torch.empty((nQ, n_scored), dtype=torch.float32, device=self.device)
                   if want_scores and n_visible > 0 else None)
         k_eff = self._check(lib().rekv_retrieve_external(self._h, _ptr(q_emb, torch.float32), nQ, top_k, n_visible,
@@ -308,6 +310,10 @@ class ReKV:
         """Event records around the attention kernel on or off for the calls that follow (see rekv_set_timing)."""
         self._check(lib().rekv_set_timing(self._h, 1 if enable else 0))
 
+    def test_set_wait_limit(self, iterations: int, skip_copy_entry: int = -1) -> None:
+        """Test-only: shortens the kernels' bounded waits and makes one tile copy go missing (rekv_test_set_wait_limit)."""
+        self._check(lib().rekv_test_set_wait_limit(self._h, iterations, skip_copy_entry))
+
     def launch_count(self) -> int:
         return int(lib().rekv_launch_count(self._h))
 
@@ -321,12 +327,6 @@ class ReKV:
         v = torch.empty_like(k)
         self._check(lib().rekv_get_page(self._h, frame, layer, _ptr(k), _ptr(v), self._stream()))
         return k, v
-
-
-def kv_cache_bytes(n_layers: int, n_frames: int, tokens_per_frame: int, n_kv_heads: int, head_dim: int,
-                   bytes_per_element: int = 2) -> int:
-    """K/V bytes of a stream: 2 * L * T * M * H * D * bytes (the paper's cache-size expression)."""
-    return 2 * n_layers * n_frames * tokens_per_frame * n_kv_heads * head_dim * bytes_per_element
 
 
 def score_frames_static(q: torch.Tensor, cu_q: Sequence[int], n_kv_heads: int, reps: torch.Tensor,

