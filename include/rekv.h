@@ -147,7 +147,9 @@ int rekv_retrieve(rekv_ctx* ctx, const void* q, const int32_t* cu_q, int nQ, int
  * rekv_check_status as REKV_ERR_ARG).  Builds the context of every (layer, question):
  * the selected frames in list order, then frames max(n_visible - W, 0) .. n_visible-1.  Pages that
  * live only in pinned host memory are pulled over the host link into an HBM staging area (on an
- * internal stream, layer by layer).  rekv_attend reads this context.
+ * internal stream, layer by layer); on an offloaded context the frames still in the HBM tail are
+ * copied there too, so the context keeps its bytes when later appends recycle the tail's slots
+ * (an append enqueued after the gather waits for those copies).  rekv_attend reads this context.
  *   k_ctx, v_ctx (nullable, both or neither): device bf16 [L][nQ][H_kv][(k_eff+W')*N_f][D] with
  *   W' = min(W, n_visible); when given, the context is also written out contiguously, token rows
  *   in context order -- a bit-exact copy of the stored K/V.
@@ -218,7 +220,10 @@ int rekv_question(rekv_ctx* ctx, const void* q, const int32_t* cu_q, int nQ, int
  * allocated and the host is not synchronised; on a context whose cache is all in HBM the call may be
  * captured into a CUDA graph (one graph per layer, replayed while the stored frames, n_visible and the
  * buffers stay the same); an offloaded context uses the internal side stream and must not be captured.
- * The context built for the layer stays valid for rekv_attend_layer until the next gather of that layer.
+ * The context built for the layer stays valid for rekv_attend_layer until the next gather of that layer, or
+ * until a gather of ANY layer with another number of questions or context frames (top_k, n_visible): all
+ * layers share one context table, whose layout follows those counts; rekv_attend_layer, rekv_attend and
+ * rekv_attend_full then return REKV_ERR_STATE for the layers that were not gathered again.
  * Returns the number of context frames, or a negative error code. */
 int rekv_question_layer(rekv_ctx* ctx, int layer, const void* q, const int32_t* cu_q, int nQ, int top_k, int n_visible,
                         int32_t* idx_out, void* out, void* stream);

@@ -131,23 +131,26 @@ __global__ void __launch_bounds__(256) page_table_pull_kernel(StoreView s, const
   }
   const long long slot = ((long long)l * nQ + qi) * ncf + j;
   char* page;
-  bool pull = false;
+  bool pull = false, from_ring = false;
   if (s.tail == 0) {
     page = s.hbm + rekv_hbm_page_offset(s, frame, l);
-  } else if (frame >= frames_now - s.tail) {
-    page = s.hbm + rekv_hbm_page_offset(s, frame, l);
   } else {
+    // Offloaded context: the context owns its bytes.  A frame that is still in the HBM ring is copied into the
+    // staging page as well (HBM to HBM), because the ring slot is recycled by a later append while the context --
+    // decode steps reuse it -- must stay what it was at gather time.
     page = s.staging + slot * s.page_bytes;
     pull = true;
+    from_ring = frame >= frames_now - s.tail;
   }
   if (threadIdx.x == 0 && part == 0) {
     tbl[slot] = page;
-    if (pull) atomicAdd(link_bytes, (unsigned long long)s.host_page_bytes);
+    if (pull && !from_ring) atomicAdd(link_bytes, (unsigned long long)s.host_page_bytes);
   }
   if (!pull) return;
-  const char* src = s.host_arenas[frame / s.frames_per_arena] +
-                    ((long long)(frame % s.frames_per_arena) * s.L + l) * s.host_page_bytes;
-  if (s.host_fp8) {  // codes and scales cross the link; the staging page receives bf16
+  const char* src = from_ring ? s.hbm + rekv_hbm_page_offset(s, frame, l)
+                              : s.host_arenas[frame / s.frames_per_arena] +
+                                    ((long long)(frame % s.frames_per_arena) * s.L + l) * s.host_page_bytes;
+  if (s.host_fp8 && !from_ring) {  // codes and scales cross the link; the staging page receives bf16
     __shared__ float s_scale[DEQ_MAX_ROWS];
     const long long g16 = (long long)s.Hkv * 2 * s.Nf * 8;
     const long long gper = ((g16 + parts - 1) / parts + 7) & ~7ll;  // whole rows per part

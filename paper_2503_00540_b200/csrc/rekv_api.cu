@@ -161,6 +161,8 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   c->ev_t0 = c->ev_t1 = nullptr;
   c->timing_valid = false;
   c->d2h_pending = false;
+  c->ring_reader_ev = nullptr;
+  c->layer_ctx_valid.assign(cfg->n_layers, 0);
   c->gathered = false;
   c->gather_layerwise = false;
   memset(&c->sv, 0, sizeof(c->sv));
@@ -318,6 +320,11 @@ int rekv_append_frame(rekv_ctx* c, const void* k, const void* v, void* stream) {
     // the ring slot is reused: its previous occupant's write-through must have left HBM
     const int slot = f % s.tail;
     if (c->slot_event_valid[slot]) REKV_CUDA(c, cudaStreamWaitEvent(st, c->slot_events[slot], 0));
+    // ... and a gather that is still copying ring pages into its context (side stream) must have read them
+    if (c->ring_reader_ev) {
+      REKV_CUDA(c, cudaStreamWaitEvent(st, c->ring_reader_ev, 0));
+      c->ring_reader_ev = nullptr;
+    }
   }
   REKV_CUDA(c, rekv_launch_append(c, k, v, f, st));
   if (s.tail > 0) {
@@ -391,9 +398,11 @@ int rekv_gather(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, int n_visibl
       REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, geom, n_visible, l, l + 1, c->frames, c->side));
       REKV_CUDA(c, cudaEventRecord(c->layer_events[l], c->side));
     }
+    c->ring_reader_ev = c->layer_events[s.L - 1];
     c->gather_layerwise = true;
   }
   c->gathered = true;
+  c->layer_ctx_valid.assign(s.L, 1);
   c->g_nQ = nQ;
   c->g_ncf = ncf;
   c->g_keff = k_eff;
@@ -410,6 +419,9 @@ int rekv_attend(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, void* o
   if (!c) return REKV_ERR_ARG;
   if (!q || !out) REKV_FAIL(c, REKV_ERR_ARG, "null q or out");
   if (!c->gathered) REKV_FAIL(c, REKV_ERR_STATE, "rekv_attend needs a preceding rekv_gather");
+  for (int l = 0; l < c->sv.L; ++l)
+    if (!c->layer_ctx_valid[l])
+      REKV_FAIL(c, REKV_ERR_STATE, "layer %d has no context with the geometry of the latest gather", l);
   if (nQ != c->g_nQ) REKV_FAIL(c, REKV_ERR_STATE, "nQ=%d differs from the gathered batch (%d)", nQ, c->g_nQ);
   QBatch qb;
   int rc = build_qbatch(c, cu_q, nQ, &qb);
@@ -464,6 +476,7 @@ int rekv_question(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, int t
   const CtxGeom geom = rekv_geom(n_visible, c->cfg.window_frames, c->cfg.block_frames, top_k);
   REKV_CUDA(c, rekv_launch_retrieve(c, q, qb, top_k, geom, n_visible, 0, s.L, idx, c->scores, st, true));
   c->gathered = true;
+  c->layer_ctx_valid.assign(s.L, 1);
   c->gather_layerwise = false;
   c->g_nQ = nQ;
   c->g_ncf = geom.ncf;
@@ -507,8 +520,13 @@ int rekv_question_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu
     REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_main, 0));
     REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, geom, n_visible, layer, layer + 1, c->frames, c->side));
     REKV_CUDA(c, cudaEventRecord(c->layer_events[layer], c->side));
+    c->ring_reader_ev = c->layer_events[layer];
     REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[layer], 0));
   }
+  // the table's row pitch follows (nQ, context frames): a layer call with another geometry re-lays it out, and the
+  // contexts the other layers built under the old one are gone
+  if (!c->gathered || c->g_nQ != nQ || c->g_ncf != geom.ncf) c->layer_ctx_valid.assign(s.L, 0);
+  c->layer_ctx_valid[layer] = 1;
   c->gathered = true;
   c->gather_layerwise = s.tail > 0;
   c->g_nQ = nQ;
@@ -524,7 +542,9 @@ int rekv_attend_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu_q
   if (!c) return REKV_ERR_ARG;
   if (!q || !out) REKV_FAIL(c, REKV_ERR_ARG, "null q or out");
   if (layer < 0 || layer >= c->sv.L) REKV_FAIL(c, REKV_ERR_ARG, "layer=%d outside [0, %d)", layer, c->sv.L);
-  if (!c->gathered) REKV_FAIL(c, REKV_ERR_STATE, "rekv_attend_layer needs a preceding gather of the layer");
+  if (!c->gathered || !c->layer_ctx_valid[layer])
+    REKV_FAIL(c, REKV_ERR_STATE, "rekv_attend_layer needs a preceding gather of the layer (with the geometry of the "
+                                 "latest gather: a layer call with other question or frame counts re-lays the table out)");
   if (nQ != c->g_nQ) REKV_FAIL(c, REKV_ERR_STATE, "nQ=%d differs from the gathered batch (%d)", nQ, c->g_nQ);
   QBatch qb;
   int rc = build_qbatch(c, cu_q, nQ, &qb);
@@ -577,6 +597,9 @@ int rekv_attend_full(rekv_ctx* c, const void* q, const void* k_self, const void*
   if (!q || !k_self || !v_self || !out) REKV_FAIL(c, REKV_ERR_ARG, "null q, k_self, v_self or out");
   if (c->cfg.max_self_tokens <= 0) REKV_FAIL(c, REKV_ERR_STATE, "the context was created with max_self_tokens == 0");
   if (!c->gathered) REKV_FAIL(c, REKV_ERR_STATE, "rekv_attend_full needs a preceding rekv_gather");
+  for (int l = 0; l < c->sv.L; ++l)
+    if (!c->layer_ctx_valid[l])
+      REKV_FAIL(c, REKV_ERR_STATE, "layer %d has no context with the geometry of the latest gather", l);
   if (nQ != c->g_nQ) REKV_FAIL(c, REKV_ERR_STATE, "nQ=%d differs from the gathered batch (%d)", nQ, c->g_nQ);
   QBatch qb, sb;
   int rc = build_qbatch(c, cu_q, nQ, &qb);

@@ -98,6 +98,8 @@ struct rekv_ctx {
   cudaEvent_t ev_side;              // side stream -> caller stream fence
   std::vector<cudaEvent_t> layer_events;  // per layer: its host-tier gather finished
   bool d2h_pending;
+  cudaEvent_t ring_reader_ev;       // offloaded: the last gather on the side stream, which reads ring pages; the next
+                                    // append (it recycles a ring slot on the caller's stream) waits for it once
   cudaEvent_t ev_t0, ev_t1;         // REKV_FLAG_TIMING: around the attention kernel
   bool timing_valid;
 
@@ -132,7 +134,9 @@ struct rekv_ctx {
   unsigned test_wait_limit;
   int test_skip_copy_entry;
 
-  // state of the last gather
+  // state of the last gather.  The context table has one geometry (questions x context frames) for all layers; a
+  // layer's context is valid while the table still has the geometry it was built with (layer_ctx_valid).
+  std::vector<char> layer_ctx_valid;
   bool gathered;
   bool gather_layerwise;            // layer events are pending (offloaded context)
   int g_nQ, g_ncf, g_keff, g_nvis, g_topk;

@@ -167,3 +167,29 @@ def test_all_layer_question_replayed_from_one_cuda_graph():
     g.check_status()
     assert torch.equal(out, eager2)
     g.close()
+
+
+def test_a_layer_context_built_under_another_geometry_is_refused():
+    """All layers share one context table laid out by (questions, context frames).  A layer gathered with fewer
+    visible frames (a shorter context) re-lays it out: the other layers' contexts are gone, and using them must fail
+    with REKV_ERR_STATE instead of attending over the wrong pages; gathering the layer again makes it usable."""
+    s = H.Shape(L=2, Hq=8, Hkv=2, Nf=16, T=20, W=4, k=8, seed=7)
+    g = H.build_gpu(s, max_q_tokens=16)
+    o = H.build_oracle(s)
+    q, cu = H.questions(s, [16], device="cuda")
+    ref = o.question(q.cpu(), s.k, s.T)
+    out0 = g.question_layer(0, q[0], cu, s.k, s.T)
+    g.question_layer(1, q[1], cu, s.k, 6)      # 2 candidates + 4 window frames: 6 context frames instead of 12
+    g.check_status()
+    with pytest.raises(rekv.RekvError) as e:
+        g.attend_layer(0, q[0], cu)
+    assert e.value.code == rekv.ERR_STATE
+    with pytest.raises(rekv.RekvError) as e:
+        g.attend(q, cu)
+    assert e.value.code == rekv.ERR_STATE
+    g.attend_layer(1, q[1], cu)                # the layer gathered last is fine
+    out0b = g.question_layer(0, q[0], cu, s.k, s.T)
+    g.check_status()
+    assert torch.equal(out0, out0b)
+    H.assert_attention(out0b[None], ref["out"][0:1], "layer 0 gathered again")
+    g.close()

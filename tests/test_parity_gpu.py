@@ -208,3 +208,29 @@ def test_host_tier_pages_survive_the_round_trip():
             vr = synth.frame(s.seed, synth.V, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale)[l].permute(1, 0, 2)
             assert torch.equal(k.cpu(), kr) and torch.equal(v.cpu(), vr), (f, l)
     g.close()
+
+
+def test_offloaded_context_keeps_its_frames_when_appends_recycle_the_hbm_tail():
+    """A context gathered on an offloaded stream references frames that were in the HBM tail at gather time (the
+    window always is).  The stream keeps growing while the answer is decoded: `tail` appends after the gather recycle
+    every ring slot.  The attention -- all layers, then one layer again as a decode step would -- must still see the
+    frames of gather time."""
+    s = H.Shape(L=2, Hq=8, Hkv=2, Nf=48, T=34, W=3, k=6, tail=5, seed=540)
+    n0 = s.T - s.tail                      # frames when the question is asked
+    g = H.build_gpu(s, max_q_tokens=16, n_frames=n0)
+    o = H.build_oracle(s, n_frames=n0)
+    q, cu = H.questions(s, [16], device="cuda")
+    ref = o.question(q.cpu(), s.k, n0)
+    idx_ref = ref["idx"][:, None].contiguous().cuda()
+    g.gather(idx_ref, 1, s.k, n0)
+    for f in range(n0, s.T):               # the stream goes on: every ring slot gets a new frame
+        k = synth.frame(s.seed, synth.K, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale, device="cuda")
+        v = synth.frame(s.seed, synth.V, f, s.L, s.Nf, s.Hkv, s.D, s.off_scale, device="cuda")
+        assert g.append_frame(k, v) == f
+    out = g.attend(q, cu)
+    g.check_status()
+    H.assert_attention(out, ref["out"], "attention after the tail was recycled")
+    out_l = g.attend_layer(1, q[1].contiguous(), cu)
+    g.check_status()
+    assert torch.equal(out_l, out[1])
+    g.close()
