@@ -398,12 +398,16 @@ def run_cuda(args, w):
     # attention-kernel duration (library-internal events on the launching stream) and bytes over the host link
     # (the event records stand between the attention kernel and its neighbours, so they are on only here)
     att_us, link_bytes = [], 0
+    stage_us = {"retrieve": [], "pull": [], "merge": []}
     g.set_timing(True)
     for i in range(min(K, 8)):
         ask(qs[i % N_ROTATE], g.stats().frames, out)
         torch.cuda.synchronize()
         st = g.stats()
         att_us.append(st.last_attend_kernel_us)
+        stage_us["retrieve"].append(st.last_retrieve_us)
+        stage_us["pull"].append(st.last_pull_us)
+        stage_us["merge"].append(st.last_merge_us)
         link_bytes = st.last_link_bytes
     g.set_timing(False)
 
@@ -580,6 +584,9 @@ def run_cuda(args, w):
                                                           / (retrieve_us * 1e-6)),
                          "questions_per_s_all_gpus": world * 1e6 / q_lat},
             "append_us": app_us,
+            # the library's own stage timings of a question (rekv_stats with the event records on; each record stands
+            # between two kernels, so the stages add up to a little more than the untimed question)
+            "stages_us": {k: (sum(v) / len(v) if v else None) for k, v in stage_us.items()},
             "e2e": {"value": e2e_lat, "unit": "us",
                     "h2d_bytes_per_step": dq.numel() * 2,
                     "d2h_bytes_per_step": out.numel() * 2,

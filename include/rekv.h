@@ -103,6 +103,12 @@ typedef struct {
   int32_t last_ctx_frames;   /* k_eff + window frames of the last gather */
   double last_attend_kernel_us; /* device time of the last attention kernel launch (REKV_FLAG_TIMING, HBM
                                    tier), without the split-KV merge; 0 when not measured */
+  double last_retrieve_us;      /* REKV_FLAG_TIMING: steps 2-3 of the last question (question vectors, scores,
+                                   selection) on the caller's stream; 0 when not measured or not finished yet */
+  double last_pull_us;          /* REKV_FLAG_TIMING, offloaded contexts: the last gather's pulls over the host
+                                   link, all layers, on the internal stream; 0 when not measured or not finished */
+  double last_merge_us;         /* REKV_FLAG_TIMING: the merge kernel that followed the last attention kernel
+                                   (units cut at CTA boundaries, half-streams); 0 when none ran or not measured */
 } rekv_stats_t;
 
 /* Creates a context on cfg->device: allocates the frame store (HBM tier, and the pinned-host tier
@@ -252,7 +258,9 @@ int rekv_load(const char* path, int device, rekv_ctx** out);
  * top_k that is not a multiple of block_frames. */
 int rekv_geometry(rekv_ctx* ctx, int n_visible, int top_k, int32_t* n_scored, int32_t* k_eff, int32_t* w_eff);
 
-/* Fills *out with store accounting and the last call's counters. */
+/* Fills *out with store accounting and the last call's counters.  Never waits for the device: the byte counter
+ * of the host link and the stage timings describe work that has COMPLETED (synchronise the stream first for the
+ * figures of the call just enqueued); a stage whose events have not completed yet reads 0. */
 int rekv_stats(rekv_ctx* ctx, rekv_stats_t* out);
 
 /* Switches REKV_FLAG_TIMING on (enable != 0) or off for the calls that follow.  The two event records around

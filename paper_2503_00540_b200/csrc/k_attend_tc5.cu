@@ -731,12 +731,17 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     if (timed) {
       cudaEventRecord(c->ev_t1, st);
       c->timing_valid = true;
+      c->merge_timed = false;
     }
     c->launches += 1;
     if (p.per != ncf && !p.unit_cnt) {
       cudaError_t e2 = rekv_launch_pdl(combine_tc5_kernel, dim3((unsigned)units, 2, 32), dim3(128), 0, st, p);
       if (e2 != cudaSuccess) return e2;
       c->launches += 1;
+      if (timed) {
+        cudaEventRecord(c->ev_t2, st);
+        c->merge_timed = true;
+      }
     }
     return cudaGetLastError();
   }
@@ -771,12 +776,17 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   if (timed) {
     cudaEventRecord(c->ev_t1, st);
     c->timing_valid = true;
+    c->merge_timed = false;
   }
   c->launches += 1;
   if (p.per != ncf || p.n_split > 0) {
     cudaError_t e2 = rekv_launch_pdl(combine_tc5_kernel, dim3((unsigned)units, 2, 32), dim3(128), 0, st, p);
     if (e2 != cudaSuccess) return e2;
     c->launches += 1;
+    if (timed) {
+      cudaEventRecord(c->ev_t2, st);
+      c->merge_timed = true;
+    }
   }
   return cudaGetLastError();
 }

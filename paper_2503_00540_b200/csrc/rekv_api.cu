@@ -79,8 +79,9 @@ void free_ctx(rekv_ctx* c) {
   for (cudaEvent_t e : c->layer_events) cudaEventDestroy(e);
   if (c->ev_main) cudaEventDestroy(c->ev_main);
   if (c->ev_side) cudaEventDestroy(c->ev_side);
-  if (c->ev_t0) cudaEventDestroy(c->ev_t0);
-  if (c->ev_t1) cudaEventDestroy(c->ev_t1);
+  for (cudaEvent_t e : {c->ev_t0, c->ev_t1, c->ev_t2, c->ev_r0, c->ev_r1, c->ev_p0, c->ev_p1})
+    if (e) cudaEventDestroy(e);
+  if (c->h_link_bytes) cudaFreeHost(c->h_link_bytes);
   if (c->side) cudaStreamDestroy(c->side);
   delete c;
 }
@@ -158,8 +159,9 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   c->d_host_arenas = nullptr;
   c->side = nullptr;
   c->ev_main = c->ev_side = nullptr;
-  c->ev_t0 = c->ev_t1 = nullptr;
-  c->timing_valid = false;
+  c->ev_t0 = c->ev_t1 = c->ev_t2 = c->ev_r0 = c->ev_r1 = c->ev_p0 = c->ev_p1 = nullptr;
+  c->timing_valid = c->merge_timed = c->retrieve_timed = c->pull_timed = false;
+  c->h_link_bytes = nullptr;
   c->d2h_pending = false;
   c->ring_reader_ev = nullptr;
   c->layer_ctx_valid.assign(cfg->n_layers, 0);
@@ -259,8 +261,10 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
   CREATE_CUDA(cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking), "creating the side stream");
   CREATE_CUDA(cudaEventCreateWithFlags(&c->ev_main, cudaEventDisableTiming), "creating events");
   CREATE_CUDA(cudaEventCreateWithFlags(&c->ev_side, cudaEventDisableTiming), "creating events");
-  CREATE_CUDA(cudaEventCreate(&c->ev_t0), "creating events");
-  CREATE_CUDA(cudaEventCreate(&c->ev_t1), "creating events");
+  for (cudaEvent_t* e : {&c->ev_t0, &c->ev_t1, &c->ev_t2, &c->ev_r0, &c->ev_r1, &c->ev_p0, &c->ev_p1})
+    CREATE_CUDA(cudaEventCreate(e), "creating events");
+  CREATE_CUDA(cudaHostAlloc((void**)&c->h_link_bytes, sizeof(unsigned long long), cudaHostAllocDefault), "allocating counters");
+  *c->h_link_bytes = 0;
 
   if (s.tail > 0) {
     // pinned-host tier: arenas of whole frames, allocated up front so that append never blocks
@@ -363,8 +367,12 @@ int rekv_retrieve(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, int t
     REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d must be a multiple of block_frames=%d", top_k, c->cfg.block_frames);
   DeviceGuard guard(c->device);
   const CtxGeom geom = rekv_geom(n_visible, c->cfg.window_frames, c->cfg.block_frames, top_k);
+  const bool timed = (c->cfg.flags & REKV_FLAG_TIMING) != 0;
+  if (timed) REKV_CUDA(c, cudaEventRecord(c->ev_r0, (cudaStream_t)stream));
   REKV_CUDA(c, rekv_launch_retrieve(c, q, qb, top_k, geom, n_visible, 0, c->sv.L, idx_out, scores_out ? scores_out : c->scores,
                                     (cudaStream_t)stream));
+  if (timed) REKV_CUDA(c, cudaEventRecord(c->ev_r1, (cudaStream_t)stream));
+  c->retrieve_timed = timed;
   return geom.k_eff;
 }
 
@@ -388,16 +396,24 @@ int rekv_gather(rekv_ctx* c, const int32_t* idx, int nQ, int top_k, int n_visibl
   if (s.tail == 0) {
     REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, geom, n_visible, 0, s.L, c->frames, st));
     c->gather_layerwise = false;
+    c->pull_timed = false;
+    *c->h_link_bytes = 0;
   } else {
     // host tier: the pulls run layer by layer on the side stream (behind every write-through that is
     // still in flight there); attention of layer l only waits for layer l's event
     REKV_CUDA(c, cudaMemsetAsync(c->link_bytes, 0, sizeof(unsigned long long), st));
     REKV_CUDA(c, cudaEventRecord(c->ev_main, st));
     REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_main, 0));
+    const bool timed = (c->cfg.flags & REKV_FLAG_TIMING) != 0;
+    if (timed) REKV_CUDA(c, cudaEventRecord(c->ev_p0, c->side));
     for (int l = 0; l < s.L; ++l) {
       REKV_CUDA(c, rekv_launch_page_table(c, idx, nQ, top_k, geom, n_visible, l, l + 1, c->frames, c->side));
       REKV_CUDA(c, cudaEventRecord(c->layer_events[l], c->side));
     }
+    if (timed) REKV_CUDA(c, cudaEventRecord(c->ev_p1, c->side));
+    c->pull_timed = timed;
+    // the bytes that crossed the link, mirrored to pinned host memory behind the pulls (rekv_stats reads the mirror)
+    REKV_CUDA(c, cudaMemcpyAsync(c->h_link_bytes, c->link_bytes, sizeof(unsigned long long), cudaMemcpyDeviceToHost, c->side));
     c->ring_reader_ev = c->layer_events[s.L - 1];
     c->gather_layerwise = true;
   }
@@ -474,7 +490,12 @@ int rekv_question(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, int t
   DeviceGuard guard(c->device);
   cudaStream_t st = (cudaStream_t)stream;
   const CtxGeom geom = rekv_geom(n_visible, c->cfg.window_frames, c->cfg.block_frames, top_k);
+  const bool timed = (c->cfg.flags & REKV_FLAG_TIMING) != 0;
+  if (timed) REKV_CUDA(c, cudaEventRecord(c->ev_r0, st));
   REKV_CUDA(c, rekv_launch_retrieve(c, q, qb, top_k, geom, n_visible, 0, s.L, idx, c->scores, st, true));
+  if (timed) REKV_CUDA(c, cudaEventRecord(c->ev_r1, st));
+  c->retrieve_timed = timed;
+  c->pull_timed = false;
   c->gathered = true;
   c->layer_ctx_valid.assign(s.L, 1);
   c->gather_layerwise = false;
@@ -663,15 +684,20 @@ int rekv_stats(rekv_ctx* c, rekv_stats_t* out) {
   out->kv_bytes_host = s.tail > 0 ? (long long)c->frames * s.host_page_bytes * s.L : 0;
   out->kv_bytes_logical = 2ll * s.L * c->frames * s.Nf * s.Hkv * REKV_HEAD_DIM * 2;
   out->rep_bytes = (long long)s.L * c->frames * s.Dp * (long long)sizeof(float);
-  unsigned long long lb = 0;
-  REKV_CUDA(c, cudaDeviceSynchronize());
-  REKV_CUDA(c, cudaMemcpy(&lb, c->link_bytes, sizeof(lb), cudaMemcpyDeviceToHost));
-  out->last_link_bytes = (int64_t)lb;
-  if (c->timing_valid) {
+  // nothing here waits for the device: counters and timings are those of the work that has completed
+  out->last_link_bytes = (int64_t)*c->h_link_bytes;
+  auto elapsed_us = [](cudaEvent_t a, cudaEvent_t b) -> double {
     float ms = 0.f;
-    if (cudaEventElapsedTime(&ms, c->ev_t0, c->ev_t1) == cudaSuccess) out->last_attend_kernel_us = 1e3 * ms;
-    cudaGetLastError();
-  }
+    if (cudaEventQuery(b) != cudaSuccess || cudaEventElapsedTime(&ms, a, b) != cudaSuccess) {
+      cudaGetLastError();
+      return 0.0;
+    }
+    return 1e3 * ms;
+  };
+  if (c->timing_valid) out->last_attend_kernel_us = elapsed_us(c->ev_t0, c->ev_t1);
+  if (c->timing_valid && c->merge_timed) out->last_merge_us = elapsed_us(c->ev_t1, c->ev_t2);
+  if (c->retrieve_timed) out->last_retrieve_us = elapsed_us(c->ev_r0, c->ev_r1);
+  if (c->pull_timed) out->last_pull_us = elapsed_us(c->ev_p0, c->ev_p1);
   out->last_k_eff = c->gathered ? c->g_keff : 0;
   out->last_ctx_frames = c->gathered ? c->g_ncf : 0;
   return REKV_OK;
@@ -683,7 +709,7 @@ int rekv_set_timing(rekv_ctx* c, int enable) {
     c->cfg.flags |= REKV_FLAG_TIMING;
   } else {
     c->cfg.flags &= ~(uint32_t)REKV_FLAG_TIMING;
-    c->timing_valid = false;
+    c->timing_valid = c->merge_timed = c->retrieve_timed = c->pull_timed = false;
   }
   return REKV_OK;
 }

@@ -100,8 +100,12 @@ struct rekv_ctx {
   bool d2h_pending;
   cudaEvent_t ring_reader_ev;       // offloaded: the last gather on the side stream, which reads ring pages; the next
                                     // append (it recycles a ring slot on the caller's stream) waits for it once
-  cudaEvent_t ev_t0, ev_t1;         // REKV_FLAG_TIMING: around the attention kernel
-  bool timing_valid;
+  // REKV_FLAG_TIMING: event pairs around the stages of the last question; rekv_stats reads the pairs that have
+  // completed (cudaEventQuery) and never waits.  ev_t0/ev_t1 around the attention kernel, ev_t2 after its merge kernel;
+  // ev_r0/ev_r1 around steps 2-3; ev_p0/ev_p1 (on the side stream) around the host-tier pulls of a gather.
+  cudaEvent_t ev_t0, ev_t1, ev_t2, ev_r0, ev_r1, ev_p0, ev_p1;
+  bool timing_valid, merge_timed, retrieve_timed, pull_timed;
+  unsigned long long* h_link_bytes; // pinned host mirror of link_bytes, refreshed (asynchronously) after each gather
 
   // scratch (device)
   float* qa;                        // [L][max_questions][Dp] fp32 question vectors

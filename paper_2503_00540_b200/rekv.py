@@ -37,7 +37,8 @@ class rekv_stats_t(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in (
         "frames", "kv_bytes_hbm", "kv_bytes_host", "kv_bytes_logical", "rep_bytes", "page_bytes",
         "last_link_bytes")] + [("last_k_eff", ctypes.c_int32), ("last_ctx_frames", ctypes.c_int32),
-                                       ("last_attend_kernel_us", ctypes.c_double)]
+                                       ("last_attend_kernel_us", ctypes.c_double), ("last_retrieve_us", ctypes.c_double),
+                                       ("last_pull_us", ctypes.c_double), ("last_merge_us", ctypes.c_double)]
 
 
 EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", "rekv_gather", "rekv_attend",

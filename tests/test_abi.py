@@ -35,7 +35,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_config_struct_matches_header_layout():
     assert ctypes.sizeof(rekv.rekv_config) == 17 * 4
-    assert ctypes.sizeof(rekv.rekv_stats_t) == 7 * 8 + 2 * 4 + 8
+    assert ctypes.sizeof(rekv.rekv_stats_t) == 7 * 8 + 2 * 4 + 4 * 8  # seven counters, two ints, four stage timings
 
 
 def test_create_rejects_bad_shapes_before_touching_a_device():

@@ -200,6 +200,7 @@ def _offloaded(s: H.Shape, q_tokens: int, layers, need_gb: float):
     assert st.kv_bytes_host == st.kv_bytes_logical == orc.kv_cache_bytes(s.L, s.T, s.Nf, s.Hkv, s.D)
     assert st.kv_bytes_hbm == st.kv_bytes_logical * s.tail // s.T
     worst = _sampled_parity(g, s, [q_tokens], layers=layers, n_visible=s.T)
+    g.check_status()
     st = g.stats()
     # every selected frame outside the HBM tail crossed the host link exactly once
     assert 0 < st.last_link_bytes <= s.L * s.k * st.page_bytes

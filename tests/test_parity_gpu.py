@@ -115,11 +115,14 @@ def test_timing_switch_reports_the_kernel_and_leaves_results_alone():
     g.set_timing(True)
     out_timed = g.question(q, cu, s.k, s.T).clone()
     torch.cuda.synchronize()
-    assert g.stats().last_attend_kernel_us > 0.0
+    st = g.stats()
+    assert st.last_attend_kernel_us > 0.0 and st.last_retrieve_us > 0.0 and st.last_merge_us > 0.0
+    assert st.last_pull_us == 0.0  # nothing crosses the host link on a cache that is all in HBM
     g.set_timing(False)
     out_again = g.question(q, cu, s.k, s.T).clone()
     torch.cuda.synchronize()
-    assert g.stats().last_attend_kernel_us == 0.0
+    st = g.stats()
+    assert st.last_attend_kernel_us == 0.0 and st.last_retrieve_us == 0.0 and st.last_merge_us == 0.0
     assert torch.equal(out_plain, out_timed) and torch.equal(out_plain, out_again)
     g.check_status()
     g.close()
@@ -233,4 +236,19 @@ def test_offloaded_context_keeps_its_frames_when_appends_recycle_the_hbm_tail():
     out_l = g.attend_layer(1, q[1].contiguous(), cu)
     g.check_status()
     assert torch.equal(out_l, out[1])
+    g.close()
+
+
+def test_stats_report_the_pull_stage_of_an_offloaded_question_without_waiting():
+    """rekv_stats never synchronises: right after the call is enqueued the pull stage may read 0; once the streams
+    have drained it reports the host-link bytes and the duration of the pulls."""
+    s = H.Shape(L=3, Hq=8, Hkv=2, Nf=48, T=30, W=3, k=6, tail=5, seed=7)
+    g = H.build_gpu(s, max_q_tokens=16, flags=rekv.FLAG_TIMING)
+    q, cu = H.questions(s, [16], device="cuda")
+    g.question(q, cu, s.k, s.T)
+    g.stats()                      # must return at once, whatever it reads
+    g.check_status()               # drains the caller's and the library's streams
+    st = g.stats()
+    assert st.last_pull_us > 0.0 and st.last_retrieve_us > 0.0
+    assert 0 < st.last_link_bytes <= s.L * s.k * st.page_bytes
     g.close()
