@@ -27,6 +27,7 @@ struct TcParams {
   // producer of CTA 0 leaves out so that a wait runs out with nothing in flight
   unsigned wait_limit;
   int skip_copy_entry;
+  long long part_slots;   // capacity of part_o / part_ml in 128-row partial slots (checks build)
   int per;          // (unit, frame) steps per CTA
   // A unit with one row tile has no second tile to overlap with; it is run as two half-streams on the two tile
   // slots instead -- the same rows, the frame's token chunks dealt alternately -- whose (max, sum, O) partials the

@@ -10,7 +10,9 @@ namespace {
 __global__ void __launch_bounds__(256) append_pool_kernel(const uint4* __restrict__ k_in,
                                                           const uint4* __restrict__ v_in, char* __restrict__ page0,
                                                           float* __restrict__ reps, int frame, int L, int Hkv,
-                                                          int Nf, int max_frames, long long page_bytes) {
+                                                          int Nf, int max_frames, long long page_bytes,
+                                                          long long store_bytes, char* __restrict__ store,
+                                                          int* __restrict__ status) {
   const int kv = blockIdx.x & 1;
   const int h = (blockIdx.x >> 1) % Hkv;
   const int l = (blockIdx.x >> 1) / Hkv;
@@ -36,7 +38,11 @@ __global__ void __launch_bounds__(256) append_pool_kernel(const uint4* __restric
     for (int u = 0; u < 4; ++u) {
       const int t = t0 + 16 * u;
       if (t < Nf) {
-        *reinterpret_cast<uint4*>(tile + t * 128 + ((cc ^ (t & 7)) << 4)) = x[u];
+        char* dst = tile + t * 128 + ((cc ^ (t & 7)) << 4);
+        if (!REKV_CHECK(dst >= store && dst + 16 <= store + store_bytes && (reinterpret_cast<uintptr_t>(dst) & 15) == 0,
+                        status, 1))
+          continue;
+        *reinterpret_cast<uint4*>(dst) = x[u];
         if (kv == 0) {
           const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&x[u]);
 #pragma unroll
@@ -58,7 +64,8 @@ __global__ void __launch_bounds__(256) append_pool_kernel(const uint4* __restric
       float s = 0.f;
 #pragma unroll
       for (int r = 0; r < 16; ++r) s += red[r][threadIdx.x];
-      reps[((long long)l * max_frames + frame) * (Hkv * 128) + h * 128 + threadIdx.x] = __fdiv_rn(s, (float)Nf);
+      if (REKV_CHECK(frame >= 0 && frame < max_frames && l < L, status, 2))
+        reps[((long long)l * max_frames + frame) * (Hkv * 128) + h * 128 + threadIdx.x] = __fdiv_rn(s, (float)Nf);
     }
   }
 }
@@ -86,7 +93,9 @@ cudaError_t rekv_launch_append(rekv_ctx* c, const void* k, const void* v, int fr
   const StoreView& s = c->sv;
   char* page0 = s.hbm + rekv_hbm_page_offset(s, frame, 0);
   append_pool_kernel<<<s.L * s.Hkv * 2, 256, 0, st>>>((const uint4*)k, (const uint4*)v, page0, s.reps, frame, s.L,
-                                                      s.Hkv, s.Nf, s.max_frames, s.page_bytes);
+                                                      s.Hkv, s.Nf, s.max_frames, s.page_bytes,
+                                                      (long long)(s.tail > 0 ? s.tail : s.max_frames) * s.L * s.page_bytes,
+                                                      s.hbm, c->status);
   c->launches += 1;
   return cudaGetLastError();
 }

@@ -252,6 +252,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
               if (FULL && kv == 0 && pages_k) src = pages_k[fi] + (long long)ui.g * 2 * page_half_bytes;  // rotated K tiles
               const uint32_t d = dst + (uint32_t)(fi * p.Ns + ta - row0) * 128u;
               const uint32_t nb = (uint32_t)(tb - ta) * 128u;
+              // (checks build) a piece must lie inside its ring tile half and start on 16 bytes at both ends; a piece
+              // that does not is left out, and the wait for the tile then runs out and reports it
+              if (!REKV_CHECK(pages[fi] != nullptr && (reinterpret_cast<uintptr_t>(src) & 15) == 0 && d >= dst &&
+                                  d + nb <= dst + HALF_BYTES && fi * p.Ns + ta - row0 >= 0,
+                              p.status, 31))
+                continue;
               bulk_g2s(d, src + (long long)ta * 128, nb, bars.full(b));
               bulk_g2s(d + HALF_BYTES, src + page_half_bytes + (long long)ta * 128, nb, bars.full(b));
             }
@@ -583,10 +589,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
               __syncwarp();
             }
           } else {
-            const long long slot = (p.per == p.ncf ? (long long)ui.srank : (long long)blockIdx.x + u) * 2 + t;
+            const long long slot_raw = (p.per == p.ncf ? (long long)ui.srank : (long long)blockIdx.x + u) * 2 + t;
+            const bool slot_ok = REKV_CHECK(slot_raw >= 0 && slot_raw < p.part_slots, p.status, 32);  // (checks build)
+            const long long slot = slot_ok ? slot_raw : 0;
             // rows this lane stores: r = 4 k + (lane >> 3), 16 bytes (4 floats) at chunk (lane & 7) of the quarter
             float* po = p.part_o + ((slot * 128 + ((warp & 3) << 5) + (lane >> 3)) * 128 + (lane & 7) * 4);
-            const int nrows_w = ui.rows_q - rr0;  // valid rows of this warp (may exceed 32)
+            const int nrows_w = slot_ok ? ui.rows_q - rr0 : 0;  // valid rows of this warp (may exceed 32)
 #pragma unroll 1
             for (int qd = 0; qd < 4; ++qd) {
               uint32_t o[2][16];
@@ -612,7 +620,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
               }
               __syncwarp();
             }
-            if (valid) {
+            if (valid && slot_ok) {
               p.part_ml[(slot * 128 + row) * 2] = m_used;
               p.part_ml[(slot * 128 + row) * 2 + 1] = l_sum;
             }
@@ -687,6 +695,7 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   p.Ns = (s.Nf + 7) & ~7;
   p.wait_limit = c->test_wait_limit;
   p.skip_copy_entry = c->test_skip_copy_entry;
+  p.part_slots = (long long)c->part_units * 2;
   p.ncf = ncf;
   p.layer0 = layer0;
   p.n_split = 0;

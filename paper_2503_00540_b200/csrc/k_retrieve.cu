@@ -71,7 +71,7 @@ template <int SCORE_MAX_V4>
 __global__ void __launch_bounds__(256, SCORE_MAX_V4 <= 4 ? 4 : 2)
     score_kernel(const float* __restrict__ reps, const float* __restrict__ qa, const float* __restrict__ qsq, int nQ,
                  int maxQ, int Dp, int Hkv, int max_frames, int n_visible, int q_group, float* __restrict__ scores,
-                 int block, int layer0, int fpc) {
+                 int block, int layer0, int fpc, int* __restrict__ status) {
   extern __shared__ float4 s_q[];  // [q_group][Dp/4]
   __shared__ float s_qn[REKV_MAX_QUESTIONS];
   rekv_ptx::grid_dep_wait();
@@ -97,6 +97,7 @@ __global__ void __launch_bounds__(256, SCORE_MAX_V4 <= 4 ? 4 : 2)
     // two frames per iteration: twice the loads in flight per warp
     for (int f = f0 + warp * 2; f < f1; f += 16) {
       const bool two = f + 1 < f1;
+      if (!REKV_CHECK((long long)(f + (two ? 2 : 1)) * block <= max_frames && f >= 0, status, 11)) continue;
       const float4* row0 = reinterpret_cast<const float4*>(reps + ((long long)l * max_frames + (long long)f * block) * Dp);
       const float4* row1 = row0 + (two ? (long long)block * (Dp / 4) : 0);
       float4 r0[SCORE_MAX_V4], r1[SCORE_MAX_V4];
@@ -201,7 +202,7 @@ __device__ __forceinline__ void topk_write_table(const TopkTable& t, const int32
 
 __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ scores, int nQ, int n_visible,
                                                    int n_cand, int top_k, int k_eff, int32_t* __restrict__ idx_out,
-                                                   int block, int layer0, TopkTable tt) {
+                                                   int block, int layer0, TopkTable tt, int* __restrict__ status) {
   const int qi = blockIdx.x, l = layer0 + blockIdx.y;
   const float* s = scores + ((long long)l * nQ + qi) * n_visible;
   int32_t* out = idx_out + ((long long)l * nQ + qi) * top_k;
@@ -304,7 +305,7 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
     int pos = -1;
     if (gt) pos = rank_gt + min(rank_eq, need_eq);
     if (eq && rank_eq < need_eq) pos = rank_gt + rank_eq;
-    if (pos >= 0)
+    if (pos >= 0 && REKV_CHECK(pos < k_eff && i < n_cand, status, 21))
       for (int j = 0; j < block; ++j) out[pos * block + j] = i * block + j;
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -414,7 +415,7 @@ __global__ void replicate_idx_kernel(int32_t* __restrict__ idx, int per_layer, i
 template <int V4>
 cudaError_t launch_score_v4(bool pdl, cudaStream_t st, size_t smem, int nl, int n_scored, const float* reps, const float* qa,
                             const float* qsq, int nQ, int maxQ, int Dp, int Hkv, int max_frames, int q_group, float* scores,
-                            int block, int layer0) {
+                            int block, int layer0, int* status) {
   static PerDeviceOnce attr;
   cudaError_t ea = attr.run([] {
     return cudaFuncSetAttribute(score_kernel<V4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
@@ -430,18 +431,18 @@ cudaError_t launch_score_v4(bool pdl, cudaStream_t st, size_t smem, int nl, int 
   dim3 grid((n_scored + fpc - 1) / fpc, nl);
   if (pdl)
     return rekv_launch_pdl(score_kernel<V4>, grid, dim3(256), smem, st, reps, qa, qsq, nQ, maxQ, Dp, Hkv, max_frames,
-                           n_scored, q_group, scores, block, layer0, fpc);
+                           n_scored, q_group, scores, block, layer0, fpc, status);
   score_kernel<V4><<<grid, 256, smem, st>>>(reps, qa, qsq, nQ, maxQ, Dp, Hkv, max_frames, n_scored, q_group, scores, block,
-                                            layer0, fpc);
+                                            layer0, fpc, status);
   return cudaGetLastError();
 }
 cudaError_t launch_score(bool pdl, cudaStream_t st, size_t smem, int nl, int n_scored, const float* reps, const float* qa,
                          const float* qsq, int nQ, int maxQ, int Dp, int Hkv, int max_frames, int q_group, float* scores,
-                         int block, int layer0) {
+                         int block, int layer0, int* status) {
   return Dp <= 512 ? launch_score_v4<4>(pdl, st, smem, nl, n_scored, reps, qa, qsq, nQ, maxQ, Dp, Hkv, max_frames, q_group,
-                                        scores, block, layer0)
+                                        scores, block, layer0, status)
                    : launch_score_v4<8>(pdl, st, smem, nl, n_scored, reps, qa, qsq, nQ, maxQ, Dp, Hkv, max_frames, q_group,
-                                        scores, block, layer0);
+                                        scores, block, layer0, status);
 }
 
 }  // namespace
@@ -465,7 +466,7 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
   const int n_scored = b == 1 ? n_visible : geom.n_items;
   if (n_scored > 0) {
     cudaError_t e1 = launch_score(true, st, smem, nl, n_scored, s.reps, c->qa, c->qnorm, qb.nQ, maxQ, s.Dp, s.Hkv,
-                                  s.max_frames, q_group, scores, b, layer0);
+                                  s.max_frames, q_group, scores, b, layer0, c->status);
     if (e1 != cudaSuccess) return e1;
     c->launches += 1;
   }
@@ -480,7 +481,7 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
       tt.n_vis_frames = n_visible;
     }
     cudaError_t e2 = rekv_launch_pdl(topk_kernel, dim3(qb.nQ, nl), dim3(512), 0, st, scores, qb.nQ, n_scored,
-                                     geom.n_items, top_k, geom.k_items, idx_out, b, layer0, tt);
+                                     geom.n_items, top_k, geom.k_items, idx_out, b, layer0, tt, c->status);
     if (e2 != cudaSuccess) return e2;
     c->launches += 1;
   }
@@ -507,7 +508,7 @@ cudaError_t rekv_launch_retrieve_external(rekv_ctx* c, const float* q_emb, int n
   }
   if (top_k > 0) {
     cudaError_t e2 = rekv_launch_pdl(topk_kernel, dim3(nQ, 1), dim3(512), 0, st, (const float*)scores, nQ, n_scored,
-                                     geom.n_items, top_k, geom.k_items, idx_out, b, 0, TopkTable{});
+                                     geom.n_items, top_k, geom.k_items, idx_out, b, 0, TopkTable{}, c->status);
     if (e2 != cudaSuccess) return e2;
     const int per_layer = nQ * top_k;
     if (s.L > 1) {
@@ -613,7 +614,7 @@ extern "C" int rekv_score_frames_static(const void* q, const int32_t* cu_q, int 
   int q_group = (int)((96 * 1024) / (Dp * sizeof(float)));
   if (q_group > nQ) q_group = nQ;
   e = launch_score(false, st, (size_t)q_group * Dp * sizeof(float), 1, n_frames, reps, qa, qsq, nQ, STATIC_MAX_QUESTIONS, Dp,
-                   n_kv_heads, n_frames, q_group, scores_out, 1, 0);
+                   n_kv_heads, n_frames, q_group, scores_out, 1, 0, nullptr);
   if (e != cudaSuccess) {
     rekv_set_error(nullptr, cudaGetErrorString(e));
     return REKV_ERR_CUDA;

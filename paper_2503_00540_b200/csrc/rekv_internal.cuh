@@ -164,6 +164,16 @@ struct rekv_ctx {
 
 void rekv_set_error(rekv_ctx* ctx, const char* msg);
 
+// Checks build (-DREKV_CHECKS): the stand-in for a memory checker on machines where none can run.  Index and address
+// computations of the kernels are tested before use; a violation is recorded in the context's status word as
+// -(2000 + site) -- rekv_check_status then fails with that code -- and the access is skipped.  Nothing traps or faults.
+// In the shipped build the tests compile to nothing.
+#ifdef REKV_CHECKS
+#define REKV_CHECK(cond, status, site) ((cond) ? true : ((status) ? (atomicExch((status), -(2000 + (site))), false) : false))
+#else
+#define REKV_CHECK(cond, status, site) (true)
+#endif
+
 // Launch state that belongs to one device: a function attribute (the dynamic shared-memory limit) is set on the
 // function of the CURRENT device only, so "already set" is kept per device ordinal, and the SM count is asked of
 // each device once.  A context created on a second device of the same process gets its own settings.

@@ -7,6 +7,7 @@ There is no CPU fallback: loading fails loudly if the shared library is missing 
 built, and creating a context fails without a CUDA device.
 """
 import ctypes
+import os
 from dataclasses import dataclass
 from typing import Optional, Sequence, Tuple
 
@@ -55,7 +56,11 @@ def lib() -> ctypes.CDLL:
     """Loads (building in-tree if stale) librekv.so.  Raises if that is impossible."""
     global _lib
     if _lib is None:
-        path = _build.build_librekv()
+        # REKV_CHECKS=1 in the environment selects the self-checking build of the same sources (test runs only)
+        # REKV_SANITIZE=1 selects the build whose host code runs under AddressSanitizer/UBSan (the process must have
+        # the sanitizer runtime preloaded)
+        path = _build.build_librekv(checks=os.environ.get("REKV_CHECKS", "") == "1",
+                                    sanitize=os.environ.get("REKV_SANITIZE", "") == "1")
         L = ctypes.CDLL(path)
         vp, i32, ip = ctypes.c_void_p, ctypes.c_int, ctypes.POINTER(ctypes.c_int32)
         L.rekv_create.argtypes = [ctypes.POINTER(rekv_config), ctypes.POINTER(vp)]
