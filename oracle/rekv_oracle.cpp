@@ -292,7 +292,10 @@ void oracle_rope(const double* x, int head_dim, long pos, double theta, double* 
  * rounded to bf16.  rope_theta == 0: no positional term.  Outputs as oracle_attend. */
 void oracle_attend_full(const uint16_t* q, int n_q, int n_q_heads, int n_kv_heads, int head_dim, const uint16_t* k_ctx,
                         const uint16_t* v_ctx, long n_ctx, const uint16_t* k_self, const uint16_t* v_self, int n_self,
-                        double rope_theta, float* out_f32, uint16_t* out_bf16) {
+                        double rope_theta, int static_ctx, float* out_f32, uint16_t* out_bf16) {
+  /* static_ctx != 0: the static variant named in the "Positional Encoding" paragraph (taken from Inf-LLM): all
+   * retrieved tokens are assigned the same position.  Reading: every context token has position 0 and token s of X
+   * has position 1 + s (X follows the context's single position).  static_ctx == 0: consecutive positions. */
   const int G = n_q_heads / n_kv_heads;
   const double scale = 1.0 / std::sqrt((double)head_dim);
   const long rows = (long)n_q * n_q_heads;
@@ -314,12 +317,12 @@ void oracle_attend_full(const uint16_t* q, int n_q, int n_q_heads, int n_kv_head
     const int x_tok = n_self - n_q + n;        // this row's token index inside X
     const long n_seen = n_ctx + x_tok + 1;     // all of R, then X up to and including itself
     std::vector<double> qd(head_dim), kd(head_dim), logit((size_t)n_seen), acc(head_dim, 0.0);
-    load(q + row * head_dim, n_ctx + x_tok, qd);
+    load(q + row * head_dim, static_ctx ? 1 + x_tok : n_ctx + x_tok, qd);
     double m = -std::numeric_limits<double>::infinity();
     for (long j = 0; j < n_seen; ++j) {
       const uint16_t* kj = j < n_ctx ? k_ctx + ((long)g * n_ctx + j) * head_dim
                                      : k_self + ((j - n_ctx) * n_kv_heads + g) * head_dim;
-      load(kj, j, kd);
+      load(kj, static_ctx ? (j < n_ctx ? 0 : 1 + (j - n_ctx)) : j, kd);
       double s = 0.0;
       for (int d = 0; d < head_dim; ++d) s += qd[d] * kd[d];
       logit[j] = s * scale;

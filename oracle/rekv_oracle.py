@@ -46,7 +46,7 @@ _lib.oracle_fp8_roundtrip.restype = None
 _lib.oracle_rope.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_long, ctypes.c_double, ctypes.c_void_p]
 _lib.oracle_rope.restype = None
 _lib.oracle_attend_full.argtypes = [_u16p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, _u16p, _u16p,
-                                    ctypes.c_long, _u16p, _u16p, ctypes.c_int, ctypes.c_double, ctypes.c_void_p,
+                                    ctypes.c_long, _u16p, _u16p, ctypes.c_int, ctypes.c_double, ctypes.c_int, ctypes.c_void_p,
                                     ctypes.c_void_p]
 _lib.oracle_attend_full.restype = None
 _lib.oracle_kv_cache_bytes.argtypes = [ctypes.c_int, ctypes.c_long, ctypes.c_int, ctypes.c_int, ctypes.c_int,
@@ -208,9 +208,10 @@ def rope(x: torch.Tensor, pos: int, theta: float) -> torch.Tensor:
 
 
 def attend_full(q: torch.Tensor, k_ctx: torch.Tensor, v_ctx: torch.Tensor, k_self: torch.Tensor, v_self: torch.Tensor,
-                rope_theta: float = 0.0):
+                rope_theta: float = 0.0, static_ctx: bool = False):
     """The whole of Eq. 3.  q: bf16 [N_q][H_q][D]; k_ctx, v_ctx: bf16 [H_kv][n_ctx][D] (n_ctx may be 0);
-    k_self, v_self: bf16 [N_self][H_kv][D], N_self >= N_q.  -> (out float32, out bf16) [N_q][H_q][D]."""
+    k_self, v_self: bf16 [N_self][H_kv][D], N_self >= N_q.  -> (out float32, out bf16) [N_q][H_q][D].
+    static_ctx: the static position variant (every context token at position 0, token s of X at 1 + s)."""
     for t in (q, k_ctx, v_ctx, k_self, v_self):
         _chk(t, torch.bfloat16)
     n_q, n_qh, d = q.shape
@@ -220,7 +221,8 @@ def attend_full(q: torch.Tensor, k_ctx: torch.Tensor, v_ctx: torch.Tensor, k_sel
     out = torch.empty(n_q, n_qh, d, dtype=torch.float32)
     out_b = torch.empty(n_q, n_qh, d, dtype=torch.bfloat16)
     _lib.oracle_attend_full(q.data_ptr(), n_q, n_qh, n_kv, d, k_ctx.data_ptr(), v_ctx.data_ptr(), n_ctx,
-                            k_self.data_ptr(), v_self.data_ptr(), n_self, rope_theta, out.data_ptr(), out_b.data_ptr())
+                            k_self.data_ptr(), v_self.data_ptr(), n_self, rope_theta, 1 if static_ctx else 0, out.data_ptr(),
+                            out_b.data_ptr())
     return out, out_b
 
 

@@ -454,7 +454,7 @@ def test_rope_closed_forms():
     assert abs(d1 - d2) < 1e-9
 
 
-def _sdpa_full(q, k_ctx, v_ctx, k_self, v_self, theta):
+def _sdpa_full(q, k_ctx, v_ctx, k_self, v_self, theta, static_ctx=False):
     """torch's scaled_dot_product_attention in fp64 on [R, X] with an explicit mask, GQA by head repetition,
     rotary embedding by the complex-number form, rotated vectors rounded to bf16."""
     n_q, hq, d = q.shape
@@ -474,8 +474,13 @@ def _sdpa_full(q, k_ctx, v_ctx, k_self, v_self, theta):
     k_all = torch.cat([k_ctx.permute(1, 0, 2), k_self], dim=0)          # [n_ctx + n_self][hkv][d]
     v_all = torch.cat([v_ctx.permute(1, 0, 2), v_self], dim=0).double()
     n_all = n_ctx + n_self
-    pos_k = np.broadcast_to(np.arange(n_all)[:, None], (n_all, hkv))
-    pos_q = np.broadcast_to((n_ctx + n_self - n_q + np.arange(n_q))[:, None], (n_q, hq))
+    if static_ctx:  # every context token at position 0, token s of X at 1 + s
+        pos_1d = np.concatenate([np.zeros(n_ctx, dtype=np.int64), 1 + np.arange(n_self)])
+        pos_q1 = 1 + n_self - n_q + np.arange(n_q)
+    else:
+        pos_1d, pos_q1 = np.arange(n_all), n_ctx + n_self - n_q + np.arange(n_q)
+    pos_k = np.broadcast_to(pos_1d[:, None], (n_all, hkv))
+    pos_q = np.broadcast_to(pos_q1[:, None], (n_q, hq))
     kr, qr = rot(k_all, pos_k), rot(q, pos_q)
     kh = kr.permute(1, 0, 2).repeat_interleave(G, dim=0)                # [hq][n_all][d]
     vh = v_all.permute(1, 0, 2).repeat_interleave(G, dim=0)
@@ -557,3 +562,27 @@ def test_synthetic_inputs_have_the_stated_distribution():
     assert torch.equal(k1[0], synth.frame(2503, synth.K, 0, 2, 196, 4, 128, off_scale=0.5)[1])
     lens = synth.question_lengths(7, 64, 24, 64)
     assert min(lens) >= 24 and max(lens) <= 64 and len(set(lens)) > 10
+
+
+def test_attend_full_static_positions_match_masked_sdpa_and_forget_the_context_order():
+    """The static variant of the "Positional Encoding" paragraph: all retrieved tokens share one position.  Against
+    fp64 SDPA with the complex-number rotation at positions (0, ..., 0, 1, 2, ...); and, unlike consecutive positions,
+    the result must not change when the context tokens are permuted (with consecutive positions it does)."""
+    theta = 1e6
+    for seed, (n_q, n_self, n_ctx) in enumerate([(5, 5, 12), (1, 9, 7), (6, 6, 40)]):
+        q, kc, vc, ks, vs = _full_inputs(100 + seed, n_q, n_self, n_ctx)
+        o, _ = orc.attend_full(q, kc, vc, ks, vs, theta, static_ctx=True)
+        ref = _sdpa_full(q, kc, vc, ks, vs, theta, static_ctx=True)
+        assert (o.double() - ref).abs().max().item() < 2e-6
+        perm = torch.randperm(n_ctx, generator=torch.Generator().manual_seed(seed))
+        o_p, _ = orc.attend_full(q, kc[:, perm].contiguous(), vc[:, perm].contiguous(), ks, vs, theta, static_ctx=True)
+        assert (o - o_p).abs().max().item() < 1e-6
+        o_c, _ = orc.attend_full(q, kc, vc, ks, vs, theta)
+        o_cp, _ = orc.attend_full(q, kc[:, perm].contiguous(), vc[:, perm].contiguous(), ks, vs, theta)
+        assert (o_c - o_cp).abs().max().item() > 1e-3      # consecutive positions do depend on the order
+        assert (o - o_c).abs().max().item() > 1e-3         # and the two variants differ
+    # without a rotation the flag changes nothing
+    q, kc, vc, ks, vs = _full_inputs(7, 4, 6, 9)
+    a, _ = orc.attend_full(q, kc, vc, ks, vs, 0.0, static_ctx=True)
+    b, _ = orc.attend_full(q, kc, vc, ks, vs, 0.0)
+    assert torch.equal(a, b)
