@@ -48,6 +48,10 @@ WORKLOADS = {
     # retrieved tokens at consecutive positions (base 1e6, the paper's Qwen2-based models)
     "7b_hbm_full_eq3_rope": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503,
                                  off_scale=0.5, tail=0, nQ=1, appends_per_step=1, full=True, rope_theta=1e6),
+    # the same with the paragraph's static variant: all context tokens at one position, no rotated copies of the keys
+    "7b_hbm_full_eq3_rope_static": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=64, Nq=32, seed=2503,
+                                        off_scale=0.5, tail=0, nQ=1, appends_per_step=1, full=True, rope_theta=1e6,
+                                        rope_static=True),
     # Eq. 1, one step of stream encoding: the incoming frame's tokens attend the local window (the last W stored
     # frames, nothing retrieved) and themselves causally, then the frame's K/V are appended
     "7b_encode_frame_w8": dict(L=28, Hq=28, Hkv=4, D=128, Nf=196, T=1800, W=8, k=0, Nq=196, seed=2503,
@@ -292,7 +296,7 @@ def run_cuda(args, w):
 
     g = rekv.ReKV(w["L"], w["Hq"], w["Hkv"], w["D"], w["Nf"], w["T"] + 8, w["W"], hbm_tail_frames=w["tail"],
                   max_q_tokens=cu[-1], max_topk=w["k"], max_questions=nQ, device=local,
-                  flags=(rekv.FLAG_HOST_FP8 if w.get("host_fp8") else 0),
+                  flags=(rekv.FLAG_HOST_FP8 if w.get("host_fp8") else 0) | (rekv.FLAG_ROPE_STATIC if w.get("rope_static") else 0),
                   max_self_tokens=cu[-1] if w.get("full") else 0, rope_theta=w.get("rope_theta", 0.0),
                   ext_embed_dim=w.get("ext_dim", 0), block_frames=w.get("b", 1))
     kf = torch.empty((w["L"], w["Nf"], w["Hkv"], w["D"]), dtype=torch.bfloat16, device=dev)

@@ -54,6 +54,11 @@ enum {
 enum {
   REKV_FLAG_TIMING = 1u << 2,                   /* bracket the attention kernel with CUDA events on the caller's
                                                   stream; rekv_stats then reports its duration */
+  REKV_FLAG_ROPE_STATIC = 1u << 4,              /* rekv_attend_full with rope_theta > 0: the static position variant of
+                                                  the "Positional Encoding" paragraph -- every context token gets the
+                                                  same position (0) and token s of X position 1 + s -- instead of
+                                                  consecutive positions.  The stored keys are then used as they are
+                                                  (no rotated copies of the context), only the queries and X rotate */
   REKV_FLAG_HOST_FP8 = 1u << 3                  /* offloaded contexts only: the pinned-host tier holds each page row
                                                   (128 dims of one token of one KV head) as 128 FP8 E4M3 codes and
                                                   one float scale = amax / 448; pages pulled from it come back as

@@ -322,7 +322,10 @@ cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const vo
                                             const QBatch& qb, const QBatch& sb, int ncf, cudaStream_t st) {
   const StoreView& s = c->sv;
   const bool rope = c->cfg.rope_theta > 0.f;
-  const int n_ctx_tokens = ncf * s.Nf;
+  // positions: context token j at j and token s of X at n_ctx + s; with REKV_FLAG_ROPE_STATIC every context token
+  // at 0 -- its rotation is the identity, the stored keys are used as they are -- and token s of X at 1 + s
+  const bool static_ctx = rope && (c->cfg.flags & REKV_FLAG_ROPE_STATIC) != 0;
+  const int n_ctx_tokens = static_ctx ? 1 : ncf * s.Nf;   // position of X's first token
   const __nv_bfloat16* q_eff = (const __nv_bfloat16*)q;
   if (rope) {
     dim3 grid((qb.sumNq * s.Hq + 31) / 32, s.L);
@@ -332,7 +335,7 @@ cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const vo
   }
   // the part over X (latency-bound) runs on the side stream beside the pass over the context's keys
   // (bandwidth-bound); both are joined before the attention kernel
-  const bool fork = rope && ncf > 0;
+  const bool fork = rope && !static_ctx && ncf > 0;
   cudaStream_t st_self = fork ? c->side : st;
   cudaError_t e;
   if (fork) {

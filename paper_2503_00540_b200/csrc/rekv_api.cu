@@ -245,13 +245,16 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
     CREATE_CUDA(cudaMalloc(&c->self_o, rows * 128 * sizeof(float)), "allocating the self-attention partials");
     CREATE_CUDA(cudaMalloc(&c->self_ml, rows * 2 * sizeof(float)), "allocating the self-attention partials");
     if (c->cfg.rope_theta > 0.f) {
-      c->rope_positions = ctx_frames_max * s.Nf + c->cfg.max_self_tokens;
+      const bool static_ctx = (cfg->flags & REKV_FLAG_ROPE_STATIC) != 0;
+      c->rope_positions = (static_ctx ? 1 : ctx_frames_max * s.Nf) + c->cfg.max_self_tokens;
       CREATE_CUDA(cudaMalloc(&c->q_rot, rows * 128 * sizeof(__nv_bfloat16)), "allocating rotated queries");
       CREATE_CUDA(cudaMalloc(&c->rope_tab, (size_t)c->rope_positions * 64 * sizeof(float2)), "allocating the rotary table");
-      CREATE_CUDA(cudaMalloc(&c->k_rot, (size_t)s.L * maxQ * ctx_frames_max * (s.page_bytes / 2)),
-                  "allocating rotated key tiles");
-      CREATE_CUDA(cudaMalloc(&c->tbl_k, (size_t)s.L * maxQ * (ctx_frames_max + 1) * sizeof(char*)),
-                  "allocating the rotated-key table");
+      if (!static_ctx) {
+        CREATE_CUDA(cudaMalloc(&c->k_rot, (size_t)s.L * maxQ * ctx_frames_max * (s.page_bytes / 2)),
+                    "allocating rotated key tiles");
+        CREATE_CUDA(cudaMalloc(&c->tbl_k, (size_t)s.L * maxQ * (ctx_frames_max + 1) * sizeof(char*)),
+                    "allocating the rotated-key table");
+      }
       CREATE_CUDA(rekv_launch_rope_table(c, 0), "building the rotary table");
       CREATE_CUDA(cudaDeviceSynchronize(), "building the rotary table");
     }
@@ -641,7 +644,8 @@ int rekv_attend_full(rekv_ctx* c, const void* q, const void* k_self, const void*
   // an offloaded context: every layer's pages must have arrived before the keys are rotated
   if (c->gather_layerwise) REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[s.L - 1], 0));
   REKV_CUDA(c, rekv_launch_attend_full_prepare(c, q, k_self, v_self, qb, sb, c->g_ncf, st));
-  const bool rope = c->cfg.rope_theta > 0.f;
+  const bool rope = c->cfg.rope_theta > 0.f && !(c->cfg.flags & REKV_FLAG_ROPE_STATIC);  // rotated copies of the context's keys
+  const bool rope_q = c->cfg.rope_theta > 0.f;
   if (c->g_ncf == 0) {
     REKV_CUDA(c, rekv_launch_self_finalize(c, qb, out, st));
   } else {
@@ -649,7 +653,7 @@ int rekv_attend_full(rekv_ctx* c, const void* q, const void* k_self, const void*
     fa.tbl_k = rope ? c->tbl_k : nullptr;
     fa.self_o = c->self_o;
     fa.self_ml = c->self_ml;
-    REKV_CUDA(c, rekv_launch_attend_tc5(c, rope ? (const void*)c->q_rot : q, qb, c->g_ncf, 0, s.L, out, st,
+    REKV_CUDA(c, rekv_launch_attend_tc5(c, rope_q ? (const void*)c->q_rot : q, qb, c->g_ncf, 0, s.L, out, st,
                                         (c->cfg.flags & REKV_FLAG_TIMING) != 0, &fa));
   }
   if (c->gather_layerwise) {

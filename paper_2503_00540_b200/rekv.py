@@ -18,6 +18,7 @@ from . import _build
 OK, ERR_ARG, ERR_FULL, ERR_EMPTY, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT, ERR_STATE = 0, -1, -2, -3, -4, -5, -6, -7
 FLAG_TIMING = 1 << 2
 FLAG_HOST_FP8 = 1 << 3
+FLAG_ROPE_STATIC = 1 << 4
 
 
 class RekvError(RuntimeError):

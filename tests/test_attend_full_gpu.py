@@ -12,12 +12,12 @@ pytestmark = pytest.mark.gpu
 THETAS = [pytest.param(0.0, id="no_rope"), pytest.param(1e6, id="rope_1e6")]
 
 
-def _run(s: H.Shape, nq_lengths, ns_lengths, theta, n_visible=None, top_k=None):
+def _run(s: H.Shape, nq_lengths, ns_lengths, theta, n_visible=None, top_k=None, static_ctx=False):
     n_visible = s.T if n_visible is None else n_visible
     top_k = s.k if top_k is None else top_k
     nQ = len(nq_lengths)
     g = H.build_gpu(s, max_questions=nQ, max_q_tokens=sum(nq_lengths), max_self_tokens=sum(ns_lengths),
-                    rope_theta=theta)
+                    rope_theta=theta, flags=rekv.FLAG_ROPE_STATIC if static_ctx else 0)
     o = H.build_oracle(s)
     q, cu = H.questions(s, nq_lengths, device="cuda")
     ks, vs, cus = H.self_kv(s, ns_lengths, device="cuda")
@@ -33,7 +33,7 @@ def _run(s: H.Shape, nq_lengths, ns_lengths, theta, n_visible=None, top_k=None):
         for l in range(s.L):
             ref, _ = orc.attend_full(q_cpu[l, cu[i]:cu[i + 1]].contiguous(), refs[i]["k_ctx"][l].contiguous(),
                                      refs[i]["v_ctx"][l].contiguous(), ks_cpu[l, cus[i]:cus[i + 1]].contiguous(),
-                                     vs_cpu[l, cus[i]:cus[i + 1]].contiguous(), theta)
+                                     vs_cpu[l, cus[i]:cus[i + 1]].contiguous(), theta, static_ctx=static_ctx)
             H.assert_attention(out[l:l + 1, cu[i]:cu[i + 1]], ref[None], f"Eq. 3 in full, layer {l} question {i}")
             worst = max(worst, (out[l, cu[i]:cu[i + 1]].float().cpu() - ref).abs().max().item())
     # the plain call must differ (the self part matters) unless nothing of X is visible -- never the case
@@ -165,3 +165,11 @@ def test_stream_encoding_step_is_the_same_computation(theta):
                                  kx[l].cpu().contiguous(), vx[l].cpu().contiguous(), theta)
         H.assert_attention(out[l:l + 1], ref[None], f"encode step, layer {l}")
     g.close()
+
+
+def test_static_position_variant():
+    """REKV_FLAG_ROPE_STATIC: every context token at one position (the paragraph's static variant), X after it;
+    prefill over two row tiles with cut units, a mixed batch with generated tokens, and decode steps."""
+    _run(H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=40, W=8, k=12), [32], [32], 1e6, static_ctx=True)
+    _run(H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=30, W=4, k=6, seed=540), [24, 64, 1, 5], [24, 80, 37, 9], 1e6, static_ctx=True)
+    _run(H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=24, W=4, k=8, seed=7), [1, 1], [150, 65], 1e6, static_ctx=True)
