@@ -72,8 +72,10 @@ typedef struct {
   int32_t n_q_heads;         /* H_q; must be a multiple of n_kv_heads */
   int32_t n_kv_heads;        /* H_kv */
   int32_t head_dim;          /* D; must be 128 */
-  int32_t tokens_per_frame;  /* N_f, fixed per context (the paper's M); 1..208 (three K/V head tiles and two
-                                query tiles share one SM's shared memory in the attention kernel) */
+  int32_t tokens_per_frame;  /* N_f, fixed per context (the paper's M); 1..1024.  The attention kernel streams the
+                                context in 128-token chunks whatever N_f is; the load-bound decode kernel needs two
+                                whole frames of a KV head in shared memory and hands frames of more than 224 tokens
+                                to the tensor-core kernel */
   int32_t max_frames;        /* stream capacity; an append past it returns REKV_ERR_FULL */
   int32_t hbm_tail_frames;   /* 0: the whole cache lives in HBM.  n > 0: every page lives in pinned host
                                 memory and only the most recent n frames are also kept in HBM */

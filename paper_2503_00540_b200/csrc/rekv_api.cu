@@ -122,8 +122,8 @@ int rekv_create(const rekv_config* cfg, rekv_ctx** out) {
       cfg->n_q_heads % cfg->n_kv_heads)
     REKV_FAIL(nullptr, REKV_ERR_ARG, "unsupported head counts: %d query / %d kv (kv <= 8, query a multiple of kv)",
               cfg->n_q_heads, cfg->n_kv_heads);
-  if (cfg->tokens_per_frame < 1 || cfg->tokens_per_frame > 208)
-    REKV_FAIL(nullptr, REKV_ERR_ARG, "tokens_per_frame=%d outside [1, 208]", cfg->tokens_per_frame);
+  if (cfg->tokens_per_frame < 1 || cfg->tokens_per_frame > 1024)
+    REKV_FAIL(nullptr, REKV_ERR_ARG, "tokens_per_frame=%d outside [1, 1024]", cfg->tokens_per_frame);
   if (cfg->max_frames < 1) REKV_FAIL(nullptr, REKV_ERR_ARG, "max_frames must be positive");
   if (cfg->block_frames < 1 || cfg->block_frames > 64)
     REKV_FAIL(nullptr, REKV_ERR_ARG, "block_frames=%d outside [1, 64]", cfg->block_frames);

@@ -43,7 +43,7 @@ def test_create_rejects_bad_shapes_before_touching_a_device():
         (dict(head_dim=64), "head_dim"),
         (dict(n_q_heads=7), "head counts"),
         (dict(tokens_per_frame=0), "tokens_per_frame"),
-        (dict(tokens_per_frame=209), "tokens_per_frame"),
+        (dict(tokens_per_frame=1025), "tokens_per_frame"),
         (dict(block_frames=0), "block_frames"),
         (dict(block_frames=3, max_topk=64), "multiple of block_frames"),
         (dict(hbm_tail_frames=2, window_frames=4), "window_frames"),

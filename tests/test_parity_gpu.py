@@ -252,3 +252,13 @@ def test_stats_report_the_pull_stage_of_an_offloaded_question_without_waiting():
     assert st.last_pull_us > 0.0 and st.last_retrieve_us > 0.0
     assert 0 < st.last_link_bytes <= s.L * s.k * st.page_bytes
     g.close()
+
+
+@pytest.mark.parametrize("nf", [224, 256, 400, 1000])
+def test_frames_longer_than_a_chunk_or_two(nf):
+    """Tokens per frame beyond the 128-token chunk of the attention kernel and beyond what the decode kernel can hold:
+    several chunks per frame, frame boundaries at any place of a chunk; a 2-token question takes the decode-shaped
+    path (or its fallback), a 19-token one the tensor-core path."""
+    s = H.Shape(L=2, Hq=8, Hkv=2, Nf=nf, T=9, W=2, k=3, seed=7)
+    _run_question_parity(s, [19, 2])
+    _run_question_parity(s, [2])
