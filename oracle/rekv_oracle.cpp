@@ -155,8 +155,8 @@ void oracle_score_external(const float* q, const float* embs, int dim, int n_ite
   }
 }
 
-/* Step 2, block variant (Eq. 2 paragraph: "group b consecutive frames into blocks by averaging their frame
- * vectors").  Block j averages the representatives of frames [j*b, (j+1)*b); only complete blocks exist.
+/* Step 2, block variant (Eq. 2 paragraph: b consecutive frames form a block whose vector is the average of the
+ * frames' vectors).  Block j averages the representatives of frames [j*b, (j+1)*b); only complete blocks exist.
  * scores[j] = cosine(question vector, block vector), tau = 1.  The block mean is kept in double. */
 void oracle_score_blocks(const uint16_t* q, int n_q, int n_q_heads, int n_kv_heads, int head_dim, const float* reps,
                          int n_blocks, int b, float* scores) {
