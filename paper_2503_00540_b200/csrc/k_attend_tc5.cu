@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   // ---- one-time set-up -------------------------------------------------------------------------
   if (tid == 0) {
     for (int i = 0; i < KV_BUFS; ++i) {
-      mbar_init(bars.full(i), 1);
+      mbar_init(bars.full(i), 2);   // the copies' byte count (with its arrival) and the producer's zeroed rows
       mbar_init(bars.empty(i), 1);
     }
     for (int t = 0; t < 2; ++t) {
@@ -222,26 +222,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
             break;
           }
           const uint32_t dst = s_kv + b * TILE_BYTES;
-          {  // rows without a token
-            int x = pos0 + lane;
-            for (int rr = lane; rr < N; rr += 32, x += 32) {
-              if (p.Ns >= CHUNK) {
-                if (x >= p.Ns) x -= p.Ns;
-              } else {
-                x %= p.Ns;
-              }
-              if (rr >= nrows || x >= p.Nf) {
-                unsigned char* row_ptr = smem + (dst - s_base) + rr * 128;
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                  *reinterpret_cast<uint4*>(row_ptr + c * 16) = make_uint4(0, 0, 0, 0);
-                  *reinterpret_cast<uint4*>(row_ptr + HALF_BYTES + c * 16) = make_uint4(0, 0, 0, 0);
-                }
-              }
-            }
-            fence_proxy_async();
-            __syncwarp();
-          }
+          // copies first: nothing stands between the slot becoming free and its next tile being on its way
           const bool skip = p.skip_copy_entry >= 0 && blockIdx.x == 0 && (int)r == p.skip_copy_entry;  // test-only
           if (elect_one() && !skip) {
             mbar_expect_tx(bars.full(b), bytes);
@@ -261,6 +242,29 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
               bulk_g2s(d, src + (long long)ta * 128, nb, bars.full(b));
               bulk_g2s(d + HALF_BYTES, src + page_half_bytes + (long long)ta * 128, nb, bars.full(b));
             }
+          }
+          {  // then the rows without a token (the copies do not touch them); the tile's second arrival follows them
+            int x = pos0 + lane;
+            // (no such row in a chunk that lies inside one frame's tokens and is full)
+            const bool all_covered = nrows == N && pos0 + nrows <= p.Nf;
+            for (int rr = all_covered ? N : lane; rr < N; rr += 32, x += 32) {
+              if (p.Ns >= CHUNK) {
+                if (x >= p.Ns) x -= p.Ns;
+              } else {
+                x %= p.Ns;
+              }
+              if (rr >= nrows || x >= p.Nf) {
+                unsigned char* row_ptr = smem + (dst - s_base) + rr * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                  *reinterpret_cast<uint4*>(row_ptr + c * 16) = make_uint4(0, 0, 0, 0);
+                  *reinterpret_cast<uint4*>(row_ptr + HALF_BYTES + c * 16) = make_uint4(0, 0, 0, 0);
+                }
+              }
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0 && !skip) mbar_arrive(bars.full(b));
           }
           ring_issued = r + 1;
           __syncwarp();
