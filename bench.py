@@ -232,8 +232,14 @@ def run_reference(args, w):
         "impl": "reference", "metric": "question_latency_us", "value": val, "unit": "us", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": val / 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w["name"], "layers": w["L"], "frames": w["T"], "tokens_per_frame": w["Nf"],
-                   "q_tokens": w["Nq"], "top_k": w["k"], "window": w["W"]},
+        # the same keys as the CUDA arm's config (the workload is the same; what a CPU run has no use for says so)
+        "config": {"workload": w["name"], "layers": w["L"], "q_heads": w["Hq"], "kv_heads": w["Hkv"],
+                   "frames": w["T"], "tokens_per_frame": w["Nf"], "questions_per_batch": w["nQ"],
+                   "q_tokens": w["Nq"], "top_k": w["k"], "window": w["W"], "hbm_tail_frames": w["tail"],
+                   "cache_gb": 2 * w["L"] * w["T"] * w["Nf"] * w["Hkv"] * w["D"] * 2 / 1e9,
+                   "l2": "not applicable: CPU oracle, inputs regenerated from the seed",
+                   "parallelism": "host cores (OpenMP)",
+                   "step": f"1 question (retrieve, gather, attend) on {Ls} of {w['L']} layers, scaled to all layers"},
         "cpu_baseline": {"value": val, "unit": "us", "cores": cores, "kind": "oracle",
                          "sample": f"steps 2-5 of one question on {Ls} of {w['L']} layers per step, "
                                    f"scaled x{w['L'] // Ls}"},
