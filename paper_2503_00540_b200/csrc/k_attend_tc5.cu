@@ -795,7 +795,8 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   if (p.per != ncf || p.n_split > 0) {
     // units cut at CTA boundaries: a block group per unit; whole units: only those with half-stream partials
     const long long merge_units = p.per != ncf ? units : (long long)(layer1 - layer0) * s.Hkv * p.n_split;
-    cudaError_t e2 = rekv_launch_pdl(combine_tc5_kernel, dim3((unsigned)merge_units, 2, 32), dim3(128), 0, st, p);
+    // (units with half-streams have one row tile)
+    cudaError_t e2 = rekv_launch_pdl(combine_tc5_kernel, dim3((unsigned)merge_units, p.per != ncf ? 2 : 1, 32), dim3(128), 0, st, p);
     if (e2 != cudaSuccess) return e2;
     c->launches += 1;
     if (timed) {
