@@ -15,13 +15,15 @@
 //   warp 0      assembles K/V chunk tiles in a 5-deep shared-memory ring (bulk copies, one lane)
 //   warp 1      tcgen05.mma issue (one lane): S = Q K^T into TMEM, O += P V with P read from TMEM
 //               (warps 2, 3 idle: the service warps form one warpgroup and give their registers up)
-//   warps 4-7   softmax of row tile 0: one thread per row (= TMEM lane), fp32, lazy rescaling of O
+//   warps 4-7   softmax of row tile 0: one thread per row (= TMEM lane), fp32
 //   warps 8-11  softmax of row tile 1 -- the two tiles alternate on the tensor core, so one tile's
 //               softmax overlaps the other's matrix products
 // After set-up the service warpgroup shrinks to 88 registers per thread and the softmax warpgroups grow to
 // 208 (setmaxnreg), so that a softmax thread holds a whole S row chunk (128 values) at once: one TMEM load
-// instruction, one wait, one maximum and one rescaling decision per chunk, and two TMEM stores for P.  Columns
-// without a token are masked piece by piece (16 columns) behind a warp-uniform test of the piece's mask bits.
+// instruction and one wait per chunk, and two TMEM stores for P.  The exponentials take the row maximum of the
+// range's first chunk as their reference; later chunks look for no maximum, and only a row sum beyond 2^60 raises the
+// reference and rescales O (rare).  Columns without a token are masked in the one 16-column piece that has some,
+// behind a warp-uniform switch.
 // TMEM (512 columns): O0 [0,128)  O1 [128,256)  S0/P0 [256,384)  S1/P1 [384,512); P (bf16) overwrites
 // the front of its S.
 // A range that does not cover a whole unit leaves (max, sum, O) partials for the combine kernel.

@@ -262,3 +262,32 @@ def test_frames_longer_than_a_chunk_or_two(nf):
     s = H.Shape(L=2, Hq=8, Hkv=2, Nf=nf, T=9, W=2, k=3, seed=7)
     _run_question_parity(s, [19, 2])
     _run_question_parity(s, [2])
+
+
+@pytest.mark.parametrize("n_tokens", [16, 40])
+def test_logits_far_above_the_first_chunk_raise_the_reference_maximum(n_tokens):
+    """The attention kernel keeps the row maximum of a range's first 128-token chunk as the reference of its
+    exponentials and only checks that a chunk's row sum stays below 2^60.  Here the last context frame holds keys whose
+    logits lie about 80 octaves above everything before them: the rare path (true maximum, rescaling of O and of the
+    running sum, second pass) must give the oracle's answer.  16 tokens: one row tile, two half-streams; 40 tokens: two
+    row tiles."""
+    s = H.Shape(L=1, Hq=8, Hkv=2, Nf=48, T=12, W=2, k=6, seed=7)
+    g = rekv.ReKV(s.L, s.Hq, s.Hkv, s.D, s.Nf, s.T, s.W, max_q_tokens=n_tokens, max_topk=s.k)
+    o = orc.OracleCache(s.L, s.Hq, s.Hkv, s.D, s.Nf, s.W)
+    gen = torch.Generator().manual_seed(11)
+    sign = (torch.randint(0, 2, (s.D,), generator=gen) * 2 - 1).float()
+    for f in range(s.T):
+        k = (0.1 * torch.randn(s.L, s.Nf, s.Hkv, s.D, generator=gen)).to(torch.bfloat16)
+        v = torch.randn(s.L, s.Nf, s.Hkv, s.D, generator=gen).to(torch.bfloat16)
+        if f == s.T - 1:  # the last window frame: keys along the query direction, 2.5 per dimension
+            k[:, 5:40] = (2.5 * sign).to(torch.bfloat16)
+        assert g.append_frame(k.cuda(), v.cuda()) == f
+        o.append(k, v)
+    q = (2.0 * sign).to(torch.bfloat16).expand(s.L, n_tokens, s.Hq, s.D).contiguous()
+    cu = [0, n_tokens]
+    ref = o.question(q, s.k, s.T)
+    out = g.question(q.cuda(), cu, s.k, s.T, idx=ref["idx"][:, None].contiguous().cuda())
+    g.check_status()
+    # the big logits are 2.0 * 2.5 * 128 / sqrt(128) = 56.6 nats = 81.6 octaves above the others' (about 0)
+    H.assert_attention(out, ref["out"], "attention with a late, very large logit")
+    g.close()
