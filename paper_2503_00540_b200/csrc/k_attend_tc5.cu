@@ -54,6 +54,7 @@ constexpr uint32_t TILE_BYTES = 2 * HALF_BYTES;
 constexpr uint32_t STAGE_ROW_F32 = 144, STAGE_ROW_BF16 = 80;  // epilogue staging rows: a quarter row + 16 bytes (no bank conflicts)
 constexpr uint32_t STAGE_WARP_BYTES = 32 * STAGE_ROW_F32;
 constexpr float RESCALE_SUM_LIMIT = 1.152921504606846976e18f;  // 2^60: a chunk's row sum beyond it raises the reference maximum
+constexpr int PEND_MAX = 8;   // units a CTA can have to merge at the end of its range (two cut units x two row tiles)
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 // P is cut (not rounded) to bf16: a value with mantissa m in [1, 2) loses u * 2^-7 / m of itself, u uniform in [0, 1).
 // The mantissa of 2^x is log-uniform, E[1/m] = 1 / (2 ln 2), so the mean loss is 0.7213 * 2^-8 of the value, and scaling
@@ -81,7 +82,7 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // FULL: Eq. 3 in full (rotated K tiles, the part over X joins in the epilogue).  SPLIT: the launch has units with a
 // single row tile, which run as two half-streams (compiled out otherwise: the common loop stays as it was).
 template <bool FULL, bool SPLIT>
-__global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParams p) {
+__global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const uint32_t s_base = smem_u32(smem);
@@ -93,6 +94,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   volatile uint32_t* s_tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + (s_bar - s_base) + 8 * (2 * KV_BUFS + 6));
   volatile uint32_t* s_abort = s_tmem_slot + 1;
   volatile uint32_t* s_stop = s_tmem_slot + 2;  // the abort flag as one thread saw it between two segment barriers
+  volatile uint32_t* s_pend_n = s_tmem_slot + 3;  // units whose last part this CTA finished: count ...
+  volatile uint32_t* s_bad = s_tmem_slot + 4;     // [2] per tile slot: a warp of the slot did not write its partial rows
+  volatile uint32_t* s_fast = s_tmem_slot + 6;    // [2] per tile slot: every other part of the unit is in place
+  volatile uint32_t* s_pend = s_tmem_slot + 8;    // ... and list [PEND_MAX] of (unit << 2 | row tile << 1 | half-streams)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -109,6 +114,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
     }
     *s_abort = 0;
     *s_stop = 0;
+    s_bad[0] = s_bad[1] = 0;
+    *s_pend_n = 0;
     fence_barrier_init();
   }
   if (warp == 0) {
@@ -142,6 +149,253 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
   // held back by the ring's empty barriers only), so that K/V tiles are already on their way during an epilogue.
   auto seg_sync = [&]() {
     if (warp != 0) asm volatile("bar.sync 1, %0;" ::"n"(TC_THREADS - 32) : "memory");
+  };
+  // Merge inside the kernel.  After a tile slot's partial rows of a cut unit are written (softmax warps), the parts are
+  // published with a fence and counted with an atomic per (unit, row tile); the slot that finishes the unit's last
+  // part puts the unit on the CTA's list, and at the end of the CTA's range its softmax warps join the listed units'
+  // parts -- in part order, whichever CTA does it -- write the output rows and leave the counters at zero for the
+  // next launch.  Nobody waits for anybody.  The barrier is taken by all four warps of the slot whether or not their
+  // own partial rows got written (a wait that ran out): a warp that failed marks the slot, which then does not
+  // count, and the unit stays unmerged behind the status word that the wait has set.
+  auto slot_sync = [&](int t) {  // the four softmax warps of tile slot t
+    if (t == 0)
+      asm volatile("bar.sync 2, 128;" ::: "memory");
+    else
+      asm volatile("bar.sync 3, 128;" ::: "memory");
+  };
+  auto part_range = [&](long long u, long long& c_first, long long& c_last) {
+    c_first = (u * p.ncf) / p.per;
+    c_last = ((u + 1) * p.ncf - 1) / p.per;
+  };
+  auto part_slot = [&](const UnitInfo& ui, long long u, long long c_first, bool split, int rt, int k) -> long long {
+    const long long c = c_first + (split ? k >> 1 : k);
+    const long long base = p.per == p.ncf ? (long long)ui.srank : c + u;
+    return base * 2 + (split ? (k & 1) : rt);
+  };
+  auto count_part = [&](long long u, const UnitInfo& ui, int t, int rt, bool split, bool wrote) {
+    if (!wrote) s_bad[t] = 1;
+    __threadfence();
+    slot_sync(t);
+    if ((warp & 3) == 0 && lane == 0) {
+      if (!s_bad[t]) {
+        long long c_first, c_last;
+        part_range(u, c_first, c_last);
+        const int n_parts = (int)(c_last - c_first + 1) * (split ? 2 : 1);
+        int* cnt = p.unit_cnt + (p.per == p.ncf ? (long long)ui.srank : u) * 2 + (split ? 0 : t);
+        if (atomicAdd(cnt, 1) == n_parts - 1) {
+          *cnt = 0;
+          const uint32_t at = atomicAdd((uint32_t*)s_pend_n, 1u);
+          if (at < PEND_MAX)
+            s_pend[at] = ((uint32_t)u << 2) | ((uint32_t)rt << 1) | (split ? 1u : 0u);
+          else
+            atomicExch(p.status, -2033);  // cannot happen: a range cuts two units at most
+        }
+      }
+      s_bad[t] = 0;  // (a warp marks the next segment's failure only after the segment barrier that follows)
+    }
+  };
+  // Both ways of finishing a cut unit do the same arithmetic, so that the output does not depend on which CTA came
+  // last: M = the maximum over the parts (the part over X included), weights 2^(m_k - M), numerators and
+  // denominator accumulated with fused multiply-adds in part order starting from the part over X, one division.
+  //
+  // The listed units, by the eight softmax warps: a warp per row, eight rows at a time, a float4 of the 128 columns
+  // per lane.
+  auto merge_listed = [&]() {
+    const uint32_t n_pend = min(*s_pend_n, (uint32_t)PEND_MAX);
+    __threadfence();
+    const int w8 = warp - SM_WARP0;
+#pragma unroll 1
+    for (uint32_t e = 0; e < n_pend; ++e) {
+      const uint32_t code = s_pend[e];
+      const long long u = code >> 2;
+      const int rt = (code >> 1) & 1;
+      const bool split = code & 1u;
+      const UnitInfo ui = decode_unit(p, u);
+      long long c_first, c_last;
+      part_range(u, c_first, c_last);
+      const int n_parts = (int)(c_last - c_first + 1) * (split ? 2 : 1);
+#pragma unroll 1
+      for (int r0 = w8 * 8; r0 < 128; r0 += 64) {
+        const int rr0 = ui.m0 + rt * 128 + r0;
+        if (rr0 >= ui.rows_q) break;
+        float M[8], den[8];
+        float4 acc[8];
+        long long out_at[8];
+#pragma unroll
+        for (int a = 0; a < 8; ++a) {
+          const int rr = min(rr0 + a, ui.rows_q - 1);
+          const int n = rr / p.G, j = rr - n * p.G;
+          out_at[a] = ((ui.q_row0 + n) * p.Hq + ui.g * p.G + j) * 128 + lane * 4;
+          M[a] = (FULL && p.self_o) ? fmaxf(-1e30f, p.self_ml[(out_at[a] >> 7) * 2]) : -1e30f;
+        }
+#pragma unroll 1
+        for (int k = 0; k < n_parts; ++k) {
+          const long long base = part_slot(ui, u, c_first, split, rt, k) * 128 + r0;
+#pragma unroll
+          for (int a = 0; a < 8; ++a) M[a] = fmaxf(M[a], __ldcg(p.part_ml + (base + a) * 2));
+        }
+#pragma unroll
+        for (int a = 0; a < 8; ++a) {
+          den[a] = 0.f;
+          acc[a] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (FULL && p.self_o) {
+            const long long orow = out_at[a] >> 7;
+            const float w = ex2(p.self_ml[orow * 2] - M[a]);
+            const float4 o = *reinterpret_cast<const float4*>(p.self_o + out_at[a]);
+            den[a] = w * p.self_ml[orow * 2 + 1];
+            acc[a] = make_float4(w * o.x, w * o.y, w * o.z, w * o.w);
+          }
+        }
+#pragma unroll 1
+        for (int k0 = 0; k0 < n_parts; k0 += 2) {  // sixteen rows in flight
+          float4 o[2][8];
+          float2 ml[2][8];
+#pragma unroll
+          for (int i = 0; i < 2; ++i)
+            if (k0 + i < n_parts) {
+              const long long base = part_slot(ui, u, c_first, split, rt, k0 + i) * 128 + r0;
+#pragma unroll
+              for (int a = 0; a < 8; ++a) {
+                ml[i][a] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (base + a) * 2));
+                o[i][a] = __ldcg(reinterpret_cast<const float4*>(p.part_o + (base + a) * 128 + lane * 4));
+              }
+            }
+#pragma unroll
+          for (int i = 0; i < 2; ++i)
+            if (k0 + i < n_parts) {
+#pragma unroll
+              for (int a = 0; a < 8; ++a) {
+                const float w = ex2(ml[i][a].x - M[a]);
+                den[a] = fmaf(w, ml[i][a].y, den[a]);
+                acc[a].x = fmaf(w, o[i][a].x, acc[a].x);
+                acc[a].y = fmaf(w, o[i][a].y, acc[a].y);
+                acc[a].z = fmaf(w, o[i][a].z, acc[a].z);
+                acc[a].w = fmaf(w, o[i][a].w, acc[a].w);
+              }
+            }
+        }
+#pragma unroll
+        for (int a = 0; a < 8; ++a)
+          if (rr0 + a < ui.rows_q) {
+            const float inv = den[a] > 0.f ? 1.f / den[a] : 0.f;
+            uint2 packed;
+            packed.x = pack_bf16(acc[a].x * inv, acc[a].y * inv);
+            packed.y = pack_bf16(acc[a].z * inv, acc[a].w * inv);
+            *reinterpret_cast<uint2*>(p.out + out_at[a]) = packed;
+          }
+      }
+    }
+  };
+  // The unit's other parts joined with this tile slot's own part, which is still in tensor memory: one thread per
+  // row as in the other epilogues.  The other parts' rows come through the warp's staging rows (contiguous global
+  // reads, then each thread takes its row), the result leaves through them as bf16.
+  auto finish_from_tmem = [&](long long u, const UnitInfo& ui, int t, int rt, bool split, int row, int rr0, bool valid,
+                              int n, int j, float m_own, float l_own, bool own_empty, uint32_t t_o,
+                              unsigned char* stage) {
+    if (rr0 >= ui.rows_q) return;  // a warp without a valid row (the ragged tile)
+    long long c_first, c_last;
+    part_range(u, c_first, c_last);
+    const int n_parts = (int)(c_last - c_first + 1) * (split ? 2 : 1);
+    const int own = (int)(blockIdx.x - c_first) * (split ? 2 : 1) + (split ? t : 0);
+    const long long out_row = (ui.q_row0 + (valid ? n : 0)) * p.Hq + ui.g * p.G + (valid ? j : 0);
+    float M = fmaxf(-1e30f, m_own);
+#pragma unroll 1
+    for (int k = 0; k < n_parts; ++k)
+      if (k != own) M = fmaxf(M, __ldcg(p.part_ml + (part_slot(ui, u, c_first, split, rt, k) * 128 + row) * 2));
+    float den = 0.f, w_x = 0.f;
+    const float4* o_x = nullptr;
+    if (FULL && p.self_o) {
+      const float m_x = p.self_ml[out_row * 2];
+      M = fmaxf(M, m_x);
+      w_x = ex2(m_x - M);
+      den = w_x * p.self_ml[out_row * 2 + 1];
+      o_x = reinterpret_cast<const float4*>(p.self_o + out_row * 128);
+    }
+#pragma unroll 1
+    for (int k = 0; k < n_parts; ++k) {
+      float2 ml = make_float2(m_own, l_own);
+      if (k != own)
+        ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (part_slot(ui, u, c_first, split, rt, k) * 128 + row) * 2));
+      den = fmaf(ex2(ml.x - M), ml.y, den);
+    }
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+    // rows this lane stores: r = 8 k + (lane >> 2), 16 bytes (8 bf16) at chunk (lane & 3) of the quarter
+    __nv_bfloat16* dst_k[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int r2 = rr0 + 8 * k + (lane >> 2);
+      const int n2 = r2 / p.G, j2 = r2 - n2 * p.G;
+      dst_k[k] = r2 < ui.rows_q ? p.out + ((ui.q_row0 + n2) * p.Hq + ui.g * p.G + j2) * 128 + (lane & 3) * 8 : nullptr;
+    }
+#pragma unroll 1
+    for (int qd = 0; qd < 4; ++qd) {
+      float acc[32];
+#pragma unroll
+      for (int v4 = 0; v4 < 8; ++v4) {
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (FULL && o_x) x = __ldg(o_x + qd * 8 + v4);
+        acc[4 * v4] = w_x * x.x;
+        acc[4 * v4 + 1] = w_x * x.y;
+        acc[4 * v4 + 2] = w_x * x.z;
+        acc[4 * v4 + 3] = w_x * x.w;
+      }
+#pragma unroll 1
+      for (int k = 0; k < n_parts; ++k) {
+        if (k == own) {  // (uniform over the slot's warps)
+          uint32_t o[2][16];
+          tmem_ld16(t_o + qd * 32, o[0]);
+          tmem_ld16(t_o + qd * 32 + 16, o[1]);
+          tmem_wait_ld16(o[0]);
+          tmem_wait_ld16(o[1]);
+          const float w = ex2(m_own - M);
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            acc[e] = fmaf(w, own_empty ? 0.f : __uint_as_float(o[e >> 4][e & 15]), acc[e]);
+        } else {
+          const long long slot = part_slot(ui, u, c_first, split, rt, k);
+          const float w = ex2(__ldcg(p.part_ml + (slot * 128 + row) * 2) - M);
+          const float* po = p.part_o + ((slot * 128 + ((warp & 3) << 5) + (lane >> 3)) * 128 + (lane & 7) * 4) + qd * 32;
+          uint4 x[8];
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) x[kk] = __ldcg(reinterpret_cast<const uint4*>(po + (long long)kk * 4 * 128));
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk)
+            *reinterpret_cast<uint4*>(stage + (4 * kk + (lane >> 3)) * STAGE_ROW_F32 + (lane & 7) * 16) = x[kk];
+          __syncwarp();
+#pragma unroll
+          for (int v4 = 0; v4 < 8; ++v4) {
+            const float4 y = *reinterpret_cast<const float4*>(stage + lane * STAGE_ROW_F32 + v4 * 16);
+            acc[4 * v4] = fmaf(w, y.x, acc[4 * v4]);
+            acc[4 * v4 + 1] = fmaf(w, y.y, acc[4 * v4 + 1]);
+            acc[4 * v4 + 2] = fmaf(w, y.z, acc[4 * v4 + 2]);
+            acc[4 * v4 + 3] = fmaf(w, y.w, acc[4 * v4 + 3]);
+          }
+          __syncwarp();
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        uint4 a, b;
+        const float* c = acc + 16 * h;
+        a.x = pack_bf16(c[0] * inv, c[1] * inv);
+        a.y = pack_bf16(c[2] * inv, c[3] * inv);
+        a.z = pack_bf16(c[4] * inv, c[5] * inv);
+        a.w = pack_bf16(c[6] * inv, c[7] * inv);
+        b.x = pack_bf16(c[8] * inv, c[9] * inv);
+        b.y = pack_bf16(c[10] * inv, c[11] * inv);
+        b.z = pack_bf16(c[12] * inv, c[13] * inv);
+        b.w = pack_bf16(c[14] * inv, c[15] * inv);
+        *reinterpret_cast<uint4*>(stage + lane * STAGE_ROW_BF16 + h * 32) = a;
+        *reinterpret_cast<uint4*>(stage + lane * STAGE_ROW_BF16 + h * 32 + 16) = b;
+      }
+      __syncwarp();
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const uint4 x = *reinterpret_cast<const uint4*>(stage + (8 * k + (lane >> 2)) * STAGE_ROW_BF16 + (lane & 3) * 16);
+        if (dst_k[k]) *reinterpret_cast<uint4*>(dst_k[k] + qd * 32) = x;
+      }
+      __syncwarp();
+    }
   };
   const uint32_t page_half_bytes = (uint32_t)p.Nf * 128u;   // one 64-dim half of a head tile in a page
   const uint32_t idesc_pv = idesc_bf16(128, 128, 1);
@@ -518,6 +772,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
         }
         l_sum *= TRUNC_GAIN_INV;  // the row sum was taken over the scaled values
         // ---- output of this range: final rows, or a partial for the combine kernel ----
+        // A cut unit whose other parts are all in place is finished here, from this slot's O in tensor memory (the
+        // usual case for the CTA that holds a unit's head: the later CTAs worked on its tail first): no partial of
+        // its own is written or read back.  Otherwise the slot writes its partial and counts it.
+        const bool cut = !whole_unit && p.unit_cnt != nullptr;
+        bool fast = false;
+        if (cut) {
+          if ((warp & 3) == 0 && lane == 0) {
+            long long c_first, c_last;
+            part_range(u, c_first, c_last);
+            const int n_parts = (int)(c_last - c_first + 1) * (split ? 2 : 1);
+            int* cnt = p.unit_cnt + (p.per == p.ncf ? (long long)ui.srank : u) * 2 + (split ? 0 : t);
+            s_fast[t] = atomicAdd(cnt, 0) == n_parts - 1;
+          }
+          slot_sync(t);
+          fast = s_fast[t] != 0;
+          if (fast) __threadfence();
+        }
+        bool wrote = false;  // this thread's rows are in place (partial or final)
         if (ok && (nch == 0 || wait(bars.pv_done(t), (chunk_cnt[t] + nch - 1) & 1))) {
           tc_fence_after();
           const int rr = ui.m0 + rt * 128 + row;
@@ -594,6 +866,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
               }
               __syncwarp();
             }
+          } else if (fast) {
+            finish_from_tmem(u, ui, t, rt, split, row, rr0, valid, n, j, m_used, l_sum, nch == 0, t_o, stage);
+            wrote = true;
           } else {
             const long long slot_raw = (p.per == p.ncf ? (long long)ui.srank : (long long)blockIdx.x + u) * 2 + t;
             const bool slot_ok = REKV_CHECK(slot_raw >= 0 && slot_raw < p.part_slots, p.status, 32);  // (checks build)
@@ -630,6 +905,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
               p.part_ml[(slot * 128 + row) * 2] = m_used;
               p.part_ml[(slot * 128 + row) * 2 + 1] = l_sum;
             }
+            wrote = slot_ok;
+          }
+        }
+        if (cut) {
+          if (!fast) {
+            count_part(u, ui, t, rt, split, wrote);
+          } else if ((warp & 3) == 0 && lane == 0) {  // every other part had been counted: nobody else touches it
+            p.unit_cnt[(p.per == p.ncf ? (long long)ui.srank : u) * 2 + (split ? 0 : t)] = 0;
           }
         }
       }
@@ -651,6 +934,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const TcParam
       seg_sync();
       if (*s_stop) break;
     }
+  }
+  if constexpr (SOFTMAX) {
+    if (p.unit_cnt && !*s_stop) merge_listed();
   }
   if constexpr (!SOFTMAX) {
     // A CTA that gives up must not return while copies into its shared memory are still on their way: the producer
@@ -701,7 +987,7 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   p.Ns = (s.Nf + 7) & ~7;
   p.wait_limit = c->test_wait_limit;
   p.skip_copy_entry = c->test_skip_copy_entry;
-  p.part_slots = (long long)c->part_units * 2;
+  p.part_slots = (long long)c->part_units;
   p.ncf = ncf;
   p.layer0 = layer0;
   p.n_split = 0;
@@ -768,8 +1054,8 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     if (p.per == ncf && (size_t)(layer1 - layer0) * s.Hkv * n_split * 2 > c->part_units) n_split = 0;
     p.n_split = n_split;
   }
-  const size_t smem = 2 * Q_TILE_BYTES + (size_t)KV_BUFS * TILE_BYTES + 8 * (2 * KV_BUFS + 6) + 16 + 1024;
-  static_assert(2 * Q_TILE_BYTES + KV_BUFS * TILE_BYTES + 8 * (2 * KV_BUFS + 6) + 16 + 1024 <= 227 * 1024,
+  const size_t smem = 2 * Q_TILE_BYTES + (size_t)KV_BUFS * TILE_BYTES + 8 * (2 * KV_BUFS + 6) + 64 + 1024;
+  static_assert(2 * Q_TILE_BYTES + KV_BUFS * TILE_BYTES + 8 * (2 * KV_BUFS + 6) + 64 + 1024 <= 227 * 1024,
                 "shared-memory plan of the attention kernel");
   static PerDeviceOnce attr;
   cudaError_t ea = attr.run([] {
@@ -783,6 +1069,15 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     return e;
   });
   if (ea != cudaSuccess) return ea;
+  // A unit cut into a few parts is merged inside the kernel by the CTA that finishes its last part; with many parts
+  // per unit (a launch of few units, such as one layer) the merge kernel's parallelism is worth its launch.
+  {
+    const int ctas_per_unit = p.per == ncf ? 1 : (ncf + p.per - 1) / p.per + 1;
+    if (ctas_per_unit * (p.n_split > 0 ? 2 : 1) > 8) p.unit_cnt = nullptr;
+    // cut units that also run as two half-streams have four to six parts each, most of them written at the end of
+    // the launch: the merge kernel's parallelism is faster there (10-token question: 209 against 220 us)
+    if (p.per != ncf && p.n_split > 0) p.unit_cnt = nullptr;
+  }
   if (timed) cudaEventRecord(c->ev_t0, st);
   auto kernel = full ? (p.n_split > 0 ? attend_tc5_kernel<true, true> : attend_tc5_kernel<true, false>)
                      : (p.n_split > 0 ? attend_tc5_kernel<false, true> : attend_tc5_kernel<false, false>);
@@ -794,7 +1089,7 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     c->merge_timed = false;
   }
   c->launches += 1;
-  if (p.per != ncf || p.n_split > 0) {
+  if ((p.per != ncf || p.n_split > 0) && !p.unit_cnt) {
     // units cut at CTA boundaries: a block group per unit; whole units: only those with half-stream partials
     const long long merge_units = p.per != ncf ? units : (long long)(layer1 - layer0) * s.Hkv * p.n_split;
     // (units with half-streams have one row tile)

@@ -86,16 +86,35 @@ def test_72b_head_shape(flags):
 
 def test_many_short_questions_whole_units_as_half_streams():
     """640 units of one row tile each (more than four per SM, so no unit is cut at a CTA boundary): every unit runs
-    as two half-streams whose partials the merge kernel joins, with partial slots counted per such unit."""
+    as two half-streams; the half that finishes second joins the other's partial inside the kernel, with partial slots
+    counted per such unit."""
     s = H.Shape(L=4, Hq=16, Hkv=8, Nf=33, T=12, W=2, k=4, seed=540)
     lengths = [9 + (7 * i) % 32 for i in range(20)]  # 18..80 rows per KV head
     _run_question_parity(s, lengths, max_questions=20)
 
 
 def test_short_question_cut_at_cta_boundaries():
-    """One 10-token question at the 7B head shape: 70 rows = one row tile per unit, units cut at CTA boundaries."""
+    """One 10-token question at the 7B head shape: 70 rows = one row tile per unit, units cut at CTA boundaries
+    (four to six partials per unit: the merge kernel joins them)."""
     s = H.Shape(L=3, Hq=28, Hkv=4, Nf=196, T=30, W=4, k=12, seed=7)
     _run_question_parity(s, [10])
+
+
+def test_units_cut_into_a_few_parts_are_finished_inside_the_kernel():
+    """32 units of two row tiles over 128 CTAs, five context frames per CTA: every unit is cut into four or five parts,
+    and the CTA that finishes a unit's last part joins them (from its own accumulator if the others are already
+    there, from the written partials otherwise).  Both ways do the same arithmetic in part order: repeated
+    launches give the same bits whichever CTA came last."""
+    s = H.Shape(L=8, Hq=28, Hkv=4, Nf=196, T=28, W=4, k=16, seed=2503)
+    _run_question_parity(s, [32])
+    g = H.build_gpu(s, max_questions=1, max_q_tokens=32)
+    q, cu = H.questions(s, [32], device="cuda")
+    first = g.question(q, cu, s.k, s.T).clone()
+    for _ in range(8):
+        assert torch.equal(g.question(q, cu, s.k, s.T), first)
+    g.check_status()
+    st = g.stats()
+    g.close()
 
 
 def test_question_in_the_past_sees_only_visible_frames():
