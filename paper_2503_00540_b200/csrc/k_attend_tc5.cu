@@ -1069,14 +1069,13 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     return e;
   });
   if (ea != cudaSuccess) return ea;
-  // A unit cut into a few parts is merged inside the kernel by the CTA that finishes its last part; with many parts
-  // per unit (a launch of few units, such as one layer) the merge kernel's parallelism is worth its launch.
+  // A unit cut into two or three parts is finished inside the kernel by the CTA that completes its last part; with more
+  // parts per unit (fewer units than SMs: 8 to 16 layers of a single question lose 2 to 13 us that way, one layer more)
+  // the merge kernel's parallelism is worth its launch.
   {
     const int ctas_per_unit = p.per == ncf ? 1 : (ncf + p.per - 1) / p.per + 1;
-    if (ctas_per_unit * (p.n_split > 0 ? 2 : 1) > 8) p.unit_cnt = nullptr;
-    // cut units that also run as two half-streams have four to six parts each, most of them written at the end of
-    // the launch: the merge kernel's parallelism is faster there (10-token question: 209 against 220 us)
-    if (p.per != ncf && p.n_split > 0) p.unit_cnt = nullptr;
+    // (cut units that also run as two half-streams have four to six parts: 10-token question 209 against 220 us)
+    if (ctas_per_unit * (p.n_split > 0 ? 2 : 1) > 3) p.unit_cnt = nullptr;
   }
   if (timed) cudaEventRecord(c->ev_t0, st);
   auto kernel = full ? (p.n_split > 0 ? attend_tc5_kernel<true, true> : attend_tc5_kernel<true, false>)

@@ -101,14 +101,14 @@ def test_short_question_cut_at_cta_boundaries():
 
 
 def test_units_cut_into_a_few_parts_are_finished_inside_the_kernel():
-    """32 units of two row tiles over 128 CTAs, five context frames per CTA: every unit is cut into four or five parts,
-    and the CTA that finishes a unit's last part joins them (from its own accumulator if the others are already
-    there, from the written partials otherwise).  Both ways do the same arithmetic in part order: repeated
-    launches give the same bits whichever CTA came last."""
-    s = H.Shape(L=8, Hq=28, Hkv=4, Nf=196, T=28, W=4, k=16, seed=2503)
-    _run_question_parity(s, [32])
-    g = H.build_gpu(s, max_questions=1, max_q_tokens=32)
-    q, cu = H.questions(s, [32], device="cuda")
+    """80 units of two row tiles over 146 CTAs (on 148 SMs), eleven of a unit's twenty context frames per CTA: every
+    unit is cut into two or three parts, and the CTA that finishes a unit's last part joins them (from its own
+    accumulator if the others are already there, from the written partials otherwise).  Both ways do the same
+    arithmetic in part order: repeated launches give the same bits whichever CTA came last."""
+    s = H.Shape(L=10, Hq=16, Hkv=8, Nf=100, T=28, W=4, k=16, seed=2503)
+    _run_question_parity(s, [80])
+    g = H.build_gpu(s, max_questions=1, max_q_tokens=80)
+    q, cu = H.questions(s, [80], device="cuda")
     first = g.question(q, cu, s.k, s.T).clone()
     for _ in range(8):
         assert torch.equal(g.question(q, cu, s.k, s.T), first)
