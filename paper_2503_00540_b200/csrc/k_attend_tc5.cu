@@ -81,7 +81,9 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 
 // FULL: Eq. 3 in full (rotated K tiles, the part over X joins in the epilogue).  SPLIT: the launch has units with a
 // single row tile, which run as two half-streams (compiled out otherwise: the common loop stays as it was).
-template <bool FULL, bool SPLIT>
+// EARLYQ: Q does not depend on the kernels just before this launch (the library's own selection kernels, which read Q
+// but do not write it): the first segment's Q tiles are loaded before the dependency wait.
+template <bool FULL, bool SPLIT, bool EARLYQ>
 __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -127,9 +129,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem_slot;
-  // everything above is independent of earlier kernels; the context table and Q are not
-  grid_dep_wait();
-  grid_dep_launch();
+  // everything above is independent of earlier kernels; the context table is not, and Q only when the launcher says
+  // so (after the library's own selection kernels, which read Q but do not write it, the first segment's Q tiles
+  // are loaded while those kernels are still running: the wait then stands after that load in the range loop)
+  if constexpr (!EARLYQ) {
+    grid_dep_wait();
+    grid_dep_launch();
+  }
   auto col_o = [](int t) { return (uint32_t)t * 128u; };
   auto col_s = [](int t) { return 256u + (uint32_t)t * 128u; };
 
@@ -447,6 +453,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_
           *reinterpret_cast<uint4*>(dst + (c >> 3) * (Q_TILE_BYTES / 2) + (((c & 7) ^ (row & 7)) << 4)) = x[c];
       }
       fence_proxy_async();
+    }
+    if constexpr (EARLYQ) {
+      if (pos == (long long)blockIdx.x * p.per) {  // first segment: only now the earlier kernels' results
+        grid_dep_wait();
+        grid_dep_launch();
+      }
     }
     seg_sync();
 
@@ -1059,14 +1071,14 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
                 "shared-memory plan of the attention kernel");
   static PerDeviceOnce attr;
   cudaError_t ea = attr.run([] {
-    cudaError_t e = cudaFuncSetAttribute(attend_tc5_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attend_tc5_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attend_tc5_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(attend_tc5_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    return e;
+    const void* kernels[] = {(const void*)attend_tc5_kernel<false, false, false>, (const void*)attend_tc5_kernel<true, false, false>,
+                             (const void*)attend_tc5_kernel<false, true, false>,  (const void*)attend_tc5_kernel<true, true, false>,
+                             (const void*)attend_tc5_kernel<false, false, true>,  (const void*)attend_tc5_kernel<false, true, true>};
+    for (const void* k : kernels) {
+      cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
   });
   if (ea != cudaSuccess) return ea;
   // A unit cut into two or three parts is finished inside the kernel by the CTA that completes its last part; with more
@@ -1078,8 +1090,10 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     if (ctas_per_unit * (p.n_split > 0 ? 2 : 1) > 3) p.unit_cnt = nullptr;
   }
   if (timed) cudaEventRecord(c->ev_t0, st);
-  auto kernel = full ? (p.n_split > 0 ? attend_tc5_kernel<true, true> : attend_tc5_kernel<true, false>)
-                     : (p.n_split > 0 ? attend_tc5_kernel<false, true> : attend_tc5_kernel<false, false>);
+  const bool early_q = c->q_early_ok && !full;
+  auto kernel = full ? (p.n_split > 0 ? attend_tc5_kernel<true, true, false> : attend_tc5_kernel<true, false, false>)
+                : early_q ? (p.n_split > 0 ? attend_tc5_kernel<false, true, true> : attend_tc5_kernel<false, false, true>)
+                          : (p.n_split > 0 ? attend_tc5_kernel<false, true, false> : attend_tc5_kernel<false, false, false>);
   cudaError_t e1 = rekv_launch_pdl(kernel, dim3((unsigned)grid), dim3(TC_THREADS), smem, st, p);
   if (e1 != cudaSuccess) return e1;
   if (timed) {

@@ -558,7 +558,9 @@ int rekv_question_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu
   c->g_keff = geom.k_eff;
   c->g_nvis = n_visible;
   c->g_topk = top_k;
+  c->q_early_ok = fused_table;  // the selection kernel, which only reads Q, is directly before the attention
   rc = attend_one_layer(c, layer, q, qb, out, st);
+  c->q_early_ok = false;
   return rc ? rc : geom.ncf;
 }
 

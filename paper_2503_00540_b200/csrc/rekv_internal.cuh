@@ -137,6 +137,7 @@ struct rekv_ctx {
   // test-only knobs of the bounded device-side waits (rekv_test_set_wait_limit); 0 / -1 = off
   unsigned test_wait_limit;
   int test_skip_copy_entry;
+  bool q_early_ok = false;          // the attention launch that follows is chained to the library's own selection kernels (which only read Q)
 
   // state of the last gather.  The context table has one geometry (questions x context frames) for all layers; a
   // layer's context is valid while the table still has the geometry it was built with (layer_ctx_valid).
