@@ -206,7 +206,7 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
   const int qi = blockIdx.x, l = layer0 + blockIdx.y;
   const float* s = scores + ((long long)l * nQ + qi) * n_visible;
   int32_t* out = idx_out + ((long long)l * nQ + qi) * top_k;
-  __shared__ unsigned hist[256];
+  __shared__ unsigned hist[4 * 256];
   __shared__ unsigned s_prefix;
   __shared__ int s_krem;
   __shared__ int warp_gt[16], warp_eq[16];
@@ -220,13 +220,14 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
     topk_write_table(tt, out, 0, l, qi, nQ);
     return;
   }
-  // up to TK_CACHE * 512 candidates keep their keys in registers: one read of the scores instead of five
+  // up to TK_CACHE * 512 candidates keep their keys in registers: one read of the scores instead of five.  A thread
+  // holds TK_CACHE consecutive candidates, so that the ordered compaction at the end is one scan over the threads.
   constexpr int TK_CACHE = 4;
   const bool cached = n_cand <= TK_CACHE * 512;
   unsigned kc[TK_CACHE];
 #pragma unroll
   for (int j = 0; j < TK_CACHE; ++j) {
-    const int i = j * 512 + threadIdx.x;
+    const int i = threadIdx.x * TK_CACHE + j;
     kc[j] = (cached && i < n_cand) ? score_key(s[i]) : 0u;
   }
   if (threadIdx.x == 0) {
@@ -235,20 +236,21 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
     s_base_gt = 0;
     s_base_eq = 0;
   }
+  for (int i = threadIdx.x; i < 4 * 256; i += blockDim.x) hist[i] = 0;  // one histogram per pass, cleared once
+  __syncthreads();
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
-    __syncthreads();
+    unsigned* h = hist + 256 * pass;
     const unsigned prefix = s_prefix;
     const unsigned mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
     if (cached) {
 #pragma unroll
       for (int j = 0; j < TK_CACHE; ++j)
-        if (j * 512 + (int)threadIdx.x < n_cand && (kc[j] & mask) == prefix) atomicAdd(&hist[(kc[j] >> shift) & 255u], 1u);
+        if ((int)threadIdx.x * TK_CACHE + j < n_cand && (kc[j] & mask) == prefix) atomicAdd(&h[(kc[j] >> shift) & 255u], 1u);
     } else {
       for (int i = threadIdx.x; i < n_cand; i += blockDim.x) {
         const unsigned key = score_key(s[i]);
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        if ((key & mask) == prefix) atomicAdd(&h[(key >> shift) & 255u], 1u);
       }
     }
     __syncthreads();
@@ -257,7 +259,7 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
       unsigned b[8], tot = 0;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        b[j] = hist[lane * 8 + j];
+        b[j] = h[lane * 8 + j];
         tot += b[j];
       }
       unsigned suf = tot;  // inclusive suffix sum over lanes >= this one
@@ -283,53 +285,80 @@ __global__ void __launch_bounds__(512) topk_kernel(const float* __restrict__ sco
   }
   const unsigned thr = s_prefix;  // key of the k_eff-th largest score
   const int need_eq = s_krem;     // how many candidates equal to it are selected (lowest indices first)
-  const int n_gt = k_eff - need_eq;
-  auto emit = [&](const int i0, const unsigned key_in) {
-    const int i = i0 + threadIdx.x;
-    const unsigned key = i < n_cand ? key_in : 0u;
-    const bool gt = i < n_cand && key > thr, eq = i < n_cand && key == thr;
-    const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
-    if (lane == 0) {
-      warp_gt[warp] = __popc(bg);
-      warp_eq[warp] = __popc(be);
+  // Ordered compaction of a stretch of blockDim.x * TK_CACHE candidates starting at i0, thread t holding candidates
+  // i0 + t * TK_CACHE + j: counts of "greater" and "equal" per thread, an exclusive scan over the block (shuffles
+  // inside a warp, the warps' totals through shared memory), then
+  // output position = selected frames before this one = (greater before) + min(equal before, need_eq).
+  auto emit = [&](const int i0, const unsigned (&key_in)[TK_CACHE]) {
+    int cg = 0, ce = 0;
+#pragma unroll
+    for (int j = 0; j < TK_CACHE; ++j) {
+      const int i = i0 + threadIdx.x * TK_CACHE + j;
+      cg += i < n_cand && key_in[j] > thr;
+      ce += i < n_cand && key_in[j] == thr;
     }
-    __syncthreads();
-    int og = s_base_gt, oe = s_base_eq;
-    for (int w = 0; w < warp; ++w) {
-      og += warp_gt[w];
-      oe += warp_eq[w];
-    }
-    const unsigned lower = (1u << lane) - 1u;
-    const int rank_gt = og + __popc(bg & lower), rank_eq = oe + __popc(be & lower);
-    // output position = selected frames before this one = (greater before) + min(equal before, need_eq)
-    int pos = -1;
-    if (gt) pos = rank_gt + min(rank_eq, need_eq);
-    if (eq && rank_eq < need_eq) pos = rank_gt + rank_eq;
-    if (pos >= 0 && REKV_CHECK(pos < k_eff && i < n_cand, status, 21))
-      for (int j = 0; j < block; ++j) out[pos * block + j] = i * block + j;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      int tg = 0, te = 0;
-      for (int w = 0; w < 16; ++w) {
-        tg += warp_gt[w];
-        te += warp_eq[w];
+    int sg = cg, se = ce;  // inclusive scans over the warp
+    for (int o = 1; o < 32; o <<= 1) {
+      const int vg = __shfl_up_sync(0xffffffffu, sg, o), ve = __shfl_up_sync(0xffffffffu, se, o);
+      if (lane >= o) {
+        sg += vg;
+        se += ve;
       }
-      s_base_gt += tg;
-      s_base_eq += te;
+    }
+    if (lane == 31) {
+      warp_gt[warp] = sg;
+      warp_eq[warp] = se;
     }
     __syncthreads();
+    int og = s_base_gt + sg - cg, oe = s_base_eq + se - ce;  // greater / equal candidates before this thread's
+    {
+      const int wg = lane < 16 ? warp_gt[lane] : 0, we = lane < 16 ? warp_eq[lane] : 0;
+      const unsigned below = lane < warp ? 0xffffffffu : 0u;
+      int ag = wg & (int)below, ae = we & (int)below;  // totals of the warps before this one
+      for (int o = 16; o; o >>= 1) {
+        ag += __shfl_xor_sync(0xffffffffu, ag, o);
+        ae += __shfl_xor_sync(0xffffffffu, ae, o);
+      }
+      og += ag;
+      oe += ae;
+    }
+#pragma unroll
+    for (int j = 0; j < TK_CACHE; ++j) {
+      const int i = i0 + threadIdx.x * TK_CACHE + j;
+      const bool gt = i < n_cand && key_in[j] > thr, eq = i < n_cand && key_in[j] == thr;
+      int pos = -1;
+      if (gt) pos = og + min(oe, need_eq);
+      if (eq && oe < need_eq) pos = og + oe;
+      if (pos >= 0 && REKV_CHECK(pos < k_eff && i < n_cand, status, 21))
+        for (int jj = 0; jj < block; ++jj) out[pos * block + jj] = i * block + jj;
+      og += gt;
+      oe += eq;
+    }
   };
   if (cached) {
-#pragma unroll
-    for (int j = 0; j < TK_CACHE; ++j)
-      if (j * 512 < n_cand) emit(j * 512, kc[j]);
+    emit(0, kc);
   } else {
-    for (int i0 = 0; i0 < n_cand; i0 += blockDim.x) {
-      const int i = i0 + threadIdx.x;
-      emit(i0, i < n_cand ? score_key(s[i]) : 0u);
+    for (int i0 = 0; i0 < n_cand; i0 += blockDim.x * TK_CACHE) {
+      unsigned key[TK_CACHE];
+#pragma unroll
+      for (int j = 0; j < TK_CACHE; ++j) {
+        const int i = i0 + threadIdx.x * TK_CACHE + j;
+        key[j] = i < n_cand ? score_key(s[i]) : 0u;
+      }
+      emit(i0, key);
+      __syncthreads();  // everybody has read the warps' totals
+      if (threadIdx.x == 0) {
+        int tg = 0, te = 0;
+        for (int w = 0; w < 16; ++w) {
+          tg += warp_gt[w];
+          te += warp_eq[w];
+        }
+        s_base_gt += tg;
+        s_base_eq += te;
+      }
+      __syncthreads();
     }
   }
-  (void)n_gt;
   topk_write_table(tt, out, k_eff * block, l, qi, nQ);
 }
 
