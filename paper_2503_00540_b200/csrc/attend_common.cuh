@@ -75,5 +75,6 @@ constexpr uint32_t DEC_SCRATCH = DEC_WARPS * 16 * (128 + 2) * 4;  // the warps' 
 __global__ void attend_decode_kernel(const TcParams p);
 // k_attend_combine.cu: joins the (max, sum, O) partials of a unit's parts
 __global__ void combine_tc5_kernel(const TcParams p);
+__global__ void combine_many_kernel(const TcParams p);  // units of many parts (launches of few units)
 
 }  // namespace rekv_att

@@ -1052,7 +1052,8 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     }
     c->launches += 1;
     if (p.per != ncf && !p.unit_cnt) {
-      cudaError_t e2 = rekv_launch_pdl(combine_tc5_kernel, dim3((unsigned)units, 2, 32), dim3(128), 0, st, p);
+      const bool many = (ncf + p.per - 1) / p.per + 1 > 8;  // parts per unit
+      cudaError_t e2 = rekv_launch_pdl(many ? combine_many_kernel : combine_tc5_kernel, dim3((unsigned)units, 2, 32), dim3(128), 0, st, p);
       if (e2 != cudaSuccess) return e2;
       c->launches += 1;
       if (timed) {
@@ -1110,7 +1111,9 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
     // units cut at CTA boundaries: a block group per unit; whole units: only those with half-stream partials
     const long long merge_units = p.per != ncf ? units : (long long)(layer1 - layer0) * s.Hkv * p.n_split;
     // (units with half-streams have one row tile)
-    cudaError_t e2 = rekv_launch_pdl(combine_tc5_kernel, dim3((unsigned)merge_units, p.per != ncf ? 2 : 1, 32), dim3(128), 0, st, p);
+    const bool many = p.per != ncf && ((ncf + p.per - 1) / p.per + 1) * (p.n_split > 0 ? 2 : 1) > 8;  // parts per unit
+    cudaError_t e2 = rekv_launch_pdl(many ? combine_many_kernel : combine_tc5_kernel,
+                                     dim3((unsigned)merge_units, p.per != ncf ? 2 : 1, 32), dim3(128), 0, st, p);
     if (e2 != cudaSuccess) return e2;
     c->launches += 1;
     if (timed) {
