@@ -1017,9 +1017,9 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
   } else {
     grid = p.total < n_sm ? p.total : n_sm;
     p.per = (int)((p.total + grid - 1) / grid);
-    // a launch of few units (one layer): at least three frames per CTA -- fewer, longer ranges leave the merge kernel
-    // two thirds of the partials and amortise a range's fixed cost (one layer of config 2: 40 against 46 us with two
-    // frames per CTA, 42 with four)
+    // a launch of few units (one layer): at least three frames per CTA -- fewer, longer ranges amortise a range's fixed
+    // cost and leave fewer partials (one layer of config 2: 37 us with two or three frames per CTA, 49 with one, 40
+    // with four)
     if (p.per < 3) p.per = ncf < 3 ? ncf : 3;
     grid = (p.total + p.per - 1) / p.per;
   }
