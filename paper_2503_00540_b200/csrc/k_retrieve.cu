@@ -14,6 +14,10 @@ constexpr int QM_SLICES = 16;
 __global__ void __launch_bounds__(QM_SLICES * 64) qmean_kernel(const __nv_bfloat162* __restrict__ q, QBatch qb, int Hq, int Hkv,
                                                     int G, float* __restrict__ qa, float* __restrict__ qsq,
                                                     int maxQ, int layer0) {
+  // launched with programmatic stream serialisation: its blocks are resident when the kernel before it ends (the
+  // caller's, which wrote the queries, or the library's own), and wait here for that kernel's results
+  rekv_ptx::grid_dep_wait();
+  rekv_ptx::grid_dep_launch();
   const int qi = blockIdx.x, l = layer0 + blockIdx.y, g = blockIdx.z;
   const int Dp = Hkv * 128;
   const int n0 = qb.cu[qi], n1 = qb.cu[qi + 1];
@@ -484,8 +488,11 @@ cudaError_t rekv_launch_retrieve(rekv_ctx* c, const void* q, const QBatch& qb, i
   const StoreView& s = c->sv;
   const int maxQ = c->cfg.max_questions;
   const int nl = layer1 - layer0;
-  qmean_kernel<<<dim3(qb.nQ, nl, s.Hkv), QM_SLICES * 64, 0, st>>>((const __nv_bfloat162*)q, qb, s.Hq, s.Hkv, s.G, c->qa,
-                                                      c->qnorm, maxQ, layer0);
+  {
+    cudaError_t e0 = rekv_launch_pdl(qmean_kernel, dim3(qb.nQ, nl, s.Hkv), dim3(QM_SLICES * 64), 0, st,
+                                     (const __nv_bfloat162*)q, qb, s.Hq, s.Hkv, s.G, c->qa, c->qnorm, maxQ, layer0);
+    if (e0 != cudaSuccess) return e0;
+  }
   int q_group = (int)((96 * 1024) / (s.Dp * sizeof(float)));
   if (q_group > qb.nQ) q_group = qb.nQ;
   size_t smem = (size_t)q_group * s.Dp * sizeof(float);
