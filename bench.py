@@ -615,7 +615,10 @@ def run_cuda(args, w):
                                 "traffic": TRAFFIC_NCU.get(w["name"]), "peak_source": peaks["source"],
                                 "kernel_us": att_kernel_us,
                                 "tensor_tflops": fl / (att_kernel_us * 1e-6) / 1e12,
-                                "tensor_frac": fl / (att_kernel_us * 1e-6) / 1e12 / peaks["bf16_tflops"]}
+                                "tensor_frac": fl / (att_kernel_us * 1e-6) / 1e12 / peaks["bf16_tflops"],
+                                "covers": ("the whole of step 5: when no merge launch follows (stages_us.merge = 0) the "
+                                           "kernel also joins the units cut between CTAs, which are not among the "
+                                           "algorithmic bytes")}
         else:
             link = pinned_h2d_gbs(dev)
             achieved = link_bytes / (q_lat * 1e-6) / 1e9

@@ -117,6 +117,15 @@ def test_units_cut_into_a_few_parts_are_finished_inside_the_kernel():
     g.close()
 
 
+@pytest.mark.parametrize("n_tokens", [40, 10, 1])
+def test_few_units_of_many_parts_each(n_tokens):
+    """Two units (one layer, two KV heads) over 48 context frames: three or four frames per CTA, 13 to 34 partials per
+    unit, joined by the merge kernel for units of many parts -- with two row tiles (40 tokens x 4 heads), as two
+    half-streams (10 tokens) and in the decode-shaped kernel (1 token)."""
+    s = H.Shape(L=1, Hq=8, Hkv=2, Nf=16, T=80, W=8, k=40, seed=7)
+    _run_question_parity(s, [n_tokens])
+
+
 def test_question_in_the_past_sees_only_visible_frames():
     s = H.Shape(L=1, Hq=8, Hkv=2, Nf=16, T=64, W=4, k=8, off_scale=0.0)
     _run_question_parity(s, [16], n_visible=37)
