@@ -109,13 +109,15 @@ typedef struct {
   int32_t last_k_eff;        /* frames actually retrieved per (layer, question) by the last question */
   int32_t last_ctx_frames;   /* k_eff + window frames of the last gather */
   double last_attend_kernel_us; /* device time of the last attention kernel launch (REKV_FLAG_TIMING, HBM
-                                   tier), without the split-KV merge; 0 when not measured */
+                                   tier): it includes the joining of units cut between CTAs when the kernel does
+                                   that itself (two or three parts per unit), not a merge kernel that followed
+                                   (last_merge_us); 0 when not measured */
   double last_retrieve_us;      /* REKV_FLAG_TIMING: steps 2-3 of the last question (question vectors, scores,
                                    selection) on the caller's stream; 0 when not measured or not finished yet */
   double last_pull_us;          /* REKV_FLAG_TIMING, offloaded contexts: the last gather's pulls over the host
                                    link, all layers, on the internal stream; 0 when not measured or not finished */
   double last_merge_us;         /* REKV_FLAG_TIMING: the merge kernel that followed the last attention kernel
-                                   (units cut at CTA boundaries, half-streams); 0 when none ran or not measured */
+                                   (units cut into more than three parts); 0 when none ran or not measured */
 } rekv_stats_t;
 
 /* Creates a context on cfg->device: allocates the frame store (HBM tier, and the pinned-host tier
