@@ -5,33 +5,33 @@ using namespace rekv_ptx;
 
 namespace rekv_att {
 
+// The unit a block of the merge kernels works on, from blockIdx.x.  When units are not cut (per == ncf) only the units
+// with one row tile have partials (their two half-streams): the grid then counts those units only -- blockIdx.x =
+// ((layer, kv head) * n_split + rank among the batch's such questions) -- instead of every unit of a large batch, most
+// of which would have nothing to do.  Returns -1 if there is none.
+__device__ __forceinline__ long long combine_unit(const TcParams& p) {
+  if (p.per != p.ncf) return blockIdx.x;
+  const int rank = (int)(blockIdx.x % p.n_split);
+  const long long lg = blockIdx.x / p.n_split;   // (layer - layer0) * H_kv + kv head
+  int mp = 0, seen = 0;
+  for (int qi = 0; qi < p.qb.nQ; ++qi) {  // the rank-th question whose last unit has one row tile: that unit
+    const int rows = (p.qb.cu[qi + 1] - p.qb.cu[qi]) * p.G;
+    const int units_q = (rows + 255) / 256;
+    if (((rows - 1) & 255) < 128) {
+      if (seen == rank) return lg * p.MP + mp + units_q - 1;
+      ++seen;
+    }
+    mp += units_q;
+  }
+  return -1;
+}
+
 // Merge the partials of the units that were cut by a CTA boundary.
 // grid = (units, 2 row tiles, 32 groups of 4 rows); a warp per row, float4 per lane: one short
 // dependent chain per warp, enough warps in flight to hide its latency.
 __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
-  // When units are not cut (per == ncf) only the units with one row tile have partials (their two half-streams): the
-  // grid then counts those units only -- blockIdx.x = ((layer, kv head) * n_split + rank among the batch's such
-  // questions) -- instead of every unit of a large batch, most of which would have nothing to do.
-  long long u = blockIdx.x;
-  if (p.per == p.ncf) {
-    const int rank = (int)(blockIdx.x % p.n_split);
-    const long long lg = blockIdx.x / p.n_split;   // (layer - layer0) * H_kv + kv head
-    int mp = 0, seen = 0, found = -1;
-    for (int qi = 0; qi < p.qb.nQ; ++qi) {  // the rank-th question whose last unit has one row tile: that unit
-      const int rows = (p.qb.cu[qi + 1] - p.qb.cu[qi]) * p.G;
-      const int units_q = (rows + 255) / 256;
-      if (((rows - 1) & 255) < 128) {
-        if (seen == rank) {
-          found = mp + units_q - 1;
-          break;
-        }
-        ++seen;
-      }
-      mp += units_q;
-    }
-    if (found < 0) return;
-    u = lg * p.MP + found;
-  }
+  const long long u = combine_unit(p);
+  if (u < 0) return;
   const int t = blockIdx.y;
   const long long c_first = (u * p.ncf) / p.per, c_last = ((u + 1) * p.ncf - 1) / p.per;
   const UnitInfo ui = decode_unit(p, u);
@@ -99,29 +99,8 @@ __global__ void __launch_bounds__(128) combine_tc5_kernel(const TcParams p) {
 // The same for units of many parts (a launch of few units, such as one layer, spreads each unit over dozens of CTAs).
 // grid = (units, 2 row tiles, 32 groups of 4 rows), 4 warps, float4 of the 128 columns per lane.
 __global__ void __launch_bounds__(128) combine_many_kernel(const TcParams p) {
-  // When units are not cut (per == ncf) only the units with one row tile have partials (their two half-streams): the
-  // grid then counts those units only -- blockIdx.x = ((layer, kv head) * n_split + rank among the batch's such
-  // questions) -- instead of every unit of a large batch, most of which would have nothing to do.
-  long long u = blockIdx.x;
-  if (p.per == p.ncf) {
-    const int rank = (int)(blockIdx.x % p.n_split);
-    const long long lg = blockIdx.x / p.n_split;   // (layer - layer0) * H_kv + kv head
-    int mp = 0, seen = 0, found = -1;
-    for (int qi = 0; qi < p.qb.nQ; ++qi) {  // the rank-th question whose last unit has one row tile: that unit
-      const int rows = (p.qb.cu[qi + 1] - p.qb.cu[qi]) * p.G;
-      const int units_q = (rows + 255) / 256;
-      if (((rows - 1) & 255) < 128) {
-        if (seen == rank) {
-          found = mp + units_q - 1;
-          break;
-        }
-        ++seen;
-      }
-      mp += units_q;
-    }
-    if (found < 0) return;
-    u = lg * p.MP + found;
-  }
+  const long long u = combine_unit(p);
+  if (u < 0) return;
   const int t = blockIdx.y;
   const long long c_first = (u * p.ncf) / p.per, c_last = ((u + 1) * p.ncf - 1) / p.per;
   const UnitInfo ui = decode_unit(p, u);
