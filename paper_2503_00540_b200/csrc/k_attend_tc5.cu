@@ -304,10 +304,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_
     const int n_parts = (int)(c_last - c_first + 1) * (split ? 2 : 1);
     const int own = (int)(blockIdx.x - c_first) * (split ? 2 : 1) + (split ? t : 0);
     const long long out_row = (ui.q_row0 + (valid ? n : 0)) * p.Hq + ui.g * p.G + (valid ? j : 0);
-    float M = fmaxf(-1e30f, m_own);
-#pragma unroll 1
-    for (int k = 0; k < n_parts; ++k)
-      if (k != own) M = fmaxf(M, __ldcg(p.part_ml + (part_slot(ui, u, c_first, split, rt, k) * 128 + row) * 2));
+    // At most three parts reach this path (the launcher sees to it): the (max, sum) of the one or two other parts
+    // come in one round of loads.
+    const int ka = own == 0 ? 1 : 0, kb = n_parts >= 3 ? (own == 2 ? 1 : 2) : -1;
+    const float2 ml_a = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (part_slot(ui, u, c_first, split, rt, ka) * 128 + row) * 2));
+    float2 ml_b = make_float2(-INFINITY, 0.f);
+    if (kb >= 0)
+      ml_b = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (part_slot(ui, u, c_first, split, rt, kb) * 128 + row) * 2));
+    float M = fmaxf(fmaxf(-1e30f, m_own), fmaxf(ml_a.x, ml_b.x));
     float den = 0.f, w_x = 0.f;
     const float4* o_x = nullptr;
     if (FULL && p.self_o) {
@@ -317,13 +321,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_
       den = w_x * p.self_ml[out_row * 2 + 1];
       o_x = reinterpret_cast<const float4*>(p.self_o + out_row * 128);
     }
-#pragma unroll 1
-    for (int k = 0; k < n_parts; ++k) {
-      float2 ml = make_float2(m_own, l_own);
-      if (k != own)
-        ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (part_slot(ui, u, c_first, split, rt, k) * 128 + row) * 2));
-      den = fmaf(ex2(ml.x - M), ml.y, den);
-    }
+#pragma unroll
+    for (int k = 0; k < 3; ++k)
+      if (k < n_parts) {
+        const float2 ml = k == own ? make_float2(m_own, l_own) : (k == ka ? ml_a : ml_b);
+        den = fmaf(ex2(ml.x - M), ml.y, den);
+      }
     const float inv = den > 0.f ? 1.f / den : 0.f;
     // rows this lane stores: r = 8 k + (lane >> 2), 16 bytes (8 bf16) at chunk (lane & 3) of the quarter
     __nv_bfloat16* dst_k[4];
@@ -359,7 +362,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_
             acc[e] = fmaf(w, own_empty ? 0.f : __uint_as_float(o[e >> 4][e & 15]), acc[e]);
         } else {
           const long long slot = part_slot(ui, u, c_first, split, rt, k);
-          const float w = ex2(__ldcg(p.part_ml + (slot * 128 + row) * 2) - M);
+          const float w = ex2((k == ka ? ml_a.x : ml_b.x) - M);
           const float* po = p.part_o + ((slot * 128 + ((warp & 3) << 5) + (lane >> 3)) * 128 + (lane & 7) * 4) + qd * 32;
           uint4 x[8];
 #pragma unroll
