@@ -336,17 +336,27 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_
       const int n2 = r2 / p.G, j2 = r2 - n2 * p.G;
       dst_k[k] = r2 < ui.rows_q ? p.out + ((ui.q_row0 + n2) * p.Hq + ui.g * p.G + j2) * 128 + (lane & 3) * 8 : nullptr;
     }
+    // The other parts' quarter rows are asked for one step ahead: the loads of the next (quarter, part) are in flight
+    // while the current one is added up and the quarter's output leaves.
+    uint4 x[8];
+#define REKV_ASK(QD, K)                                                                                              \
+  do {                                                                                                               \
+    const float* po_ = p.part_o + ((part_slot(ui, u, c_first, split, rt, (K)) * 128 + ((warp & 3) << 5) + (lane >> 3)) * 128 + \
+                                   (lane & 7) * 4) + (QD) * 32;                                                      \
+    _Pragma("unroll") for (int kk = 0; kk < 8; ++kk) x[kk] = __ldcg(reinterpret_cast<const uint4*>(po_ + (long long)kk * 4 * 128)); \
+  } while (0)
+    REKV_ASK(0, ka);
 #pragma unroll 1
     for (int qd = 0; qd < 4; ++qd) {
       float acc[32];
 #pragma unroll
       for (int v4 = 0; v4 < 8; ++v4) {
-        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (FULL && o_x) x = __ldg(o_x + qd * 8 + v4);
-        acc[4 * v4] = w_x * x.x;
-        acc[4 * v4 + 1] = w_x * x.y;
-        acc[4 * v4 + 2] = w_x * x.z;
-        acc[4 * v4 + 3] = w_x * x.w;
+        float4 y = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (FULL && o_x) y = __ldg(o_x + qd * 8 + v4);
+        acc[4 * v4] = w_x * y.x;
+        acc[4 * v4 + 1] = w_x * y.y;
+        acc[4 * v4 + 2] = w_x * y.z;
+        acc[4 * v4 + 3] = w_x * y.w;
       }
 #pragma unroll 1
       for (int k = 0; k < n_parts; ++k) {
@@ -361,16 +371,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_
           for (int e = 0; e < 32; ++e)
             acc[e] = fmaf(w, own_empty ? 0.f : __uint_as_float(o[e >> 4][e & 15]), acc[e]);
         } else {
-          const long long slot = part_slot(ui, u, c_first, split, rt, k);
           const float w = ex2((k == ka ? ml_a.x : ml_b.x) - M);
-          const float* po = p.part_o + ((slot * 128 + ((warp & 3) << 5) + (lane >> 3)) * 128 + (lane & 7) * 4) + qd * 32;
-          uint4 x[8];
-#pragma unroll
-          for (int kk = 0; kk < 8; ++kk) x[kk] = __ldcg(reinterpret_cast<const uint4*>(po + (long long)kk * 4 * 128));
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk)
             *reinterpret_cast<uint4*>(stage + (4 * kk + (lane >> 3)) * STAGE_ROW_F32 + (lane & 7) * 16) = x[kk];
           __syncwarp();
+          // the next step that reads another part: this quarter's second other part, else the next quarter's first
+          if (k == ka && kb >= 0) {
+            REKV_ASK(qd, kb);
+          } else if (qd < 3) {
+            REKV_ASK(qd + 1, ka);
+          }
 #pragma unroll
           for (int v4 = 0; v4 < 8; ++v4) {
             const float4 y = *reinterpret_cast<const float4*>(stage + lane * STAGE_ROW_F32 + v4 * 16);
@@ -382,6 +393,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_
           __syncwarp();
         }
       }
+#undef REKV_ASK
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         uint4 a, b;
