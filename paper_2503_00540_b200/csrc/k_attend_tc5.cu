@@ -208,6 +208,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_
   // per lane.
   auto merge_listed = [&]() {
     const uint32_t n_pend = min(*s_pend_n, (uint32_t)PEND_MAX);
+    if (n_pend == 0) return;  // (the usual case; the fence below would wait for the output rows just stored)
     __threadfence();
     const int w8 = warp - SM_WARP0;
 #pragma unroll 1
