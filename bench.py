@@ -149,7 +149,7 @@ class ClockSampler:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch from the committed ncu capture
 # (profiles/), scaled to the full workload by the layers processed; None where no capture exists.
-TRAFFIC_NCU = {"7b_hbm_1800f": 848.8e6, "7b_hbm_decode_1tok": 825.0e6}
+TRAFFIC_NCU = {"7b_hbm_1800f": 848.2e6, "7b_hbm_decode_1tok": 825.0e6}
 
 
 def algorithmic_bytes(w, sum_nq=None, nQ=1):
