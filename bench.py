@@ -583,7 +583,7 @@ def run_cuda(args, w):
             "question": {"bytes_per_batch": ab["total"], "gbs": ab["total"] / (q_lat * nQ * 1e-6) / 1e9,
                          "hbm_frac": ab["total"] / (q_lat * nQ * 1e-6) / 1e9 / peaks["hbm_gbs"],
                          "attention_tflops": fl / (q_lat * nQ * 1e-6) / 1e12,
-                         "median_us": q_median, "min_us": q_min,
+                         "median_us": q_median, "min_us": q_min, "per_step_us": [round(x, 1) for x in q_us],
                          "layer_sequential_us": layer_seq_us,
                          "layer_sequential_one_graph_us": layer_seq_one_graph_us,
                          "decode_token_layer_by_layer_us": decode_layers_us,
