@@ -74,6 +74,14 @@ def test_72b_head_shape(theta):
 
 
 @pytest.mark.parametrize("theta", THETAS)
+def test_units_cut_in_two_or_three_are_finished_in_the_kernel_with_the_part_over_x(theta):
+    """80 units of two row tiles over 146 CTAs: every unit is cut into two or three parts, which the CTA that completes
+    the last one joins -- together with the part over X, the first part in the fixed order."""
+    s = H.Shape(L=10, Hq=16, Hkv=8, Nf=100, T=28, W=4, k=16, seed=2503)
+    _run(s, [80], [96], theta)
+
+
+@pytest.mark.parametrize("theta", THETAS)
 def test_many_units_take_the_whole_unit_path(theta):
     """Enough (layer, head, question) units that every unit is produced whole by one CTA."""
     s = H.Shape(L=8, Hq=16, Hkv=8, Nf=64, T=12, W=2, k=4)
