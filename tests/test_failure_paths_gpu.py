@@ -51,6 +51,15 @@ def test_tensor_core_kernel_gives_up_when_a_tile_never_arrives(skip_entry):
     _expire_then_recover(s, [16], skip_entry)
 
 
+def test_a_cta_that_gives_up_leaves_its_units_unfinished_and_their_counters_are_cleared():
+    """80 units of two row tiles, each cut into two or three parts that the attention kernel joins itself by counting
+    the parts per unit.  The first CTA gives up on its first K tile: its parts are never counted, the units it shares
+    stay unfinished behind the status word, and reading the status clears the counters -- the next question would
+    otherwise join the wrong parts."""
+    s = H.Shape(L=10, Hq=16, Hkv=8, Nf=100, T=28, W=4, k=16, seed=2503)
+    _expire_then_recover(s, [80], 0)
+
+
 def test_decode_kernel_gives_up_when_a_frame_never_arrives():
     """One query token (4 rows per KV head): the load-bound decode kernel."""
     s = H.Shape(L=4, Hq=8, Hkv=2, Nf=48, T=60, W=4, k=36, seed=7)
