@@ -26,11 +26,15 @@
 // behind a warp-uniform switch.
 // TMEM (512 columns): O0 [0,128)  O1 [128,256)  S0/P0 [256,384)  S1/P1 [384,512); P (bf16) overwrites
 // the front of its S.
-// A range that does not cover a whole unit leaves (max, sum, O) partials for the combine kernel.
+// A range that does not cover a whole unit produces a part of it, (max, sum, O) per row.  When units have two or
+// three parts the kernel joins them itself: a tile slot that finds every other part of its unit counted finishes the
+// unit from its own O in tensor memory; otherwise it writes its part as a partial and counts it, and the slot whose
+// count completes a unit lists it for the end of the CTA's range (see "Merge inside the kernel" below; nobody waits
+// for anybody).  With more parts per unit the partials are left for the merge kernels.
 // A unit with a single row tile (at most 128 rows: short questions, the remainder of long ones) would leave the
 // tensor core idle during its softmax; it runs as two half-streams instead -- both tile slots work on the same rows,
-// the token chunks of the context dealt to them alternately, each with its own (max, sum, O) -- and the combine
-// kernel joins the two partials like those of any cut unit.
+// the token chunks of the context dealt to them alternately, each with its own (max, sum, O) -- which are joined
+// like the parts of a cut unit.
 // Every wait is bounded: on expiry the status word is set and the CTA leaves.
 #include <algorithm>
 #include <type_traits>
