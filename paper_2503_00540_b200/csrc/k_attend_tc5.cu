@@ -467,7 +467,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) attend_tc5_kernel(const __grid_
         unsigned char* dst = smem + t * Q_TILE_BYTES + row * 128;
         uint4 x[16];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) x[c] = valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+        // (before the dependency wait the rows are read past L1: nothing has invalidated it since an earlier launch
+        // may have read other contents at the same addresses)
+        for (int c = 0; c < 16; ++c) x[c] = valid ? (EARLYQ ? __ldcg(src + c) : __ldg(src + c)) : make_uint4(0, 0, 0, 0);
 #pragma unroll
         for (int c = 0; c < 16; ++c)
           *reinterpret_cast<uint4*>(dst + (c >> 3) * (Q_TILE_BYTES / 2) + (((c & 7) ^ (row & 7)) << 4)) = x[c];
