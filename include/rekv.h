@@ -248,6 +248,21 @@ int rekv_question_layer(rekv_ctx* ctx, int layer, const void* q, const int32_t* 
  * q, out: device bf16 [sum_Nq][H_q][D]; nQ must equal the gathered batch.  Returns 0 or an error code. */
 int rekv_attend_layer(rekv_ctx* ctx, int layer, const void* q, const int32_t* cu_q, int nQ, void* out, void* stream);
 
+/* The two layer calls with Eq. 3 in full -- what a decoder layer calls with the Q, K, V it has just made of X:
+ * rekv_question_layer_full = steps 2-4 of the layer as in rekv_question_layer, then step 5 over [R, X] as in
+ * rekv_attend_full; rekv_attend_full_layer = that step 5 alone over the layer's existing context (decode steps).
+ *   q               device bf16 [sum_Nq][H_q][D] of this layer
+ *   k_self, v_self  device bf16 [sum_Ns][H_kv][D] of this layer; cu_q, cu_self as in rekv_attend_full
+ *   idx_out, out    as in rekv_question_layer
+ * Positions under rope_theta > 0, the static variant, the validity of a layer's context and the error codes are those
+ * of rekv_attend_full and rekv_question_layer.  Needs max_self_tokens > 0 at creation.  Returns the number of context
+ * frames (rekv_question_layer_full) or 0 (rekv_attend_full_layer), or an error code. */
+int rekv_question_layer_full(rekv_ctx* ctx, int layer, const void* q, const void* k_self, const void* v_self,
+                             const int32_t* cu_q, const int32_t* cu_self, int nQ, int top_k, int n_visible,
+                             int32_t* idx_out, void* out, void* stream);
+int rekv_attend_full_layer(rekv_ctx* ctx, int layer, const void* q, const void* k_self, const void* v_self,
+                           const int32_t* cu_q, const int32_t* cu_self, int nQ, void* out, void* stream);
+
 /* Disk tier.  rekv_save synchronises the device and writes the context's stream state -- configuration, frame
  * count, representatives, frame embeddings, every page (host tier as it is held, plus the exact frames of the HBM
  * tail) -- to `path`.  rekv_load creates a context on `device` from such a file, ready for further appends and

@@ -63,8 +63,8 @@ __device__ __forceinline__ int find_question(const QBatch& qb, int n) {
 // each half per thread
 __global__ void __launch_bounds__(256) rope_q_kernel(const uint4* __restrict__ q, uint4* __restrict__ q_rot, QBatch qb,
                                                      QBatch sb, int Hq, int n_ctx_tokens,
-                                                     const float2* __restrict__ tab) {
-  const int l = blockIdx.y;
+                                                     const float2* __restrict__ tab, int layer0) {
+  const int l = layer0 + blockIdx.y;
   const int row = blockIdx.x * 32 + (threadIdx.x >> 3), c = threadIdx.x & 7;
   if (row >= qb.sumNq * Hq) return;
   const int n = row / Hq;
@@ -83,9 +83,9 @@ __global__ void __launch_bounds__(256) rope_q_kernel(const uint4* __restrict__ q
 // (i, i + 64) sits at the same swizzled offset of the two halves, so a thread moves one chunk of each.
 __global__ void __launch_bounds__(256) rope_stage_kernel(char* const* __restrict__ tbl, char** __restrict__ tbl_k,
                                                          char* __restrict__ k_rot, int nQ, int ncf, int Hkv, int Nf,
-                                                         const float2* __restrict__ tab) {
+                                                         const float2* __restrict__ tab, int layer0) {
   grid_dep_wait();
-  const int slot = blockIdx.x, qi = blockIdx.y, l = blockIdx.z;
+  const int slot = blockIdx.x, qi = blockIdx.y, l = layer0 + blockIdx.z;
   const long long e = ((long long)l * nQ + qi) * ncf + slot;
   const char* page = tbl[e];
   const long long half_bytes = (long long)Nf * 128;
@@ -133,10 +133,11 @@ __global__ void __launch_bounds__(256) self_attend_kernel(const __nv_bfloat16* _
                                                           const __nv_bfloat16* __restrict__ v_self, QBatch qb, QBatch sb,
                                                           int Hq, int Hkv, int G, int n_ctx_tokens,
                                                           const float2* __restrict__ tab, float scale_log2,
-                                                          float* __restrict__ self_o, float* __restrict__ self_ml) {
+                                                          float* __restrict__ self_o, float* __restrict__ self_ml,
+                                                          int layer0) {
   __shared__ __align__(128) unsigned char s_kv[2 * 2 * SELF_TILE * 128];  // K tile, V tile
   const int rb = blockIdx.x, h = blockIdx.y;
-  const int l = blockIdx.z / qb.nQ, qi = blockIdx.z - l * qb.nQ;
+  const int l = layer0 + blockIdx.z / qb.nQ, qi = blockIdx.z % qb.nQ;
   const int g = h / G;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int q0 = qb.cu[qi], nq = qb.cu[qi + 1] - q0;
@@ -294,10 +295,11 @@ __global__ void __launch_bounds__(256) self_attend_kernel(const __nv_bfloat16* _
 // No retrieved context at all (nothing visible but X): the output is the normalised self part.
 __global__ void __launch_bounds__(256) self_finalize_kernel(const float* __restrict__ self_o,
                                                             const float* __restrict__ self_ml,
-                                                            __nv_bfloat16* __restrict__ out, long long rows) {
-  const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+                                                            __nv_bfloat16* __restrict__ out, long long row0,
+                                                            long long rows) {
+  const long long row = row0 + (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  if (row >= rows) return;
+  if (row >= row0 + rows) return;
   const float l = self_ml[row * 2 + 1];
   const float inv = l > 0.f ? 1.f / l : 0.f;
   const float4 o = *reinterpret_cast<const float4*>(self_o + row * 128 + lane * 4);
@@ -319,8 +321,12 @@ cudaError_t rekv_launch_rope_table(rekv_ctx* c, cudaStream_t st) {
 // embedding) and the partial over the tokens of X.  q_eff receives the query pointer the attention
 // kernel must read.
 cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const void* k_self, const void* v_self,
-                                            const QBatch& qb, const QBatch& sb, int ncf, cudaStream_t st) {
+                                            const QBatch& qb, const QBatch& sb, int ncf, cudaStream_t st,
+                                            int layer0, int layer1) {
+  // layers [layer0, layer1): q, k_self, v_self are indexed with the absolute layer (a caller that holds one layer's
+  // rows passes pointers moved back by layer0 layers), as the library's own buffers are
   const StoreView& s = c->sv;
+  const int nl = layer1 - layer0;
   const bool rope = c->cfg.rope_theta > 0.f;
   // positions: context token j at j and token s of X at n_ctx + s; with REKV_FLAG_ROPE_STATIC every context token
   // at 0 -- its rotation is the identity, the stored keys are used as they are -- and token s of X at 1 + s
@@ -328,8 +334,9 @@ cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const vo
   const int n_ctx_tokens = static_ctx ? 1 : ncf * s.Nf;   // position of X's first token
   const __nv_bfloat16* q_eff = (const __nv_bfloat16*)q;
   if (rope) {
-    dim3 grid((qb.sumNq * s.Hq + 31) / 32, s.L);
-    rope_q_kernel<<<grid, 256, 0, st>>>((const uint4*)q, (uint4*)c->q_rot, qb, sb, s.Hq, n_ctx_tokens, c->rope_tab);
+    dim3 grid((qb.sumNq * s.Hq + 31) / 32, nl);
+    rope_q_kernel<<<grid, 256, 0, st>>>((const uint4*)q, (uint4*)c->q_rot, qb, sb, s.Hq, n_ctx_tokens, c->rope_tab,
+                                        layer0);
     c->launches += 1;
     q_eff = c->q_rot;
   }
@@ -344,23 +351,25 @@ cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const vo
   }
   int max_nq = 1;
   for (int i = 0; i < qb.nQ; ++i) max_nq = std::max(max_nq, qb.cu[i + 1] - qb.cu[i]);
-  self_attend_kernel<<<dim3((max_nq + 127) / 128, s.Hq, s.L * qb.nQ), 256, 0, st_self>>>(
+  self_attend_kernel<<<dim3((max_nq + 127) / 128, s.Hq, nl * qb.nQ), 256, 0, st_self>>>(
       q_eff, (const __nv_bfloat16*)k_self, (const __nv_bfloat16*)v_self, qb, sb, s.Hq, s.Hkv, s.G, n_ctx_tokens,
-      rope ? c->rope_tab : nullptr, 1.4426950408889634f / sqrtf(128.f), c->self_o, c->self_ml);
+      rope ? c->rope_tab : nullptr, 1.4426950408889634f / sqrtf(128.f), c->self_o, c->self_ml, layer0);
   c->launches += 1;
   if (fork) {
     if ((e = cudaEventRecord(c->ev_side, c->side)) != cudaSuccess) return e;
-    rope_stage_kernel<<<dim3(ncf, qb.nQ, s.L), 256, 0, st>>>(c->ctx_tbl, c->tbl_k, c->k_rot, qb.nQ, ncf, s.Hkv, s.Nf,
-                                                             c->rope_tab);
+    rope_stage_kernel<<<dim3(ncf, qb.nQ, nl), 256, 0, st>>>(c->ctx_tbl, c->tbl_k, c->k_rot, qb.nQ, ncf, s.Hkv, s.Nf,
+                                                            c->rope_tab, layer0);
     c->launches += 1;
     if ((e = cudaStreamWaitEvent(st, c->ev_side, 0)) != cudaSuccess) return e;
   }
   return cudaGetLastError();
 }
 
-cudaError_t rekv_launch_self_finalize(rekv_ctx* c, const QBatch& qb, void* out, cudaStream_t st) {
-  const long long rows = (long long)c->sv.L * qb.sumNq * c->sv.Hq;
-  self_finalize_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(c->self_o, c->self_ml, (__nv_bfloat16*)out, rows);
+cudaError_t rekv_launch_self_finalize(rekv_ctx* c, const QBatch& qb, void* out, cudaStream_t st, int layer0,
+                                      int layer1) {
+  const long long per_layer = (long long)qb.sumNq * c->sv.Hq, rows = (layer1 - layer0) * per_layer;
+  self_finalize_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(c->self_o, c->self_ml, (__nv_bfloat16*)out,
+                                                                   layer0 * per_layer, rows);
   c->launches += 1;
   return cudaGetLastError();
 }

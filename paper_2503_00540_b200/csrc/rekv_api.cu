@@ -511,8 +511,16 @@ int rekv_question(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, int t
   return rc < 0 ? rc : geom.ncf;
 }
 
-int rekv_question_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu_q, int nQ, int top_k, int n_visible,
-                        int32_t* idx_out, void* out, void* stream) {
+namespace {
+int attend_full_range(rekv_ctx* c, int layer0, int layer1, const void* q, const void* k_self, const void* v_self,
+                      const QBatch& qb, const QBatch& sb, void* out, cudaStream_t st);
+int build_self_batch(rekv_ctx* c, const QBatch& qb, const int32_t* cu_self, int nQ, QBatch* sb);
+}  // namespace
+
+// steps 2-5 of one layer; with k_self != null step 5 is Eq. 3 in full (the questions' own K/V after the context)
+static int question_layer_impl(rekv_ctx* c, int layer, const void* q, const void* k_self, const void* v_self,
+                               const int32_t* cu_q, const int32_t* cu_self, int nQ, int top_k, int n_visible,
+                               int32_t* idx_out, void* out, void* stream) {
   if (!c) return REKV_ERR_ARG;
   if (!q || !out) REKV_FAIL(c, REKV_ERR_ARG, "null q or out");
   if (layer < 0 || layer >= c->sv.L) REKV_FAIL(c, REKV_ERR_ARG, "layer=%d outside [0, %d)", layer, c->sv.L);
@@ -522,9 +530,13 @@ int rekv_question_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu
   if (n_visible == 0) REKV_FAIL(c, REKV_ERR_EMPTY, "no visible frame");
   if (top_k % c->cfg.block_frames)
     REKV_FAIL(c, REKV_ERR_ARG, "top_k=%d must be a multiple of block_frames=%d", top_k, c->cfg.block_frames);
-  QBatch qb;
+  QBatch qb, sb;
   int rc = build_qbatch(c, cu_q, nQ, &qb);
   if (rc) return rc;
+  if (k_self) {
+    rc = build_self_batch(c, qb, cu_self, nQ, &sb);
+    if (rc) return rc;
+  }
   DeviceGuard guard(c->device);
   cudaStream_t st = (cudaStream_t)stream;
   const StoreView& s = c->sv;
@@ -558,10 +570,31 @@ int rekv_question_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu
   c->g_keff = geom.k_eff;
   c->g_nvis = n_visible;
   c->g_topk = top_k;
+  if (k_self) {
+    const long long kv_layer = (long long)sb.sumNq * s.Hkv * REKV_HEAD_DIM * 2;
+    rc = attend_full_range(c, layer, layer + 1, layer_view(q, layer, qb.sumNq * row_bytes),
+                           layer_view(k_self, layer, kv_layer), layer_view(v_self, layer, kv_layer), qb, sb,
+                           layer_view(out, layer, qb.sumNq * row_bytes), st);
+    return rc ? rc : geom.ncf;
+  }
   c->q_early_ok = fused_table;  // the selection kernel, which only reads Q, is directly before the attention
   rc = attend_one_layer(c, layer, q, qb, out, st);
   c->q_early_ok = false;
   return rc ? rc : geom.ncf;
+}
+
+int rekv_question_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu_q, int nQ, int top_k, int n_visible,
+                        int32_t* idx_out, void* out, void* stream) {
+  return question_layer_impl(c, layer, q, nullptr, nullptr, cu_q, nullptr, nQ, top_k, n_visible, idx_out, out, stream);
+}
+
+int rekv_question_layer_full(rekv_ctx* c, int layer, const void* q, const void* k_self, const void* v_self,
+                             const int32_t* cu_q, const int32_t* cu_self, int nQ, int top_k, int n_visible,
+                             int32_t* idx_out, void* out, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (!k_self || !v_self) REKV_FAIL(c, REKV_ERR_ARG, "null k_self or v_self");
+  if (c->cfg.max_self_tokens <= 0) REKV_FAIL(c, REKV_ERR_STATE, "the context was created with max_self_tokens == 0");
+  return question_layer_impl(c, layer, q, k_self, v_self, cu_q, cu_self, nQ, top_k, n_visible, idx_out, out, stream);
 }
 
 int rekv_attend_layer(rekv_ctx* c, int layer, const void* q, const int32_t* cu_q, int nQ, void* out, void* stream) {
@@ -617,6 +650,52 @@ int rekv_retrieve_external(rekv_ctx* c, const float* q_emb, int nQ, int top_k, i
   return geom.k_eff;
 }
 
+namespace {
+
+// the batch's own K/V lengths, checked against the query lengths and the context's capacity
+int build_self_batch(rekv_ctx* c, const QBatch& qb, const int32_t* cu_self, int nQ, QBatch* sb) {
+  if (!cu_self || cu_self[0] != 0) REKV_FAIL(c, REKV_ERR_ARG, "cu_self must start at 0");
+  sb->nQ = nQ;
+  for (int i = 0; i <= nQ; ++i) sb->cu[i] = cu_self[i];
+  sb->sumNq = cu_self[nQ];
+  for (int i = 0; i < nQ; ++i)
+    if (sb->cu[i + 1] - sb->cu[i] < qb.cu[i + 1] - qb.cu[i])
+      REKV_FAIL(c, REKV_ERR_ARG, "question %d: %d tokens of its own K/V for %d query rows", i, sb->cu[i + 1] - sb->cu[i],
+                qb.cu[i + 1] - qb.cu[i]);
+  if (sb->sumNq > c->cfg.max_self_tokens)
+    REKV_FAIL(c, REKV_ERR_ARG, "%d tokens of own K/V exceed max_self_tokens=%d", sb->sumNq, c->cfg.max_self_tokens);
+  return REKV_OK;
+}
+
+// Eq. 3 in full for layers [layer0, layer1).  q, k_self, v_self and out are indexed with the absolute layer: a caller
+// that holds one layer's rows passes pointers moved back by layer0 layers (layer_view).
+int attend_full_range(rekv_ctx* c, int layer0, int layer1, const void* q, const void* k_self, const void* v_self,
+                      const QBatch& qb, const QBatch& sb, void* out, cudaStream_t st) {
+  // an offloaded context: the range's pages must have arrived before the keys are rotated
+  if (c->gather_layerwise) REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[layer1 - 1], 0));
+  REKV_CUDA(c, rekv_launch_attend_full_prepare(c, q, k_self, v_self, qb, sb, c->g_ncf, st, layer0, layer1));
+  const bool rope = c->cfg.rope_theta > 0.f && !(c->cfg.flags & REKV_FLAG_ROPE_STATIC);  // rotated copies of the context's keys
+  const bool rope_q = c->cfg.rope_theta > 0.f;
+  if (c->g_ncf == 0) {
+    REKV_CUDA(c, rekv_launch_self_finalize(c, qb, out, st, layer0, layer1));
+  } else {
+    AttendFullArgs fa;
+    fa.tbl_k = rope ? c->tbl_k : nullptr;
+    fa.self_o = c->self_o;
+    fa.self_ml = c->self_ml;
+    REKV_CUDA(c, rekv_launch_attend_tc5(c, rope_q ? (const void*)c->q_rot : q, qb, c->g_ncf, layer0, layer1, out, st,
+                                        (c->cfg.flags & REKV_FLAG_TIMING) != 0 && layer1 - layer0 == c->sv.L, &fa));
+  }
+  if (c->gather_layerwise || (c->sv.tail > 0 && layer1 - layer0 < c->sv.L)) {
+    // later appends (ring slots) and gathers (staging) on the side stream must not overtake this read
+    REKV_CUDA(c, cudaEventRecord(c->ev_side, st));
+    REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_side, 0));
+  }
+  return REKV_OK;
+}
+
+}  // namespace
+
 int rekv_attend_full(rekv_ctx* c, const void* q, const void* k_self, const void* v_self, const int32_t* cu_q,
                      const int32_t* cu_self, int nQ, void* out, void* stream) {
   if (!c) return REKV_ERR_ARG;
@@ -630,39 +709,34 @@ int rekv_attend_full(rekv_ctx* c, const void* q, const void* k_self, const void*
   QBatch qb, sb;
   int rc = build_qbatch(c, cu_q, nQ, &qb);
   if (rc) return rc;
-  if (!cu_self || cu_self[0] != 0) REKV_FAIL(c, REKV_ERR_ARG, "cu_self must start at 0");
-  sb.nQ = nQ;
-  for (int i = 0; i <= nQ; ++i) sb.cu[i] = cu_self[i];
-  sb.sumNq = cu_self[nQ];
-  for (int i = 0; i < nQ; ++i)
-    if (sb.cu[i + 1] - sb.cu[i] < qb.cu[i + 1] - qb.cu[i])
-      REKV_FAIL(c, REKV_ERR_ARG, "question %d: %d tokens of its own K/V for %d query rows", i, sb.cu[i + 1] - sb.cu[i],
-                qb.cu[i + 1] - qb.cu[i]);
-  if (sb.sumNq > c->cfg.max_self_tokens)
-    REKV_FAIL(c, REKV_ERR_ARG, "%d tokens of own K/V exceed max_self_tokens=%d", sb.sumNq, c->cfg.max_self_tokens);
+  rc = build_self_batch(c, qb, cu_self, nQ, &sb);
+  if (rc) return rc;
   DeviceGuard guard(c->device);
-  cudaStream_t st = (cudaStream_t)stream;
+  return attend_full_range(c, 0, c->sv.L, q, k_self, v_self, qb, sb, out, (cudaStream_t)stream);
+}
+
+int rekv_attend_full_layer(rekv_ctx* c, int layer, const void* q, const void* k_self, const void* v_self,
+                           const int32_t* cu_q, const int32_t* cu_self, int nQ, void* out, void* stream) {
+  if (!c) return REKV_ERR_ARG;
+  if (!q || !k_self || !v_self || !out) REKV_FAIL(c, REKV_ERR_ARG, "null q, k_self, v_self or out");
+  if (layer < 0 || layer >= c->sv.L) REKV_FAIL(c, REKV_ERR_ARG, "layer=%d outside [0, %d)", layer, c->sv.L);
+  if (c->cfg.max_self_tokens <= 0) REKV_FAIL(c, REKV_ERR_STATE, "the context was created with max_self_tokens == 0");
+  if (!c->gathered || !c->layer_ctx_valid[layer])
+    REKV_FAIL(c, REKV_ERR_STATE, "rekv_attend_full_layer needs a preceding gather of the layer (with the geometry of "
+                                 "the latest gather)");
+  if (nQ != c->g_nQ) REKV_FAIL(c, REKV_ERR_STATE, "nQ=%d differs from the gathered batch (%d)", nQ, c->g_nQ);
+  QBatch qb, sb;
+  int rc = build_qbatch(c, cu_q, nQ, &qb);
+  if (rc) return rc;
+  rc = build_self_batch(c, qb, cu_self, nQ, &sb);
+  if (rc) return rc;
+  DeviceGuard guard(c->device);
   const StoreView& s = c->sv;
-  // an offloaded context: every layer's pages must have arrived before the keys are rotated
-  if (c->gather_layerwise) REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[s.L - 1], 0));
-  REKV_CUDA(c, rekv_launch_attend_full_prepare(c, q, k_self, v_self, qb, sb, c->g_ncf, st));
-  const bool rope = c->cfg.rope_theta > 0.f && !(c->cfg.flags & REKV_FLAG_ROPE_STATIC);  // rotated copies of the context's keys
-  const bool rope_q = c->cfg.rope_theta > 0.f;
-  if (c->g_ncf == 0) {
-    REKV_CUDA(c, rekv_launch_self_finalize(c, qb, out, st));
-  } else {
-    AttendFullArgs fa;
-    fa.tbl_k = rope ? c->tbl_k : nullptr;
-    fa.self_o = c->self_o;
-    fa.self_ml = c->self_ml;
-    REKV_CUDA(c, rekv_launch_attend_tc5(c, rope_q ? (const void*)c->q_rot : q, qb, c->g_ncf, 0, s.L, out, st,
-                                        (c->cfg.flags & REKV_FLAG_TIMING) != 0, &fa));
-  }
-  if (c->gather_layerwise) {
-    REKV_CUDA(c, cudaEventRecord(c->ev_side, st));
-    REKV_CUDA(c, cudaStreamWaitEvent(c->side, c->ev_side, 0));
-  }
-  return REKV_OK;
+  const long long q_layer = (long long)qb.sumNq * s.Hq * REKV_HEAD_DIM * 2;
+  const long long kv_layer = (long long)sb.sumNq * s.Hkv * REKV_HEAD_DIM * 2;
+  return attend_full_range(c, layer, layer + 1, layer_view(q, layer, q_layer), layer_view(k_self, layer, kv_layer),
+                           layer_view(v_self, layer, kv_layer), qb, sb, layer_view(out, layer, q_layer),
+                           (cudaStream_t)stream);
 }
 
 int rekv_geometry(rekv_ctx* c, int n_visible, int top_k, int32_t* n_scored, int32_t* k_eff, int32_t* w_eff) {

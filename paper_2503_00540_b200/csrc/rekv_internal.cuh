@@ -253,5 +253,7 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
 // k_attend_full.cu: the pieces of Eq. 3 in full around the attention kernel
 cudaError_t rekv_launch_rope_table(rekv_ctx* c, cudaStream_t st);
 cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const void* k_self, const void* v_self,
-                                            const QBatch& qb, const QBatch& sb, int ncf, cudaStream_t st);
-cudaError_t rekv_launch_self_finalize(rekv_ctx* c, const QBatch& qb, void* out, cudaStream_t st);
+                                            const QBatch& qb, const QBatch& sb, int ncf, cudaStream_t st, int layer0,
+                                            int layer1);
+cudaError_t rekv_launch_self_finalize(rekv_ctx* c, const QBatch& qb, void* out, cudaStream_t st, int layer0,
+                                      int layer1);

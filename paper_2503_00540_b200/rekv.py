@@ -46,6 +46,7 @@ class rekv_stats_t(ctypes.Structure):
 EXPORTS = ("rekv_create", "rekv_destroy", "rekv_append_frame", "rekv_retrieve", "rekv_gather", "rekv_attend",
            "rekv_stats", "rekv_check_status", "rekv_last_error", "rekv_get_reps", "rekv_get_page",
            "rekv_launch_count", "rekv_score_frames_static", "rekv_question_layer", "rekv_attend_layer", "rekv_attend_full",
+           "rekv_question_layer_full", "rekv_attend_full_layer",
            "rekv_set_frame_embedding", "rekv_retrieve_external", "rekv_question",
            "rekv_save", "rekv_load", "rekv_set_timing", "rekv_geometry",
            "rekv_test_set_wait_limit")
@@ -76,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.rekv_load.argtypes = [ctypes.c_char_p, i32, ctypes.POINTER(vp)]
         L.rekv_attend_layer.argtypes = [vp, i32, vp, ip, i32, vp, vp]
         L.rekv_attend_full.argtypes = [vp, vp, vp, vp, ip, ip, i32, vp, vp]
+        L.rekv_question_layer_full.argtypes = [vp, i32, vp, vp, vp, ip, ip, i32, i32, i32, vp, vp, vp]
+        L.rekv_attend_full_layer.argtypes = [vp, i32, vp, vp, vp, ip, ip, i32, vp, vp]
         L.rekv_set_frame_embedding.argtypes = [vp, i32, vp, vp]
         L.rekv_retrieve_external.argtypes = [vp, vp, i32, i32, i32, ctypes.c_float, vp, vp, vp]
         L.rekv_stats.argtypes = [vp, ctypes.POINTER(rekv_stats_t)]
@@ -292,6 +295,41 @@ class ReKV:
                                               n_visible, _ptr(idx, torch.int32), _ptr(out, torch.bfloat16),
                                               self._stream()))
         return out
+
+    def question_layer_full(self, layer: int, q: torch.Tensor, k_self: torch.Tensor, v_self: torch.Tensor,
+                            cu_q: Sequence[int], cu_self: Sequence[int], top_k: int, n_visible: int,
+                            out: Optional[torch.Tensor] = None, idx: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """retrieve -> gather of one layer, then Eq. 3 in full over [R, X].  q: bf16 [sum_Nq][H_q][D];
+        k_self, v_self: bf16 [sum_Ns][H_kv][D], all of this layer -> bf16 like q."""
+        nQ = len(cu_q) - 1
+        self._check_layer_full_shapes(q, k_self, v_self, cu_q, cu_self)
+        if idx is not None and tuple(idx.shape) != (nQ, top_k):
+            raise ValueError("idx must be [nQ][top_k]")
+        if out is None:
+            out = torch.empty_like(q)
+        self._check(lib().rekv_question_layer_full(self._h, layer, _ptr(q, torch.bfloat16), _ptr(k_self, torch.bfloat16),
+                                                   _ptr(v_self, torch.bfloat16), _cu_array(cu_q), _cu_array(cu_self),
+                                                   nQ, top_k, n_visible, _ptr(idx, torch.int32),
+                                                   _ptr(out, torch.bfloat16), self._stream()))
+        return out
+
+    def attend_full_layer(self, layer: int, q: torch.Tensor, k_self: torch.Tensor, v_self: torch.Tensor,
+                          cu_q: Sequence[int], cu_self: Sequence[int],
+                          out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Eq. 3 in full of one layer over the context its last question_layer(_full) (or gather) built."""
+        self._check_layer_full_shapes(q, k_self, v_self, cu_q, cu_self)
+        if out is None:
+            out = torch.empty_like(q)
+        self._check(lib().rekv_attend_full_layer(self._h, layer, _ptr(q, torch.bfloat16), _ptr(k_self, torch.bfloat16),
+                                                 _ptr(v_self, torch.bfloat16), _cu_array(cu_q), _cu_array(cu_self),
+                                                 len(cu_q) - 1, _ptr(out, torch.bfloat16), self._stream()))
+        return out
+
+    def _check_layer_full_shapes(self, q, k_self, v_self, cu_q, cu_self):
+        if tuple(q.shape) != (cu_q[-1], self.Hq, self.D):
+            raise ValueError("q must be [sum_Nq][H_q][D]")
+        if tuple(k_self.shape) != (cu_self[-1], self.Hkv, self.D) or k_self.shape != v_self.shape:
+            raise ValueError("k_self and v_self must be [sum_Ns][H_kv][D]")
 
     def attend_layer(self, layer: int, q: torch.Tensor, cu_q: Sequence[int],
                      out: Optional[torch.Tensor] = None) -> torch.Tensor:

@@ -181,3 +181,48 @@ def test_static_position_variant():
     _run(H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=40, W=8, k=12), [32], [32], 1e6, static_ctx=True)
     _run(H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=30, W=4, k=6, seed=540), [24, 64, 1, 5], [24, 80, 37, 9], 1e6, static_ctx=True)
     _run(H.Shape(L=2, Hq=28, Hkv=4, Nf=196, T=24, W=4, k=8, seed=7), [1, 1], [150, 65], 1e6, static_ctx=True)
+
+
+@pytest.mark.parametrize("theta", THETAS)
+@pytest.mark.parametrize("tail", [0, 8])
+def test_layer_calls_of_eq3_in_full(theta, tail):
+    """What a decoder layer calls with the Q, K, V it has just made of X: rekv_question_layer_full per layer (steps 2-5
+    with Eq. 3 in full), then decode steps through rekv_attend_full_layer over the layer's context -- against the
+    oracle per layer, and against the all-layer calls on the same selection."""
+    s = H.Shape(L=3, Hq=28, Hkv=4, Nf=196, T=40, W=4, k=8, seed=540, tail=tail)
+    nq, ns = [24, 33], [24, 40]
+    g = H.build_gpu(s, max_questions=2, max_q_tokens=sum(nq), max_self_tokens=sum(ns) + 2, rope_theta=theta)
+    o = H.build_oracle(s)
+    q, cu = H.questions(s, nq, device="cuda")
+    ks, vs, cus = H.self_kv(s, ns, device="cuda")
+    out = torch.empty_like(q)
+    idx = torch.zeros((s.L, 2, s.k), dtype=torch.int32, device="cuda")
+    for l in range(s.L):
+        g.question_layer_full(l, q[l], ks[l], vs[l], cu, cus, s.k, s.T, out=out[l], idx=idx[l])
+    g.check_status()
+    q_cpu, ks_cpu, vs_cpu = q.cpu(), ks.cpu(), vs.cpu()
+    refs = [o.question(q_cpu[:, cu[i]:cu[i + 1]].contiguous(), s.k, s.T) for i in range(2)]
+    for i in range(2):
+        for l in range(s.L):
+            if not torch.equal(idx[l, i].cpu(), refs[i]["idx"][l]):
+                continue  # (a near-tie: another selection is as correct; the all-layer comparison below still holds)
+            ref, _ = orc.attend_full(q_cpu[l, cu[i]:cu[i + 1]].contiguous(), refs[i]["k_ctx"][l].contiguous(),
+                                     refs[i]["v_ctx"][l].contiguous(), ks_cpu[l, cus[i]:cus[i + 1]].contiguous(),
+                                     vs_cpu[l, cus[i]:cus[i + 1]].contiguous(), theta)
+            H.assert_attention(out[l:l + 1, cu[i]:cu[i + 1]], ref[None], f"layer call of Eq. 3 in full, layer {l} question {i}")
+    # decode steps: one more token of X per question, over the same contexts, layer by layer
+    qd, cud = H.questions(s, [1, 1], device="cuda", first_id=11)
+    ks2, vs2, cus2 = H.self_kv(s, [ns[0] + 1, ns[1] + 1], device="cuda")
+    outd = torch.empty_like(qd)
+    for l in range(s.L):
+        g.attend_full_layer(l, qd[l], ks2[l], vs2[l], cud, cus2, out=outd[l])
+    g.check_status()
+    # the all-layer calls on the same selection give the same rows (other launch shapes: close, not bit-equal)
+    g.gather(idx, 2, s.k, s.T)
+    all_prefill = g.attend_full(q, ks, vs, cu, cus)
+    all_decode = g.attend_full(qd, ks2, vs2, cud, cus2)
+    g.check_status()
+    for a, b, what in ((out, all_prefill, "prefill"), (outd, all_decode, "decode")):
+        d = (a.float() - b.float()).abs()
+        assert d.max().item() <= 4e-3 and d.mean().item() <= 2e-4, f"layer calls vs all-layer calls, {what}: {d.max().item()}"
+    g.close()
