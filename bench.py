@@ -489,7 +489,11 @@ def run_cuda(args, w):
     # work between layers), offloaded caches issue the calls eagerly (their side stream is not capturable)
     q_l = qs[0].clone()
     layer_calls = []
-    if w["tail"] == 0:
+    if w.get("full"):  # Eq. 3 in full, layer by layer: the decoder layer's call with its own Q, K, V (eager calls)
+        for l in range(w["L"]):
+            layer_calls.append(lambda l=l: g.question_layer_full(l, q_l[l], ks_self[l], vs_self[l], cu, cu, w["k"],
+                                                                 n_vis, out=out[l]))
+    elif w["tail"] == 0:
         cap = torch.cuda.Stream(dev)
         cap.wait_stream(stream)
         with torch.cuda.stream(cap):
@@ -501,7 +505,7 @@ def run_cuda(args, w):
             # the same 28 calls as consecutive nodes of ONE graph: what a decoder captured whole (its own
             # kernels between the layers) pays for the path, without a graph launch per layer
             gr_all = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gr_all, stream=cap):
+            with torch.cuda.graph(gr_all, stream=cap):  # (used below for workloads without Eq. 3 in full)
                 for l in range(w["L"]):
                     g.question_layer(l, q_l[l], cu, w["k"], n_vis, out=out[l])
         stream.wait_stream(cap)
@@ -546,7 +550,7 @@ def run_cuda(args, w):
         ev_r[1].record(stream)
         torch.cuda.synchronize()
         decode_layers_us = ev_r[0].elapsed_time(ev_r[1]) * 1e3 / 20
-    if w["tail"] == 0:
+    if w["tail"] == 0 and not w.get("full"):
         for i in range(2 + n_seq):
             if i == 2:
                 torch.cuda.synchronize()
@@ -587,7 +591,8 @@ def run_cuda(args, w):
                          "layer_sequential_us": layer_seq_us,
                          "layer_sequential_one_graph_us": layer_seq_one_graph_us,
                          "decode_token_layer_by_layer_us": decode_layers_us,
-                         "layer_sequential_mode": ("one CUDA graph replay per layer" if w["tail"] == 0
+                         "layer_sequential_mode": ("one eager rekv_question_layer_full call per layer" if w.get("full")
+                                                   else "one CUDA graph replay per layer" if w["tail"] == 0
                                                    else "one eager call per layer"),
                          "retrieve_us_per_batch": retrieve_us,
                          "frames_scored_per_s_all_gpus": (world * (1 if w.get("ext_dim") else w["L"]) * n_vis * nQ
