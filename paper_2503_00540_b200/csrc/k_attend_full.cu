@@ -317,14 +317,15 @@ cudaError_t rekv_launch_rope_table(rekv_ctx* c, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-// Everything the attention kernel needs for Eq. 3 in full: rotated queries and K copies (with rotary
-// embedding) and the partial over the tokens of X.  q_eff receives the query pointer the attention
-// kernel must read.
-cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const void* k_self, const void* v_self,
-                                            const QBatch& qb, const QBatch& sb, int ncf, cudaStream_t st,
-                                            int layer0, int layer1) {
-  // layers [layer0, layer1): q, k_self, v_self are indexed with the absolute layer (a caller that holds one layer's
-  // rows passes pointers moved back by layer0 layers), as the library's own buffers are
+// What the attention kernel needs for Eq. 3 in full, in two halves.
+// First half, independent of the retrieval: rotated queries (with rotary embedding) and the partial over the tokens
+// of X.  Layers [layer0, layer1): q, k_self, v_self are indexed with the absolute layer (a caller that holds one
+// layer's rows passes pointers moved back by layer0 layers), as the library's own buffers are.  The part over X
+// (latency-bound) goes to the internal stream when something runs beside it on the caller's: the pass over the
+// context's keys (consecutive positions), or -- early -- the layer's retrieval kernels.
+cudaError_t rekv_launch_attend_full_self(rekv_ctx* c, const void* q, const void* k_self, const void* v_self,
+                                         const QBatch& qb, const QBatch& sb, int ncf, cudaStream_t st, int layer0,
+                                         int layer1, bool early) {
   const StoreView& s = c->sv;
   const int nl = layer1 - layer0;
   const bool rope = c->cfg.rope_theta > 0.f;
@@ -340,9 +341,7 @@ cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const vo
     c->launches += 1;
     q_eff = c->q_rot;
   }
-  // the part over X (latency-bound) runs on the side stream beside the pass over the context's keys
-  // (bandwidth-bound); both are joined before the attention kernel
-  const bool fork = rope && !static_ctx && ncf > 0;
+  const bool fork = (rope && !static_ctx && ncf > 0) || early;
   cudaStream_t st_self = fork ? c->side : st;
   cudaError_t e;
   if (fork) {
@@ -355,12 +354,27 @@ cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const vo
       q_eff, (const __nv_bfloat16*)k_self, (const __nv_bfloat16*)v_self, qb, sb, s.Hq, s.Hkv, s.G, n_ctx_tokens,
       rope ? c->rope_tab : nullptr, 1.4426950408889634f / sqrtf(128.f), c->self_o, c->self_ml, layer0);
   c->launches += 1;
-  if (fork) {
-    if ((e = cudaEventRecord(c->ev_side, c->side)) != cudaSuccess) return e;
-    rope_stage_kernel<<<dim3(ncf, qb.nQ, nl), 256, 0, st>>>(c->ctx_tbl, c->tbl_k, c->k_rot, qb.nQ, ncf, s.Hkv, s.Nf,
-                                                            c->rope_tab, layer0);
+  if (fork && (e = cudaEventRecord(c->ev_side, c->side)) != cudaSuccess) return e;
+  c->self_forked = fork;
+  return cudaGetLastError();
+}
+
+// Second half, after the context table is there: rotated copies of the context's keys (consecutive positions), and
+// the join with the part over X if that went to the internal stream.
+cudaError_t rekv_launch_attend_full_ctx(rekv_ctx* c, const QBatch& qb, int ncf, cudaStream_t st, int layer0,
+                                        int layer1) {
+  const StoreView& s = c->sv;
+  const bool rope = c->cfg.rope_theta > 0.f;
+  const bool static_ctx = rope && (c->cfg.flags & REKV_FLAG_ROPE_STATIC) != 0;
+  if (rope && !static_ctx && ncf > 0) {
+    rope_stage_kernel<<<dim3(ncf, qb.nQ, layer1 - layer0), 256, 0, st>>>(c->ctx_tbl, c->tbl_k, c->k_rot, qb.nQ, ncf,
+                                                                        s.Hkv, s.Nf, c->rope_tab, layer0);
     c->launches += 1;
-    if ((e = cudaStreamWaitEvent(st, c->ev_side, 0)) != cudaSuccess) return e;
+  }
+  if (c->self_forked) {
+    c->self_forked = false;
+    cudaError_t e = cudaStreamWaitEvent(st, c->ev_side, 0);
+    if (e != cudaSuccess) return e;
   }
   return cudaGetLastError();
 }

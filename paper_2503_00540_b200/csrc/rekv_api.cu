@@ -513,7 +513,7 @@ int rekv_question(rekv_ctx* c, const void* q, const int32_t* cu_q, int nQ, int t
 
 namespace {
 int attend_full_range(rekv_ctx* c, int layer0, int layer1, const void* q, const void* k_self, const void* v_self,
-                      const QBatch& qb, const QBatch& sb, void* out, cudaStream_t st);
+                      const QBatch& qb, const QBatch& sb, void* out, cudaStream_t st, bool self_done);
 int build_self_batch(rekv_ctx* c, const QBatch& qb, const int32_t* cu_self, int nQ, QBatch* sb);
 }  // namespace
 
@@ -544,6 +544,15 @@ static int question_layer_impl(rekv_ctx* c, int layer, const void* q, const void
   const long long row_bytes = (long long)s.Hq * REKV_HEAD_DIM * 2;
   // the selection goes to the caller's buffer if there is one, else to the context's own
   int32_t* idx = idx_out ? layer_view(idx_out, layer, (long long)nQ * top_k * 4) : c->idx_own;
+  // Eq. 3 in full on an HBM-resident cache: the part over X needs nothing of the retrieval, so it starts on the internal
+  // stream now and runs beside the layer's retrieval kernels (it joins before the attention kernel)
+  const bool self_early = k_self != nullptr && s.tail == 0 && geom.ncf > 0;
+  if (self_early) {
+    const long long kv_layer = (long long)sb.sumNq * s.Hkv * REKV_HEAD_DIM * 2;
+    REKV_CUDA(c, rekv_launch_attend_full_self(c, layer_view(q, layer, qb.sumNq * row_bytes),
+                                              layer_view(k_self, layer, kv_layer), layer_view(v_self, layer, kv_layer),
+                                              qb, sb, geom.ncf, st, layer, layer + 1, true));
+  }
   // cache all in HBM: the selection kernel writes the layer's context table itself (top_k > 0 launches it)
   const bool fused_table = s.tail == 0 && top_k > 0;
   REKV_CUDA(c, rekv_launch_retrieve(c, layer_view(q, layer, qb.sumNq * row_bytes), qb, top_k, geom, n_visible, layer,
@@ -574,7 +583,7 @@ static int question_layer_impl(rekv_ctx* c, int layer, const void* q, const void
     const long long kv_layer = (long long)sb.sumNq * s.Hkv * REKV_HEAD_DIM * 2;
     rc = attend_full_range(c, layer, layer + 1, layer_view(q, layer, qb.sumNq * row_bytes),
                            layer_view(k_self, layer, kv_layer), layer_view(v_self, layer, kv_layer), qb, sb,
-                           layer_view(out, layer, qb.sumNq * row_bytes), st);
+                           layer_view(out, layer, qb.sumNq * row_bytes), st, self_early);
     return rc ? rc : geom.ncf;
   }
   c->q_early_ok = fused_table;  // the selection kernel, which only reads Q, is directly before the attention
@@ -670,10 +679,12 @@ int build_self_batch(rekv_ctx* c, const QBatch& qb, const int32_t* cu_self, int 
 // Eq. 3 in full for layers [layer0, layer1).  q, k_self, v_self and out are indexed with the absolute layer: a caller
 // that holds one layer's rows passes pointers moved back by layer0 layers (layer_view).
 int attend_full_range(rekv_ctx* c, int layer0, int layer1, const void* q, const void* k_self, const void* v_self,
-                      const QBatch& qb, const QBatch& sb, void* out, cudaStream_t st) {
+                      const QBatch& qb, const QBatch& sb, void* out, cudaStream_t st, bool self_done) {
   // an offloaded context: the range's pages must have arrived before the keys are rotated
   if (c->gather_layerwise) REKV_CUDA(c, cudaStreamWaitEvent(st, c->layer_events[layer1 - 1], 0));
-  REKV_CUDA(c, rekv_launch_attend_full_prepare(c, q, k_self, v_self, qb, sb, c->g_ncf, st, layer0, layer1));
+  if (!self_done)
+    REKV_CUDA(c, rekv_launch_attend_full_self(c, q, k_self, v_self, qb, sb, c->g_ncf, st, layer0, layer1, false));
+  REKV_CUDA(c, rekv_launch_attend_full_ctx(c, qb, c->g_ncf, st, layer0, layer1));
   const bool rope = c->cfg.rope_theta > 0.f && !(c->cfg.flags & REKV_FLAG_ROPE_STATIC);  // rotated copies of the context's keys
   const bool rope_q = c->cfg.rope_theta > 0.f;
   if (c->g_ncf == 0) {
@@ -712,7 +723,7 @@ int rekv_attend_full(rekv_ctx* c, const void* q, const void* k_self, const void*
   rc = build_self_batch(c, qb, cu_self, nQ, &sb);
   if (rc) return rc;
   DeviceGuard guard(c->device);
-  return attend_full_range(c, 0, c->sv.L, q, k_self, v_self, qb, sb, out, (cudaStream_t)stream);
+  return attend_full_range(c, 0, c->sv.L, q, k_self, v_self, qb, sb, out, (cudaStream_t)stream, false);
 }
 
 int rekv_attend_full_layer(rekv_ctx* c, int layer, const void* q, const void* k_self, const void* v_self,
@@ -736,7 +747,7 @@ int rekv_attend_full_layer(rekv_ctx* c, int layer, const void* q, const void* k_
   const long long kv_layer = (long long)sb.sumNq * s.Hkv * REKV_HEAD_DIM * 2;
   return attend_full_range(c, layer, layer + 1, layer_view(q, layer, q_layer), layer_view(k_self, layer, kv_layer),
                            layer_view(v_self, layer, kv_layer), qb, sb, layer_view(out, layer, q_layer),
-                           (cudaStream_t)stream);
+                           (cudaStream_t)stream, false);
 }
 
 int rekv_geometry(rekv_ctx* c, int n_visible, int top_k, int32_t* n_scored, int32_t* k_eff, int32_t* w_eff) {

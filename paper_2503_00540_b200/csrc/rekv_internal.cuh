@@ -137,6 +137,7 @@ struct rekv_ctx {
   // test-only knobs of the bounded device-side waits (rekv_test_set_wait_limit); 0 / -1 = off
   unsigned test_wait_limit;
   int test_skip_copy_entry;
+  bool self_forked = false;         // Eq. 3 in full: the part over X is on the internal stream, ev_side marks its end
   bool q_early_ok = false;          // the attention launch that follows is chained to the library's own selection kernels (which only read Q)
 
   // state of the last gather.  The context table has one geometry (questions x context frames) for all layers; a
@@ -252,8 +253,10 @@ cudaError_t rekv_launch_attend_tc5(rekv_ctx* c, const void* q, const QBatch& qb,
                                    void* out, cudaStream_t st, bool timed, const AttendFullArgs* full = nullptr);
 // k_attend_full.cu: the pieces of Eq. 3 in full around the attention kernel
 cudaError_t rekv_launch_rope_table(rekv_ctx* c, cudaStream_t st);
-cudaError_t rekv_launch_attend_full_prepare(rekv_ctx* c, const void* q, const void* k_self, const void* v_self,
-                                            const QBatch& qb, const QBatch& sb, int ncf, cudaStream_t st, int layer0,
-                                            int layer1);
+cudaError_t rekv_launch_attend_full_self(rekv_ctx* c, const void* q, const void* k_self, const void* v_self,
+                                         const QBatch& qb, const QBatch& sb, int ncf, cudaStream_t st, int layer0,
+                                         int layer1, bool early);
+cudaError_t rekv_launch_attend_full_ctx(rekv_ctx* c, const QBatch& qb, int ncf, cudaStream_t st, int layer0,
+                                        int layer1);
 cudaError_t rekv_launch_self_finalize(rekv_ctx* c, const QBatch& qb, void* out, cudaStream_t st, int layer0,
                                       int layer1);
