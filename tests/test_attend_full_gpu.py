@@ -226,3 +226,44 @@ def test_layer_calls_of_eq3_in_full(theta, tail):
         d = (a.float() - b.float()).abs()
         assert d.max().item() <= 4e-3 and d.mean().item() <= 2e-4, f"layer calls vs all-layer calls, {what}: {d.max().item()}"
     g.close()
+
+
+@pytest.mark.parametrize("theta", THETAS)
+def test_layer_calls_of_eq3_in_full_replayed_from_a_cuda_graph(theta):
+    """A decoder captured whole: the layers' rekv_question_layer_full calls as nodes of one graph (the part over X forks
+    to the library's internal stream and joins again inside the capture).  The replay gives the eager calls' bits,
+    also after the buffers were given another question."""
+    s = H.Shape(L=3, Hq=28, Hkv=4, Nf=196, T=40, W=4, k=8, seed=7)
+    g = H.build_gpu(s, max_questions=1, max_q_tokens=32, max_self_tokens=32, rope_theta=theta)
+    q, cu = H.questions(s, [32], device="cuda")
+    ks, vs, cus = H.self_kv(s, [32], device="cuda")
+    q2, _ = H.questions(s, [32], device="cuda", first_id=5)
+    ks2, vs2, _ = H.self_kv(s, [32], device="cuda", first_id=5)
+
+    def eager(qq, kk, vv):
+        o = torch.empty_like(qq)
+        for l in range(s.L):
+            g.question_layer_full(l, qq[l], kk[l], vv[l], cu, cus, s.k, s.T, out=o[l])
+        return o
+
+    ref1, ref2 = eager(q, ks, vs), eager(q2, ks2, vs2)
+    qb, kb, vb, out = q.clone(), ks.clone(), vs.clone(), torch.zeros_like(q)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=side):
+            for l in range(s.L):
+                g.question_layer_full(l, qb[l], kb[l], vb[l], cu, cus, s.k, s.T, out=out[l])
+    torch.cuda.current_stream().wait_stream(side)
+    gr.replay()
+    torch.cuda.synchronize()
+    g.check_status()
+    assert torch.equal(out, ref1)
+    qb.copy_(q2)
+    kb.copy_(ks2)
+    vb.copy_(vs2)
+    gr.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, ref2)
+    g.close()
