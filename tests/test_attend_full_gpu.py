@@ -184,12 +184,14 @@ def test_static_position_variant():
 
 
 @pytest.mark.parametrize("theta", THETAS)
-@pytest.mark.parametrize("tail", [0, 8])
-def test_layer_calls_of_eq3_in_full(theta, tail):
+@pytest.mark.parametrize("tail,k", [(0, 8), (8, 8), (0, 26)])
+def test_layer_calls_of_eq3_in_full(theta, tail, k):
     """What a decoder layer calls with the Q, K, V it has just made of X: rekv_question_layer_full per layer (steps 2-5
     with Eq. 3 in full), then decode steps through rekv_attend_full_layer over the layer's context -- against the
     oracle per layer, and against the all-layer calls on the same selection."""
-    s = H.Shape(L=3, Hq=28, Hkv=4, Nf=196, T=40, W=4, k=8, seed=540, tail=tail)
+    # (k = 26: 30 context frames, ten or eleven partials per unit of a one-layer launch -- the merge kernel for units of
+    # many parts takes the part over X in)
+    s = H.Shape(L=3, Hq=28, Hkv=4, Nf=196, T=40, W=4, k=k, seed=540, tail=tail)
     nq, ns = [24, 33], [24, 40]
     g = H.build_gpu(s, max_questions=2, max_q_tokens=sum(nq), max_self_tokens=sum(ns) + 2, rope_theta=theta)
     o = H.build_oracle(s)
