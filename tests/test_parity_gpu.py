@@ -93,6 +93,14 @@ def test_many_short_questions_whole_units_as_half_streams():
     _run_question_parity(s, lengths, max_questions=20)
 
 
+def test_half_streams_over_a_context_of_a_single_chunk():
+    """As above with three context frames of 33 tokens (113 stream rows: one chunk): the second half-stream of every
+    unit has no chunk at all and contributes the neutral part."""
+    s = H.Shape(L=4, Hq=16, Hkv=8, Nf=33, T=12, W=1, k=2, seed=7)
+    lengths = [9 + (7 * i) % 32 for i in range(20)]
+    _run_question_parity(s, lengths, max_questions=20)
+
+
 def test_short_question_cut_at_cta_boundaries():
     """One 10-token question at the 7B head shape: 70 rows = one row tile per unit, units cut at CTA boundaries
     (four to six partials per unit: the merge kernel joins them)."""
