@@ -108,6 +108,13 @@ def test_short_question_cut_at_cta_boundaries():
     _run_question_parity(s, [10])
 
 
+def test_units_of_two_questions_cut_into_a_few_parts():
+    """The same regime with a batch: 80 units of two questions (160 and 144 rows per KV head), cut into two or three
+    parts and finished inside the kernel."""
+    s = H.Shape(L=5, Hq=16, Hkv=8, Nf=100, T=28, W=4, k=16, seed=540)
+    _run_question_parity(s, [80, 72])
+
+
 def test_units_cut_into_a_few_parts_are_finished_inside_the_kernel():
     """80 units of two row tiles over 146 CTAs (on 148 SMs), eleven of a unit's twenty context frames per CTA: every
     unit is cut into two or three parts, and the CTA that finishes a unit's last part joins them (from its own
