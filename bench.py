@@ -106,12 +106,18 @@ class ClockSampler:
         except Exception:
             self.p = None
 
-    def mark_begin(self):
+    def wait_first_sample(self):
+        """Called before the barrier that opens the timed region, so that nothing here keeps the device idle
+        between that barrier and the first timed step."""
         if self.p is None:
             return
         t0 = time.time()
-        while not self._lines() and time.time() - t0 < 3.0:  # wait for the first sample
+        while not self._lines() and time.time() - t0 < 3.0:
             time.sleep(0.02)
+
+    def mark_begin(self):
+        if self.p is None:
+            return
         self.begin = len(self._lines())
 
     def mark_end(self):
@@ -387,11 +393,12 @@ def run_cuda(args, w):
     for i in range(Wu):
         step_device(i)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    barrier()
-    sampler.mark_begin()
-    l0 = g.launch_count()
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
+    sampler.wait_first_sample()
+    l0 = g.launch_count()
+    barrier()
+    sampler.mark_begin()
     t_begin.record(stream)
     for i in range(K):
         step_device(i, evs[i])
